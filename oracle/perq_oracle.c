@@ -1,0 +1,352 @@
+/*
+ * PeRQ rotate+quantize -- CPU ORACLE.  TEST INFRASTRUCTURE ONLY.
+ *
+ * A plain, slow, fp64 statement of what the online path computes, written from the
+ * paper's definitions.  It exists so that tests (and the benchmark's CPU-baseline leg)
+ * have something independent to compare the CUDA library against.  It shares no code
+ * with the CUDA library, is never linked into it, and the product never calls it.
+ *
+ * Every function cites the passage it follows.  Inputs are bf16 bit patterns (uint16),
+ * widened exactly to double; all arithmetic is double unless stated.
+ *
+ * Parity pins (see tests/test_oracle_*.py): every function here is pinned by closed
+ * forms / invariants / brute force except the storage conventions the paper does not
+ * fix -- "parity unpinned" for: nibble order inside a byte, the all-zero-range
+ * convention (scale 0, codes 0), sign of values that quantise to zero in E2M1, the
+ * MX shared-exponent reading floor(log2 amax) - 2 versus 2^floor(log2(amax/6)), and the
+ * tie-breaks of the greedy permutation.
+ *
+ * Rows are independent; `#pragma omp parallel for` over rows is the only parallelism.
+ */
+#include <fenv.h>
+#include <math.h>
+#include <stdint.h>
+#include <stdlib.h>
+#include <string.h>
+#ifdef _OPENMP
+#include <omp.h>
+#endif
+
+/* ---------------------------------------------------------------- helpers */
+
+static double bf16_to_double(uint16_t h)
+{
+    uint32_t w = (uint32_t)h << 16; /* bf16 is the upper half of an IEEE binary32 */
+    float f;
+    memcpy(&f, &w, sizeof f);
+    return (double)f;
+}
+
+static int popcount32(uint32_t v)
+{
+    int c = 0;
+    while (v) { c += (int)(v & 1u); v >>= 1; }
+    return c;
+}
+
+int perq_oracle_num_threads(void)
+{
+#ifdef _OPENMP
+    return omp_get_max_threads();
+#else
+    return 1;
+#endif
+}
+
+/* ---------------------------------------------------------------- Hadamard matrix
+ * Notation paragraph: R is a normalised Hadamard matrix, columns of unit l2 norm and
+ * entries +-1/sqrt(k).  The Sylvester construction in natural order has entry (k,i)
+ * equal to (-1)^{popcount(k AND i)}.  This writes the UNNORMALISED +-1 matrix, b*b
+ * signed bytes, row-major. */
+int perq_oracle_hadamard_pm1(int32_t b, int8_t *H)
+{
+    if (b < 1 || (b & (b - 1)) != 0 || !H) return 1;
+    for (int32_t k = 0; k < b; ++k)
+        for (int32_t i = 0; i < b; ++i)
+            H[(size_t)k * b + i] = (popcount32((uint32_t)(k & i)) & 1) ? -1 : 1;
+    return 0;
+}
+
+/* ---------------------------------------------------------------- permute + rotate
+ * Notation paragraph: X is a row vector, d = n*b; P e_i = e_{pi(i)} so (X P)_i =
+ * X_{pi(i)} (a gather); R~ = I_n (x) R acts on each contiguous block of b coordinates
+ * (proof of the probabilistic proposition, coordinate form: X~_i = sum over k in the
+ * block of i of X_k R~_{k,i}).
+ *
+ * y[t, j*b + i] = (1/sqrt(b)) * sum_{k<b} x'[t, j*b + k] * H[k][i],  x'[i] = x[perm[i]].
+ * The sum is an explicit matrix-vector product (k ascending), no butterfly.
+ * perm == NULL is the identity.  b may be any power of two >= 1 that divides d. */
+int perq_oracle_rotate(const uint16_t *x, const int32_t *perm, int64_t T, int32_t d,
+                       int32_t b, double *y)
+{
+    if (!x || !y || T < 0 || d <= 0 || b < 1 || (b & (b - 1)) != 0 || d % b != 0) return 1;
+    if (perm)
+        for (int32_t i = 0; i < d; ++i)
+            if (perm[i] < 0 || perm[i] >= d) return 2;
+    int8_t *H = (int8_t *)malloc((size_t)b * b);
+    if (!H) return 3;
+    perq_oracle_hadamard_pm1(b, H);
+    const double sqrt_b = sqrt((double)b);
+    int fail = 0;
+#pragma omp parallel
+    {
+        double *xp = (double *)malloc(sizeof(double) * (size_t)d);
+        double *u = (double *)malloc(sizeof(double) * (size_t)b);
+        if (!xp || !u) {
+#pragma omp atomic write
+            fail = 1;
+        } else {
+#pragma omp for schedule(static)
+            for (int64_t t = 0; t < T; ++t) {
+                const uint16_t *row = x + (size_t)t * d;
+                for (int32_t i = 0; i < d; ++i)
+                    xp[i] = bf16_to_double(row[perm ? perm[i] : i]);
+                for (int32_t j = 0; j < d / b; ++j) {
+                    for (int32_t i = 0; i < b; ++i) u[i] = 0.0;
+                    for (int32_t k = 0; k < b; ++k) {
+                        const double xk = xp[(size_t)j * b + k];
+                        const int8_t *Hk = H + (size_t)k * b;
+                        for (int32_t i = 0; i < b; ++i) u[i] += xk * (double)Hk[i];
+                    }
+                    for (int32_t i = 0; i < b; ++i)
+                        y[(size_t)t * d + (size_t)j * b + i] = u[i] / sqrt_b;
+                }
+            }
+        }
+        free(xp);
+        free(u);
+    }
+    free(H);
+    return fail ? 3 : 0;
+}
+
+/* ---------------------------------------------------------------- packing
+ * The paper has no storage format.  Two 4-bit codes per byte: byte k of a row holds
+ * code[2k] in its low nibble and code[2k+1] in its high nibble. */
+static void pack_row(const uint8_t *codes, int32_t d, uint8_t *out)
+{
+    for (int32_t k = 0; k < d / 2; ++k)
+        out[k] = (uint8_t)((codes[2 * k] & 0xF) | ((codes[2 * k + 1] & 0xF) << 4));
+}
+
+/* ---------------------------------------------------------------- INT4
+ * Sec. 3: step size s = ||X||_inf / (2^{q-1} - 1), q = 4, taken over the scale range
+ * (the whole token when group == 0, else each contiguous `group` coordinates of the
+ * rotated row).  Appendix B quantiser with zero point 0: q_i = clip(round(y_i / s),
+ * -8, 7), round = nearest, ties to even.  The division uses the real (double) s; the
+ * stored scale is s rounded to binary32.  A range whose max is 0 stores scale 0 and
+ * codes 0.
+ *
+ * codes: packed [T, d/2]; scales: float [T] or [T, d/group];
+ * v_pre (optional, may be NULL): the pre-rounding values y_i / s, [T, d]. */
+int perq_oracle_quantize_int4(const double *y, int64_t T, int32_t d, int32_t group,
+                              uint8_t *codes, float *scales, double *v_pre)
+{
+    if (!y || !codes || !scales || T < 0 || d <= 0 || d % 2 != 0 || group < 0) return 1;
+    const int32_t g = group == 0 ? d : group;
+    if (d % g != 0) return 1;
+    if (fegetround() != FE_TONEAREST) return 4;
+    const int32_t ng = d / g;
+#pragma omp parallel
+    {
+        uint8_t *c = (uint8_t *)malloc((size_t)d);
+#pragma omp for schedule(static)
+        for (int64_t t = 0; t < T; ++t) {
+            const double *yr = y + (size_t)t * d;
+            for (int32_t r = 0; r < ng; ++r) {
+                double a = 0.0;
+                for (int32_t i = 0; i < g; ++i) {
+                    const double m = fabs(yr[(size_t)r * g + i]);
+                    if (m > a) a = m;
+                }
+                const double s = a / 7.0;
+                scales[(size_t)t * ng + r] = (a == 0.0) ? 0.0f : (float)s;
+                for (int32_t i = 0; i < g; ++i) {
+                    const size_t idx = (size_t)r * g + i;
+                    double v = 0.0, q = 0.0;
+                    if (a != 0.0) {
+                        v = yr[idx] / s;
+                        q = nearbyint(v); /* FE_TONEAREST: ties to even */
+                        if (q > 7.0) q = 7.0;
+                        if (q < -8.0) q = -8.0;
+                    }
+                    if (v_pre) v_pre[(size_t)t * d + idx] = v;
+                    c[idx] = (uint8_t)((int)q & 0xF); /* two's complement nibble */
+                }
+            }
+            pack_row(c, d, codes + (size_t)t * (d / 2));
+        }
+        free(c);
+    }
+    return 0;
+}
+
+/* ---------------------------------------------------------------- MXFP4
+ * Appendix B, "(MX)FP4 Quantization": elements are E2M1 (e = 2, m = 1, per the OCP MX
+ * specification the paper cites), one shared scale per 32 elements, rounded down to a
+ * power of two.  Reading of the shared exponent (the printed formula is garbled):
+ * E = floor(log2(max |y|)) - 2, where 2 is the exponent of the largest E2M1 value
+ * 6 = 1.5 * 2^2; stored as E8M0 = clamp(E, -127, 127) + 127.
+ * Elements: v = y * 2^-E (exact), magnitude rounded to the nearest of
+ * {0, .5, 1, 1.5, 2, 3, 4, 6}, ties to the even code, |v| > 6 saturates to 6; the sign
+ * bit of y is kept (code = sign << 3 | index).  An all-zero group stores E8M0 = 0.
+ *
+ * codes: packed [T, d/2]; e8m0: uint8 [T, d/32];
+ * v_pre (optional): the pre-rounding scaled values y_i * 2^-E, [T, d]. */
+static const double E2M1_GRID[8] = {0.0, 0.5, 1.0, 1.5, 2.0, 3.0, 4.0, 6.0};
+
+static int e2m1_nearest_index(double mag)
+{
+    if (mag >= 6.0) return 7;
+    for (int k = 0; k < 7; ++k) {
+        const double lo = E2M1_GRID[k], hi = E2M1_GRID[k + 1];
+        if (mag >= lo && mag <= hi) {
+            const double mid = 0.5 * (lo + hi); /* exact: grid values are dyadic */
+            if (mag < mid) return k;
+            if (mag > mid) return k + 1;
+            return (k % 2 == 0) ? k : k + 1; /* tie: the even code */
+        }
+    }
+    return 7;
+}
+
+int perq_oracle_quantize_mxfp4(const double *y, int64_t T, int32_t d, uint8_t *codes,
+                               uint8_t *e8m0, double *v_pre)
+{
+    if (!y || !codes || !e8m0 || T < 0 || d <= 0 || d % 32 != 0) return 1;
+    const int32_t ng = d / 32;
+#pragma omp parallel
+    {
+        uint8_t *c = (uint8_t *)malloc((size_t)d);
+#pragma omp for schedule(static)
+        for (int64_t t = 0; t < T; ++t) {
+            const double *yr = y + (size_t)t * d;
+            for (int32_t r = 0; r < ng; ++r) {
+                double a = 0.0;
+                for (int32_t i = 0; i < 32; ++i) {
+                    const double m = fabs(yr[(size_t)r * 32 + i]);
+                    if (m > a) a = m;
+                }
+                int E = -127;
+                if (a != 0.0) {
+                    int e;
+                    (void)frexp(a, &e);  /* a = m * 2^e, m in [0.5, 1)  =>  floor(log2 a) = e - 1 */
+                    E = (e - 1) - 2;
+                    if (E < -127) E = -127;
+                    if (E > 127) E = 127;
+                }
+                e8m0[(size_t)t * ng + r] = (a == 0.0) ? 0 : (uint8_t)(E + 127);
+                for (int32_t i = 0; i < 32; ++i) {
+                    const size_t idx = (size_t)r * 32 + i;
+                    const double v = ldexp(yr[idx], -E);
+                    if (v_pre) v_pre[(size_t)t * d + idx] = v;
+                    const int k = e2m1_nearest_index(fabs(v));
+                    c[idx] = (uint8_t)((signbit(yr[idx]) ? 8 : 0) | k);
+                }
+            }
+            pack_row(c, d, codes + (size_t)t * (d / 2));
+        }
+        free(c);
+    }
+    return 0;
+}
+
+/* ---------------------------------------------------------------- whole path
+ * (X P) R~ then Q(.), Fig. "perq-pipeline" / Sec. 4 overview.  fmt: 0 = INT4, 1 = MXFP4.
+ * y_out (optional) receives the rotated row, v_pre (optional) the pre-rounding values. */
+int perq_oracle_rotate_quantize(const uint16_t *x, const int32_t *perm, int64_t T, int32_t d,
+                                int32_t b, int32_t fmt, int32_t group, uint8_t *codes,
+                                void *scales, double *y_out, double *v_pre)
+{
+    if (T < 0 || d <= 0) return 1;
+    double *y = y_out ? y_out : (double *)malloc(sizeof(double) * (size_t)(T > 0 ? T : 1) * d);
+    if (!y) return 3;
+    int rc = perq_oracle_rotate(x, perm, T, d, b, y);
+    if (rc == 0) {
+        if (fmt == 0) rc = perq_oracle_quantize_int4(y, T, d, group, codes, (float *)scales, v_pre);
+        else if (fmt == 1) rc = perq_oracle_quantize_mxfp4(y, T, d, codes, (uint8_t *)scales, v_pre);
+        else rc = 1;
+    }
+    if (!y_out) free(y);
+    return rc;
+}
+
+/* ---------------------------------------------------------------- calibration statistic
+ * Algorithm 1 (MassDiff) uses the per-coordinate mean magnitude (1/m) sum_k |X_i^(k)|
+ * and the per-block mean l1 norm (1/m) sum_k ||X^(k)_{B_j}||_1; the block proposition
+ * bounds ||X R~||_inf by max_j ||X_{j}||_1 / sqrt(b).
+ *
+ * chan_abs_sum[c]        = sum_t |x[t, c]|                 (original channel order)
+ * block_l1_mean[j]       = (1/T) sum_t L[t, j]             L[t, j] = sum_{i<b} |x'[t, j*b+i]|
+ * token_max_block_l1[t]  = max_j L[t, j]                   x' = gather(x, perm)
+ * Any output pointer may be NULL. */
+int perq_oracle_block_l1_stats(const uint16_t *x, const int32_t *perm, int64_t T, int32_t d,
+                               int32_t b, double *chan_abs_sum, double *block_l1_mean,
+                               double *token_max_block_l1)
+{
+    if (!x || T < 0 || d <= 0 || b < 1 || d % b != 0) return 1;
+    if (perm)
+        for (int32_t i = 0; i < d; ++i)
+            if (perm[i] < 0 || perm[i] >= d) return 2;
+    const int32_t n = d / b;
+    if (chan_abs_sum) for (int32_t c = 0; c < d; ++c) chan_abs_sum[c] = 0.0;
+    if (block_l1_mean) for (int32_t j = 0; j < n; ++j) block_l1_mean[j] = 0.0;
+    for (int64_t t = 0; t < T; ++t) {
+        const uint16_t *row = x + (size_t)t * d;
+        if (chan_abs_sum)
+            for (int32_t c = 0; c < d; ++c) chan_abs_sum[c] += fabs(bf16_to_double(row[c]));
+        double mx = 0.0;
+        for (int32_t j = 0; j < n; ++j) {
+            double L = 0.0;
+            for (int32_t i = 0; i < b; ++i) {
+                const int32_t src = perm ? perm[(size_t)j * b + i] : j * b + i;
+                L += fabs(bf16_to_double(row[src]));
+            }
+            if (block_l1_mean) block_l1_mean[j] += L;
+            if (L > mx) mx = L;
+        }
+        if (token_max_block_l1) token_max_block_l1[t] = mx;
+    }
+    if (block_l1_mean && T > 0)
+        for (int32_t j = 0; j < n; ++j) block_l1_mean[j] /= (double)T;
+    return 0;
+}
+
+/* ---------------------------------------------------------------- MassDiff (Algorithm 1)
+ * Visit coordinates in descending mean magnitude; put each into the not-yet-full block
+ * whose running mean l1 norm is smallest; drop a block from the candidates once it holds
+ * b coordinates; return the blocks concatenated.  The argmin's "+ |X_i|" term is common
+ * to all blocks, so only the running block sums matter, and since the mean is a positive
+ * multiple of the sum the channel sums can stand in for the means.
+ * Unfixed by the paper: sort ties -> lower channel index first; argmin ties -> lower
+ * block index.  perm[j*b + r] = the r-th coordinate assigned to block j. */
+int perq_oracle_massdiff_perm(const double *chan_abs_sum, int32_t d, int32_t b, int32_t *perm)
+{
+    if (!chan_abs_sum || !perm || d <= 0 || b < 1 || d % b != 0) return 1;
+    const int32_t n = d / b;
+    int32_t *order = (int32_t *)malloc(sizeof(int32_t) * (size_t)d);
+    double *mass = (double *)calloc((size_t)n, sizeof(double));
+    int32_t *fill = (int32_t *)calloc((size_t)n, sizeof(int32_t));
+    if (!order || !mass || !fill) { free(order); free(mass); free(fill); return 3; }
+    for (int32_t i = 0; i < d; ++i) order[i] = i;
+    /* stable insertion sort, descending: equal values keep ascending index order */
+    for (int32_t i = 1; i < d; ++i) {
+        const int32_t c = order[i];
+        int32_t p = i - 1;
+        while (p >= 0 && chan_abs_sum[order[p]] < chan_abs_sum[c]) { order[p + 1] = order[p]; --p; }
+        order[p + 1] = c;
+    }
+    for (int32_t s = 0; s < d; ++s) {
+        const int32_t c = order[s];
+        int32_t best = -1;
+        for (int32_t j = 0; j < n; ++j) {
+            if (fill[j] >= b) continue;              /* block j is full: not in J */
+            if (best < 0 || mass[j] < mass[best]) best = j;
+        }
+        perm[(size_t)best * b + fill[best]] = c;
+        fill[best] += 1;
+        mass[best] += chan_abs_sum[c];
+    }
+    free(order); free(mass); free(fill);
+    return 0;
+}
