@@ -1,0 +1,165 @@
+/*
+ * perq.h -- C ABI of the PeRQ online path for NVIDIA B200 (sm_100a).
+ *
+ * PeRQ = Permute, Rotate, then Quantize.  For activation rows X[T, d] (bf16) the path is
+ *
+ *     (X P)  ->  (X P) R~  ->  Q((X P) R~)
+ *
+ * with P a channel permutation applied as a gather, R~ = I_n (x) R a block-diagonal
+ * rotation whose b x b block R is the normalised Sylvester Hadamard matrix, and Q a 4-bit
+ * quantiser (symmetric INT4 or MXFP4).  Citations below are to the paper's sections,
+ * equations and algorithms.
+ *
+ * Conventions for every entry point
+ *   - "device" pointers are CUDA device memory, "host" pointers ordinary host memory.
+ *   - The caller owns every buffer; nothing is allocated, freed or retained by the
+ *     library.
+ *   - Work is enqueued on `stream` (a cudaStream_t passed as void*, NULL = default
+ *     stream); no call synchronises the device unless it says so.  Outputs are valid
+ *     once the caller has synchronised `stream`.
+ *   - The return value is a perq_status_t.  Arguments are checked on the host before
+ *     anything is launched; on an error nothing has been enqueued.
+ *   - Device pointers must be 16-byte aligned.  Rows are dense (row stride = d).
+ *   - Inputs are assumed finite.  NaN/Inf give unspecified codes but never a fault.
+ */
+#ifndef PERQ_H
+#define PERQ_H
+
+#include <stddef.h>
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+typedef enum {
+    PERQ_FMT_INT4 = 0,      /* symmetric INT4, absmax scale (fp32) per token or per group */
+    PERQ_FMT_MXFP4 = 1,     /* E2M1 elements, one E8M0 scale per 32 elements */
+    PERQ_FMT_F32_DEBUG = 2  /* no quantisation: the rotated row as fp32 (test hook) */
+} perq_fmt_t;
+
+typedef enum {
+    PERQ_OK = 0,
+    PERQ_ERR_NULL = 1,   /* a required pointer is NULL */
+    PERQ_ERR_SHAPE = 2,  /* T < 0, d <= 0, d % 32 != 0 or d > PERQ_MAX_D */
+    PERQ_ERR_BLOCK = 3,  /* b is not one of 16/32/64/128 dividing d, nor b == d with d a power of two */
+    PERQ_ERR_GROUP = 4,  /* INT4: group not 0 and (d % group != 0 or group % 8 != 0); MXFP4: group not 0/32 */
+    PERQ_ERR_FMT = 5,    /* unknown format */
+    PERQ_ERR_ALIGN = 6,  /* a device pointer is not 16-byte aligned */
+    PERQ_ERR_CUDA = 7,   /* the CUDA runtime reported an error (launch, copy, attribute) */
+    PERQ_ERR_PERM = 8,   /* host-side permutation argument is not a permutation */
+    PERQ_ERR_WORKSPACE = 9 /* workspace missing or too small */
+} perq_status_t;
+
+#define PERQ_MAX_D 32768
+
+/*
+ * perq_rotate_quantize -- the online hot path, one fused pass.
+ *
+ * Defined by: Notation paragraph of Sec. 1 (row vector X, d = n*b, block rotation
+ * R~ = I_n (x) R, permutation P e_i = e_pi(i)); the block proposition of Sec. 3 and the
+ * coordinate form in the proof of the probabilistic proposition (blocks are contiguous
+ * index ranges of the permuted row); Sec. 3 for the INT step size
+ * s = ||X||_inf / (2^{q-1} - 1); Appendix B for the INT4 and (MX)FP4 quantisers.
+ *
+ * For every token row t:
+ *   1. x'_i = x[t, perm[i]]                       (perm == NULL: x' = x)
+ *   2. y_{j*b+i} = b^{-1/2} * sum_{k<b} (-1)^{popcount(i & k)} x'_{j*b+k}   for each block j
+ *   3. INT4:  per scale range G (whole row if group == 0, else each `group` consecutive
+ *             coordinates of y): a = max_G |y|, s = a / 7, code_i = clip(rne(y_i / s), -8, 7),
+ *             stored scale = s as fp32.  a == 0 gives scale 0 and codes 0.
+ *      MXFP4: per 32 consecutive coordinates: a = max |y|, E = floor(log2 a) - 2 clamped to
+ *             [-127, 127], stored scale byte = E + 127 (0 if a == 0); element code =
+ *             sign(y_i) << 3 | index of the nearest of {0, .5, 1, 1.5, 2, 3, 4, 6} to
+ *             |y_i| * 2^-E, ties to the even index, saturating at 6.
+ *   4. byte k of the output row = code[2k] | code[2k+1] << 4  (INT4 nibbles are two's complement).
+ *
+ * x          device, bf16 [T, d] row-major.
+ * perm       device, int32 [d], a permutation of 0..d-1, or NULL.  Out-of-range entries
+ *            are clamped into range (wrong numbers, never a fault); use
+ *            perq_validate_perm to check a permutation beforehand.
+ * T, d       rows and channels.  T == 0 is a no-op.  d % 32 == 0, d <= PERQ_MAX_D.
+ * b          16, 32, 64 or 128 with d % b == 0; or b == d when d is a power of two.
+ * fmt        perq_fmt_t.
+ * group      INT4: 0 (per token) or a multiple of 8 dividing d.  MXFP4: 0 or 32 (always 32).
+ *            Scale ranges are consecutive coordinates of the ROTATED row, independent of b.
+ * out_codes  device.  INT4/MXFP4: uint8 [T, d/2].  F32_DEBUG: float [T, d] (the rotated row y).
+ * out_scales device.  INT4: float [T] or [T, d/group].  MXFP4: uint8 [T, d/32].  F32_DEBUG: unused, may be NULL.
+ *
+ * Codes and scales are deterministic (bit-identical from run to run).
+ */
+int perq_rotate_quantize(const void *x, const int32_t *perm, int64_t T, int32_t d, int32_t b,
+                         int32_t fmt, int32_t group, void *out_codes, void *out_scales,
+                         void *stream);
+
+/*
+ * perq_out_sizes -- bytes of out_codes and out_scales for a call.  Host only, no CUDA.
+ * Either output pointer may be NULL.
+ */
+int perq_out_sizes(int64_t T, int32_t d, int32_t fmt, int32_t group, size_t *codes_bytes,
+                   size_t *scales_bytes);
+
+/*
+ * perq_rotate_quantize_host -- the same operation on HOST buffers.
+ *
+ * Copies x from host memory (pinned memory makes the copies asynchronous), runs
+ * perq_rotate_quantize on the device and copies codes and scales back, all on `stream`,
+ * then synchronises `stream` before returning.  `workspace` is device memory provided
+ * by the caller, at least perq_host_workspace_bytes(...) long; the library allocates
+ * nothing.  perm stays a DEVICE pointer (it is reused across calls) or NULL.
+ */
+int perq_rotate_quantize_host(const void *x_host, const int32_t *perm, int64_t T, int32_t d,
+                              int32_t b, int32_t fmt, int32_t group, void *out_codes_host,
+                              void *out_scales_host, void *workspace, size_t workspace_bytes,
+                              void *stream);
+int perq_host_workspace_bytes(int64_t T, int32_t d, int32_t fmt, int32_t group, size_t *bytes);
+
+/*
+ * perq_block_l1_stats -- the calibration statistic of the greedy mass-diffusion
+ * permutation (Algorithm 1: per-coordinate mean magnitude and per-block mean l1 norm)
+ * and of the block proposition's bound ||X R~||_inf <= max_j ||X_{j}||_1 / sqrt(b).
+ *
+ *   chan_abs_sum[c]       = sum_t |x[t, c]|                         (original channel order)
+ *   block_l1_mean[j]      = (1/T) sum_t L[t, j],   L[t, j] = sum_{i<b} |x[t, perm[j*b+i]]|
+ *   token_max_block_l1[t] = max_j L[t, j]
+ *
+ * x, perm, T, d as above (T >= 1 here unless all outputs are NULL); b any power of two
+ * >= 8 dividing d (or b == d).  Each output is device fp32 and may be NULL: [d], [d/b], [T].
+ * workspace  device, perq_block_l1_stats_workspace_bytes(...) bytes: per-CTA partial sums
+ *            that a second kernel adds in a fixed order, so results are deterministic.
+ * Accumulation is fp32: sums agree with exact arithmetic to about 1e-6 relative.
+ */
+int perq_block_l1_stats(const void *x, const int32_t *perm, int64_t T, int32_t d, int32_t b,
+                        float *chan_abs_sum, float *block_l1_mean, float *token_max_block_l1,
+                        void *workspace, size_t workspace_bytes, void *stream);
+int perq_block_l1_stats_workspace_bytes(int64_t T, int32_t d, int32_t b, size_t *bytes);
+
+/*
+ * perq_validate_perm -- checks on the device that perm[0..d) is a permutation.
+ * Writes one int32 to status_dev: 0 = valid, bit 0 = an entry out of range,
+ * bit 1 = a duplicate entry.  (Algorithm 1 returns such a permutation; this guards
+ * perq_rotate_quantize against a corrupted one.)
+ */
+int perq_validate_perm(const int32_t *perm, int32_t d, int32_t *status_dev, void *stream);
+
+/*
+ * perq_massdiff_perm -- Algorithm 1 (MassDiff), host only, no CUDA.
+ *
+ * Visits channels in descending chan_abs_sum (ties: lower channel first), assigns each
+ * to the not-yet-full block with the smallest running sum (ties: lower block first), and
+ * returns the blocks concatenated: perm[j*b + r] = r-th channel assigned to block j.  The
+ * result is the `perm` argument of perq_rotate_quantize / perq_block_l1_stats.
+ * chan_abs_sum_host: float [d] (e.g. copied back from perq_block_l1_stats; the mean is a
+ * positive multiple of the sum, so sums give the same permutation).  perm_host: int32 [d].
+ * Running sums are kept in double.  b >= 1, d % b == 0.
+ */
+int perq_massdiff_perm(const float *chan_abs_sum_host, int32_t d, int32_t b, int32_t *perm_host);
+
+/* Text for a status code (static storage).  Library version = major*10000 + minor*100 + patch. */
+const char *perq_status_string(int status);
+int perq_version(void);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* PERQ_H */

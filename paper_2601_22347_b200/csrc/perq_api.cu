@@ -1,0 +1,299 @@
+// C ABI of the PeRQ online path: argument validation, kernel selection, launches.
+// Nothing here allocates device memory or synchronises, except where perq.h says so.
+#include "perq.h"
+
+#include <algorithm>
+#include <cmath>
+#include <cstdint>
+#include <queue>
+#include <utility>
+#include <vector>
+
+#include <cuda_runtime.h>
+
+#include "perq_generic.cuh"
+#include "perq_stats.cuh"
+
+namespace {
+
+constexpr int kVersion = 100;   // 0.1.0
+constexpr size_t kMaxSmem = 227 * 1024;
+
+inline bool is_pow2(long long v) { return v > 0 && (v & (v - 1)) == 0; }
+inline int ilog2(int v) { int l = 0; while ((1 << l) < v) ++l; return l; }
+inline bool aligned16(const void *p) { return (reinterpret_cast<uintptr_t>(p) & 15u) == 0; }
+
+// Common shape checks.  On success *g_out is the effective scale-range length.
+int check_shape(int64_t T, int32_t d, int32_t b, int32_t fmt, int32_t group, int *g_out)
+{
+    if (T < 0 || d <= 0 || d % 32 != 0 || d > PERQ_MAX_D) return PERQ_ERR_SHAPE;
+    if (fmt != PERQ_FMT_INT4 && fmt != PERQ_FMT_MXFP4 && fmt != PERQ_FMT_F32_DEBUG) return PERQ_ERR_FMT;
+    const bool small_block = (b == 16 || b == 32 || b == 64 || b == 128) && d % b == 0;
+    const bool full_vector = (b == d) && is_pow2(d);
+    if (!small_block && !full_vector) return PERQ_ERR_BLOCK;
+    int g = d;
+    if (fmt == PERQ_FMT_INT4) {
+        if (group < 0) return PERQ_ERR_GROUP;
+        if (group > 0) {
+            if (d % group != 0 || group % 8 != 0) return PERQ_ERR_GROUP;
+            g = group;
+        }
+    } else if (fmt == PERQ_FMT_MXFP4) {
+        if (group != 0 && group != 32) return PERQ_ERR_GROUP;
+        g = 32;
+    }
+    if (g_out) *g_out = g;
+    return PERQ_OK;
+}
+
+int sm_count()
+{
+    static int cached = 0;
+    if (cached == 0) {
+        int dev = 0, n = 0;
+        if (cudaGetDevice(&dev) != cudaSuccess) return 0;
+        if (cudaDeviceGetAttribute(&n, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess) return 0;
+        cached = n;
+    }
+    return cached;
+}
+
+template <typename K>
+int allow_smem(K kernel, size_t bytes)
+{
+    if (bytes > 48 * 1024) {
+        if (cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)bytes) != cudaSuccess) {
+            (void)cudaGetLastError();
+            return PERQ_ERR_CUDA;
+        }
+    }
+    return PERQ_OK;
+}
+
+int launch_generic(const void *x, const int32_t *perm, int64_t T, int32_t d, int32_t b, int32_t fmt, int g,
+                   void *out_codes, void *out_scales, cudaStream_t st)
+{
+    perq::GenParams p;
+    p.x = static_cast<const uint16_t *>(x);
+    p.perm = perm;
+    p.T = T;
+    p.d = d;
+    p.log2b = ilog2(b);
+    p.fmt = fmt;
+    p.g = g;
+    p.out_codes = out_codes;
+    p.out_scales = out_scales;
+    p.sqrt_b = std::sqrt((double)b);
+    p.inv_sqrt_b = (float)(1.0 / p.sqrt_b);
+    const perq::GenSmem lay(d, g, p.log2b);
+    if (lay.total > kMaxSmem) return PERQ_ERR_SHAPE;
+    if (int rc = allow_smem(perq::perq_generic_kernel, lay.total)) return rc;
+    const int sms = sm_count();
+    if (sms <= 0) return PERQ_ERR_CUDA;
+    const int per_sm = (int)std::max<size_t>(1, std::min<size_t>(2048 / perq::GEN_THREADS, kMaxSmem / lay.total));
+    const long long grid = std::min<long long>(T, (long long)sms * per_sm);
+    perq::perq_generic_kernel<<<(unsigned)grid, perq::GEN_THREADS, lay.total, st>>>(p);
+    return cudaGetLastError() == cudaSuccess ? PERQ_OK : PERQ_ERR_CUDA;
+}
+
+struct StatsPlan {
+    int n_cta;
+    int rows_per_cta;
+    size_t smem;
+    size_t ws_bytes;
+};
+
+int plan_stats(int64_t T, int32_t d, int32_t b, StatsPlan *plan)
+{
+    if (T < 0 || d <= 0 || d % 32 != 0 || d > PERQ_MAX_D) return PERQ_ERR_SHAPE;
+    if (!is_pow2(b) || b < 8 || d % b != 0) return PERQ_ERR_BLOCK;
+    // The CTA count is a fixed function of the shape (not of the device) so that the
+    // order of additions, and with it every output bit, is the same everywhere.
+    const int max_cta = 148;
+    const long long rows = std::max<long long>(1, (T + max_cta - 1) / max_cta);
+    plan->rows_per_cta = (int)std::min<long long>(rows, 1 << 30);
+    plan->n_cta = (int)std::max<long long>(1, (T + rows - 1) / rows);
+    plan->smem = (size_t)d * 4 + (size_t)(d / 8) * 4 + 32 * 4;
+    plan->ws_bytes = (size_t)plan->n_cta * ((size_t)d + (size_t)(d / b)) * sizeof(float);
+    return PERQ_OK;
+}
+
+}  // namespace
+
+extern "C" {
+
+int perq_version(void) { return kVersion; }
+
+const char *perq_status_string(int status)
+{
+    switch (status) {
+    case PERQ_OK: return "ok";
+    case PERQ_ERR_NULL: return "a required pointer is NULL";
+    case PERQ_ERR_SHAPE: return "bad shape: need T >= 0, 0 < d <= 32768, d % 32 == 0 (and the row must fit in shared memory)";
+    case PERQ_ERR_BLOCK: return "bad block size: need b in {16,32,64,128} dividing d, or b == d with d a power of two";
+    case PERQ_ERR_GROUP: return "bad group: INT4 needs 0 or a multiple of 8 dividing d; MXFP4 needs 0 or 32";
+    case PERQ_ERR_FMT: return "unknown format";
+    case PERQ_ERR_ALIGN: return "device pointers must be 16-byte aligned";
+    case PERQ_ERR_CUDA: return "CUDA runtime error";
+    case PERQ_ERR_PERM: return "not a permutation";
+    case PERQ_ERR_WORKSPACE: return "workspace missing or too small";
+    default: return "unknown status";
+    }
+}
+
+int perq_out_sizes(int64_t T, int32_t d, int32_t fmt, int32_t group, size_t *codes_bytes, size_t *scales_bytes)
+{
+    if (T < 0 || d <= 0 || d % 32 != 0 || d > PERQ_MAX_D) return PERQ_ERR_SHAPE;
+    size_t cb = 0, sb = 0;
+    if (fmt == PERQ_FMT_INT4) {
+        if (group < 0 || (group > 0 && (d % group != 0 || group % 8 != 0))) return PERQ_ERR_GROUP;
+        cb = (size_t)T * (size_t)(d / 2);
+        sb = (size_t)T * (size_t)(group == 0 ? 1 : d / group) * sizeof(float);
+    } else if (fmt == PERQ_FMT_MXFP4) {
+        if (group != 0 && group != 32) return PERQ_ERR_GROUP;
+        cb = (size_t)T * (size_t)(d / 2);
+        sb = (size_t)T * (size_t)(d / 32);
+    } else if (fmt == PERQ_FMT_F32_DEBUG) {
+        cb = (size_t)T * (size_t)d * sizeof(float);
+        sb = 0;
+    } else {
+        return PERQ_ERR_FMT;
+    }
+    if (codes_bytes) *codes_bytes = cb;
+    if (scales_bytes) *scales_bytes = sb;
+    return PERQ_OK;
+}
+
+int perq_rotate_quantize(const void *x, const int32_t *perm, int64_t T, int32_t d, int32_t b, int32_t fmt,
+                         int32_t group, void *out_codes, void *out_scales, void *stream)
+{
+    int g = 0;
+    if (int rc = check_shape(T, d, b, fmt, group, &g)) return rc;
+    if (!x || !out_codes || (fmt != PERQ_FMT_F32_DEBUG && !out_scales)) return PERQ_ERR_NULL;
+    if (!aligned16(x) || !aligned16(out_codes) || !aligned16(out_scales) || !aligned16(perm)) return PERQ_ERR_ALIGN;
+    if (T == 0) return PERQ_OK;
+    return launch_generic(x, perm, T, d, b, fmt, g, out_codes, out_scales, static_cast<cudaStream_t>(stream));
+}
+
+int perq_host_workspace_bytes(int64_t T, int32_t d, int32_t fmt, int32_t group, size_t *bytes)
+{
+    size_t cb = 0, sb = 0;
+    if (int rc = perq_out_sizes(T, d, fmt, group, &cb, &sb)) return rc;
+    if (!bytes) return PERQ_ERR_NULL;
+    auto up = [](size_t v) { return (v + 255) & ~(size_t)255; };
+    *bytes = up((size_t)T * (size_t)d * 2) + up(cb) + up(sb) + 256;
+    return PERQ_OK;
+}
+
+int perq_rotate_quantize_host(const void *x_host, const int32_t *perm, int64_t T, int32_t d, int32_t b,
+                              int32_t fmt, int32_t group, void *out_codes_host, void *out_scales_host,
+                              void *workspace, size_t workspace_bytes, void *stream)
+{
+    int g = 0;
+    if (int rc = check_shape(T, d, b, fmt, group, &g)) return rc;
+    if (!x_host || !out_codes_host || (fmt != PERQ_FMT_F32_DEBUG && !out_scales_host)) return PERQ_ERR_NULL;
+    size_t need = 0, cb = 0, sb = 0;
+    perq_host_workspace_bytes(T, d, fmt, group, &need);
+    perq_out_sizes(T, d, fmt, group, &cb, &sb);
+    if (T == 0) return PERQ_OK;
+    if (!workspace || workspace_bytes < need) return PERQ_ERR_WORKSPACE;
+    if (!aligned16(workspace) || !aligned16(perm)) return PERQ_ERR_ALIGN;
+    auto up = [](size_t v) { return (v + 255) & ~(size_t)255; };
+    cudaStream_t st = static_cast<cudaStream_t>(stream);
+    unsigned char *base = static_cast<unsigned char *>(workspace);
+    base = reinterpret_cast<unsigned char *>((reinterpret_cast<uintptr_t>(base) + 255) & ~(uintptr_t)255);
+    unsigned char *x_dev = base;
+    unsigned char *codes_dev = x_dev + up((size_t)T * (size_t)d * 2);
+    unsigned char *scales_dev = codes_dev + up(cb);
+    if (cudaMemcpyAsync(x_dev, x_host, (size_t)T * (size_t)d * 2, cudaMemcpyHostToDevice, st) != cudaSuccess)
+        return PERQ_ERR_CUDA;
+    if (int rc = launch_generic(x_dev, perm, T, d, b, fmt, g, codes_dev, scales_dev, st)) return rc;
+    if (cudaMemcpyAsync(out_codes_host, codes_dev, cb, cudaMemcpyDeviceToHost, st) != cudaSuccess) return PERQ_ERR_CUDA;
+    if (sb && cudaMemcpyAsync(out_scales_host, scales_dev, sb, cudaMemcpyDeviceToHost, st) != cudaSuccess)
+        return PERQ_ERR_CUDA;
+    return cudaStreamSynchronize(st) == cudaSuccess ? PERQ_OK : PERQ_ERR_CUDA;
+}
+
+int perq_block_l1_stats_workspace_bytes(int64_t T, int32_t d, int32_t b, size_t *bytes)
+{
+    StatsPlan plan;
+    if (int rc = plan_stats(T, d, b, &plan)) return rc;
+    if (!bytes) return PERQ_ERR_NULL;
+    *bytes = plan.ws_bytes;
+    return PERQ_OK;
+}
+
+int perq_block_l1_stats(const void *x, const int32_t *perm, int64_t T, int32_t d, int32_t b, float *chan_abs_sum,
+                        float *block_l1_mean, float *token_max_block_l1, void *workspace, size_t workspace_bytes,
+                        void *stream)
+{
+    StatsPlan plan;
+    if (int rc = plan_stats(T, d, b, &plan)) return rc;
+    if (!chan_abs_sum && !block_l1_mean && !token_max_block_l1) return PERQ_OK;
+    if (!x) return PERQ_ERR_NULL;
+    if (T == 0) return PERQ_ERR_SHAPE;
+    if (!workspace || workspace_bytes < plan.ws_bytes) return PERQ_ERR_WORKSPACE;
+    if (!aligned16(x) || !aligned16(perm) || !aligned16(workspace)) return PERQ_ERR_ALIGN;
+    cudaStream_t st = static_cast<cudaStream_t>(stream);
+    perq::StatsParams p;
+    p.x = static_cast<const uint16_t *>(x);
+    p.perm = perm;
+    p.T = T;
+    p.d = d;
+    p.log2b = ilog2(b);
+    p.rows_per_cta = plan.rows_per_cta;
+    float *ws = static_cast<float *>(workspace);
+    p.ws_chan = chan_abs_sum ? ws : nullptr;
+    p.ws_block = block_l1_mean ? ws + (size_t)plan.n_cta * d : nullptr;
+    p.token_max = token_max_block_l1;
+    if (int rc = allow_smem(perq::perq_stats_partial_kernel, plan.smem)) return rc;
+    perq::perq_stats_partial_kernel<<<plan.n_cta, perq::ST_THREADS, plan.smem, st>>>(p);
+    if (cudaGetLastError() != cudaSuccess) return PERQ_ERR_CUDA;
+    if (chan_abs_sum || block_l1_mean) {
+        const int threads = 256;
+        perq::perq_stats_reduce_kernel<<<(d + threads - 1) / threads, threads, 0, st>>>(
+            p.ws_chan, p.ws_block, plan.n_cta, d, d / b, (float)(1.0 / (double)T), chan_abs_sum, block_l1_mean);
+        if (cudaGetLastError() != cudaSuccess) return PERQ_ERR_CUDA;
+    }
+    return PERQ_OK;
+}
+
+int perq_validate_perm(const int32_t *perm, int32_t d, int32_t *status_dev, void *stream)
+{
+    if (!perm || !status_dev) return PERQ_ERR_NULL;
+    if (d <= 0 || d > PERQ_MAX_D) return PERQ_ERR_SHAPE;
+    const size_t smem = (size_t)((d + 31) / 32) * sizeof(uint32_t);
+    perq::perq_validate_perm_kernel<<<1, 1024, smem, static_cast<cudaStream_t>(stream)>>>(perm, d, status_dev);
+    return cudaGetLastError() == cudaSuccess ? PERQ_OK : PERQ_ERR_CUDA;
+}
+
+int perq_massdiff_perm(const float *chan_abs_sum_host, int32_t d, int32_t b, int32_t *perm_host)
+{
+    if (!chan_abs_sum_host || !perm_host) return PERQ_ERR_NULL;
+    if (d <= 0) return PERQ_ERR_SHAPE;
+    if (b < 1 || d % b != 0) return PERQ_ERR_BLOCK;
+    const int n = d / b;
+    // channels by descending mass, equal masses by ascending index
+    std::vector<int32_t> order(d);
+    for (int i = 0; i < d; ++i) order[i] = i;
+    std::stable_sort(order.begin(), order.end(), [&](int32_t l, int32_t r) {
+        return chan_abs_sum_host[l] > chan_abs_sum_host[r];
+    });
+    // open blocks keyed by (running mass, block index): the top is the lightest, lowest-index block
+    using Key = std::pair<double, int32_t>;
+    std::priority_queue<Key, std::vector<Key>, std::greater<Key>> open;
+    for (int j = 0; j < n; ++j) open.push(Key(0.0, j));
+    std::vector<int32_t> fill(n, 0);
+    for (int s = 0; s < d; ++s) {
+        const int32_t c = order[s];
+        Key top = open.top();
+        open.pop();
+        const int32_t j = top.second;
+        perm_host[(size_t)j * b + fill[j]] = c;
+        fill[j] += 1;
+        if (fill[j] < b) open.push(Key(top.first + (double)chan_abs_sum_host[c], j));
+    }
+    return PERQ_OK;
+}
+
+}  // extern "C"

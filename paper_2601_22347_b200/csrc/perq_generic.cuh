@@ -1,0 +1,391 @@
+// Generic rotate+quantize kernel: any supported (d, b, fmt, group, perm) combination.
+//
+// One CTA owns one token row at a time (grid-stride over rows).  The (permuted) bf16 row
+// stays in shared memory for the whole row so that single output coordinates can be
+// re-evaluated exactly; the butterfly runs in fp32 through registers and shared memory.
+//
+// Numerical contract (what makes scales and codes reproducible against exact arithmetic):
+//   * the fp32 butterfly result u32 carries a small rounding error, bounded here by
+//     ERR_K * log2(b) * 2^-24 * (largest |u32| of the Hadamard block);
+//   * every quantity that decides an output bit is therefore re-derived in fp64 from the
+//     bf16 inputs whenever the fp32 value is within that bound of a decision boundary:
+//       - the absmax of an INT4 scale range (always: the stored scale must be exact),
+//       - the absmax of an MX group when it is close to a power-of-two boundary,
+//       - any element whose scaled value is close to a rounding tie.
+//     An fp64 sum of <= 32768 bf16 terms is exact unless their exponents span more than
+//     ~30 binades, so these re-derived values are the true ones.
+#pragma once
+#include <cuda_runtime.h>
+#include <stdint.h>
+
+namespace perq {
+
+constexpr int GEN_THREADS = 256;
+constexpr int GEN_WARPS = GEN_THREADS / 32;
+constexpr int TIE_CAP = 1024;
+constexpr float ERR_K = 8.0f;                 // safety factor on the fp32 butterfly error model
+constexpr float TWO_M24 = 5.9604644775390625e-8f;
+
+struct GenParams {
+    const uint16_t *x;
+    const int32_t *perm;
+    long long T;
+    int d;
+    int log2b;
+    int fmt;          // 0 INT4, 1 MXFP4, 2 F32 debug
+    int g;            // effective scale-range length (d for per-token, 32 for MX)
+    void *out_codes;
+    void *out_scales;
+    float inv_sqrt_b;
+    double sqrt_b;
+};
+
+// Shared-memory carve-up, computed identically on host (for the launch) and device.
+struct GenSmem {
+    size_t xs, ub, codes, r_max, r_thr, r_mul, r_aux, r_E, b_max, ties, total;
+    __host__ __device__ GenSmem(int d, int g, int log2b)
+    {
+        const size_t nr = (size_t)(d / g), nb = (size_t)(d >> log2b);
+        size_t o = 0;
+        xs = o;    o += (size_t)d * 2;
+        ub = o;    o += (size_t)d * 4;
+        codes = o; o += (size_t)d / 2;
+        o = (o + 15) & ~(size_t)15;
+        r_aux = o; o += nr * 8;
+        r_max = o; o += nr * 4;
+        r_thr = o; o += nr * 4;
+        r_mul = o; o += nr * 4;
+        r_E = o;   o += nr * 4;
+        b_max = o; o += nb * 4;
+        ties = o;  o += (size_t)TIE_CAP * 4 + 16;
+        total = o;
+    }
+};
+
+__device__ __forceinline__ float bf16lo(uint32_t w) { return __uint_as_float(w << 16); }
+__device__ __forceinline__ float bf16hi(uint32_t w) { return __uint_as_float(w & 0xffff0000u); }
+__device__ __forceinline__ double bf16_to_f64(uint16_t h) { return (double)__uint_as_float((uint32_t)h << 16); }
+
+// In-register butterfly over the low `R` index bits of v[0..2^R).
+template <int R>
+__device__ __forceinline__ void butterfly_regs(float (&v)[1 << R])
+{
+#pragma unroll
+    for (int t = 0; t < R; ++t) {
+#pragma unroll
+        for (int e = 0; e < (1 << R); ++e) {
+            if ((e & (1 << t)) == 0) {
+                const float a = v[e], c = v[e | (1 << t)];
+                v[e] = a + c;
+                v[e | (1 << t)] = a - c;
+            }
+        }
+    }
+}
+
+// One pass of R butterfly stages on index bits [s, s+R) of the fp32 row in shared memory.
+template <int R>
+__device__ __forceinline__ void radix_pass(float *ub, int d, int s, int tid)
+{
+    const int nsets = d >> R;
+    for (int q = tid; q < nsets; q += GEN_THREADS) {
+        const int base = ((q >> s) << (s + R)) | (q & ((1 << s) - 1));
+        float v[1 << R];
+#pragma unroll
+        for (int e = 0; e < (1 << R); ++e) v[e] = ub[base + (e << s)];
+        butterfly_regs<R>(v);
+#pragma unroll
+        for (int e = 0; e < (1 << R); ++e) ub[base + (e << s)] = v[e];
+    }
+}
+
+// Exact value of one unnormalised output coordinate, sum_k (-1)^{popcount(ii & k)} x'_k over
+// the coordinate's block, evaluated by a whole warp in fp64.
+__device__ __forceinline__ double exact_coord_warp(const uint16_t *xs, int blk_base, int b, int ii, int lane)
+{
+    double acc = 0.0;
+    for (int k = lane; k < b; k += 32) {
+        const double v = bf16_to_f64(xs[blk_base + k]);
+        acc += (__popc(ii & k) & 1) ? -v : v;
+    }
+#pragma unroll
+    for (int o = 16; o > 0; o >>= 1) acc += __shfl_xor_sync(0xffffffffu, acc, o);
+    return acc;
+}
+
+__device__ __forceinline__ double exact_coord_thread(const uint16_t *xs, int blk_base, int b, int ii)
+{
+    double acc = 0.0;
+    for (int k = 0; k < b; ++k) {
+        const double v = bf16_to_f64(xs[blk_base + k]);
+        acc += (__popc(ii & k) & 1) ? -v : v;
+    }
+    return acc;
+}
+
+// E2M1 code (sign << 3 | magnitude index) of an exactly known scaled value; ties to the even index.
+__device__ __forceinline__ uint32_t e2m1_code_exact(double v, bool negative)
+{
+    const double m = fabs(v);
+    uint32_t k;
+    if (m <= 0.25) k = 0;
+    else if (m < 0.75) k = 1;
+    else if (m <= 1.25) k = 2;
+    else if (m < 1.75) k = 3;
+    else if (m <= 2.5) k = 4;
+    else if (m < 3.5) k = 5;
+    else if (m <= 5.0) k = 6;
+    else k = 7;
+    return (negative ? 8u : 0u) | k;
+}
+
+// Distance from |v| to the nearest E2M1 rounding midpoint {.25,.75,1.25,1.75,2.5,3.5,5}.
+__device__ __forceinline__ float e2m1_tie_distance(float m)
+{
+    if (m < 2.0f) {
+        const float t = 2.0f * m - 0.5f;             // midpoints at t = 0, 1, 2, 3
+        const float r = fminf(rintf(t), 3.0f);
+        return 0.5f * fabsf(t - r);
+    }
+    if (m < 4.0f) {
+        const float t = m - 0.5f;                    // midpoints at t = 2, 3
+        const float r = fminf(fmaxf(rintf(t), 2.0f), 3.0f);
+        return fabsf(t - r);
+    }
+    return fabsf(m - 5.0f);
+}
+
+// Two fp32 values -> one byte of two E2M1 codes (first operand in the low nibble), RNE, saturating.
+__device__ __forceinline__ uint32_t cvt_e2m1x2(float lo, float hi)
+{
+    uint16_t r;
+    asm("{ .reg .b8 t; cvt.rn.satfinite.e2m1x2.f32 t, %1, %2; cvt.u16.u8 %0, t; }" : "=h"(r) : "f"(hi), "f"(lo));
+    return (uint32_t)r;
+}
+
+// Exact code of element i (row-relative index) from its exact unnormalised value u.
+__device__ __forceinline__ uint32_t exact_code(const GenParams &p, double u, double s64, int E)
+{
+    const double y = u / p.sqrt_b;
+    if (p.fmt == 0) {
+        if (s64 == 0.0) return 0u;
+        double q = rint(y / s64);
+        q = fmin(fmax(q, -8.0), 7.0);
+        return (uint32_t)((int)q) & 0xFu;
+    }
+    return e2m1_code_exact(scalbn(y, -E), signbit(y));
+}
+
+__global__ void __launch_bounds__(GEN_THREADS) perq_generic_kernel(GenParams p)
+{
+    extern __shared__ __align__(16) unsigned char smem[];
+    const int d = p.d, L = p.log2b, b = 1 << L, g = p.g;
+    const int nr = d / g, nb = d >> L, nchunks = d >> 3;
+    const GenSmem lay(d, g, L);
+    uint16_t *xs = (uint16_t *)(smem + lay.xs);
+    float *ub = (float *)(smem + lay.ub);
+    uint32_t *codes = (uint32_t *)(smem + lay.codes);
+    unsigned long long *r_aux = (unsigned long long *)(smem + lay.r_aux);  // exact amax bits, then s64 bits
+    uint32_t *r_max = (uint32_t *)(smem + lay.r_max);
+    float *r_thr = (float *)(smem + lay.r_thr);
+    float *r_mul = (float *)(smem + lay.r_mul);
+    int *r_E = (int *)(smem + lay.r_E);
+    uint32_t *b_max = (uint32_t *)(smem + lay.b_max);
+    int *tie_list = (int *)(smem + lay.ties);
+    int *tie_count = tie_list + TIE_CAP;
+
+    const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+    const float err_rel = ERR_K * (float)L * TWO_M24;   // |u32 - u| <= err_rel * (block max |u32|)
+
+    for (long long row = blockIdx.x; row < p.T; row += gridDim.x) {
+        // ---- A. row -> shared memory, through the permutation gather if there is one
+        const uint4 *src = (const uint4 *)(p.x + (size_t)row * d);
+        if (p.perm == nullptr) {
+            for (int c = tid; c < nchunks; c += GEN_THREADS) ((uint4 *)xs)[c] = __ldcs(src + c);
+        } else {
+            uint16_t *raw = (uint16_t *)ub;
+            for (int c = tid; c < nchunks; c += GEN_THREADS) ((uint4 *)raw)[c] = __ldcs(src + c);
+            __syncthreads();
+            for (int i = tid; i < d; i += GEN_THREADS) {
+                int q = __ldg(p.perm + i);
+                q = min(max(q, 0), d - 1);
+                xs[i] = raw[q];
+            }
+        }
+        for (int r = tid; r < nr; r += GEN_THREADS) { r_max[r] = 0u; r_aux[r] = 0ull; }
+        for (int j = tid; j < nb; j += GEN_THREADS) b_max[j] = 0u;
+        if (tid == 0) *tie_count = 0;
+        __syncthreads();
+
+        // ---- B. butterfly: index bits 0..2 in registers, the rest in passes over shared memory
+        for (int c = tid; c < nchunks; c += GEN_THREADS) {
+            const uint4 w = ((const uint4 *)xs)[c];
+            float v[8] = {bf16lo(w.x), bf16hi(w.x), bf16lo(w.y), bf16hi(w.y),
+                          bf16lo(w.z), bf16hi(w.z), bf16lo(w.w), bf16hi(w.w)};
+            butterfly_regs<3>(v);
+            ((float4 *)ub)[2 * c] = make_float4(v[0], v[1], v[2], v[3]);
+            ((float4 *)ub)[2 * c + 1] = make_float4(v[4], v[5], v[6], v[7]);
+        }
+        __syncthreads();
+        for (int s = 3; s < L; s += 3) {
+            const int R = min(3, L - s);
+            if (R == 3) radix_pass<3>(ub, d, s, tid);
+            else if (R == 2) radix_pass<2>(ub, d, s, tid);
+            else radix_pass<1>(ub, d, s, tid);
+            __syncthreads();
+        }
+
+        if (p.fmt == 2) {   // debug: the rotated row itself
+            float4 *dst = (float4 *)((float *)p.out_codes + (size_t)row * d);
+            const float k = p.inv_sqrt_b;
+            for (int c = tid; c < d / 4; c += GEN_THREADS) {
+                float4 v = ((const float4 *)ub)[c];
+                dst[c] = make_float4(v.x * k, v.y * k, v.z * k, v.w * k);
+            }
+            __syncthreads();
+            continue;
+        }
+
+        // ---- C. fp32 absmax per scale range and per Hadamard block
+        for (int c = tid; c < nchunks; c += GEN_THREADS) {
+            const float4 a = ((const float4 *)ub)[2 * c], e = ((const float4 *)ub)[2 * c + 1];
+            const float m = fmaxf(fmaxf(fmaxf(fabsf(a.x), fabsf(a.y)), fmaxf(fabsf(a.z), fabsf(a.w))),
+                                  fmaxf(fmaxf(fabsf(e.x), fabsf(e.y)), fmaxf(fabsf(e.z), fabsf(e.w))));
+            atomicMax(&r_max[(c * 8) / g], __float_as_uint(m));
+            atomicMax(&b_max[(c * 8) >> L], __float_as_uint(m));
+        }
+        __syncthreads();
+
+        // ---- D. which ranges need their absmax re-derived exactly, and from which elements
+        for (int r = tid; r < nr; r += GEN_THREADS) {
+            const float rm = __uint_as_float(r_max[r]);
+            const float bm = (g >= b) ? rm : __uint_as_float(b_max[(r * g) >> L]);
+            const float err = err_rel * bm;
+            bool need = rm > 0.0f;
+            if (need && p.fmt == 1) {
+                // MX only needs floor(log2(amax / sqrt(b))): exact only near a power of two
+                int e;
+                const double mant = frexp((double)rm / p.sqrt_b, &e);       // [0.5, 1)
+                const double rho = (double)err / (double)rm + 2.4e-7;
+                need = (mant * (1.0 + rho) >= 1.0) || (mant * (1.0 - rho) < 0.5);
+            }
+            r_thr[r] = need ? fmaxf(rm - 2.0f * err, 0.0f) : __int_as_float(0x7f800000);
+        }
+        __syncthreads();
+        {
+            const int parts = (g + 255) >> 8;
+            const int units = nr * parts;
+            for (int unit = warp; unit < units; unit += GEN_WARPS) {
+                const int r = unit / parts, part = unit - r * parts;
+                const float thr = r_thr[r];
+                if (!(thr < __int_as_float(0x7f800000))) continue;
+                const int start = r * g + (part << 8);
+                const int end = min(r * g + g, start + 256);
+                for (int i0 = start; i0 < end; i0 += 32) {
+                    const int i = i0 + lane;
+                    const bool cand = (i < end) && (fabsf(ub[i]) >= thr);
+                    unsigned m = __ballot_sync(0xffffffffu, cand);
+                    while (m) {
+                        const int ic = i0 + (__ffs(m) - 1);
+                        m &= m - 1;
+                        const double u = exact_coord_warp(xs, (ic >> L) << L, b, ic & (b - 1), lane);
+                        if (lane == 0) atomicMax(&r_aux[r], (unsigned long long)__double_as_longlong(fabs(u)));
+                    }
+                }
+            }
+        }
+        __syncthreads();
+
+        // ---- E. scales
+        for (int r = tid; r < nr; r += GEN_THREADS) {
+            const float rm = __uint_as_float(r_max[r]);
+            const bool exact = r_thr[r] < __int_as_float(0x7f800000);
+            const double au = exact ? __longlong_as_double((long long)r_aux[r]) : (double)rm;
+            const double yd = au / p.sqrt_b;
+            if (p.fmt == 0) {
+                const double s = yd / 7.0;
+                ((float *)p.out_scales)[(size_t)row * nr + r] = (au == 0.0) ? 0.0f : (float)s;
+                r_mul[r] = (au == 0.0) ? 0.0f : fminf((float)(7.0 / au), 3.0e38f);
+                r_aux[r] = (unsigned long long)__double_as_longlong(s);
+            } else {
+                int E = -127;
+                if (au != 0.0) {
+                    int e;
+                    (void)frexp(yd, &e);
+                    E = min(max(e - 3, -127), 127);
+                }
+                ((uint8_t *)p.out_scales)[(size_t)row * nr + r] = (au == 0.0) ? 0 : (uint8_t)(E + 127);
+                r_mul[r] = (au == 0.0) ? 0.0f : (float)(scalbn(1.0, -E) / p.sqrt_b);
+                r_E[r] = E;
+            }
+        }
+        __syncthreads();
+
+        // ---- F. quantise in fp32, flagging elements too close to a rounding tie
+        for (int c = tid; c < nchunks; c += GEN_THREADS) {
+            const int i0 = c * 8, r = i0 / g;
+            const float mul = r_mul[r];
+            const float tau_abs = err_rel * __uint_as_float(b_max[i0 >> L]) * mul;
+            const float4 a = ((const float4 *)ub)[2 * c], e = ((const float4 *)ub)[2 * c + 1];
+            const float u[8] = {a.x, a.y, a.z, a.w, e.x, e.y, e.z, e.w};
+            uint32_t word = 0u, flags = 0u;
+            if (p.fmt == 0) {
+#pragma unroll
+                for (int k = 0; k < 8; ++k) {
+                    const float v = u[k] * mul;
+                    const float q = fminf(fmaxf(rintf(v), -8.0f), 7.0f);
+                    if (fabsf(v - q) > 0.5f - (tau_abs + 4.0e-6f)) flags |= 1u << k;
+                    word |= ((uint32_t)((int)q) & 0xFu) << (4 * k);
+                }
+            } else {
+#pragma unroll
+                for (int k = 0; k < 8; k += 2) {
+                    const float v0 = fmaf(u[k], mul, 0.0f), v1 = fmaf(u[k + 1], mul, 0.0f);
+                    word |= cvt_e2m1x2(v0, v1) << (4 * k);
+                    if (e2m1_tie_distance(fabsf(v0)) < tau_abs + fabsf(v0) * 1.0e-6f) flags |= 1u << k;
+                    if (e2m1_tie_distance(fabsf(v1)) < tau_abs + fabsf(v1) * 1.0e-6f) flags |= 2u << k;
+                }
+            }
+            while (flags) {
+                const int k = __ffs(flags) - 1;
+                flags &= flags - 1;
+                const int pos = atomicAdd(tie_count, 1);
+                if (pos < TIE_CAP) {
+                    tie_list[pos] = i0 + k;
+                } else {   // list full: resolve here, single-threaded
+                    const int i = i0 + k;
+                    const double ue = exact_coord_thread(xs, (i >> L) << L, b, i & (b - 1));
+                    const uint32_t code = exact_code(p, ue, __longlong_as_double((long long)r_aux[r]), r_E[r]);
+                    word = (word & ~(0xFu << (4 * k))) | (code << (4 * k));
+                }
+            }
+            codes[c] = word;
+        }
+        __syncthreads();
+
+        // ---- G. resolve the flagged elements exactly
+        {
+            const int n = min(*tie_count, TIE_CAP);
+            for (int t = warp; t < n; t += GEN_WARPS) {
+                const int i = tie_list[t], r = i / g;
+                const double ue = exact_coord_warp(xs, (i >> L) << L, b, i & (b - 1), lane);
+                if (lane == 0) {
+                    const uint32_t code = exact_code(p, ue, __longlong_as_double((long long)r_aux[r]), r_E[r]);
+                    const int sh = 4 * (i & 7);
+                    atomicAnd(&codes[i >> 3], ~(0xFu << sh));
+                    atomicOr(&codes[i >> 3], code << sh);
+                }
+            }
+        }
+        __syncthreads();
+
+        // ---- H. packed codes out
+        {
+            uint4 *dst = (uint4 *)((uint8_t *)p.out_codes + (size_t)row * (d / 2));
+            for (int c = tid; c < d / 32; c += GEN_THREADS) __stcs(dst + c, ((const uint4 *)codes)[c]);
+        }
+        __syncthreads();
+    }
+}
+
+}  // namespace perq

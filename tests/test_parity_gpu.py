@@ -1,0 +1,298 @@
+"""Parity of the CUDA path (called through the C ABI) with the CPU oracle, on a B200."""
+import numpy as np
+import pytest
+import torch
+
+from paper_2601_22347_b200 import inputs
+
+from parity import compare_quantized, compare_rotated, unpack_nibbles, int4_values
+
+pytestmark = pytest.mark.gpu
+
+FMT = {"int4": 0, "mxfp4": 1}
+
+
+@pytest.fixture(scope="module")
+def B():
+    assert torch.cuda.is_available(), "GPU tests need a CUDA device"
+    from paper_2601_22347_b200 import binding, build
+    build.build()
+    binding.load()
+    return binding
+
+
+def to_dev(bits: np.ndarray) -> torch.Tensor:
+    return torch.from_numpy(bits.view(np.int16).copy()).cuda().view(torch.bfloat16)
+
+
+def run_gpu(B, w: inputs.Workload, x_dev=None):
+    x = to_dev(w.x) if x_dev is None else x_dev
+    perm = None if w.perm is None else torch.from_numpy(w.perm).cuda()
+    codes, scales = B.perq_rotate_quantize(x, perm, w.b, FMT[w.fmt], w.group)
+    torch.cuda.synchronize()
+    return codes.cpu().numpy(), scales.cpu().numpy()
+
+
+def check(B, oracle, w: inputs.Workload, rows=None):
+    """Full comparison when rows is None, else the GPU runs everything and the oracle the sampled rows."""
+    codes, scales = run_gpu(B, w)
+    xs = w.x if rows is None else w.x[rows]
+    ora = oracle.rotate_quantize(xs, w.perm, w.b, FMT[w.fmt], w.group, want_pre=True)
+    if rows is not None:
+        codes, scales = codes[rows], scales[rows]
+    rep = compare_quantized(w.fmt, codes, scales, ora)
+    print("%s T=%d d=%d b=%d %s g=%d: %d elements, %d tie-window exemptions, scale ulp max %d"
+          % (w.name, w.T, w.d, w.b, w.fmt, w.group, rep["elements"], rep["code_mismatch_exempt"],
+             rep["scale_ulp_max"]))
+    return rep
+
+
+# ------------------------------------------------------------------ the five workloads
+
+def test_config1_full(B, oracle):
+    check(B, oracle, inputs.config1())
+
+
+@pytest.mark.parametrize("b", [16, 32, 64, 128, 2048])
+def test_config2(B, oracle, b):
+    check(B, oracle, inputs.config2(T=768 if b <= 128 else 96, b=b))
+
+
+def test_config3_with_massdiff_permutation(B, oracle):
+    w = inputs.config3(T=320)
+    x = to_dev(w.x)
+    chan, _, _ = B.perq_block_l1_stats(x, None, w.b, want=("chan",))
+    torch.cuda.synchronize()
+    w.perm = B.perq_massdiff_perm(chan.cpu().numpy(), w.b)
+    assert sorted(w.perm.tolist()) == list(range(w.d))
+    status = B.perq_validate_perm(torch.from_numpy(w.perm).cuda())
+    assert int(status.item()) == 0
+    check(B, oracle, w)
+    # the permutation does what it is for: it lowers the largest per-block l1 mass
+    _, blk_id, _ = B.perq_block_l1_stats(x, None, w.b, want=("block",))
+    _, blk_md, _ = B.perq_block_l1_stats(x, torch.from_numpy(w.perm).cuda(), w.b, want=("block",))
+    assert float(blk_md.max()) < float(blk_id.max())
+
+
+@pytest.mark.parametrize("fmt", ["int4", "mxfp4"])
+@pytest.mark.parametrize("b", [16, 32, 128, 4096])
+def test_config4_full_size_sampled(B, oracle, b, fmt):
+    w = inputs.config4(T=16384, b=b, fmt=fmt)
+    rows = np.sort(np.random.default_rng(4).choice(w.T, 96 if b < 4096 else 24, replace=False))
+    rows[0], rows[-1] = 0, w.T - 1
+    check(B, oracle, w, rows=rows)
+
+
+@pytest.mark.parametrize("T", [1, 16, 128])
+@pytest.mark.parametrize("b", [16, 32, 64, 128])
+def test_config5_small_T(B, oracle, T, b):
+    check(B, oracle, inputs.config5(T=T, b=b))
+
+
+def test_config5_large_T_sampled(B, oracle):
+    w = inputs.config5(T=1024, b=128)
+    rows = np.sort(np.random.default_rng(5).choice(w.T, 64, replace=False))
+    check(B, oracle, w, rows=rows)
+
+
+# ------------------------------------------------------------------ rotated values (debug format)
+
+@pytest.mark.parametrize("d,b,perm", [(2048, 16, False), (2048, 128, True), (4096, 4096, False),
+                                      (14336, 64, True), (8192, 32, False), (2048, 2048, True)])
+def test_rotated_values(B, oracle, d, b, perm):
+    bits, _ = inputs.laplace_outliers(48, d, 4, 200.0, seed=77 + d + b)
+    p = inputs.random_perm(d, 78) if perm else None
+    x = to_dev(bits)
+    y, _ = B.perq_rotate_quantize(x, None if p is None else torch.from_numpy(p).cuda(), b, B.PERQ_FMT_F32_DEBUG, 0)
+    torch.cuda.synchronize()
+    rep = compare_rotated(y.cpu().numpy(), oracle.rotate(bits, p, b), b)
+    print("rotated d=%d b=%d: max %.2e rms %.2e of block max" % (d, b, rep["max_rel_to_block_max"], rep["rms_rel"]))
+
+
+# ------------------------------------------------------------------ edge cases
+
+def test_empty_and_tiny_T(B, oracle):
+    x = torch.empty((0, 2048), dtype=torch.bfloat16, device="cuda")
+    codes, scales = B.perq_rotate_quantize(x, None, 16, 0, 0)
+    assert codes.shape == (0, 1024) and scales.shape == (0, 1)
+    for T in (1, 3):
+        w = inputs.config1(T=T, variant=T)
+        check(B, oracle, w)
+        w.fmt, w.group = "mxfp4", 32
+        check(B, oracle, w)
+
+
+def test_zero_rows_and_zero_groups(B, oracle):
+    w = inputs.config2(T=8, b=32)
+    w.x[1] = 0
+    w.x[2, :] = 0
+    w.x[3, 256:512] = 0           # two whole groups of 128 (under the identity permutation)
+    w.perm = None
+    check(B, oracle, w)
+    w.fmt, w.group = "mxfp4", 32
+    check(B, oracle, w)
+    codes, scales = run_gpu(B, w)
+    assert not codes[1].any() and not scales[1].any()
+
+
+def test_single_huge_outlier_and_basis_rows(B, oracle):
+    d = 2048
+    x = np.zeros((6, d), np.float32)
+    x[0, 77] = 3.0e4                      # one nonzero: every output of its block has the same magnitude
+    x[1, 5] = 1.0
+    x[1, 1029] = -2.5
+    x[2] = 1.0                            # constant row: all mass lands on the first coordinate of each block
+    x[3] = np.random.default_rng(1).standard_normal(d) * 1e-3
+    x[3, 100] = 6.0e4
+    x[4] = np.random.default_rng(2).standard_normal(d)
+    x[4, 1000:1016] = 0
+    x[5, ::2] = 1.0
+    x[5, 1::2] = -1.0
+    bits = inputs.f32_to_bf16_bits(x)
+    for b in (16, 128, 2048):
+        for fmt, g in (("int4", 0), ("int4", 128), ("mxfp4", 32)):
+            check(B, oracle, inputs.Workload("edge", bits, None, b, fmt, g, 0))
+
+
+def test_constructed_exact_ties(B, oracle):
+    """Rows built so that the rotated values are exact k + 1/2 multiples of the step: the
+    CUDA path has to resolve them like exact arithmetic does (round half to even)."""
+    import scipy.linalg
+    H = scipy.linalg.hadamard(16)
+    rng = np.random.default_rng(8)
+    rows = []
+    for _ in range(32):
+        blocks = []
+        for j in range(8):
+            ystar = rng.integers(-13, 14, size=16) * 0.5          # halves in [-6.5, 6.5]
+            ystar[rng.integers(0, 16)] = 7.0 if j == 0 else ystar[0]
+            blocks.append((ystar @ H) / 4.0)
+        rows.append(np.concatenate(blocks))
+    x = np.array(rows, np.float32)
+    bits = inputs.f32_to_bf16_bits(x)
+    assert np.array_equal(inputs.bf16_bits_to_f32(bits), x)
+    w = inputs.Workload("ties", bits, None, 16, "int4", 0, 0)
+    rep = check(B, oracle, w)
+    assert rep["code_mismatch_exempt"] == 0          # exact ties are not approximated: they must match
+    ora = oracle.rotate_quantize(bits, None, 16, 0, 0, want_pre=True)
+    assert (np.abs(ora["pre"] - np.floor(ora["pre"])) == 0.5).sum() > 500
+    # the same rows scaled so that MX midpoints are hit: amax 7 -> E = 0, halves/quarters are midpoints
+    w2 = inputs.Workload("ties-mx", inputs.f32_to_bf16_bits(x * 0.5), None, 16, "mxfp4", 32, 0)
+    rep2 = check(B, oracle, w2)
+    assert rep2["code_mismatch_exempt"] == 0
+
+
+def test_mx_saturation_band(B, oracle):
+    """Values in (6, 8) * 2^E must saturate to the largest E2M1 magnitude."""
+    d = 64
+    x = np.zeros((4, d), np.float32)
+    x[:, 0] = [7.5 * 4, 6.5 * 4, 7.0 * 4, 4.0 * 4]     # with b = 16 a lone entry spreads as x/4 over its block
+    bits = inputs.f32_to_bf16_bits(x)
+    w = inputs.Workload("sat", bits, None, 16, "mxfp4", 32, 0)
+    check(B, oracle, w)
+    codes, scales = run_gpu(B, w)
+    nib = unpack_nibbles(codes)
+    assert np.all(nib[:3, :16] == 7) and np.all(nib[3, :16] == 6)
+
+
+@pytest.mark.parametrize("kind", ["reversal", "interleave", "random"])
+def test_permutations(B, oracle, kind):
+    d = 2048
+    if kind == "reversal":
+        perm = np.arange(d - 1, -1, -1, dtype=np.int32)
+    elif kind == "interleave":
+        perm = np.arange(d, dtype=np.int32).reshape(32, 64).T.reshape(-1).copy()
+    else:
+        perm = inputs.random_perm(d, 99)
+    w = inputs.config2(T=64, b=64)
+    w.perm = perm
+    check(B, oracle, w)
+
+
+def test_group_smaller_than_block_and_other_groups(B, oracle):
+    for b, g in ((128, 32), (2048, 64), (16, 8), (64, 256), (32, 1024)):
+        w = inputs.config2(T=32, b=b)
+        w.group = g
+        check(B, oracle, w)
+
+
+def test_outputs_are_deterministic_and_stay_inside_their_buffers(B):
+    w = inputs.config2(T=200, b=128)
+    x = to_dev(w.x)
+    perm = torch.from_numpy(w.perm).cuda()
+    cb, sb = B.perq_out_sizes(w.T, w.d, 0, 128)
+    guard = 4096
+    bufc = torch.full((cb + guard,), 0xA5, dtype=torch.uint8, device="cuda")
+    bufs = torch.full((sb + guard,), 0x5A, dtype=torch.uint8, device="cuda")
+    outs = []
+    for _ in range(2):
+        bufc.fill_(0xA5); bufs.fill_(0x5A)
+        B.perq_rotate_quantize(x, perm, 128, 0, 128, out_codes=bufc, out_scales=bufs)
+        torch.cuda.synchronize()
+        assert bool((bufc[cb:] == 0xA5).all()) and bool((bufs[sb:] == 0x5A).all())
+        outs.append((bufc[:cb].clone(), bufs[:sb].clone()))
+    assert torch.equal(outs[0][0], outs[1][0]) and torch.equal(outs[0][1], outs[1][1])
+
+
+def test_row_sharding_gives_identical_bytes(B):
+    """Rows are independent: running two halves separately (as two ranks would) must
+    reproduce the unsharded call byte for byte."""
+    w = inputs.config4(T=512, b=32, fmt="mxfp4")
+    x = to_dev(w.x)
+    c_all, s_all = B.perq_rotate_quantize(x, None, 32, 1, 32)
+    c0, s0 = B.perq_rotate_quantize(x[:200].contiguous(), None, 32, 1, 32)
+    c1, s1 = B.perq_rotate_quantize(x[200:].contiguous(), None, 32, 1, 32)
+    torch.cuda.synchronize()
+    assert torch.equal(torch.cat([c0, c1]), c_all) and torch.equal(torch.cat([s0, s1]), s_all)
+
+
+def test_host_buffer_entry_point(B, oracle):
+    w = inputs.config1(T=64)
+    xh = torch.from_numpy(w.x.view(np.int16).copy()).view(torch.bfloat16).pin_memory()
+    ws = torch.empty(B.perq_host_workspace_bytes(w.T, w.d, 0, 0), dtype=torch.uint8, device="cuda")
+    codes = torch.empty((w.T, w.d // 2), dtype=torch.uint8).pin_memory()
+    scales = torch.empty((w.T, 1), dtype=torch.float32).pin_memory()
+    B.perq_rotate_quantize_host(xh, None, 16, 0, 0, codes, scales, ws)
+    ora = oracle.rotate_quantize(w.x, None, 16, 0, 0, want_pre=True)
+    compare_quantized("int4", codes.numpy(), scales.numpy(), ora)
+
+
+def test_invalid_permutation_is_reported_not_faulted(B):
+    d = 2048
+    bad = inputs.random_perm(d, 3)
+    bad[10] = bad[11]
+    assert int(B.perq_validate_perm(torch.from_numpy(bad).cuda()).item()) == 2
+    bad2 = inputs.random_perm(d, 3)
+    bad2[0] = d + 5
+    bad2[1] = -1
+    st = int(B.perq_validate_perm(torch.from_numpy(bad2).cuda()).item())
+    assert st & 1
+    # out-of-range entries are clamped by the main kernel: it must finish without an error
+    w = inputs.config2(T=16, b=32)
+    x = to_dev(w.x)
+    B.perq_rotate_quantize(x, torch.from_numpy(bad2).cuda(), 32, 0, 128)
+    torch.cuda.synchronize()
+
+
+# ------------------------------------------------------------------ statistic
+
+@pytest.mark.parametrize("T,d,b,perm", [(320, 8192, 32, True), (1000, 2048, 16, False), (37, 14336, 128, True),
+                                        (5, 4096, 4096, False), (700, 4096, 8, True)])
+def test_block_l1_stats(B, oracle, T, d, b, perm):
+    bits, _ = inputs.swiglu_outliers(T, d, 32, 30.0, seed=300 + T)
+    p = inputs.random_perm(d, 301) if perm else None
+    x = to_dev(bits)
+    pd = None if p is None else torch.from_numpy(p).cuda()
+    chan, block, token = B.perq_block_l1_stats(x, pd, b)
+    chan2, block2, token2 = B.perq_block_l1_stats(x, pd, b)
+    torch.cuda.synchronize()
+    assert torch.equal(chan, chan2) and torch.equal(block, block2) and torch.equal(token, token2)
+    cas, blm, tmx = oracle.block_l1_stats(bits, p, b)
+    # fp32 accumulation in a fixed order: 1e-5 relative covers T up to a few thousand rows
+    assert np.allclose(chan.cpu().numpy(), cas, rtol=1e-5, atol=0)
+    assert np.allclose(block.cpu().numpy(), blm, rtol=1e-5, atol=0)
+    assert np.allclose(token.cpu().numpy(), tmx, rtol=1e-5, atol=0)
+    # only some outputs requested
+    only_tok = B.perq_block_l1_stats(x, pd, b, want=("token",))
+    torch.cuda.synchronize()
+    assert only_tok[0] is None and only_tok[1] is None and torch.equal(only_tok[2], token)
