@@ -1,0 +1,324 @@
+#!/usr/bin/env python
+"""Benchmark of the PeRQ online path (permute -> block Hadamard -> INT4/MXFP4) on B200.
+
+    python bench.py [--gpus N] [--steps K] [--warmup W] [--impl reference]
+
+One step = one perq_rotate_quantize call over the headline workload (Llama-3-8B-shaped
+hidden activations, T=16384 x d=4096 bf16, block Hadamard b=32, INT4 per-token scale).
+`value` is the effective bandwidth: algorithmic bytes (bf16 row in + packed codes +
+scales out) per second, inputs resident in HBM.  Prints ONE JSON line (rank 0).
+
+The other variants of the same workload (b in {16,32,128,4096} x {INT4, MXFP4}) and the
+calibration statistic are timed after the K steps and reported under "sweep".
+`--impl reference` times the CPU oracle instead (a deliberately plain fp64 program).
+"""
+from __future__ import annotations
+
+import argparse
+import json
+import os
+import statistics
+import subprocess
+import sys
+import time
+
+ROOT = os.path.dirname(os.path.abspath(__file__))
+if ROOT not in sys.path:
+    sys.path.insert(0, ROOT)
+
+METRIC = "rotate_quantize_effective_hbm_bandwidth"
+UNIT = "GB/s"
+NOMINAL_HBM_GBS = 8000.0
+FALLBACK_HBM_GBS = 6650.0
+
+# headline workload
+T_HEAD, D_HEAD, B_HEAD, FMT_HEAD, GROUP_HEAD = 16384, 4096, 32, "int4", 0
+
+# DRAM traffic per token (dram__bytes_read.sum + dram__bytes_write.sum) / T of the headline
+# kernel from an ncu capture; None until a capture of the current kernel exists.  See profiles/.
+NCU_TRAFFIC_BYTES_PER_TOKEN = None
+
+
+def measured_peak():
+    path = os.path.join(ROOT, "MEASURED_PEAKS.json")
+    try:
+        with open(path) as f:
+            return float(json.load(f)["hbm_gbs"]), "measured"
+    except Exception:
+        return FALLBACK_HBM_GBS, "fallback"
+
+
+class ClockSampler:
+    """Samples SM clocks and throttle reasons with nvidia-smi while the timed region runs."""
+    FIELDS = ("clocks.sm,clocks.max.sm,power.draw,clocks_event_reasons.hw_slowdown,"
+              "clocks_event_reasons.hw_thermal_slowdown,clocks_event_reasons.sw_thermal_slowdown,"
+              "clocks_event_reasons.sw_power_cap")
+
+    def __init__(self, index: int):
+        self.index = index
+        self.proc = None
+
+    def start(self):
+        try:
+            self.proc = subprocess.Popen(
+                ["nvidia-smi", "-i", str(self.index), "--query-gpu=" + self.FIELDS, "--format=csv,noheader,nounits",
+                 "-lms", "50"], stdout=subprocess.PIPE, stderr=subprocess.DEVNULL, text=True)
+        except Exception:
+            self.proc = None
+
+    def stop(self):
+        out = {"sm_mhz": None, "sm_max_mhz": None, "reasons": [], "samples": 0}
+        if self.proc is None:
+            return out
+        time.sleep(0.06)
+        self.proc.terminate()
+        try:
+            text, _ = self.proc.communicate(timeout=5)
+        except Exception:
+            self.proc.kill()
+            return out
+        sm, mx, reasons = [], [], set()
+        for line in text.strip().splitlines():
+            f = [s.strip() for s in line.split(",")]
+            if len(f) < 7:
+                continue
+            try:
+                sm.append(float(f[0])); mx.append(float(f[1]))
+            except ValueError:
+                continue
+            for name, v in zip(("hw_slowdown", "hw_thermal_slowdown", "sw_thermal_slowdown", "sw_power_cap"), f[3:7]):
+                if v.lower().startswith("active"):
+                    reasons.add(name)
+        if sm:
+            out.update(sm_mhz=statistics.median(sm), sm_max_mhz=max(mx), reasons=sorted(reasons), samples=len(sm))
+        return out
+
+
+def bytes_per_token(d, fmt, group):
+    from paper_2601_22347_b200.roofline import algorithmic_bytes_per_token
+    return algorithmic_bytes_per_token(d, fmt, group)
+
+
+# ------------------------------------------------------------------------------ reference arm (CPU oracle)
+
+def run_reference(args):
+    """Times the oracle, as it stands, on the host cores; each step is a bounded row sample."""
+    rank = int(os.environ.get("RANK", "0"))
+    if rank != 0:
+        return 0
+    import numpy as np
+    from oracle import perq_oracle
+    from paper_2601_22347_b200 import inputs
+    perq_oracle.build()
+    rows = 2048
+    w = inputs.config4(T=rows, b=B_HEAD, fmt=FMT_HEAD)
+    fmt = perq_oracle.FMT_INT4
+    for _ in range(max(1, min(args.warmup, 2))):
+        perq_oracle.rotate_quantize(w.x, None, w.b, fmt, w.group)
+    t0 = time.perf_counter()
+    for _ in range(args.steps):
+        perq_oracle.rotate_quantize(w.x, None, w.b, fmt, w.group)
+    dt = (time.perf_counter() - t0) / args.steps
+    bpt = bytes_per_token(D_HEAD, FMT_HEAD, GROUP_HEAD)
+    value = rows * bpt / dt / 1e9
+    sample = "%d of %d rows per step (rows are independent)" % (rows, T_HEAD)
+    line = {
+        "impl": "reference", "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": args.gpus,
+        "steps": args.steps, "warmup": args.warmup, "ms_per_step": dt * 1e3, "higher_is_better": True,
+        "scaling": "weak", "vs_baseline": None, "dtype": "f64", "data": "synthetic",
+        "config": {"workload": "cfg4 Llama-3-8B hidden: T=%d d=%d bf16 Laplace+4 outlier channels, b=%d, INT4 per-token"
+                               % (T_HEAD, D_HEAD, B_HEAD), "sample": sample},
+        "mtokens_per_s": rows / dt / 1e6,
+        "cpu_baseline": {"value": value, "unit": UNIT, "cores": perq_oracle.num_threads(), "kind": "oracle",
+                         "sample": sample},
+        "e2e": {"value": value, "unit": UNIT, "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
+        "gpu_launches": 0,
+    }
+    print(json.dumps(line))
+    return 0
+
+
+# ------------------------------------------------------------------------------ CUDA arm
+
+def main():
+    ap = argparse.ArgumentParser()
+    ap.add_argument("--gpus", type=int, default=1)
+    ap.add_argument("--steps", type=int, default=200)
+    ap.add_argument("--warmup", type=int, default=10)
+    ap.add_argument("--impl", default="perq", choices=["perq", "reference"])
+    ap.add_argument("--no-sweep", action="store_true", help="skip the per-variant sweep after the timed steps")
+    ap.add_argument("--no-cpu-baseline", action="store_true")
+    args = ap.parse_args()
+    args.warmup = max(args.warmup, 3)
+    if args.impl == "reference":
+        return run_reference(args)
+
+    import numpy as np
+    import torch
+    from paper_2601_22347_b200 import binding as B, inputs
+
+    world = int(os.environ.get("WORLD_SIZE", "1"))
+    rank = int(os.environ.get("RANK", "0"))
+    local_rank = int(os.environ.get("LOCAL_RANK", "0"))
+    assert torch.cuda.is_available(), "bench.py needs a CUDA device (no CPU fallback)"
+    torch.cuda.set_device(local_rank)
+    dist = None
+    if world > 1:
+        import torch.distributed as dist
+        dist.init_process_group("nccl", device_id=torch.device("cuda", local_rank))
+    B.load()
+
+    # Every rank holds the same-shaped workload with its own seed: rows are independent, so the
+    # path shards over T with no data-path collective (weak scaling).
+    w = inputs.config4(T=T_HEAD, b=B_HEAD, fmt=FMT_HEAD, variant=rank % 10)
+    fmt = B.FMT_BY_NAME[FMT_HEAD]
+    RING = 4   # 4 x 134 MB of inputs: every call reads rows that are not in the 126 MB L2
+    base = torch.from_numpy(w.x.view(np.int16).copy()).cuda().view(torch.bfloat16)
+    xs = [base] + [torch.roll(base, shifts=17 * (i + 1), dims=0).contiguous() for i in range(RING - 1)]
+    outs = [B.alloc_outputs(T_HEAD, D_HEAD, fmt, GROUP_HEAD, base.device) for _ in range(RING)]
+    bpt = bytes_per_token(D_HEAD, FMT_HEAD, GROUP_HEAD)
+    bytes_per_step = bpt * T_HEAD
+
+    def step(i):
+        k = i % RING
+        B.perq_rotate_quantize(xs[k], None, B_HEAD, fmt, GROUP_HEAD, out_codes=outs[k][0], out_scales=outs[k][1])
+
+    def barrier():
+        torch.cuda.synchronize()
+        if dist is not None:
+            dist.barrier()
+        torch.cuda.synchronize()
+
+    for i in range(args.warmup):
+        step(i)
+    barrier()
+    sampler = ClockSampler(local_rank)
+    if rank == 0:
+        sampler.start()
+    ev = [torch.cuda.Event(enable_timing=True) for _ in range(args.steps + 1)]
+    ev[0].record()
+    for i in range(args.steps):
+        step(i)
+        ev[i + 1].record()
+    barrier()
+    clocks = sampler.stop() if rank == 0 else None
+    total_ms = ev[0].elapsed_time(ev[-1])
+    per_launch_ms = [ev[i].elapsed_time(ev[i + 1]) for i in range(args.steps)]
+    t = torch.tensor([total_ms], dtype=torch.float64, device="cuda")
+    if dist is not None:
+        dist.all_reduce(t, op=dist.ReduceOp.MAX)
+    total_ms = float(t.item())
+    ms_per_step = total_ms / args.steps
+    value = world * bytes_per_step / (ms_per_step * 1e-3) / 1e9
+
+    # ---- end to end through the host-buffer entry point (pinned host memory, copies inside the timed region)
+    xh = torch.from_numpy(w.x.view(np.int16).copy()).view(torch.bfloat16).pin_memory()
+    ch = torch.empty((T_HEAD, D_HEAD // 2), dtype=torch.uint8).pin_memory()
+    sh = torch.empty((T_HEAD, 1), dtype=torch.float32).pin_memory()
+    ws = torch.empty(B.perq_host_workspace_bytes(T_HEAD, D_HEAD, fmt, GROUP_HEAD), dtype=torch.uint8, device="cuda")
+    e2e_steps = max(3, min(args.steps, 20))
+    for _ in range(3):
+        B.perq_rotate_quantize_host(xh, None, B_HEAD, fmt, GROUP_HEAD, ch, sh, ws)
+    barrier()
+    t0 = time.perf_counter()
+    for _ in range(e2e_steps):
+        B.perq_rotate_quantize_host(xh, None, B_HEAD, fmt, GROUP_HEAD, ch, sh, ws)   # synchronises its stream
+    e2e_s = (time.perf_counter() - t0) / e2e_steps
+    t = torch.tensor([e2e_s], dtype=torch.float64, device="cuda")
+    if dist is not None:
+        dist.all_reduce(t, op=dist.ReduceOp.MAX)
+    e2e_s = float(t.item())
+    e2e = {"value": world * bytes_per_step / e2e_s / 1e9, "unit": UNIT,
+           "h2d_bytes_per_step": int(xh.numel() * 2), "d2h_bytes_per_step": int(ch.numel() + sh.numel() * 4),
+           "ms_per_step": e2e_s * 1e3, "api": "perq_rotate_quantize_host"}
+    del ws
+
+    if rank != 0:
+        if dist is not None:
+            dist.barrier()
+            dist.destroy_process_group()
+        return 0
+
+    peak, peak_kind = measured_peak()
+    launch_ms = statistics.fmean(per_launch_ms)
+    achieved = bytes_per_step / (launch_ms * 1e-3) / 1e9
+    roofline = {"bound": "hbm", "achieved": achieved, "peak": peak, "unit": "GB/s", "frac": achieved / peak,
+                "peak_kind": "of " + peak_kind, "frac_of_nominal_8TBs": achieved / NOMINAL_HBM_GBS,
+                "traffic": None if NCU_TRAFFIC_BYTES_PER_TOKEN is None else NCU_TRAFFIC_BYTES_PER_TOKEN * T_HEAD,
+                "algorithmic_bytes_per_launch": bytes_per_step, "kernel_ms": launch_ms}
+
+    sweep = []
+    if not args.no_sweep:
+        def time_calls(fn, n=30, warm=5):
+            for i in range(warm):
+                fn(i)
+            torch.cuda.synchronize()
+            a, b_ = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+            a.record()
+            for i in range(n):
+                fn(i)
+            b_.record()
+            torch.cuda.synchronize()
+            return a.elapsed_time(b_) / n
+
+        for f in ("int4", "mxfp4"):
+            fcode = B.FMT_BY_NAME[f]
+            grp = 0 if f == "int4" else 32
+            o = [B.alloc_outputs(T_HEAD, D_HEAD, fcode, grp, base.device) for _ in range(RING)]
+            for bb in (16, 32, 128, 4096):
+                ms = time_calls(lambda i: B.perq_rotate_quantize(xs[i % RING], None, bb, fcode, grp,
+                                                                 out_codes=o[i % RING][0], out_scales=o[i % RING][1]))
+                by = bytes_per_token(D_HEAD, f, grp) * T_HEAD
+                gbs = by / (ms * 1e-3) / 1e9
+                sweep.append({"call": "perq_rotate_quantize", "T": T_HEAD, "d": D_HEAD, "b": bb, "fmt": f, "group": grp,
+                              "ms": ms, "GB/s": gbs, "frac_of_" + peak_kind: gbs / peak,
+                              "frac_of_nominal_8TBs": gbs / NOMINAL_HBM_GBS, "Mtokens/s": T_HEAD / ms / 1e3})
+            del o
+        # the calibration statistic on the MLP down-projection shape (T=4096 x d=8192, b=32)
+        w3 = inputs.config3(T=4096)
+        x3 = [torch.from_numpy(w3.x.view(np.int16).copy()).cuda().view(torch.bfloat16)]
+        x3 += [torch.roll(x3[0], shifts=5 * (i + 1), dims=0).contiguous() for i in range(RING - 1)]
+        wsb = torch.empty(B.perq_block_l1_stats_workspace_bytes(4096, 8192, 32), dtype=torch.uint8, device="cuda")
+        ms = time_calls(lambda i: B.perq_block_l1_stats(x3[i % RING], None, 32, workspace=wsb))
+        by = 4096 * 8192 * 2
+        sweep.append({"call": "perq_block_l1_stats", "T": 4096, "d": 8192, "b": 32, "ms": ms,
+                      "GB/s": by / (ms * 1e-3) / 1e9, "frac_of_" + peak_kind: by / (ms * 1e-3) / 1e9 / peak})
+
+    cpu_baseline = None
+    if not args.no_cpu_baseline:
+        from oracle import perq_oracle
+        perq_oracle.build()
+        rows = 4096
+        wb = inputs.config4(T=rows, b=B_HEAD, fmt=FMT_HEAD)
+        perq_oracle.rotate_quantize(wb.x[:256], None, B_HEAD, perq_oracle.FMT_INT4, GROUP_HEAD)
+        t0 = time.perf_counter()
+        reps = 0
+        while time.perf_counter() - t0 < 10.0:
+            perq_oracle.rotate_quantize(wb.x, None, B_HEAD, perq_oracle.FMT_INT4, GROUP_HEAD)
+            reps += 1
+        dt = (time.perf_counter() - t0) / reps
+        cpu_baseline = {"value": rows * bpt / dt / 1e9, "unit": UNIT, "cores": perq_oracle.num_threads(),
+                        "kind": "oracle", "mtokens_per_s": rows / dt / 1e6,
+                        "sample": "%d of %d rows of the same workload, repeated for ~10 s (%d passes)" % (rows, T_HEAD, reps)}
+
+    line = {
+        "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps, "warmup": args.warmup,
+        "ms_per_step": ms_per_step, "higher_is_better": True, "scaling": "weak", "vs_baseline": None,
+        "dtype": "f32", "data": "synthetic",
+        "config": {"workload": "cfg4 Llama-3-8B hidden: T=%d d=%d bf16 Laplace(0,1)+4 outlier channels x200, no perm, "
+                               "block Hadamard b=%d, INT4 per-token absmax scale" % (T_HEAD, D_HEAD, B_HEAD),
+                   "per_gpu_tokens": T_HEAD, "l2": "ring of %d input sets, each 134 MB > 126 MB L2" % RING},
+        "mtokens_per_s": world * T_HEAD / ms_per_step / 1e3,
+        "pct_of_nominal_8TBs": 100.0 * value / world / NOMINAL_HBM_GBS,
+        "clocks": clocks, "e2e": e2e, "gpu_launches": args.steps,
+        "roofline": roofline, "cpu_baseline": cpu_baseline, "sweep": sweep,
+    }
+    print(json.dumps(line))
+    if dist is not None:
+        dist.barrier()
+        dist.destroy_process_group()
+    return 0
+
+
+if __name__ == "__main__":
+    sys.exit(main())

@@ -78,7 +78,8 @@ typedef enum {
  * perm       device, int32 [d], a permutation of 0..d-1, or NULL.  Out-of-range entries
  *            are clamped into range (wrong numbers, never a fault); use
  *            perq_validate_perm to check a permutation beforehand.
- * T, d       rows and channels.  T == 0 is a no-op.  d % 32 == 0, d <= PERQ_MAX_D.
+ * T, d       rows and channels.  T == 0 is a no-op (pointers are then not looked at).
+ *            d % 32 == 0, d <= PERQ_MAX_D.
  * b          16, 32, 64 or 128 with d % b == 0; or b == d when d is a power of two.
  * fmt        perq_fmt_t.
  * group      INT4: 0 (per token) or a multiple of 8 dividing d.  MXFP4: 0 or 32 (always 32).

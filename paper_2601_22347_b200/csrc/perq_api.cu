@@ -169,9 +169,9 @@ int perq_rotate_quantize(const void *x, const int32_t *perm, int64_t T, int32_t 
 {
     int g = 0;
     if (int rc = check_shape(T, d, b, fmt, group, &g)) return rc;
+    if (T == 0) return PERQ_OK;   // nothing to read or write: pointers may be anything
     if (!x || !out_codes || (fmt != PERQ_FMT_F32_DEBUG && !out_scales)) return PERQ_ERR_NULL;
     if (!aligned16(x) || !aligned16(out_codes) || !aligned16(out_scales) || !aligned16(perm)) return PERQ_ERR_ALIGN;
-    if (T == 0) return PERQ_OK;
     return launch_generic(x, perm, T, d, b, fmt, g, out_codes, out_scales, static_cast<cudaStream_t>(stream));
 }
 
@@ -191,11 +191,11 @@ int perq_rotate_quantize_host(const void *x_host, const int32_t *perm, int64_t T
 {
     int g = 0;
     if (int rc = check_shape(T, d, b, fmt, group, &g)) return rc;
+    if (T == 0) return PERQ_OK;
     if (!x_host || !out_codes_host || (fmt != PERQ_FMT_F32_DEBUG && !out_scales_host)) return PERQ_ERR_NULL;
     size_t need = 0, cb = 0, sb = 0;
     perq_host_workspace_bytes(T, d, fmt, group, &need);
     perq_out_sizes(T, d, fmt, group, &cb, &sb);
-    if (T == 0) return PERQ_OK;
     if (!workspace || workspace_bytes < need) return PERQ_ERR_WORKSPACE;
     if (!aligned16(workspace) || !aligned16(perm)) return PERQ_ERR_ALIGN;
     auto up = [](size_t v) { return (v + 255) & ~(size_t)255; };
