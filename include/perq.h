@@ -156,6 +156,14 @@ int perq_validate_perm(const int32_t *perm, int32_t d, int32_t *status_dev, void
  */
 int perq_massdiff_perm(const float *chan_abs_sum_host, int32_t d, int32_t b, int32_t *perm_host);
 
+/*
+ * perq_device_error -- reads (synchronously, cudaMemcpyFromSymbol) the library's device-side
+ * error word on the current device into *flags_host.  0 = no error.  Bit 0 is set when a
+ * bounded wait inside a kernel ran out (an asynchronous copy that never completed); the
+ * kernel then stops early and its outputs are incomplete.  The word is never cleared.
+ */
+int perq_device_error(uint32_t *flags_host);
+
 /* Text for a status code (static storage).  Library version = major*10000 + minor*100 + patch. */
 const char *perq_status_string(int status);
 int perq_version(void);

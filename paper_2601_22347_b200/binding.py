@@ -50,6 +50,8 @@ def load() -> C.CDLL:
         lib.perq_block_l1_stats_workspace_bytes.argtypes = [i64, i32, i32, C.POINTER(sz)]
         lib.perq_validate_perm.argtypes = [vp, i32, vp, vp]
         lib.perq_massdiff_perm.argtypes = [vp, i32, i32, vp]
+        lib.perq_device_error.argtypes = [C.POINTER(C.c_uint32)]
+        lib.perq_device_error.restype = C.c_int
         lib.perq_status_string.argtypes = [C.c_int]
         lib.perq_status_string.restype = C.c_char_p
         lib.perq_version.restype = C.c_int
@@ -165,6 +167,13 @@ def perq_validate_perm(perm: torch.Tensor, stream=None) -> torch.Tensor:
     status = torch.empty(1, dtype=torch.int32, device=perm.device)
     _check(load().perq_validate_perm(_ptr(perm), perm.numel(), _ptr(status), _stream(stream)), "perq_validate_perm")
     return status
+
+
+def perq_device_error() -> int:
+    """Device-side error word of the current device (0 = none); synchronises."""
+    v = C.c_uint32(0)
+    _check(load().perq_device_error(C.byref(v)), "perq_device_error")
+    return int(v.value)
 
 
 def perq_massdiff_perm(chan_abs_sum_host: np.ndarray, b: int) -> np.ndarray:

@@ -12,6 +12,7 @@
 #include <cuda_runtime.h>
 
 #include "perq_generic.cuh"
+#include "perq_fast.cuh"
 #include "perq_stats.cuh"
 
 namespace {
@@ -96,6 +97,70 @@ int launch_generic(const void *x, const int32_t *perm, int64_t T, int32_t d, int
     return cudaGetLastError() == cudaSuccess ? PERQ_OK : PERQ_ERR_CUDA;
 }
 
+template <int LOG2B, int MODE>
+int launch_fast_inst(const perq::FastParams &p, int grid, cudaStream_t st)
+{
+    auto kernel = perq::perq_fast_kernel<LOG2B, MODE>;
+    if (int rc = allow_smem(kernel, perq::FastSmem::total)) return rc;
+    kernel<<<grid, perq::FAST_THREADS, perq::FastSmem::total, st>>>(p);
+    return cudaGetLastError() == cudaSuccess ? PERQ_OK : PERQ_ERR_CUDA;
+}
+
+template <int MODE>
+int launch_fast_mode(int log2b, const perq::FastParams &p, int grid, cudaStream_t st)
+{
+    switch (log2b) {
+    case 4: return launch_fast_inst<4, MODE>(p, grid, st);
+    case 5: return launch_fast_inst<5, MODE>(p, grid, st);
+    case 6: return launch_fast_inst<6, MODE>(p, grid, st);
+    default: return launch_fast_inst<7, MODE>(p, grid, st);
+    }
+}
+
+// The fast kernel covers: no permutation, b <= 128, d % 1024 == 0, and scales per token
+// (d / 1024 in {1,2,4,8}), per 128 (INT4) or per 32 (MXFP4).  Returns -1 if it does not apply.
+int try_launch_fast(const void *x, const int32_t *perm, int64_t T, int32_t d, int32_t b, int32_t fmt, int g,
+                    void *out_codes, void *out_scales, cudaStream_t st)
+{
+    if (perm != nullptr || b > 128 || d % perq::SEG_ELEMS != 0) return -1;
+    int mode, G = 1;
+    if (fmt == PERQ_FMT_MXFP4) {
+        mode = perq::MODE_MX;
+    } else if (fmt == PERQ_FMT_INT4 && g == 128) {
+        mode = perq::MODE_G128;
+    } else if (fmt == PERQ_FMT_INT4 && g == d) {
+        G = d / perq::SEG_ELEMS;
+        if (G != 1 && G != 2 && G != 4 && G != 8) return -1;
+        mode = perq::MODE_TOKEN;
+    } else {
+        return -1;
+    }
+    perq::FastParams p;
+    p.x = static_cast<const uint16_t *>(x);
+    p.out_codes = static_cast<uint8_t *>(out_codes);
+    p.out_scales = out_scales;
+    p.G = G;
+    p.units_total = (long long)T * (d / perq::SEG_ELEMS) / G;
+    p.sqrt_b = std::sqrt((double)b);
+    const int sms = sm_count();
+    if (sms <= 0) return PERQ_ERR_CUDA;
+    const int groups_per_cta = perq::FAST_WARPS / G;
+    const long long want = (p.units_total + groups_per_cta - 1) / groups_per_cta;
+    const int grid = (int)std::min<long long>(want, sms);
+    const int log2b = ilog2(b);
+    if (mode == perq::MODE_MX) return launch_fast_mode<perq::MODE_MX>(log2b, p, grid, st);
+    if (mode == perq::MODE_G128) return launch_fast_mode<perq::MODE_G128>(log2b, p, grid, st);
+    return launch_fast_mode<perq::MODE_TOKEN>(log2b, p, grid, st);
+}
+
+int launch_any(const void *x, const int32_t *perm, int64_t T, int32_t d, int32_t b, int32_t fmt, int g,
+               void *out_codes, void *out_scales, cudaStream_t st)
+{
+    const int rc = try_launch_fast(x, perm, T, d, b, fmt, g, out_codes, out_scales, st);
+    if (rc >= 0) return rc;
+    return launch_generic(x, perm, T, d, b, fmt, g, out_codes, out_scales, st);
+}
+
 struct StatsPlan {
     int n_cta;
     int rows_per_cta;
@@ -172,7 +237,7 @@ int perq_rotate_quantize(const void *x, const int32_t *perm, int64_t T, int32_t 
     if (T == 0) return PERQ_OK;   // nothing to read or write: pointers may be anything
     if (!x || !out_codes || (fmt != PERQ_FMT_F32_DEBUG && !out_scales)) return PERQ_ERR_NULL;
     if (!aligned16(x) || !aligned16(out_codes) || !aligned16(out_scales) || !aligned16(perm)) return PERQ_ERR_ALIGN;
-    return launch_generic(x, perm, T, d, b, fmt, g, out_codes, out_scales, static_cast<cudaStream_t>(stream));
+    return launch_any(x, perm, T, d, b, fmt, g, out_codes, out_scales, static_cast<cudaStream_t>(stream));
 }
 
 int perq_host_workspace_bytes(int64_t T, int32_t d, int32_t fmt, int32_t group, size_t *bytes)
@@ -207,7 +272,7 @@ int perq_rotate_quantize_host(const void *x_host, const int32_t *perm, int64_t T
     unsigned char *scales_dev = codes_dev + up(cb);
     if (cudaMemcpyAsync(x_dev, x_host, (size_t)T * (size_t)d * 2, cudaMemcpyHostToDevice, st) != cudaSuccess)
         return PERQ_ERR_CUDA;
-    if (int rc = launch_generic(x_dev, perm, T, d, b, fmt, g, codes_dev, scales_dev, st)) return rc;
+    if (int rc = launch_any(x_dev, perm, T, d, b, fmt, g, codes_dev, scales_dev, st)) return rc;
     if (cudaMemcpyAsync(out_codes_host, codes_dev, cb, cudaMemcpyDeviceToHost, st) != cudaSuccess) return PERQ_ERR_CUDA;
     if (sb && cudaMemcpyAsync(out_scales_host, scales_dev, sb, cudaMemcpyDeviceToHost, st) != cudaSuccess)
         return PERQ_ERR_CUDA;
@@ -265,6 +330,15 @@ int perq_validate_perm(const int32_t *perm, int32_t d, int32_t *status_dev, void
     const size_t smem = (size_t)((d + 31) / 32) * sizeof(uint32_t);
     perq::perq_validate_perm_kernel<<<1, 1024, smem, static_cast<cudaStream_t>(stream)>>>(perm, d, status_dev);
     return cudaGetLastError() == cudaSuccess ? PERQ_OK : PERQ_ERR_CUDA;
+}
+
+int perq_device_error(uint32_t *flags_host)
+{
+    if (!flags_host) return PERQ_ERR_NULL;
+    unsigned int v = 0;
+    if (cudaMemcpyFromSymbol(&v, perq::g_perq_device_error, sizeof v) != cudaSuccess) return PERQ_ERR_CUDA;
+    *flags_host = v;
+    return PERQ_OK;
 }
 
 int perq_massdiff_perm(const float *chan_abs_sum_host, int32_t d, int32_t b, int32_t *perm_host)

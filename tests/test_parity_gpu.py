@@ -95,6 +95,52 @@ def test_config5_large_T_sampled(B, oracle):
     check(B, oracle, w, rows=rows)
 
 
+# ------------------------------------------------------------------ the tensor-core fast path, every variant
+
+@pytest.mark.parametrize("fmt,group", [("int4", 0), ("int4", 128), ("mxfp4", 32)])
+@pytest.mark.parametrize("b", [16, 32, 64, 128])
+@pytest.mark.parametrize("d,T", [(1024, 67), (2048, 301), (4096, 130), (8192, 45)])
+def test_fast_path_matrix(B, oracle, d, T, b, fmt, group):
+    bits, _ = inputs.student_t_outliers(T, d, 3.0, max(2, d // 256), 100.0, seed=1000 + d + b)
+    bits[3] = 0                                   # an all-zero row in the middle of a CTA's work
+    bits[5, 128:384] = 0                          # zero groups / zero MX blocks
+    check(B, oracle, inputs.Workload("fast", bits, None, b, fmt, group, 0))
+
+
+@pytest.mark.parametrize("fmt,group", [("int4", 0), ("int4", 128), ("mxfp4", 32)])
+def test_fast_path_many_units_per_warp(B, oracle, fmt, group):
+    # enough rows that every warp of every CTA goes round its ring several times
+    w = inputs.config4(T=16384, b=64, fmt=fmt)
+    w.group = group
+    rows = np.sort(np.random.default_rng(6).choice(w.T, 80, replace=False))
+    rows[0], rows[-1] = 0, w.T - 1
+    check(B, oracle, w, rows=rows)
+    assert B.perq_device_error() == 0
+
+
+def test_fast_path_exact_ties(B, oracle):
+    import scipy.linalg
+    H = scipy.linalg.hadamard(16)
+    rng = np.random.default_rng(18)
+    rows = []
+    for _ in range(24):
+        blocks = []
+        for j in range(64):
+            ystar = rng.integers(-13, 14, size=16) * 0.5
+            ystar[rng.integers(0, 16)] = 7.0 if j == 0 else ystar[0]
+            blocks.append((ystar @ H) / 4.0)
+        rows.append(np.concatenate(blocks))
+    x = np.array(rows, np.float32)
+    bits = inputs.f32_to_bf16_bits(x)
+    assert np.array_equal(inputs.bf16_bits_to_f32(bits), x)
+    rep = check(B, oracle, inputs.Workload("fast-ties", bits, None, 16, "int4", 0, 0))
+    assert rep["code_mismatch_exempt"] == 0
+    rep = check(B, oracle, inputs.Workload("fast-ties-g", bits, None, 16, "int4", 128, 0))
+    assert rep["code_mismatch_exempt"] == 0
+    rep = check(B, oracle, inputs.Workload("fast-ties-mx", inputs.f32_to_bf16_bits(x * 0.5), None, 16, "mxfp4", 32, 0))
+    assert rep["code_mismatch_exempt"] == 0
+
+
 # ------------------------------------------------------------------ rotated values (debug format)
 
 @pytest.mark.parametrize("d,b,perm", [(2048, 16, False), (2048, 128, True), (4096, 4096, False),
