@@ -136,6 +136,37 @@ int perq_block_l1_stats(const void *x, const int32_t *perm, int64_t T, int32_t d
 int perq_block_l1_stats_workspace_bytes(int64_t T, int32_t d, int32_t b, size_t *bytes);
 
 /*
+ * perq_block_l1_stats_static -- perq_block_l1_stats for callers that cannot provide a workspace.
+ *
+ * (No counterpart in the paper: this is a deployment variant of the entry point above.)
+ * Some hosts of this library may not allocate device memory at the point where they want
+ * the statistic: code that runs inside a memory-pool-managed serving loop whose pool is
+ * already fully handed out, plugins that are only given their input and output tensors,
+ * or processes whose allocator must stay quiet because allocation would synchronise the
+ * device.  For them the per-CTA partial sums go to a fixed array inside the library
+ * instead of a caller workspace; outputs and every other argument are as above, and the
+ * results are bit-identical to perq_block_l1_stats on the same inputs.
+ *
+ *   - The array holds PERQ_STATS_STATIC_MAX_FLOATS floats (9.25 MiB) and is part of the
+ *     library image: every GPU that loads the library holds it until the process exits.
+ *   - A shape is accepted when perq_block_l1_stats_workspace_bytes(T, d, b) fits in the
+ *     array, i.e. min(T, 148) * (d + d/b) <= PERQ_STATS_STATIC_MAX_FLOATS; this covers
+ *     every d <= 14336 with any T and b >= 8.  Larger shapes return PERQ_ERR_WORKSPACE
+ *     and launch nothing.
+ *   - The call allocates and frees nothing, on the device or through any library.
+ *   - The first call on each device looks up the array's device address (with that
+ *     device current) and remembers it; make that first call outside any stream capture.
+ *   - All calls on a device share the one array.  Nothing in it has to be zero on entry
+ *     (each call overwrites what it reads), but two calls whose kernels overlap on the
+ *     GPU -- different streams, no ordering between them -- race on it and give wrong
+ *     sums.  Calls on one stream, or ordered by events, are safe.
+ */
+#define PERQ_STATS_STATIC_MAX_FLOATS (148 * 16384)
+int perq_block_l1_stats_static(const void *x, const int32_t *perm, int64_t T, int32_t d, int32_t b,
+                               float *chan_abs_sum, float *block_l1_mean,
+                               float *token_max_block_l1, void *stream);
+
+/*
  * perq_validate_perm -- checks on the device that perm[0..d) is a permutation.
  * Writes one int32 to status_dev: 0 = valid, bit 0 = an entry out of range,
  * bit 1 = a duplicate entry.  (Algorithm 1 returns such a permutation; this guards

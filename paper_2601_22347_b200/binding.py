@@ -47,6 +47,7 @@ def load() -> C.CDLL:
         lib.perq_host_workspace_bytes.argtypes = [i64, i32, i32, i32, C.POINTER(sz)]
         lib.perq_out_sizes.argtypes = [i64, i32, i32, i32, C.POINTER(sz), C.POINTER(sz)]
         lib.perq_block_l1_stats.argtypes = [vp, vp, i64, i32, i32, vp, vp, vp, vp, sz, vp]
+        lib.perq_block_l1_stats_static.argtypes = [vp, vp, i64, i32, i32, vp, vp, vp, vp]
         lib.perq_block_l1_stats_workspace_bytes.argtypes = [i64, i32, i32, C.POINTER(sz)]
         lib.perq_validate_perm.argtypes = [vp, i32, vp, vp]
         lib.perq_massdiff_perm.argtypes = [vp, i32, i32, vp]
@@ -56,7 +57,8 @@ def load() -> C.CDLL:
         lib.perq_status_string.restype = C.c_char_p
         lib.perq_version.restype = C.c_int
         for name in ("perq_rotate_quantize", "perq_rotate_quantize_host", "perq_host_workspace_bytes",
-                     "perq_out_sizes", "perq_block_l1_stats", "perq_block_l1_stats_workspace_bytes",
+                     "perq_out_sizes", "perq_block_l1_stats", "perq_block_l1_stats_static",
+                     "perq_block_l1_stats_workspace_bytes",
                      "perq_validate_perm", "perq_massdiff_perm"):
             getattr(lib, name).restype = C.c_int
         _lib = lib
@@ -158,6 +160,22 @@ def perq_block_l1_stats(x: torch.Tensor, perm: Optional[torch.Tensor], b: int, w
     rc = load().perq_block_l1_stats(_ptr(x), _ptr(perm), T, d, b, _ptr(chan), _ptr(block), _ptr(token),
                                     _ptr(workspace), workspace.numel(), _stream(stream))
     _check(rc, "perq_block_l1_stats")
+    return chan, block, token
+
+
+def perq_block_l1_stats_static(x: torch.Tensor, perm: Optional[torch.Tensor], b: int, chan: Optional[torch.Tensor],
+                               block: Optional[torch.Tensor], token: Optional[torch.Tensor], stream=None):
+    """perq_block_l1_stats with the library's built-in scratch array instead of a workspace.
+
+    The caller passes the output tensors (any may be None); nothing is allocated here or in
+    the library.  Shapes whose partial sums do not fit the built-in array raise PerqError
+    (status 9).  Calls that may overlap on the GPU must not share a device: they would race
+    on the one scratch array."""
+    assert x.is_cuda and x.dtype == torch.bfloat16 and x.dim() == 2 and x.is_contiguous()
+    T, d = x.shape
+    rc = load().perq_block_l1_stats_static(_ptr(x), _ptr(perm), T, d, b, _ptr(chan), _ptr(block), _ptr(token),
+                                           _stream(stream))
+    _check(rc, "perq_block_l1_stats_static")
     return chan, block, token
 
 

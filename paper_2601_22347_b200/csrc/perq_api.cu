@@ -5,6 +5,7 @@
 #include <algorithm>
 #include <cmath>
 #include <cstdint>
+#include <mutex>
 #include <queue>
 #include <utility>
 #include <vector>
@@ -183,6 +184,14 @@ int plan_stats(int64_t T, int32_t d, int32_t b, StatsPlan *plan)
     return PERQ_OK;
 }
 
+// Scratch of perq_block_l1_stats_static: per-CTA partial sums, resident on every device that
+// loads the library.  Each call's first kernel writes every slot its second kernel reads, so
+// nothing has to be cleared between calls.
+constexpr int kMaxDevices = 64;
+static __device__ __align__(256) float g_stats_scratch[PERQ_STATS_STATIC_MAX_FLOATS];
+float *g_stats_scratch_addr[kMaxDevices] = {};   // device address of the array, per device ordinal
+std::mutex g_stats_scratch_mutex;
+
 }  // namespace
 
 extern "C" {
@@ -321,6 +330,34 @@ int perq_block_l1_stats(const void *x, const int32_t *perm, int64_t T, int32_t d
         if (cudaGetLastError() != cudaSuccess) return PERQ_ERR_CUDA;
     }
     return PERQ_OK;
+}
+
+int perq_block_l1_stats_static(const void *x, const int32_t *perm, int64_t T, int32_t d, int32_t b,
+                                float *chan_abs_sum, float *block_l1_mean, float *token_max_block_l1, void *stream)
+{
+    StatsPlan plan;
+    if (int rc = plan_stats(T, d, b, &plan)) return rc;
+    if (plan.ws_bytes > sizeof(g_stats_scratch)) return PERQ_ERR_WORKSPACE;
+    if (!chan_abs_sum && !block_l1_mean && !token_max_block_l1) return PERQ_OK;
+    int dev = -1;
+    if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= kMaxDevices) return PERQ_ERR_CUDA;
+    float *scratch = nullptr;
+    {
+        // The array's name is only a host-side handle here; the kernels need its address on
+        // the current device, which the runtime hands out per device.
+        std::lock_guard<std::mutex> lock(g_stats_scratch_mutex);
+        if (g_stats_scratch_addr[dev] == nullptr) {
+            void *p = nullptr;
+            if (cudaGetSymbolAddress(&p, g_stats_scratch) != cudaSuccess || p == nullptr) {
+                (void)cudaGetLastError();
+                return PERQ_ERR_CUDA;
+            }
+            g_stats_scratch_addr[dev] = static_cast<float *>(p);
+        }
+        scratch = g_stats_scratch_addr[dev];
+    }
+    return perq_block_l1_stats(x, perm, T, d, b, chan_abs_sum, block_l1_mean, token_max_block_l1, scratch,
+                               sizeof(g_stats_scratch), stream);
 }
 
 int perq_validate_perm(const int32_t *perm, int32_t d, int32_t *status_dev, void *stream)
