@@ -51,6 +51,7 @@ struct FastParams {
     long long units_total;   // units of G segments
     int G;                   // warps (segments) per unit: 1 unless per-token scales
     double sqrt_b;
+    double inv_7_sqrt_b;     // 1 / (7 sqrt(b)): INT4 scale = exact |u|max times this
 };
 
 // Set (never cleared by kernels) when a bounded wait inside a kernel ran out.
@@ -60,9 +61,9 @@ struct FastSmem {
     static constexpr size_t stages = 0;
     static constexpr size_t codes = stages + (size_t)FAST_WARPS * FAST_NSTAGE * SEG_BYTES;
     static constexpr size_t full = codes + (size_t)FAST_WARPS * 2 * SEG_CODE_BYTES;
-    static constexpr size_t wmax = full + (size_t)FAST_WARPS * FAST_NSTAGE * 8;
-    static constexpr size_t exact = wmax + (size_t)FAST_WARPS * 2 * 4;
-    static constexpr size_t total = exact + (size_t)FAST_WARPS * 2 * 8;
+    static constexpr size_t wexact = full + (size_t)FAST_WARPS * FAST_NSTAGE * 8;   // [2][FAST_WARPS] u64
+    static constexpr size_t wmax = wexact + (size_t)FAST_WARPS * 2 * 8;             // [2][FAST_WARPS] f32
+    static constexpr size_t total = wmax + (size_t)FAST_WARPS * 2 * 4;
 };
 
 // ---------------------------------------------------------------- PTX wrappers
@@ -110,12 +111,62 @@ __device__ __forceinline__ void ldmatrix_x4(uint32_t (&r)[4], uint32_t addr)
     asm volatile("ldmatrix.sync.aligned.m8n8.x4.shared.b16 {%0,%1,%2,%3}, [%4];"
                  : "=r"(r[0]), "=r"(r[1]), "=r"(r[2]), "=r"(r[3]) : "r"(addr));
 }
+// c = a * b with a zero accumulator input (no registers are cleared for it)
 __device__ __forceinline__ void mma_bf16(float (&c)[4], const uint32_t (&a)[4], uint32_t b0, uint32_t b1)
 {
-    asm volatile("mma.sync.aligned.m16n8k16.row.col.f32.bf16.bf16.f32 {%0,%1,%2,%3}, {%4,%5,%6,%7}, {%8,%9}, {%0,%1,%2,%3};"
-                 : "+f"(c[0]), "+f"(c[1]), "+f"(c[2]), "+f"(c[3])
-                 : "r"(a[0]), "r"(a[1]), "r"(a[2]), "r"(a[3]), "r"(b0), "r"(b1));
+    asm volatile("mma.sync.aligned.m16n8k16.row.col.f32.bf16.bf16.f32 {%0,%1,%2,%3}, {%4,%5,%6,%7}, {%8,%9}, {%10,%10,%10,%10};"
+                 : "=f"(c[0]), "=f"(c[1]), "=f"(c[2]), "=f"(c[3])
+                 : "r"(a[0]), "r"(a[1]), "r"(a[2]), "r"(a[3]), "r"(b0), "r"(b1), "f"(0.0f));
 }
+
+// Two fp32 values in one 64-bit register pair, for the packed add/sub/mul/fma of sm_100.
+typedef unsigned long long f32x2;
+__device__ __forceinline__ f32x2 pack2(float lo, float hi)
+{
+    f32x2 r;
+    asm("mov.b64 %0, {%1, %2};" : "=l"(r) : "f"(lo), "f"(hi));
+    return r;
+}
+__device__ __forceinline__ void unpack2(f32x2 v, float &lo, float &hi)
+{
+    asm("mov.b64 {%0, %1}, %2;" : "=f"(lo), "=f"(hi) : "l"(v));
+}
+__device__ __forceinline__ void unpack2u(f32x2 v, uint32_t &lo, uint32_t &hi)
+{
+    asm("mov.b64 {%0, %1}, %2;" : "=r"(lo), "=r"(hi) : "l"(v));
+}
+__device__ __forceinline__ f32x2 add2(f32x2 a, f32x2 b)
+{
+    f32x2 r;
+    asm("add.rn.f32x2 %0, %1, %2;" : "=l"(r) : "l"(a), "l"(b));
+    return r;
+}
+__device__ __forceinline__ f32x2 sub2(f32x2 a, f32x2 b)
+{
+    f32x2 r;
+    asm("sub.rn.f32x2 %0, %1, %2;" : "=l"(r) : "l"(a), "l"(b));
+    return r;
+}
+__device__ __forceinline__ f32x2 fma2(f32x2 a, f32x2 b, f32x2 c)
+{
+    f32x2 r;
+    asm("fma.rn.f32x2 %0, %1, %2, %3;" : "=l"(r) : "l"(a), "l"(b), "l"(c));
+    return r;
+}
+__device__ __forceinline__ f32x2 mul2(f32x2 a, f32x2 b)
+{
+    f32x2 r;
+    asm("mul.rn.f32x2 %0, %1, %2;" : "=l"(r) : "l"(a), "l"(b));
+    return r;
+}
+// max over the warp of a non-negative fp32 value (one instruction on sm_100a)
+__device__ __forceinline__ float warp_max_f32(float v)
+{
+    float r;
+    asm volatile("redux.sync.max.f32 %0, %1, 0xffffffff;" : "=f"(r) : "f"(v));
+    return r;
+}
+__device__ __forceinline__ float max3abs(float acc, float a, float b) { return fmaxf(fmaxf(acc, fabsf(a)), fabsf(b)); }
 __device__ __forceinline__ void named_barrier(int id, int threads)
 {
     asm volatile("bar.sync %0, %1;" ::"r"(id), "r"(threads) : "memory");
@@ -124,6 +175,15 @@ __device__ __forceinline__ void named_barrier(int id, int threads)
 __device__ __forceinline__ uint32_t hadamard_bf16(int k, int n) { return (__popc(k & n) & 1) ? 0xBF80u : 0x3F80u; }
 
 // ---------------------------------------------------------------- exact re-evaluation
+
+// bf16 bit pattern (low 16 bits of h) -> double, exactly, with integer operations (the
+// fp32->fp64 conversion instruction is slow); zero and subnormals take the conversion.
+__device__ __forceinline__ double bf16_bits_to_f64(uint32_t h)
+{
+    const uint32_t mag = h & 0x7fffu;
+    if (mag < 0x80u) return (double)__uint_as_float(h << 16);
+    return __hiloint2double((int)(((mag << 13) + 0x38000000u) | ((h & 0x8000u) << 16)), 0);
+}
 
 // Exact unnormalised output i of the block starting at `blk` (bf16 in shared memory), evaluated
 // by the 4 lanes of a quad: each lane reduces a quarter of the block with a signed pairwise
@@ -137,8 +197,8 @@ __device__ __forceinline__ double exact_coord_quad(const uint16_t *blk, int i, i
 #pragma unroll
     for (int r = 0; r < PER / 2; ++r) {
         const uint32_t w = src[r];
-        v[2 * r] = (double)bf16lo(w);
-        v[2 * r + 1] = (double)bf16hi(w);
+        v[2 * r] = bf16_bits_to_f64(w);
+        v[2 * r + 1] = bf16_bits_to_f64(w >> 16);
     }
 #pragma unroll
     for (int t = 0; (1 << t) < PER; ++t) {
@@ -165,16 +225,56 @@ __device__ __forceinline__ void locate(int g, int q, int e, int &blk_elem, int &
     i = elem - blk_elem;
 }
 
+
+// Exact unnormalised output i of the B-element block at blk (bf16 in shared memory), by a whole warp.
+template <int B>
+__device__ __forceinline__ double exact_coord_fast(const uint16_t *blk, int i, int lane)
+{
+    double acc = 0.0;
+#pragma unroll
+    for (int k0 = 0; k0 < B; k0 += 32) {
+        const int k = k0 + lane;
+        if (B >= 32 || k < B) {
+            const double v = bf16_bits_to_f64(blk[k]);
+            acc += (__popc(i & k) & 1) ? -v : v;
+        }
+    }
+#pragma unroll
+    for (int o = 16; o > 0; o >>= 1) acc += __shfl_xor_sync(0xffffffffu, acc, o);
+    return acc;
+}
+
+// Bit mask of the lane's 32 held values (bit s*4+j) whose magnitude reaches thr; ms[s] is the
+// magnitude maximum of slot s, used to skip slots.
+__device__ __forceinline__ uint32_t candidate_mask(const f32x2 (&v)[8][2], const float (&ms)[8], float thr)
+{
+    uint32_t cm = 0u;
+#pragma unroll
+    for (int s = 0; s < 8; ++s) {
+        if (ms[s] >= thr) {
+            float a, b, c, d;
+            unpack2(v[s][0], a, b);
+            unpack2(v[s][1], c, d);
+            cm |= (fabsf(a) >= thr ? 1u : 0u) << (4 * s);
+            cm |= (fabsf(b) >= thr ? 2u : 0u) << (4 * s);
+            cm |= (fabsf(c) >= thr ? 4u : 0u) << (4 * s);
+            cm |= (fabsf(d) >= thr ? 8u : 0u) << (4 * s);
+        }
+    }
+    return cm;
+}
+
 // ---------------------------------------------------------------- the kernel
 
 template <int LOG2B, int MODE>
 __global__ void __launch_bounds__(FAST_THREADS, 1) perq_fast_kernel(FastParams p)
 {
     constexpr int B = 1 << LOG2B;
-    constexpr int CB = LOG2B - 4;
-    constexpr int PM = (1 << CB) - 1;
+    constexpr int CB = LOG2B - 4;                 // butterfly stages left after the tensor-core H_16
+    constexpr int PM = (1 << CB) - 1;             // slot bits inside a Hadamard block
+    constexpr int NCLS = (PM & 3) + 1;            // sign classes of the slot relabelling
     constexpr float MAGIC = 12582920.0f;          // 1.5 * 2^23 + 8: low nibble of the sum = code + 8
-    extern __shared__ __align__(128) unsigned char smem[];
+    extern __shared__ __align__(128) unsigned char fsmem[];
 
     const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
     const int g = lane >> 2, q = lane & 3;
@@ -184,25 +284,24 @@ __global__ void __launch_bounds__(FAST_THREADS, 1) perq_fast_kernel(FastParams p
     const unsigned qmask = 0xFu << (lane & 28);
     const float err_rel = FAST_ERR_K * (float)LOG2B * TWO_M24;
 
-    unsigned char *stage_base = smem + FastSmem::stages + (size_t)group * G * FAST_NSTAGE * SEG_BYTES;
-    unsigned char *code_base = smem + FastSmem::codes + (size_t)warp * 2 * SEG_CODE_BYTES;
-    uint64_t *full = reinterpret_cast<uint64_t *>(smem + FastSmem::full) + group * FAST_NSTAGE;
-    float *wmax = reinterpret_cast<float *>(smem + FastSmem::wmax) + group * G * 2;      // [parity][G]
-    unsigned long long *exact = reinterpret_cast<unsigned long long *>(smem + FastSmem::exact) + group * 2;
+    unsigned char *stage_base = fsmem + FastSmem::stages + (size_t)group * G * FAST_NSTAGE * SEG_BYTES;
+    unsigned char *code_base = fsmem + FastSmem::codes + (size_t)warp * 2 * SEG_CODE_BYTES;
+    uint64_t *full = reinterpret_cast<uint64_t *>(fsmem + FastSmem::full) + group * FAST_NSTAGE;
+    unsigned long long *wexact = reinterpret_cast<unsigned long long *>(fsmem + FastSmem::wexact);   // [2][FAST_WARPS]
+    float *wmax = reinterpret_cast<float *>(fsmem + FastSmem::wmax);                                 // [2][FAST_WARPS]
     const bool leader = (w_in_g == 0) && (lane == 0);
     const uint32_t unit_bytes = (uint32_t)G * SEG_BYTES;
 
     if (tid == 0) {
         for (int i = 0; i < FAST_WARPS * FAST_NSTAGE; ++i)
-            mbar_init(smem_u32(reinterpret_cast<uint64_t *>(smem + FastSmem::full) + i), 1);
+            mbar_init(smem_u32(reinterpret_cast<uint64_t *>(fsmem + FastSmem::full) + i), 1);
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
     }
-    if (MODE == MODE_TOKEN && leader) { exact[0] = 0ull; exact[1] = 0ull; }
     __syncthreads();
 
     const long long first = (long long)blockIdx.x * groups_per_cta + group;
     const long long stride = (long long)gridDim.x * groups_per_cta;
-    if (first >= p.units_total) return;      // whole groups leave together (no barrier is shared across groups)
+    if (group >= groups_per_cta || first >= p.units_total) return;   // whole groups leave together
 
     // Hadamard operand of the tensor-core stage: column n of MMA m is output 4*(n/2) + (n%2) + 2m.
     uint32_t hb[2][2];
@@ -247,11 +346,11 @@ __global__ void __launch_bounds__(FAST_THREADS, 1) perq_fast_kernel(FastParams p
         }
     }
 
-    long long it = 0;
+    uint32_t it = 0;
     for (long long unit = first; unit < p.units_total; unit += stride, ++it) {
-        const int stage = (int)(it % FAST_NSTAGE);
-        const uint32_t parity = (uint32_t)((it / FAST_NSTAGE) & 1);
-        const int par2 = (int)(it & 1);
+        const uint32_t stage = it % FAST_NSTAGE;
+        const uint32_t parity = (it / FAST_NSTAGE) & 1u;
+        const uint32_t par2 = it & 1u;
         if (!mbar_wait(smem_u32(&full[stage]), parity)) {
             if (lane == 0) atomicOr(&g_perq_device_error, 1u);
             return;
@@ -261,25 +360,27 @@ __global__ void __launch_bounds__(FAST_THREADS, 1) perq_fast_kernel(FastParams p
         const uint32_t seg_addr = smem_u32(seg);
         const long long seg_index = unit * G + w_in_g;
 
-        // ---- H_16 on the tensor cores
-        float v[8][4];
+        // ---- H_16 on the tensor cores; v[s][h] = outputs (2h, 2h+1) of this lane's four of slot s
+        f32x2 v[8][2];
 #pragma unroll
         for (int t = 0; t < 4; ++t) {
             uint32_t a[4];
             ldmatrix_x4(a, seg_addr + lm_off[t]);
-            float c0[4] = {0.f, 0.f, 0.f, 0.f}, c1[4] = {0.f, 0.f, 0.f, 0.f};
+            float c0[4], c1[4];
             mma_bf16(c0, a, hb[0][0], hb[0][1]);
             mma_bf16(c1, a, hb[1][0], hb[1][1]);
-            v[2 * t][0] = c0[0]; v[2 * t][1] = c0[1]; v[2 * t][2] = c1[0]; v[2 * t][3] = c1[1];
-            v[2 * t + 1][0] = c0[2]; v[2 * t + 1][1] = c0[3]; v[2 * t + 1][2] = c1[2]; v[2 * t + 1][3] = c1[3];
+            v[2 * t][0] = pack2(c0[0], c0[1]);
+            v[2 * t][1] = pack2(c1[0], c1[1]);
+            v[2 * t + 1][0] = pack2(c0[2], c0[3]);
+            v[2 * t + 1][1] = pack2(c1[2], c1[3]);
         }
         // refill the stage the previous iteration used (every warp of the group is past it now:
-        // for G == 1 because this warp is, for G > 1 after the first named barrier below)
+        // for G == 1 because this warp is, for G > 1 after the named barrier below)
         auto refill = [&]() {
             if (leader && it > 0) {
                 const long long u = unit + (long long)(FAST_NSTAGE - 1) * stride;
                 if (u < p.units_total) {
-                    const int ps = (int)((it - 1) % FAST_NSTAGE);
+                    const uint32_t ps = (it - 1) % FAST_NSTAGE;
                     mbar_expect_tx(smem_u32(&full[ps]), unit_bytes);
                     bulk_load(smem_u32(stage_base + (size_t)ps * unit_bytes), p.x + (size_t)u * G * SEG_ELEMS,
                               unit_bytes, smem_u32(&full[ps]));
@@ -288,299 +389,32 @@ __global__ void __launch_bounds__(FAST_THREADS, 1) perq_fast_kernel(FastParams p
         };
         if (MODE != MODE_TOKEN) refill();
 
-        // ---- remaining butterfly stages over the slot bits inside a block
+        // ---- remaining butterfly stages over the slot bits inside a block (packed add/sub)
 #pragma unroll
         for (int t = 0; t < CB; ++t) {
 #pragma unroll
             for (int s = 0; s < 8; ++s) {
                 if ((s & (1 << t)) == 0) {
 #pragma unroll
-                    for (int j = 0; j < 4; ++j) {
-                        const float a = v[s][j], c = v[s | (1 << t)][j];
-                        v[s][j] = a + c;
-                        v[s | (1 << t)][j] = a - c;
+                    for (int h = 0; h < 2; ++h) {
+                        const f32x2 a = v[s][h], c = v[s | (1 << t)][h];
+                        v[s][h] = add2(a, c);
+                        v[s | (1 << t)][h] = sub2(a, c);
                     }
                 }
             }
         }
 
-        // ---- fp32 maxima
+        // ---- fp32 maxima per slot
         float ms[8];
 #pragma unroll
-        for (int s = 0; s < 8; ++s)
-            ms[s] = fmaxf(fmaxf(fabsf(v[s][0]), fabsf(v[s][1])), fmaxf(fabsf(v[s][2]), fabsf(v[s][3])));
-
-        uint8_t *code_buf = code_base + (size_t)(it & 1) * SEG_CODE_BYTES;
-        bulk_store_wait_read<1>();           // the store that last read this staging buffer has drained
-        __syncwarp();
-
-        uint32_t tie_any = 0u;
-        double a_exact = 0.0;                // exact range maximum (INT4 modes)
-        int E_pack = 0;                      // MX: E + 127 of the lane's four groups, one per byte
-        float mul_p[4], mul_m[4];            // per sign class: +-multiplier * (1 +- delta)
-
-        if (MODE == MODE_TOKEN || MODE == MODE_G128) {
-            float a32 = fmaxf(fmaxf(fmaxf(ms[0], ms[1]), fmaxf(ms[2], ms[3])), fmaxf(fmaxf(ms[4], ms[5]), fmaxf(ms[6], ms[7])));
-            const float lane_max = a32;
-            a32 = fmaxf(a32, __shfl_xor_sync(0xffffffffu, a32, 1));
-            a32 = fmaxf(a32, __shfl_xor_sync(0xffffffffu, a32, 2));
-            if (MODE == MODE_TOKEN) {
-                a32 = fmaxf(a32, __shfl_xor_sync(0xffffffffu, a32, 4));
-                a32 = fmaxf(a32, __shfl_xor_sync(0xffffffffu, a32, 8));
-                a32 = fmaxf(a32, __shfl_xor_sync(0xffffffffu, a32, 16));
-                if (G > 1) {
-                    if (lane == 0) wmax[par2 * G + w_in_g] = a32;
-                    named_barrier(1 + group, G * 32);
-                    for (int w = 0; w < G; ++w) a32 = fmaxf(a32, wmax[par2 * G + w]);
-                }
-                refill();
-                if (leader) exact[par2 ^ 1] = 0ull;
-            }
-            const float thr = a32 * (1.0f - 2.0f * err_rel - 2.4e-7f);
-            const bool has_cand = (a32 > 0.0f) && (lane_max >= thr);
-            // exact range maximum from the candidates
-            if (MODE == MODE_G128) {
-                unsigned cq = __ballot_sync(0xffffffffu, has_cand) & qmask;      // candidate lanes of my quad
-                while (cq) {
-                    const int src = __ffs(cq) - 1;
-                    cq &= cq - 1;
-                    uint32_t cm = 0u;
-                    if (lane == src) {
-#pragma unroll
-                        for (int e = 0; e < 32; ++e) cm |= (fabsf(v[e >> 2][e & 3]) >= thr) ? (1u << e) : 0u;
-                    }
-                    cm = __shfl_sync(qmask, cm, src);
-                    while (cm) {
-                        const int e = __ffs(cm) - 1;
-                        cm &= cm - 1;
-                        int blk_elem, i, elem;
-                        locate<LOG2B>(src >> 2, src & 3, e, blk_elem, i, elem);
-                        a_exact = fmax(a_exact, fabs(exact_coord_quad<LOG2B>(seg + blk_elem, i, q, qmask)));
-                    }
-                }
-            } else {
-                double wbest = 0.0;
-                unsigned cw = __ballot_sync(0xffffffffu, has_cand);
-                while (cw) {
-                    const int src = __ffs(cw) - 1;
-                    cw &= cw - 1;
-                    uint32_t cm = 0u;
-                    if (lane == src) {
-#pragma unroll
-                        for (int e = 0; e < 32; ++e) cm |= (fabsf(v[e >> 2][e & 3]) >= thr) ? (1u << e) : 0u;
-                    }
-                    cm = __shfl_sync(0xffffffffu, cm, src);
-                    while (cm) {
-                        const int e = __ffs(cm) - 1;
-                        cm &= cm - 1;
-                        int blk_elem, i, elem;
-                        locate<LOG2B>(src >> 2, src & 3, e, blk_elem, i, elem);
-                        wbest = fmax(wbest, fabs(exact_coord_warp(seg, blk_elem, B, i, lane)));
-                    }
-                }
-                if (G > 1) {
-                    if (lane == 0 && wbest > 0.0) atomicMax(&exact[par2], (unsigned long long)__double_as_longlong(wbest));
-                    named_barrier(1 + group, G * 32);
-                    a_exact = __longlong_as_double((long long)exact[par2]);
-                } else {
-                    a_exact = wbest;
-                }
-            }
-            // scale out
-            const double s64 = (a_exact / p.sqrt_b) / 7.0;
-            if (MODE == MODE_G128) {
-                if (q == 0) reinterpret_cast<float *>(p.out_scales)[seg_index * 8 + g] = (a_exact == 0.0) ? 0.0f : (float)s64;
-            } else if (leader) {
-                reinterpret_cast<float *>(p.out_scales)[unit] = (a_exact == 0.0) ? 0.0f : (float)s64;
-            }
-            // quantise
-            const float inv = (a32 > 0.0f) ? fminf(7.0f / a32, 3.0e38f) : 0.0f;
-            const float delta = 16.0f * err_rel + 5.0e-7f;
-#pragma unroll
-            for (int k = 0; k < 4; ++k) {
-                mul_p[k] = sgn[k] * inv * (1.0f + delta);
-                mul_m[k] = sgn[k] * inv * (1.0f - delta);
-            }
-#pragma unroll
-            for (int s = 0; s < 8; ++s) {
-                uint32_t t[4];
-#pragma unroll
-                for (int j = 0; j < 4; ++j) {
-                    const uint32_t tp = __float_as_uint(fmaf(v[s][j], mul_p[s & 3 & PM], MAGIC));
-                    const uint32_t tm = __float_as_uint(fmaf(v[s][j], mul_m[s & 3 & PM], MAGIC));
-                    tie_any |= tp ^ tm;
-                    t[j] = tp;
-                }
-                const uint32_t packed = (((t[3] * 16u + t[2]) * 16u + t[1]) * 16u + t[0]) ^ 0x8888u;
-                *reinterpret_cast<uint16_t *>(code_buf + code_off[s]) = (uint16_t)packed;
-            }
-            // ---- exact resolution of near ties
-            if (__any_sync(0xffffffffu, tie_any != 0u)) {
-                __syncwarp();
-                unsigned tl = __ballot_sync(0xffffffffu, tie_any != 0u);
-                while (tl) {
-                    const int src = __ffs(tl) - 1;
-                    tl &= tl - 1;
-                    uint32_t fm = 0u;
-#pragma unroll
-                    for (int e = 0; e < 32; ++e) {
-                        const uint32_t tp = __float_as_uint(fmaf(v[e >> 2][e & 3], mul_p[(e >> 2) & 3 & PM], MAGIC));
-                        const uint32_t tm = __float_as_uint(fmaf(v[e >> 2][e & 3], mul_m[(e >> 2) & 3 & PM], MAGIC));
-                        fm |= (tp != tm) ? (1u << e) : 0u;
-                    }
-                    fm = __shfl_sync(0xffffffffu, fm, src);
-                    const double s_src = __shfl_sync(0xffffffffu, s64, src);
-                    while (fm) {
-                        const int e = __ffs(fm) - 1;
-                        fm &= fm - 1;
-                        int blk_elem, i, elem;
-                        locate<LOG2B>(src >> 2, src & 3, e, blk_elem, i, elem);
-                        const double ue = exact_coord_warp(seg, blk_elem, B, i, lane);
-                        if (lane == 0) {
-                            uint32_t code = 0u;
-                            if (s_src != 0.0) {
-                                double qd = rint((ue / p.sqrt_b) / s_src);
-                                qd = fmin(fmax(qd, -8.0), 7.0);
-                                code = (uint32_t)((int)qd) & 0xFu;
-                            }
-                            uint8_t *bp = code_buf + (elem >> 1);
-                            *bp = (elem & 1) ? (uint8_t)((*bp & 0x0F) | (code << 4)) : (uint8_t)((*bp & 0xF0) | code);
-                        }
-                        __syncwarp();
-                    }
-                }
-            }
-        } else {   // ---------------------------------------------------------------- MXFP4
-            float cp_[4], cm_[4];
-            uint32_t word = 0u;
-#pragma unroll
-            for (int m = 0; m < 4; ++m) {
-                float a32 = fmaxf(ms[2 * m], ms[2 * m + 1]);
-                a32 = fmaxf(a32, __shfl_xor_sync(0xffffffffu, a32, 1));
-                a32 = fmaxf(a32, __shfl_xor_sync(0xffffffffu, a32, 2));
-                // error reference: the largest |u| of the Hadamard block (the group may be smaller than the block)
-                float bref = a32;
-                if (CB >= 2) {
-                    float bm = (CB == 2) ? fmaxf(fmaxf(ms[(2 * m) & 4], ms[((2 * m) & 4) + 1]), fmaxf(ms[((2 * m) & 4) + 2], ms[((2 * m) & 4) + 3]))
-                                         : fmaxf(fmaxf(fmaxf(ms[0], ms[1]), fmaxf(ms[2], ms[3])), fmaxf(fmaxf(ms[4], ms[5]), fmaxf(ms[6], ms[7])));
-                    bm = fmaxf(bm, __shfl_xor_sync(0xffffffffu, bm, 1));
-                    bm = fmaxf(bm, __shfl_xor_sync(0xffffffffu, bm, 2));
-                    bref = bm;
-                }
-                const float ratio = (a32 > 0.0f) ? bref / a32 : 1.0f;
-                const float rho = err_rel * ratio + 2.4e-7f;          // relative uncertainty of a32
-                // E = floor(log2(a / sqrt(b))) - 2 from the bits of a32; exact re-derivation near a boundary
-                const uint32_t bits = __float_as_uint(a32);
-                int eu = (int)(bits >> 23) - 127;
-                const uint32_t mant = bits & 0x7fffffu;
-                const float mrel = __uint_as_float(0x3f800000u | mant);          // [1, 2)
-                bool near;
-                int E;
-                if ((LOG2B & 1) == 0) {
-                    E = eu - LOG2B / 2 - 2;
-                    near = (mrel * (1.0f - rho) < 1.0f) || (mrel * (1.0f + rho) >= 2.0f);
-                } else {
-                    const float SQ2 = 1.41421356237f;
-                    E = eu - (LOG2B + 1) / 2 + (mant >= 0x3504f3u ? 1 : 0) - 2;
-                    near = (mrel * (1.0f - rho) < 1.0f) || (mrel * (1.0f + rho) >= 2.0f) || (fabsf(mrel - SQ2) <= rho * 2.0f);
-                }
-                if (a32 > 0.0f && (near || (bits >> 23) == 0u)) {
-                    // rare: exact maximum of the group from every element that could attain it
-                    const float thr = a32 - 2.0f * err_rel * bref - a32 * 2.4e-7f;
-                    const bool has = fmaxf(ms[2 * m], ms[2 * m + 1]) >= thr;
-                    unsigned cq = __ballot_sync(qmask, has) & qmask;
-                    double best = 0.0;
-                    while (cq) {
-                        const int src = __ffs(cq) - 1;
-                        cq &= cq - 1;
-                        uint32_t cm = 0u;
-                        if (lane == src) {
-#pragma unroll
-                            for (int e = 0; e < 8; ++e) cm |= (fabsf(v[2 * m + (e >> 2)][e & 3]) >= thr) ? (1u << e) : 0u;
-                        }
-                        cm = __shfl_sync(qmask, cm, src);
-                        while (cm) {
-                            const int e = __ffs(cm) - 1;
-                            cm &= cm - 1;
-                            int blk_elem, i, elem;
-                            locate<LOG2B>(src >> 2, src & 3, 8 * m + e, blk_elem, i, elem);
-                            best = fmax(best, fabs(exact_coord_quad<LOG2B>(seg + blk_elem, i, q, qmask)));
-                        }
-                    }
-                    int ex;
-                    (void)frexp(best / p.sqrt_b, &ex);
-                    E = ex - 3;
-                }
-                E = min(max(E, -127), 127);
-                const uint32_t byte = (a32 > 0.0f) ? (uint32_t)(E + 127) : 0u;
-                E_pack |= (int)(byte << (8 * m));
-                // multiplier 2^-E / sqrt(b)
-                float c;
-                if ((LOG2B & 1) == 0) c = __uint_as_float((uint32_t)min(max(127 - E - LOG2B / 2, 1), 254) << 23);
-                else c = __uint_as_float(0x3fb504f3u + ((uint32_t)(min(max(127 - E - (LOG2B + 1) / 2, 1), 253) - 127) << 23));
-                if (!(a32 > 0.0f)) c = 0.0f;
-                const float delta = 32.0f * err_rel * ratio + 5.0e-7f;
-                cp_[m] = c * (1.0f + delta);
-                cm_[m] = c * (1.0f - delta);
-                // scale byte position: group index inside the lane group's four groups
-                word |= byte << (8 * (m ^ ((f_g & ~PM) >> 1)));
-            }
-            if (q == 0) reinterpret_cast<uint32_t *>(p.out_scales)[seg_index * 8 + g] = word;
-#pragma unroll
-            for (int s = 0; s < 8; ++s) {
-                const float sg = sgn[s & 3 & PM];
-                const float kp = sg * cp_[s >> 1], km = sg * cm_[s >> 1];
-                const uint32_t p0 = cvt_e2m1x2(fmaf(v[s][0], kp, 0.0f), fmaf(v[s][1], kp, 0.0f));
-                const uint32_t p1 = cvt_e2m1x2(fmaf(v[s][2], kp, 0.0f), fmaf(v[s][3], kp, 0.0f));
-                const uint32_t m0 = cvt_e2m1x2(fmaf(v[s][0], km, 0.0f), fmaf(v[s][1], km, 0.0f));
-                const uint32_t m1 = cvt_e2m1x2(fmaf(v[s][2], km, 0.0f), fmaf(v[s][3], km, 0.0f));
-                tie_any |= (p0 ^ m0) | (p1 ^ m1);
-                *reinterpret_cast<uint16_t *>(code_buf + code_off[s]) = (uint16_t)(p0 | (p1 << 8));
-            }
-            if (__any_sync(0xffffffffu, tie_any != 0u)) {
-                __syncwarp();
-                unsigned tl = __ballot_sync(0xffffffffu, tie_any != 0u);
-                while (tl) {
-                    const int src = __ffs(tl) - 1;
-                    tl &= tl - 1;
-                    uint32_t fm = 0u;
-#pragma unroll
-                    for (int e = 0; e < 32; e += 2) {
-                        const int s = e >> 2;
-                        const float sg = sgn[s & 3 & PM];
-                        const float kp = sg * cp_[s >> 1], km = sg * cm_[s >> 1];
-                        const uint32_t pp = cvt_e2m1x2(fmaf(v[s][e & 3], kp, 0.0f), fmaf(v[s][(e & 3) + 1], kp, 0.0f));
-                        const uint32_t mm = cvt_e2m1x2(fmaf(v[s][e & 3], km, 0.0f), fmaf(v[s][(e & 3) + 1], km, 0.0f));
-                        const uint32_t x = pp ^ mm;
-                        fm |= ((x & 0x0Fu) ? (1u << e) : 0u) | ((x & 0xF0u) ? (2u << e) : 0u);
-                    }
-                    fm = __shfl_sync(0xffffffffu, fm, src);
-                    const int Ep = __shfl_sync(0xffffffffu, E_pack, src);
-                    while (fm) {
-                        const int e = __ffs(fm) - 1;
-                        fm &= fm - 1;
-                        int blk_elem, i, elem;
-                        locate<LOG2B>(src >> 2, src & 3, e, blk_elem, i, elem);
-                        const double ue = exact_coord_warp(seg, blk_elem, B, i, lane);
-                        if (lane == 0) {
-                            const int E = ((Ep >> (8 * (e >> 3))) & 0xFF) - 127;
-                            const double y = ue / p.sqrt_b;
-                            const uint32_t code = e2m1_code_exact(scalbn(y, -E), signbit(y));
-                            uint8_t *bp = code_buf + (elem >> 1);
-                            *bp = (elem & 1) ? (uint8_t)((*bp & 0x0F) | (code << 4)) : (uint8_t)((*bp & 0xF0) | code);
-                        }
-                        __syncwarp();
-                    }
-                }
-            }
+        for (int s = 0; s < 8; ++s) {
+            float a, b, c, d;
+            unpack2(v[s][0], a, b);
+            unpack2(v[s][1], c, d);
+            ms[s] = fmaxf(max3abs(fabsf(a), b, c), fabsf(d));
         }
 
-        // ---- packed codes: shared staging -> global
-        fence_async_smem();
+        uint8_t *code_buf = code_base + (size_t)par2 * SEG_CODE_BYTES;
+        bulk_store_wait_read<1>();           // the store that last read this staging buffer has drained
         __syncwarp();
-        if (lane == 0) bulk_store(p.out_codes + (size_t)seg_index * SEG_CODE_BYTES, smem_u32(code_buf), SEG_CODE_BYTES);
-    }
-    bulk_store_wait_read<0>();
-}
-
-}  // namespace perq
