@@ -143,6 +143,7 @@ int try_launch_fast(const void *x, const int32_t *perm, int64_t T, int32_t d, in
     p.G = G;
     p.units_total = (long long)T * (d / perq::SEG_ELEMS) / G;
     p.sqrt_b = std::sqrt((double)b);
+    p.inv_7_sqrt_b = 1.0 / (7.0 * p.sqrt_b);
     const int sms = sm_count();
     if (sms <= 0) return PERQ_ERR_CUDA;
     const int groups_per_cta = perq::FAST_WARPS / G;
