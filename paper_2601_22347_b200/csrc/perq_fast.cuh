@@ -119,46 +119,13 @@ __device__ __forceinline__ void mma_bf16(float (&c)[4], const uint32_t (&a)[4], 
                  : "r"(a[0]), "r"(a[1]), "r"(a[2]), "r"(a[3]), "r"(b0), "r"(b1), "f"(0.0f));
 }
 
-// Two fp32 values in one 64-bit register pair, for the packed add/sub/mul/fma of sm_100.
-typedef unsigned long long f32x2;
-__device__ __forceinline__ f32x2 pack2(float lo, float hi)
-{
-    f32x2 r;
-    asm("mov.b64 %0, {%1, %2};" : "=l"(r) : "f"(lo), "f"(hi));
-    return r;
-}
-__device__ __forceinline__ void unpack2(f32x2 v, float &lo, float &hi)
-{
-    asm("mov.b64 {%0, %1}, %2;" : "=f"(lo), "=f"(hi) : "l"(v));
-}
-__device__ __forceinline__ void unpack2u(f32x2 v, uint32_t &lo, uint32_t &hi)
-{
-    asm("mov.b64 {%0, %1}, %2;" : "=r"(lo), "=r"(hi) : "l"(v));
-}
-__device__ __forceinline__ f32x2 add2(f32x2 a, f32x2 b)
-{
-    f32x2 r;
-    asm("add.rn.f32x2 %0, %1, %2;" : "=l"(r) : "l"(a), "l"(b));
-    return r;
-}
-__device__ __forceinline__ f32x2 sub2(f32x2 a, f32x2 b)
-{
-    f32x2 r;
-    asm("sub.rn.f32x2 %0, %1, %2;" : "=l"(r) : "l"(a), "l"(b));
-    return r;
-}
-__device__ __forceinline__ f32x2 fma2(f32x2 a, f32x2 b, f32x2 c)
-{
-    f32x2 r;
-    asm("fma.rn.f32x2 %0, %1, %2, %3;" : "=l"(r) : "l"(a), "l"(b), "l"(c));
-    return r;
-}
-__device__ __forceinline__ f32x2 mul2(f32x2 a, f32x2 b)
-{
-    f32x2 r;
-    asm("mul.rn.f32x2 %0, %1, %2;" : "=l"(r) : "l"(a), "l"(b));
-    return r;
-}
+// Two fp32 values per operand: the packed add / fma of sm_100 (half the issue slots of scalar code).
+typedef float2 f32x2;
+__device__ __forceinline__ f32x2 pack2(float lo, float hi) { return make_float2(lo, hi); }
+__device__ __forceinline__ f32x2 add2(f32x2 a, f32x2 b) { return __fadd2_rn(a, b); }
+__device__ __forceinline__ f32x2 sub2(f32x2 a, f32x2 b) { return __ffma2_rn(b, make_float2(-1.0f, -1.0f), a); }
+__device__ __forceinline__ f32x2 fma2(f32x2 a, f32x2 b, f32x2 c) { return __ffma2_rn(a, b, c); }
+__device__ __forceinline__ f32x2 mul2(f32x2 a, f32x2 b) { return __fmul2_rn(a, b); }
 // max over the warp of a non-negative fp32 value (one instruction on sm_100a)
 __device__ __forceinline__ float warp_max_f32(float v)
 {
@@ -244,6 +211,33 @@ __device__ __forceinline__ double exact_coord_fast(const uint16_t *blk, int i, i
     return acc;
 }
 
+// Exact unnormalised outputs i0 .. i0+3 (i0 a multiple of 4) of the B-element block at blk, by a
+// whole warp: lane l returns output i0 + (l & 3).  Every lane adds its terms signed by the high
+// bits of the output index; lanes with equal l & 3 are summed, then a 4-point butterfly over
+// l & 3 applies the low two index bits.
+template <int B>
+__device__ __forceinline__ double exact_coord4(const uint16_t *blk, int i0, int lane)
+{
+    double acc = 0.0;
+#pragma unroll
+    for (int k0 = 0; k0 < B; k0 += 32) {
+        const int k = k0 + lane;
+        if (B >= 32 || k < B) {
+            const double v = bf16_bits_to_f64(blk[k]);
+            acc += (__popc(i0 & k) & 1) ? -v : v;
+        }
+    }
+    acc += __shfl_xor_sync(0xffffffffu, acc, 4);
+    acc += __shfl_xor_sync(0xffffffffu, acc, 8);
+    acc += __shfl_xor_sync(0xffffffffu, acc, 16);
+#pragma unroll
+    for (int bit = 1; bit <= 2; bit <<= 1) {
+        const double other = __shfl_xor_sync(0xffffffffu, acc, bit);
+        acc = (lane & bit) ? other - acc : acc + other;
+    }
+    return acc;
+}
+
 // Bit mask of the lane's 32 held values (bit s*4+j) whose magnitude reaches thr; ms[s] is the
 // magnitude maximum of slot s, used to skip slots.
 __device__ __forceinline__ uint32_t candidate_mask(const f32x2 (&v)[8][2], const float (&ms)[8], float thr)
@@ -252,9 +246,7 @@ __device__ __forceinline__ uint32_t candidate_mask(const f32x2 (&v)[8][2], const
 #pragma unroll
     for (int s = 0; s < 8; ++s) {
         if (ms[s] >= thr) {
-            float a, b, c, d;
-            unpack2(v[s][0], a, b);
-            unpack2(v[s][1], c, d);
+            const float a = v[s][0].x, b = v[s][0].y, c = v[s][1].x, d = v[s][1].y;
             cm |= (fabsf(a) >= thr ? 1u : 0u) << (4 * s);
             cm |= (fabsf(b) >= thr ? 2u : 0u) << (4 * s);
             cm |= (fabsf(c) >= thr ? 4u : 0u) << (4 * s);
@@ -409,10 +401,7 @@ __global__ void __launch_bounds__(FAST_THREADS, 1) perq_fast_kernel(FastParams p
         float ms[8];
 #pragma unroll
         for (int s = 0; s < 8; ++s) {
-            float a, b, c, d;
-            unpack2(v[s][0], a, b);
-            unpack2(v[s][1], c, d);
-            ms[s] = fmaxf(max3abs(fabsf(a), b, c), fabsf(d));
+            ms[s] = fmaxf(max3abs(fabsf(v[s][0].x), v[s][0].y, v[s][1].x), fabsf(v[s][1].y));
         }
 
         uint8_t *code_buf = code_base + (size_t)par2 * SEG_CODE_BYTES;
@@ -453,21 +442,33 @@ __global__ void __launch_bounds__(FAST_THREADS, 1) perq_fast_kernel(FastParams p
                 // candidates near its own fp32 maximum; the row's values are the maxima of both
                 const float aw = warp_max_f32(lane_max);
                 const float thr = aw * (1.0f - 2.0f * err_rel - 2.4e-7f);
+                // candidates: slots (four adjacent outputs of one chunk) whose maximum reaches thr;
+                // each costs one cooperative exact evaluation of its four outputs
+                uint32_t slot_mask = 0u;
+#pragma unroll
+                for (int s = 0; s < 8; ++s) slot_mask |= (ms[s] >= thr) ? (1u << s) : 0u;
                 double wbest = 0.0;
-                unsigned cw = __ballot_sync(0xffffffffu, (aw > 0.0f) && (lane_max >= thr));
+                unsigned cw = __ballot_sync(0xffffffffu, (aw > 0.0f) && (slot_mask != 0u));
                 while (cw) {
                     const int src = __ffs(cw) - 1;
                     cw &= cw - 1;
-                    uint32_t cm = 0u;
-                    if (lane == src) cm = candidate_mask(v, ms, thr);
-                    cm = __shfl_sync(0xffffffffu, cm, src);
-                    while (cm) {
-                        const int e = __ffs(cm) - 1;
-                        cm &= cm - 1;
-                        int blk_elem, i, elem;
-                        locate<LOG2B>(src >> 2, src & 3, e, blk_elem, i, elem);
-                        wbest = fmax(wbest, fabs(exact_coord_fast<B>(seg + blk_elem, i, lane)));
+                    uint32_t sm = __shfl_sync(0xffffffffu, slot_mask, src);
+                    const int sg_ = src >> 2;
+                    while (sm) {
+                        const int sl = __ffs(sm) - 1;
+                        sm &= sm - 1;
+                        const int pch = sg_ * 8 + (sl ^ ((sg_ & 3) & ~PM));      // chunk position in the segment
+                        const int blk_elem = (pch >> CB) << LOG2B;
+                        const int i0 = pch * 16 - blk_elem + 4 * (src & 3);
+                        wbest = fmax(wbest, fabs(exact_coord4<B>(seg + blk_elem, i0, lane)));
                     }
+                }
+                // the four lane classes hold different outputs: maximum over the warp, on the bit pattern
+                {
+                    const unsigned long long wb = (unsigned long long)__double_as_longlong(wbest);
+                    const uint32_t hi = __reduce_max_sync(0xffffffffu, (uint32_t)(wb >> 32));
+                    const uint32_t lo = __reduce_max_sync(0xffffffffu, ((uint32_t)(wb >> 32) == hi) ? (uint32_t)wb : 0u);
+                    wbest = __hiloint2double((int)hi, (int)lo);
                 }
                 if (G > 1) {
                     if (lane == 0) {
@@ -508,16 +509,16 @@ __global__ void __launch_bounds__(FAST_THREADS, 1) perq_fast_kernel(FastParams p
 #pragma unroll
             for (int s = 0; s < 8; ++s) {
                 const int k = s & 3 & PM;
-                uint32_t t[4], u[4];
-                unpack2u(fma2(v[s][0], mul_p[k], magic2), t[0], t[1]);
-                unpack2u(fma2(v[s][1], mul_p[k], magic2), t[2], t[3]);
-                unpack2u(fma2(v[s][0], mul_m[k], magic2), u[0], u[1]);
-                unpack2u(fma2(v[s][1], mul_m[k], magic2), u[2], u[3]);
-                tie_any |= (t[0] ^ u[0]) | (t[1] ^ u[1]);
-                tie_any |= (t[2] ^ u[2]) | (t[3] ^ u[3]);
-                const uint32_t packed = (((t[3] * 16u + t[2]) * 16u + t[1]) * 16u + t[0]) ^ 0x8888u;
-                *reinterpret_cast<uint16_t *>(code_buf + code_off[s]) = (uint16_t)packed;
+                const f32x2 tp0 = fma2(v[s][0], mul_p[k], magic2), tp1 = fma2(v[s][1], mul_p[k], magic2);
+                const f32x2 tm0 = fma2(v[s][0], mul_m[k], magic2), tm1 = fma2(v[s][1], mul_m[k], magic2);
+                const uint32_t pp = ((__float_as_uint(tp1.y) * 16u + __float_as_uint(tp1.x)) * 16u + __float_as_uint(tp0.y)) * 16u
+                                    + __float_as_uint(tp0.x);
+                const uint32_t pm = ((__float_as_uint(tm1.y) * 16u + __float_as_uint(tm1.x)) * 16u + __float_as_uint(tm0.y)) * 16u
+                                    + __float_as_uint(tm0.x);
+                tie_any |= pp ^ pm;          // low 16 bits: the four codes (offset by 8) under either multiplier
+                *reinterpret_cast<uint16_t *>(code_buf + code_off[s]) = (uint16_t)(pp ^ 0x8888u);
             }
+            tie_any &= 0xffffu;
             // ---- exact resolution of near ties (rare)
             if (__any_sync(0xffffffffu, tie_any != 0u)) {
                 uint32_t fm = 0u;
@@ -525,11 +526,9 @@ __global__ void __launch_bounds__(FAST_THREADS, 1) perq_fast_kernel(FastParams p
 #pragma unroll
                     for (int s = 0; s < 8; ++s) {
                         const int k = s & 3 & PM;
-                        uint32_t t[4], u[4];
-                        unpack2u(fma2(v[s][0], mul_p[k], magic2), t[0], t[1]);
-                        unpack2u(fma2(v[s][1], mul_p[k], magic2), t[2], t[3]);
-                        unpack2u(fma2(v[s][0], mul_m[k], magic2), u[0], u[1]);
-                        unpack2u(fma2(v[s][1], mul_m[k], magic2), u[2], u[3]);
+                        const f32x2 tp0 = fma2(v[s][0], mul_p[k], magic2), tp1 = fma2(v[s][1], mul_p[k], magic2);
+                        const f32x2 tm0 = fma2(v[s][0], mul_m[k], magic2), tm1 = fma2(v[s][1], mul_m[k], magic2);
+                        const float t[4] = {tp0.x, tp0.y, tp1.x, tp1.y}, u[4] = {tm0.x, tm0.y, tm1.x, tm1.y};
 #pragma unroll
                         for (int j = 0; j < 4; ++j) fm |= (t[j] != u[j]) ? (1u << (4 * s + j)) : 0u;
                     }
@@ -567,8 +566,8 @@ __global__ void __launch_bounds__(FAST_THREADS, 1) perq_fast_kernel(FastParams p
             float vf[8][4];
 #pragma unroll
             for (int s = 0; s < 8; ++s) {
-                unpack2(v[s][0], vf[s][0], vf[s][1]);
-                unpack2(v[s][1], vf[s][2], vf[s][3]);
+                vf[s][0] = v[s][0].x; vf[s][1] = v[s][0].y;
+                vf[s][2] = v[s][1].x; vf[s][3] = v[s][1].y;
             }
             uint32_t tie_any = 0u;
             int E_pack = 0;                      // E + 127 of the lane's four groups, one per byte
