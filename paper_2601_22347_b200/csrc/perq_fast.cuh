@@ -1,10 +1,10 @@
 // Fast rotate+quantize kernel for the common cases: no permutation, b in {16,32,64,128},
-// d a multiple of 1024, scales per token (d <= 8192), per 128 (INT4) or per 32 (MXFP4).
+// d a multiple of 1024, scales per token (d/1024 in {1,2,4,8}), per 128 (INT4) or per 32 (MXFP4).
 //
 // Data path (HBM-bound, one pass):
 //   global --cp.async.bulk + mbarrier--> shared memory ring (bf16 rows, as stored)
 //   --ldmatrix--> tensor-core H_16 (mma.sync bf16 x (+-1) -> fp32; products are exact)
-//   --fp32 add/sub on registers--> remaining log2(b)-4 butterfly stages
+//   --packed fp32 add/sub on registers--> remaining log2(b)-4 butterfly stages
 //   --absmax / scale / round / pack in registers--> shared staging --cp.async.bulk--> global
 //
 // Work is split into segments of 1024 consecutive elements, one warp each.  Within a warp,
@@ -25,6 +25,12 @@
 // are re-derived exactly in fp64 from the bf16 inputs in shared memory, MX exponents when
 // the fp32 maximum is close to a power-of-two boundary, and single elements when their
 // scaled value is close to a rounding tie.
+//
+// Per-token scales: the G = d/1024 warps of a row exchange their fp32 maxima through one
+// named barrier.  Only the warps whose maximum is within the error bound of the row's
+// (normally one) derive exact values; with one such warp it stores the scale itself, with
+// several the last one to add its value to a shared accumulator does.  Warps that need the
+// exact maximum for a tie fix-up (rare) wait for it on a flag, with a bounded spin.
 #pragma once
 #include <cuda_runtime.h>
 #include <stdint.h>
@@ -48,8 +54,7 @@ struct FastParams {
     const uint16_t *x;
     uint8_t *out_codes;
     void *out_scales;
-    long long units_total;   // units of G segments
-    int G;                   // warps (segments) per unit: 1 unless per-token scales
+    uint32_t units_total;    // units of G = 2^LOG2G segments (fewer than 2^31)
     double sqrt_b;
     double inv_7_sqrt_b;     // 1 / (7 sqrt(b)): INT4 scale = exact |u|max times this
 };
@@ -57,13 +62,18 @@ struct FastParams {
 // Set (never cleared by kernels) when a bounded wait inside a kernel ran out.
 __device__ unsigned int g_perq_device_error = 0u;
 
+// Shared-memory carve-up, relative to a 1024-byte aligned base.
 struct FastSmem {
     static constexpr size_t stages = 0;
     static constexpr size_t codes = stages + (size_t)FAST_WARPS * FAST_NSTAGE * SEG_BYTES;
     static constexpr size_t full = codes + (size_t)FAST_WARPS * 2 * SEG_CODE_BYTES;
-    static constexpr size_t wexact = full + (size_t)FAST_WARPS * FAST_NSTAGE * 8;   // [2][FAST_WARPS] u64
-    static constexpr size_t wmax = wexact + (size_t)FAST_WARPS * 2 * 8;             // [2][FAST_WARPS] f32
-    static constexpr size_t total = wmax + (size_t)FAST_WARPS * 2 * 4;
+    static constexpr size_t wacc = full + (size_t)FAST_WARPS * FAST_NSTAGE * 8;     // [2][FAST_WARPS] u64 accumulators
+    static constexpr size_t wpub = wacc + (size_t)FAST_WARPS * 2 * 8;               // [2][FAST_WARPS] u64 published row maxima
+    static constexpr size_t wmax = wpub + (size_t)FAST_WARPS * 2 * 8;               // [2][FAST_WARPS] f32 warp maxima
+    static constexpr size_t wcnt = wmax + (size_t)FAST_WARPS * 2 * 4;               // [2][FAST_WARPS] u32 arrival counts
+    static constexpr size_t wflag = wcnt + (size_t)FAST_WARPS * 2 * 4;              // [2][FAST_WARPS] u32 publication flags
+    static constexpr size_t used = wflag + (size_t)FAST_WARPS * 2 * 4;
+    static constexpr size_t total = used + 1024;                                    // room to align the base
 };
 
 // ---------------------------------------------------------------- PTX wrappers
@@ -114,9 +124,23 @@ __device__ __forceinline__ void ldmatrix_x4(uint32_t (&r)[4], uint32_t addr)
 // c = a * b with a zero accumulator input (no registers are cleared for it)
 __device__ __forceinline__ void mma_bf16(float (&c)[4], const uint32_t (&a)[4], uint32_t b0, uint32_t b1)
 {
-    asm volatile("mma.sync.aligned.m16n8k16.row.col.f32.bf16.bf16.f32 {%0,%1,%2,%3}, {%4,%5,%6,%7}, {%8,%9}, {%10,%10,%10,%10};"
-                 : "=f"(c[0]), "=f"(c[1]), "=f"(c[2]), "=f"(c[3])
-                 : "r"(a[0]), "r"(a[1]), "r"(a[2]), "r"(a[3]), "r"(b0), "r"(b1), "f"(0.0f));
+    asm("mma.sync.aligned.m16n8k16.row.col.f32.bf16.bf16.f32 {%0,%1,%2,%3}, {%4,%5,%6,%7}, {%8,%9}, {%10,%10,%10,%10};"
+        : "=f"(c[0]), "=f"(c[1]), "=f"(c[2]), "=f"(c[3])
+        : "r"(a[0]), "r"(a[1]), "r"(a[2]), "r"(a[3]), "r"(b0), "r"(b1), "f"(0.0f));
+}
+__device__ __forceinline__ void named_barrier(int id, int threads)
+{
+    asm volatile("bar.sync %0, %1;" ::"r"(id), "r"(threads) : "memory");
+}
+__device__ __forceinline__ void sts_u16(uint32_t addr, uint32_t v)
+{
+    asm volatile("st.shared.u16 [%0], %1;" ::"r"(addr), "h"((uint16_t)v) : "memory");
+}
+__device__ __forceinline__ uint32_t ld_volatile_shared_u32(const uint32_t *p)
+{
+    uint32_t v;
+    asm volatile("ld.volatile.shared.u32 %0, [%1];" : "=r"(v) : "r"(smem_u32(p)) : "memory");
+    return v;
 }
 
 // Two fp32 values per operand: the packed add / fma of sm_100 (half the issue slots of scalar code).
@@ -133,574 +157,13 @@ __device__ __forceinline__ float warp_max_f32(float v)
     asm volatile("redux.sync.max.f32 %0, %1, 0xffffffff;" : "=f"(r) : "f"(v));
     return r;
 }
-__device__ __forceinline__ float max3abs(float acc, float a, float b) { return fmaxf(fmaxf(acc, fabsf(a)), fabsf(b)); }
-__device__ __forceinline__ void named_barrier(int id, int threads)
+// max over the warp of a non-negative double, on its bit pattern
+__device__ __forceinline__ unsigned long long warp_max_u64(unsigned long long v)
 {
-    asm volatile("bar.sync %0, %1;" ::"r"(id), "r"(threads) : "memory");
+    const uint32_t hi = __reduce_max_sync(0xffffffffu, (uint32_t)(v >> 32));
+    const uint32_t lo = __reduce_max_sync(0xffffffffu, ((uint32_t)(v >> 32) == hi) ? (uint32_t)v : 0u);
+    return ((unsigned long long)hi << 32) | lo;
 }
+__device__ __forceinline__ float max3abs(float acc, float a, float b) { return fmaxf(fmaxf(acc, fabsf(a)), fabsf(b)); }
 
 __device__ __forceinline__ uint32_t hadamard_bf16(int k, int n) { return (__popc(k & n) & 1) ? 0xBF80u : 0x3F80u; }
-
-// ---------------------------------------------------------------- exact re-evaluation
-
-// bf16 bit pattern (low 16 bits of h) -> double, exactly, with integer operations (the
-// fp32->fp64 conversion instruction is slow); zero and subnormals take the conversion.
-__device__ __forceinline__ double bf16_bits_to_f64(uint32_t h)
-{
-    const uint32_t mag = h & 0x7fffu;
-    if (mag < 0x80u) return (double)__uint_as_float(h << 16);
-    return __hiloint2double((int)(((mag << 13) + 0x38000000u) | ((h & 0x8000u) << 16)), 0);
-}
-
-// Exact unnormalised output i of the block starting at `blk` (bf16 in shared memory), evaluated
-// by the 4 lanes of a quad: each lane reduces a quarter of the block with a signed pairwise
-// tree in fp64, then the quarters are combined.  q = lane % 4, qmask = the quad's lanes.
-template <int LOG2B>
-__device__ __forceinline__ double exact_coord_quad(const uint16_t *blk, int i, int q, unsigned qmask)
-{
-    constexpr int PER = (1 << LOG2B) / 4;
-    double v[PER];
-    const uint32_t *src = reinterpret_cast<const uint32_t *>(blk + q * PER);
-#pragma unroll
-    for (int r = 0; r < PER / 2; ++r) {
-        const uint32_t w = src[r];
-        v[2 * r] = bf16_bits_to_f64(w);
-        v[2 * r + 1] = bf16_bits_to_f64(w >> 16);
-    }
-#pragma unroll
-    for (int t = 0; (1 << t) < PER; ++t) {
-        const double sg = ((i >> t) & 1) ? -1.0 : 1.0;
-#pragma unroll
-        for (int m = 0; m < (PER >> (t + 1)); ++m) v[m] = fma(sg, v[2 * m + 1], v[2 * m]);
-    }
-    double part = (__popc(i & (q << (LOG2B - 2))) & 1) ? -v[0] : v[0];
-    part += __shfl_xor_sync(qmask, part, 1);
-    part += __shfl_xor_sync(qmask, part, 2);
-    return part;
-}
-
-// Element e = s*4 + j of lane (g, q): block start (in elements, segment relative) and index inside the block.
-template <int LOG2B>
-__device__ __forceinline__ void locate(int g, int q, int e, int &blk_elem, int &i, int &elem)
-{
-    constexpr int CB = LOG2B - 4;                 // chunk bits inside a block
-    constexpr int PM = (1 << CB) - 1;
-    const int s = e >> 2, j = e & 3;
-    const int p = g * 8 + (s ^ ((g & 3) & ~PM));  // chunk position inside the segment
-    elem = p * 16 + 4 * q + j;
-    blk_elem = (p >> CB) << LOG2B;
-    i = elem - blk_elem;
-}
-
-
-// Exact unnormalised output i of the B-element block at blk (bf16 in shared memory), by a whole warp.
-template <int B>
-__device__ __forceinline__ double exact_coord_fast(const uint16_t *blk, int i, int lane)
-{
-    double acc = 0.0;
-#pragma unroll
-    for (int k0 = 0; k0 < B; k0 += 32) {
-        const int k = k0 + lane;
-        if (B >= 32 || k < B) {
-            const double v = bf16_bits_to_f64(blk[k]);
-            acc += (__popc(i & k) & 1) ? -v : v;
-        }
-    }
-#pragma unroll
-    for (int o = 16; o > 0; o >>= 1) acc += __shfl_xor_sync(0xffffffffu, acc, o);
-    return acc;
-}
-
-// Exact unnormalised outputs i0 .. i0+3 (i0 a multiple of 4) of the B-element block at blk, by a
-// whole warp: lane l returns output i0 + (l & 3).  Every lane adds its terms signed by the high
-// bits of the output index; lanes with equal l & 3 are summed, then a 4-point butterfly over
-// l & 3 applies the low two index bits.
-template <int B>
-__device__ __forceinline__ double exact_coord4(const uint16_t *blk, int i0, int lane)
-{
-    double acc = 0.0;
-#pragma unroll
-    for (int k0 = 0; k0 < B; k0 += 32) {
-        const int k = k0 + lane;
-        if (B >= 32 || k < B) {
-            const double v = bf16_bits_to_f64(blk[k]);
-            acc += (__popc(i0 & k) & 1) ? -v : v;
-        }
-    }
-    acc += __shfl_xor_sync(0xffffffffu, acc, 4);
-    acc += __shfl_xor_sync(0xffffffffu, acc, 8);
-    acc += __shfl_xor_sync(0xffffffffu, acc, 16);
-#pragma unroll
-    for (int bit = 1; bit <= 2; bit <<= 1) {
-        const double other = __shfl_xor_sync(0xffffffffu, acc, bit);
-        acc = (lane & bit) ? other - acc : acc + other;
-    }
-    return acc;
-}
-
-// Bit mask of the lane's 32 held values (bit s*4+j) whose magnitude reaches thr; ms[s] is the
-// magnitude maximum of slot s, used to skip slots.
-__device__ __forceinline__ uint32_t candidate_mask(const f32x2 (&v)[8][2], const float (&ms)[8], float thr)
-{
-    uint32_t cm = 0u;
-#pragma unroll
-    for (int s = 0; s < 8; ++s) {
-        if (ms[s] >= thr) {
-            const float a = v[s][0].x, b = v[s][0].y, c = v[s][1].x, d = v[s][1].y;
-            cm |= (fabsf(a) >= thr ? 1u : 0u) << (4 * s);
-            cm |= (fabsf(b) >= thr ? 2u : 0u) << (4 * s);
-            cm |= (fabsf(c) >= thr ? 4u : 0u) << (4 * s);
-            cm |= (fabsf(d) >= thr ? 8u : 0u) << (4 * s);
-        }
-    }
-    return cm;
-}
-
-// ---------------------------------------------------------------- the kernel
-
-template <int LOG2B, int MODE>
-__global__ void __launch_bounds__(FAST_THREADS, 1) perq_fast_kernel(FastParams p)
-{
-    constexpr int B = 1 << LOG2B;
-    constexpr int CB = LOG2B - 4;                 // butterfly stages left after the tensor-core H_16
-    constexpr int PM = (1 << CB) - 1;             // slot bits inside a Hadamard block
-    constexpr int NCLS = (PM & 3) + 1;            // sign classes of the slot relabelling
-    constexpr float MAGIC = 12582920.0f;          // 1.5 * 2^23 + 8: low nibble of the sum = code + 8
-    extern __shared__ __align__(128) unsigned char fsmem[];
-
-    const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
-    const int g = lane >> 2, q = lane & 3;
-    const int G = p.G;
-    const int group = warp / G, w_in_g = warp - group * G;
-    const int groups_per_cta = FAST_WARPS / G;
-    const unsigned qmask = 0xFu << (lane & 28);
-    const float err_rel = FAST_ERR_K * (float)LOG2B * TWO_M24;
-
-    unsigned char *stage_base = fsmem + FastSmem::stages + (size_t)group * G * FAST_NSTAGE * SEG_BYTES;
-    unsigned char *code_base = fsmem + FastSmem::codes + (size_t)warp * 2 * SEG_CODE_BYTES;
-    uint64_t *full = reinterpret_cast<uint64_t *>(fsmem + FastSmem::full) + group * FAST_NSTAGE;
-    unsigned long long *wexact = reinterpret_cast<unsigned long long *>(fsmem + FastSmem::wexact);   // [2][FAST_WARPS]
-    float *wmax = reinterpret_cast<float *>(fsmem + FastSmem::wmax);                                 // [2][FAST_WARPS]
-    const bool leader = (w_in_g == 0) && (lane == 0);
-    const uint32_t unit_bytes = (uint32_t)G * SEG_BYTES;
-
-    if (tid == 0) {
-        for (int i = 0; i < FAST_WARPS * FAST_NSTAGE; ++i)
-            mbar_init(smem_u32(reinterpret_cast<uint64_t *>(fsmem + FastSmem::full) + i), 1);
-        asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
-    }
-    __syncthreads();
-
-    const long long first = (long long)blockIdx.x * groups_per_cta + group;
-    const long long stride = (long long)gridDim.x * groups_per_cta;
-    if (group >= groups_per_cta || first >= p.units_total) return;   // whole groups leave together
-
-    // Hadamard operand of the tensor-core stage: column n of MMA m is output 4*(n/2) + (n%2) + 2m.
-    uint32_t hb[2][2];
-#pragma unroll
-    for (int m = 0; m < 2; ++m) {
-        const int col = 4 * (g >> 1) + (g & 1) + 2 * m;
-        hb[m][0] = hadamard_bf16(2 * q, col) | (hadamard_bf16(2 * q + 1, col) << 16);
-        hb[m][1] = hadamard_bf16(2 * q + 8, col) | (hadamard_bf16(2 * q + 9, col) << 16);
-    }
-    // ldmatrix source offsets: lane l feeds row (l & 7) of matrix (l >> 3) of every tile.
-    uint32_t lm_off[4];
-    {
-        const int r8 = lane & 7, mi = lane >> 3;
-        const int f = r8 & 3, fh = (r8 >> 2) & 1;
-#pragma unroll
-        for (int t = 0; t < 4; ++t) {
-            const int s = 2 * t + (mi & 1);
-            lm_off[t] = (uint32_t)((r8 * 8 + (s ^ f)) * 32 + (((mi >> 1) ^ fh) * 16));
-        }
-    }
-    const int f_g = g & 3;
-    // byte offset of this lane's 16-bit code piece of slot s inside the segment's 512 code bytes
-    uint32_t code_off[8];
-#pragma unroll
-    for (int s = 0; s < 8; ++s) code_off[s] = (uint32_t)((g * 8 + (s ^ (f_g & ~PM))) * 8 + 2 * q);
-    // sign of the held value relative to the true output, per (s & 3 & PM): folded into multipliers
-    const float half_sign = ((g & 4) && q >= 2) ? -1.0f : 1.0f;
-    float sgn[4];
-#pragma unroll
-    for (int k = 0; k < 4; ++k) sgn[k] = (__popc(k & f_g & PM) & 1) ? -half_sign : half_sign;
-
-    // prologue: fill the ring
-    if (leader) {
-#pragma unroll
-        for (int s = 0; s < FAST_NSTAGE; ++s) {
-            const long long u = first + (long long)s * stride;
-            if (u < p.units_total) {
-                mbar_expect_tx(smem_u32(&full[s]), unit_bytes);
-                bulk_load(smem_u32(stage_base + (size_t)s * unit_bytes), p.x + (size_t)u * G * SEG_ELEMS, unit_bytes,
-                          smem_u32(&full[s]));
-            }
-        }
-    }
-
-    uint32_t it = 0;
-    for (long long unit = first; unit < p.units_total; unit += stride, ++it) {
-        const uint32_t stage = it % FAST_NSTAGE;
-        const uint32_t parity = (it / FAST_NSTAGE) & 1u;
-        const uint32_t par2 = it & 1u;
-        if (!mbar_wait(smem_u32(&full[stage]), parity)) {
-            if (lane == 0) atomicOr(&g_perq_device_error, 1u);
-            return;
-        }
-        const unsigned char *unit_smem = stage_base + (size_t)stage * unit_bytes;
-        const uint16_t *seg = reinterpret_cast<const uint16_t *>(unit_smem + (size_t)w_in_g * SEG_BYTES);
-        const uint32_t seg_addr = smem_u32(seg);
-        const long long seg_index = unit * G + w_in_g;
-
-        // ---- H_16 on the tensor cores; v[s][h] = outputs (2h, 2h+1) of this lane's four of slot s
-        f32x2 v[8][2];
-#pragma unroll
-        for (int t = 0; t < 4; ++t) {
-            uint32_t a[4];
-            ldmatrix_x4(a, seg_addr + lm_off[t]);
-            float c0[4], c1[4];
-            mma_bf16(c0, a, hb[0][0], hb[0][1]);
-            mma_bf16(c1, a, hb[1][0], hb[1][1]);
-            v[2 * t][0] = pack2(c0[0], c0[1]);
-            v[2 * t][1] = pack2(c1[0], c1[1]);
-            v[2 * t + 1][0] = pack2(c0[2], c0[3]);
-            v[2 * t + 1][1] = pack2(c1[2], c1[3]);
-        }
-        // refill the stage the previous iteration used (every warp of the group is past it now:
-        // for G == 1 because this warp is, for G > 1 after the named barrier below)
-        auto refill = [&]() {
-            if (leader && it > 0) {
-                const long long u = unit + (long long)(FAST_NSTAGE - 1) * stride;
-                if (u < p.units_total) {
-                    const uint32_t ps = (it - 1) % FAST_NSTAGE;
-                    mbar_expect_tx(smem_u32(&full[ps]), unit_bytes);
-                    bulk_load(smem_u32(stage_base + (size_t)ps * unit_bytes), p.x + (size_t)u * G * SEG_ELEMS,
-                              unit_bytes, smem_u32(&full[ps]));
-                }
-            }
-        };
-        if (MODE != MODE_TOKEN) refill();
-
-        // ---- remaining butterfly stages over the slot bits inside a block (packed add/sub)
-#pragma unroll
-        for (int t = 0; t < CB; ++t) {
-#pragma unroll
-            for (int s = 0; s < 8; ++s) {
-                if ((s & (1 << t)) == 0) {
-#pragma unroll
-                    for (int h = 0; h < 2; ++h) {
-                        const f32x2 a = v[s][h], c = v[s | (1 << t)][h];
-                        v[s][h] = add2(a, c);
-                        v[s | (1 << t)][h] = sub2(a, c);
-                    }
-                }
-            }
-        }
-
-        // ---- fp32 maxima per slot
-        float ms[8];
-#pragma unroll
-        for (int s = 0; s < 8; ++s) {
-            ms[s] = fmaxf(max3abs(fabsf(v[s][0].x), v[s][0].y, v[s][1].x), fabsf(v[s][1].y));
-        }
-
-        uint8_t *code_buf = code_base + (size_t)par2 * SEG_CODE_BYTES;
-        bulk_store_wait_read<1>();           // the store that last read this staging buffer has drained
-        __syncwarp();
-
-        if (MODE == MODE_TOKEN || MODE == MODE_G128) {
-            // lane maximum, then the maximum of the scale range in fp32 (a32) and exactly (a_exact)
-            const float lane_max = fmaxf(fmaxf(fmaxf(ms[0], ms[1]), fmaxf(ms[2], ms[3])),
-                                         fmaxf(fmaxf(ms[4], ms[5]), fmaxf(ms[6], ms[7])));
-            float a32;
-            double a_exact = 0.0;
-            if (MODE == MODE_G128) {
-                a32 = fmaxf(lane_max, __shfl_xor_sync(0xffffffffu, lane_max, 1));
-                a32 = fmaxf(a32, __shfl_xor_sync(0xffffffffu, a32, 2));
-                const float thr = a32 * (1.0f - 2.0f * err_rel - 2.4e-7f);
-                const bool has_cand = (a32 > 0.0f) && (lane_max >= thr);
-                unsigned cq = __ballot_sync(0xffffffffu, has_cand) & qmask;      // candidate lanes of my quad
-                while (cq) {
-                    const int src = __ffs(cq) - 1;
-                    cq &= cq - 1;
-                    uint32_t cm = 0u;
-                    if (lane == src) cm = candidate_mask(v, ms, thr);
-                    cm = __shfl_sync(qmask, cm, src);
-                    while (cm) {
-                        const int e = __ffs(cm) - 1;
-                        cm &= cm - 1;
-                        int blk_elem, i, elem;
-                        locate<LOG2B>(src >> 2, src & 3, e, blk_elem, i, elem);
-                        a_exact = fmax(a_exact, fabs(exact_coord_quad<LOG2B>(seg + blk_elem, i, q, qmask)));
-                    }
-                }
-                if (q == 0)
-                    reinterpret_cast<float *>(p.out_scales)[seg_index * 8 + g] =
-                        (a_exact == 0.0) ? 0.0f : (float)(a_exact * p.inv_7_sqrt_b);
-            } else {
-                // per token: every warp derives the exact maximum of its own segment from the
-                // candidates near its own fp32 maximum; the row's values are the maxima of both
-                const float aw = warp_max_f32(lane_max);
-                const float thr = aw * (1.0f - 2.0f * err_rel - 2.4e-7f);
-                // candidates: slots (four adjacent outputs of one chunk) whose maximum reaches thr;
-                // each costs one cooperative exact evaluation of its four outputs
-                uint32_t slot_mask = 0u;
-#pragma unroll
-                for (int s = 0; s < 8; ++s) slot_mask |= (ms[s] >= thr) ? (1u << s) : 0u;
-                double wbest = 0.0;
-                unsigned cw = __ballot_sync(0xffffffffu, (aw > 0.0f) && (slot_mask != 0u));
-                while (cw) {
-                    const int src = __ffs(cw) - 1;
-                    cw &= cw - 1;
-                    uint32_t sm = __shfl_sync(0xffffffffu, slot_mask, src);
-                    const int sg_ = src >> 2;
-                    while (sm) {
-                        const int sl = __ffs(sm) - 1;
-                        sm &= sm - 1;
-                        const int pch = sg_ * 8 + (sl ^ ((sg_ & 3) & ~PM));      // chunk position in the segment
-                        const int blk_elem = (pch >> CB) << LOG2B;
-                        const int i0 = pch * 16 - blk_elem + 4 * (src & 3);
-                        wbest = fmax(wbest, fabs(exact_coord4<B>(seg + blk_elem, i0, lane)));
-                    }
-                }
-                // the four lane classes hold different outputs: maximum over the warp, on the bit pattern
-                {
-                    const unsigned long long wb = (unsigned long long)__double_as_longlong(wbest);
-                    const uint32_t hi = __reduce_max_sync(0xffffffffu, (uint32_t)(wb >> 32));
-                    const uint32_t lo = __reduce_max_sync(0xffffffffu, ((uint32_t)(wb >> 32) == hi) ? (uint32_t)wb : 0u);
-                    wbest = __hiloint2double((int)hi, (int)lo);
-                }
-                if (G > 1) {
-                    if (lane == 0) {
-                        wmax[par2 * FAST_WARPS + warp] = aw;
-                        wexact[par2 * FAST_WARPS + warp] = (unsigned long long)__double_as_longlong(wbest);
-                    }
-                    named_barrier(1 + group, G * 32);
-                    const int src_w = group * G + lane;
-                    const float am = (lane < G) ? wmax[par2 * FAST_WARPS + src_w] : 0.0f;
-                    const unsigned long long ex = (lane < G) ? wexact[par2 * FAST_WARPS + src_w] : 0ull;
-                    a32 = warp_max_f32(am);
-                    const uint32_t hi = __reduce_max_sync(0xffffffffu, (uint32_t)(ex >> 32));
-                    const uint32_t lo = __reduce_max_sync(0xffffffffu, ((uint32_t)(ex >> 32) == hi) ? (uint32_t)ex : 0u);
-                    a_exact = __hiloint2double((int)hi, (int)lo);
-                } else {
-                    a32 = aw;
-                    a_exact = wbest;
-                }
-                refill();
-                if (leader)
-                    reinterpret_cast<float *>(p.out_scales)[unit] =
-                        (a_exact == 0.0) ? 0.0f : (float)(a_exact * p.inv_7_sqrt_b);
-            }
-
-            // ---- quantise: fp32 multiply-add against the magic constant, with the multiplier nudged
-            // up and down by the error bound; elements whose two codes differ are resolved exactly
-            const float inv = (a32 > 0.0f) ? fminf(__fdividef(7.0f, a32), 3.0e38f) : 0.0f;
-            const float delta = 16.0f * err_rel + 5.0e-7f;
-            f32x2 mul_p[NCLS], mul_m[NCLS];
-#pragma unroll
-            for (int k = 0; k < NCLS; ++k) {
-                const float mp = sgn[k] * inv * (1.0f + delta), mm = sgn[k] * inv * (1.0f - delta);
-                mul_p[k] = pack2(mp, mp);
-                mul_m[k] = pack2(mm, mm);
-            }
-            const f32x2 magic2 = pack2(MAGIC, MAGIC);
-            uint32_t tie_any = 0u;
-#pragma unroll
-            for (int s = 0; s < 8; ++s) {
-                const int k = s & 3 & PM;
-                const f32x2 tp0 = fma2(v[s][0], mul_p[k], magic2), tp1 = fma2(v[s][1], mul_p[k], magic2);
-                const f32x2 tm0 = fma2(v[s][0], mul_m[k], magic2), tm1 = fma2(v[s][1], mul_m[k], magic2);
-                const uint32_t pp = ((__float_as_uint(tp1.y) * 16u + __float_as_uint(tp1.x)) * 16u + __float_as_uint(tp0.y)) * 16u
-                                    + __float_as_uint(tp0.x);
-                const uint32_t pm = ((__float_as_uint(tm1.y) * 16u + __float_as_uint(tm1.x)) * 16u + __float_as_uint(tm0.y)) * 16u
-                                    + __float_as_uint(tm0.x);
-                tie_any |= pp ^ pm;          // low 16 bits: the four codes (offset by 8) under either multiplier
-                *reinterpret_cast<uint16_t *>(code_buf + code_off[s]) = (uint16_t)(pp ^ 0x8888u);
-            }
-            tie_any &= 0xffffu;
-            // ---- exact resolution of near ties (rare)
-            if (__any_sync(0xffffffffu, tie_any != 0u)) {
-                uint32_t fm = 0u;
-                if (tie_any != 0u) {
-#pragma unroll
-                    for (int s = 0; s < 8; ++s) {
-                        const int k = s & 3 & PM;
-                        const f32x2 tp0 = fma2(v[s][0], mul_p[k], magic2), tp1 = fma2(v[s][1], mul_p[k], magic2);
-                        const f32x2 tm0 = fma2(v[s][0], mul_m[k], magic2), tm1 = fma2(v[s][1], mul_m[k], magic2);
-                        const float t[4] = {tp0.x, tp0.y, tp1.x, tp1.y}, u[4] = {tm0.x, tm0.y, tm1.x, tm1.y};
-#pragma unroll
-                        for (int j = 0; j < 4; ++j) fm |= (t[j] != u[j]) ? (1u << (4 * s + j)) : 0u;
-                    }
-                }
-                __syncwarp();
-                unsigned tl = __ballot_sync(0xffffffffu, fm != 0u);
-                while (tl) {
-                    const int src = __ffs(tl) - 1;
-                    tl &= tl - 1;
-                    uint32_t fs = __shfl_sync(0xffffffffu, fm, src);
-                    // the same sequence of fp64 operations as the definition, so exact ties land on exact halves
-                    const double a_src = __shfl_sync(0xffffffffu, a_exact, src);
-                    const double s_src = (a_src / p.sqrt_b) / 7.0;
-                    while (fs) {
-                        const int e = __ffs(fs) - 1;
-                        fs &= fs - 1;
-                        int blk_elem, i, elem;
-                        locate<LOG2B>(src >> 2, src & 3, e, blk_elem, i, elem);
-                        const double ue = exact_coord_fast<B>(seg + blk_elem, i, lane);
-                        if (lane == 0) {
-                            uint32_t code = 0u;
-                            if (s_src != 0.0) {
-                                double qd = rint((ue / p.sqrt_b) / s_src);
-                                qd = fmin(fmax(qd, -8.0), 7.0);
-                                code = (uint32_t)((int)qd) & 0xFu;
-                            }
-                            uint8_t *bp = code_buf + (elem >> 1);
-                            *bp = (elem & 1) ? (uint8_t)((*bp & 0x0F) | (code << 4)) : (uint8_t)((*bp & 0xF0) | code);
-                        }
-                        __syncwarp();
-                    }
-                }
-            }
-        } else {   // ---------------------------------------------------------------- MXFP4
-            float vf[8][4];
-#pragma unroll
-            for (int s = 0; s < 8; ++s) {
-                vf[s][0] = v[s][0].x; vf[s][1] = v[s][0].y;
-                vf[s][2] = v[s][1].x; vf[s][3] = v[s][1].y;
-            }
-            uint32_t tie_any = 0u;
-            int E_pack = 0;                      // E + 127 of the lane's four groups, one per byte
-            float cp_[4], cm_[4];
-            uint32_t word = 0u;
-#pragma unroll
-            for (int m = 0; m < 4; ++m) {
-                float a32 = fmaxf(ms[2 * m], ms[2 * m + 1]);
-                a32 = fmaxf(a32, __shfl_xor_sync(0xffffffffu, a32, 1));
-                a32 = fmaxf(a32, __shfl_xor_sync(0xffffffffu, a32, 2));
-                // error reference: the largest |u| of the Hadamard block (the group may be smaller than the block)
-                float bref = a32;
-                if (CB >= 2) {
-                    float bm = (CB == 2) ? fmaxf(fmaxf(ms[(2 * m) & 4], ms[((2 * m) & 4) + 1]), fmaxf(ms[((2 * m) & 4) + 2], ms[((2 * m) & 4) + 3]))
-                                         : fmaxf(fmaxf(fmaxf(ms[0], ms[1]), fmaxf(ms[2], ms[3])), fmaxf(fmaxf(ms[4], ms[5]), fmaxf(ms[6], ms[7])));
-                    bm = fmaxf(bm, __shfl_xor_sync(0xffffffffu, bm, 1));
-                    bm = fmaxf(bm, __shfl_xor_sync(0xffffffffu, bm, 2));
-                    bref = bm;
-                }
-                const float ratio = (a32 > 0.0f) ? bref / a32 : 1.0f;
-                const float rho = err_rel * ratio + 2.4e-7f;          // relative uncertainty of a32
-                // E = floor(log2(a / sqrt(b))) - 2 from the bits of a32; exact re-derivation near a boundary
-                const uint32_t bits = __float_as_uint(a32);
-                int eu = (int)(bits >> 23) - 127;
-                const uint32_t mant = bits & 0x7fffffu;
-                const float mrel = __uint_as_float(0x3f800000u | mant);          // [1, 2)
-                bool near;
-                int E;
-                if ((LOG2B & 1) == 0) {
-                    E = eu - LOG2B / 2 - 2;
-                    near = (mrel * (1.0f - rho) < 1.0f) || (mrel * (1.0f + rho) >= 2.0f);
-                } else {
-                    const float SQ2 = 1.41421356237f;
-                    E = eu - (LOG2B + 1) / 2 + (mant >= 0x3504f3u ? 1 : 0) - 2;
-                    near = (mrel * (1.0f - rho) < 1.0f) || (mrel * (1.0f + rho) >= 2.0f) || (fabsf(mrel - SQ2) <= rho * 2.0f);
-                }
-                if (a32 > 0.0f && (near || (bits >> 23) == 0u)) {
-                    // rare: exact maximum of the group from every element that could attain it
-                    const float thr = a32 - 2.0f * err_rel * bref - a32 * 2.4e-7f;
-                    const bool has = fmaxf(ms[2 * m], ms[2 * m + 1]) >= thr;
-                    unsigned cq = __ballot_sync(qmask, has) & qmask;
-                    double best = 0.0;
-                    while (cq) {
-                        const int src = __ffs(cq) - 1;
-                        cq &= cq - 1;
-                        uint32_t cm = 0u;
-                        if (lane == src) {
-#pragma unroll
-                            for (int e = 0; e < 8; ++e) cm |= (fabsf(vf[2 * m + (e >> 2)][e & 3]) >= thr) ? (1u << e) : 0u;
-                        }
-                        cm = __shfl_sync(qmask, cm, src);
-                        while (cm) {
-                            const int e = __ffs(cm) - 1;
-                            cm &= cm - 1;
-                            int blk_elem, i, elem;
-                            locate<LOG2B>(src >> 2, src & 3, 8 * m + e, blk_elem, i, elem);
-                            best = fmax(best, fabs(exact_coord_quad<LOG2B>(seg + blk_elem, i, q, qmask)));
-                        }
-                    }
-                    int ex;
-                    (void)frexp(best / p.sqrt_b, &ex);
-                    E = ex - 3;
-                }
-                E = min(max(E, -127), 127);
-                const uint32_t byte = (a32 > 0.0f) ? (uint32_t)(E + 127) : 0u;
-                E_pack |= (int)(byte << (8 * m));
-                // multiplier 2^-E / sqrt(b)
-                float c;
-                if ((LOG2B & 1) == 0) c = __uint_as_float((uint32_t)min(max(127 - E - LOG2B / 2, 1), 254) << 23);
-                else c = __uint_as_float(0x3fb504f3u + ((uint32_t)(min(max(127 - E - (LOG2B + 1) / 2, 1), 253) - 127) << 23));
-                if (!(a32 > 0.0f)) c = 0.0f;
-                const float delta = 32.0f * err_rel * ratio + 5.0e-7f;
-                cp_[m] = c * (1.0f + delta);
-                cm_[m] = c * (1.0f - delta);
-                // scale byte position: group index inside the lane group's four groups
-                word |= byte << (8 * (m ^ ((f_g & ~PM) >> 1)));
-            }
-            if (q == 0) reinterpret_cast<uint32_t *>(p.out_scales)[seg_index * 8 + g] = word;
-#pragma unroll
-            for (int s = 0; s < 8; ++s) {
-                const float sg = sgn[s & 3 & PM];
-                const float kp = sg * cp_[s >> 1], km = sg * cm_[s >> 1];
-                const uint32_t p0 = cvt_e2m1x2(fmaf(vf[s][0], kp, 0.0f), fmaf(vf[s][1], kp, 0.0f));
-                const uint32_t p1 = cvt_e2m1x2(fmaf(vf[s][2], kp, 0.0f), fmaf(vf[s][3], kp, 0.0f));
-                const uint32_t m0 = cvt_e2m1x2(fmaf(vf[s][0], km, 0.0f), fmaf(vf[s][1], km, 0.0f));
-                const uint32_t m1 = cvt_e2m1x2(fmaf(vf[s][2], km, 0.0f), fmaf(vf[s][3], km, 0.0f));
-                tie_any |= (p0 ^ m0) | (p1 ^ m1);
-                *reinterpret_cast<uint16_t *>(code_buf + code_off[s]) = (uint16_t)(p0 | (p1 << 8));
-            }
-            if (__any_sync(0xffffffffu, tie_any != 0u)) {
-                __syncwarp();
-                unsigned tl = __ballot_sync(0xffffffffu, tie_any != 0u);
-                while (tl) {
-                    const int src = __ffs(tl) - 1;
-                    tl &= tl - 1;
-                    uint32_t fm = 0u;
-#pragma unroll
-                    for (int e = 0; e < 32; e += 2) {
-                        const int s = e >> 2;
-                        const float sg = sgn[s & 3 & PM];
-                        const float kp = sg * cp_[s >> 1], km = sg * cm_[s >> 1];
-                        const uint32_t pp = cvt_e2m1x2(fmaf(vf[s][e & 3], kp, 0.0f), fmaf(vf[s][(e & 3) + 1], kp, 0.0f));
-                        const uint32_t mm = cvt_e2m1x2(fmaf(vf[s][e & 3], km, 0.0f), fmaf(vf[s][(e & 3) + 1], km, 0.0f));
-                        const uint32_t x = pp ^ mm;
-                        fm |= ((x & 0x0Fu) ? (1u << e) : 0u) | ((x & 0xF0u) ? (2u << e) : 0u);
-                    }
-                    fm = __shfl_sync(0xffffffffu, fm, src);
-                    const int Ep = __shfl_sync(0xffffffffu, E_pack, src);
-                    while (fm) {
-                        const int e = __ffs(fm) - 1;
-                        fm &= fm - 1;
-                        int blk_elem, i, elem;
-                        locate<LOG2B>(src >> 2, src & 3, e, blk_elem, i, elem);
-                        const double ue = exact_coord_fast<B>(seg + blk_elem, i, lane);
-                        if (lane == 0) {
-                            const int E = ((Ep >> (8 * (e >> 3))) & 0xFF) - 127;
-                            const double y = ue / p.sqrt_b;
-                            const uint32_t code = e2m1_code_exact(scalbn(y, -E), signbit(y));
-                            uint8_t *bp = code_buf + (elem >> 1);
-                            *bp = (elem & 1) ? (uint8_t)((*bp & 0x0F) | (code << 4)) : (uint8_t)((*bp & 0xF0) | code);
-                        }
-                        __syncwarp();
-                    }
-                }
-            }
-        }
-
-        // ---- packed codes: shared staging -> global
-        fence_async_smem();
-        __syncwarp();
-        if (lane == 0) bulk_store(p.out_codes + (size_t)seg_index * SEG_CODE_BYTES, smem_u32(code_buf), SEG_CODE_BYTES);
-    }
-    bulk_store_wait_read<0>();
-}
-
-}  // namespace perq
