@@ -167,3 +167,303 @@ __device__ __forceinline__ unsigned long long warp_max_u64(unsigned long long v)
 __device__ __forceinline__ float max3abs(float acc, float a, float b) { return fmaxf(fmaxf(acc, fabsf(a)), fabsf(b)); }
 
 __device__ __forceinline__ uint32_t hadamard_bf16(int k, int n) { return (__popc(k & n) & 1) ? 0xBF80u : 0x3F80u; }
+
+// ---------------------------------------------------------------- exact re-evaluation
+
+// bf16 bit pattern (low 16 bits of h) -> double, exactly, with integer operations (the
+// fp32->fp64 conversion instruction is slow); zero and subnormals take the conversion.
+__device__ __forceinline__ double bf16_bits_to_f64(uint32_t h)
+{
+    const uint32_t mag = h & 0x7fffu;
+    if (mag < 0x80u) return (double)__uint_as_float(h << 16);
+    return __hiloint2double((int)(((mag << 13) + 0x38000000u) | ((h & 0x8000u) << 16)), 0);
+}
+
+// Exact unnormalised output i of the block starting at `blk` (bf16 in shared memory), evaluated
+// by the 4 lanes of a quad: each lane reduces a quarter of the block with a signed pairwise
+// tree in fp64, then the quarters are combined.  q = lane % 4, qmask = the quad's lanes.
+template <int LOG2B>
+__device__ __forceinline__ double exact_coord_quad(const uint16_t *blk, int i, int q, unsigned qmask)
+{
+    constexpr int PER = (1 << LOG2B) / 4;
+    double v[PER];
+    const uint32_t *src = reinterpret_cast<const uint32_t *>(blk + q * PER);
+#pragma unroll
+    for (int r = 0; r < PER / 2; ++r) {
+        const uint32_t w = src[r];
+        v[2 * r] = bf16_bits_to_f64(w);
+        v[2 * r + 1] = bf16_bits_to_f64(w >> 16);
+    }
+#pragma unroll
+    for (int t = 0; (1 << t) < PER; ++t) {
+        const double sg = ((i >> t) & 1) ? -1.0 : 1.0;
+#pragma unroll
+        for (int m = 0; m < (PER >> (t + 1)); ++m) v[m] = fma(sg, v[2 * m + 1], v[2 * m]);
+    }
+    double part = (__popc(i & (q << (LOG2B - 2))) & 1) ? -v[0] : v[0];
+    part += __shfl_xor_sync(qmask, part, 1);
+    part += __shfl_xor_sync(qmask, part, 2);
+    return part;
+}
+
+// Exact unnormalised output i of the B-element block at blk, by a whole warp.
+template <int B>
+__device__ __forceinline__ double exact_coord_fast(const uint16_t *blk, int i, int lane)
+{
+    double acc = 0.0;
+#pragma unroll
+    for (int k0 = 0; k0 < B; k0 += 32) {
+        const int k = k0 + lane;
+        if (B >= 32 || k < B) {
+            const double v = bf16_bits_to_f64(blk[k]);
+            acc += (__popc(i & k) & 1) ? -v : v;
+        }
+    }
+#pragma unroll
+    for (int o = 16; o > 0; o >>= 1) acc += __shfl_xor_sync(0xffffffffu, acc, o);
+    return acc;
+}
+
+// Exact unnormalised outputs i0 .. i0+3 (i0 a multiple of 4) of the B-element block at blk, by a
+// whole warp: lane l returns output i0 + (l & 3).  Every lane adds its terms signed by the high
+// bits of the output index; lanes with equal l & 3 are summed, then a 4-point butterfly over
+// l & 3 applies the low two index bits.
+template <int B>
+__device__ __forceinline__ double exact_coord4(const uint16_t *blk, int i0, int lane)
+{
+    double acc = 0.0;
+#pragma unroll
+    for (int k0 = 0; k0 < B; k0 += 32) {
+        const int k = k0 + lane;
+        if (B >= 32 || k < B) {
+            const double v = bf16_bits_to_f64(blk[k]);
+            acc += (__popc(i0 & k) & 1) ? -v : v;
+        }
+    }
+    acc += __shfl_xor_sync(0xffffffffu, acc, 4);
+    acc += __shfl_xor_sync(0xffffffffu, acc, 8);
+    acc += __shfl_xor_sync(0xffffffffu, acc, 16);
+#pragma unroll
+    for (int bit = 1; bit <= 2; bit <<= 1) {
+        const double other = __shfl_xor_sync(0xffffffffu, acc, bit);
+        acc = (lane & bit) ? other - acc : acc + other;
+    }
+    return acc;
+}
+
+// Element e = s*4 + j of lane (g, q): block start (in elements, segment relative) and index inside the block.
+template <int LOG2B>
+__device__ __forceinline__ void locate(int g, int q, int e, int &blk_elem, int &i, int &elem)
+{
+    constexpr int CB = LOG2B - 4;                 // chunk bits inside a block
+    constexpr int PM = (1 << CB) - 1;
+    const int s = e >> 2, j = e & 3;
+    const int p = g * 8 + (s ^ ((g & 3) & ~PM));  // chunk position inside the segment
+    elem = p * 16 + 4 * q + j;
+    blk_elem = (p >> CB) << LOG2B;
+    i = elem - blk_elem;
+}
+
+// Bit mask of the lane's 32 held values (bit s*4+j) whose magnitude reaches thr; ms[s] is the
+// magnitude maximum of slot s, used to skip slots.
+__device__ __forceinline__ uint32_t candidate_mask(const f32x2 (&v)[8][2], const float (&ms)[8], float thr)
+{
+    uint32_t cm = 0u;
+#pragma unroll
+    for (int s = 0; s < 8; ++s) {
+        if (ms[s] >= thr) {
+            const float a = v[s][0].x, b = v[s][0].y, c = v[s][1].x, d = v[s][1].y;
+            cm |= (fabsf(a) >= thr ? 1u : 0u) << (4 * s);
+            cm |= (fabsf(b) >= thr ? 2u : 0u) << (4 * s);
+            cm |= (fabsf(c) >= thr ? 4u : 0u) << (4 * s);
+            cm |= (fabsf(d) >= thr ? 8u : 0u) << (4 * s);
+        }
+    }
+    return cm;
+}
+
+// Exact maximum magnitude (bit pattern of a non-negative double, the same in every lane) over the
+// slots of this warp's segment whose fp32 maximum reaches thr.
+template <int LOG2B>
+__device__ __forceinline__ unsigned long long exact_max_of_candidates(const uint16_t *seg, const float (&ms)[8],
+                                                                      float thr, int lane)
+{
+    constexpr int CB = LOG2B - 4;
+    constexpr int PM = (1 << CB) - 1;
+    uint32_t slot_mask = 0u;
+#pragma unroll
+    for (int s = 0; s < 8; ++s) slot_mask |= (ms[s] >= thr) ? (1u << s) : 0u;
+    double best = 0.0;
+    unsigned cw = __ballot_sync(0xffffffffu, slot_mask != 0u);
+    while (cw) {
+        const int src = __ffs(cw) - 1;
+        cw &= cw - 1;
+        uint32_t sm = __shfl_sync(0xffffffffu, slot_mask, src);
+        const int sg = src >> 2;
+        while (sm) {
+            const int sl = __ffs(sm) - 1;
+            sm &= sm - 1;
+            const int pch = sg * 8 + (sl ^ ((sg & 3) & ~PM));      // chunk position in the segment
+            const int blk_elem = (pch >> CB) << LOG2B;
+            const int i0 = pch * 16 - blk_elem + 4 * (src & 3);
+            best = fmax(best, fabs(exact_coord4<(1 << LOG2B)>(seg + blk_elem, i0, lane)));
+        }
+    }
+    return warp_max_u64((unsigned long long)__double_as_longlong(best));
+}
+
+// ---------------------------------------------------------------- the kernel
+
+template <int LOG2B, int MODE, int LOG2G>
+__global__ void __launch_bounds__(FAST_THREADS, 1) perq_fast_kernel(FastParams p)
+{
+    constexpr int B = 1 << LOG2B;
+    constexpr int CB = LOG2B - 4;                 // butterfly stages left after the tensor-core H_16
+    constexpr int PM = (1 << CB) - 1;             // slot bits inside a Hadamard block
+    constexpr int NCLS = (PM & 3) + 1;            // sign classes of the slot relabelling
+    constexpr int G = 1 << LOG2G;                 // warps (segments) per unit
+    constexpr int GROUPS = FAST_WARPS / G;
+    constexpr uint32_t UNIT_BYTES = (uint32_t)G * SEG_BYTES;
+    constexpr float MAGIC = 12582920.0f;          // 1.5 * 2^23 + 8: low nibble of the sum = code + 8
+    static_assert(MODE == MODE_TOKEN || LOG2G == 0, "only per-token scales couple the warps of a row");
+    extern __shared__ __align__(128) unsigned char fsmem_raw[];
+    // 1024-byte aligned base: the ldmatrix and code-store addresses below are formed with XOR
+    unsigned char *fsmem = fsmem_raw + ((1024u - (smem_u32(fsmem_raw) & 1023u)) & 1023u);
+
+    const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+    const int g = lane >> 2, q = lane & 3;
+    const int group = warp >> LOG2G, w_in_g = warp & (G - 1);
+    const unsigned qmask = 0xFu << (lane & 28);
+    const float err_rel = FAST_ERR_K * (float)LOG2B * TWO_M24;
+
+    const uint32_t stage_base = smem_u32(fsmem + FastSmem::stages) + (uint32_t)group * (FAST_NSTAGE * UNIT_BYTES);
+    const uint32_t code_base = smem_u32(fsmem + FastSmem::codes) + (uint32_t)warp * (2 * SEG_CODE_BYTES);
+    const uint32_t full_base = smem_u32(fsmem + FastSmem::full) + (uint32_t)group * (FAST_NSTAGE * 8);
+    unsigned long long *wacc = reinterpret_cast<unsigned long long *>(fsmem + FastSmem::wacc);
+    unsigned long long *wpub = reinterpret_cast<unsigned long long *>(fsmem + FastSmem::wpub);
+    float *wmax = reinterpret_cast<float *>(fsmem + FastSmem::wmax);
+    uint32_t *wcnt = reinterpret_cast<uint32_t *>(fsmem + FastSmem::wcnt);
+    uint32_t *wflag = reinterpret_cast<uint32_t *>(fsmem + FastSmem::wflag);
+    const bool leader = (w_in_g == 0) && (lane == 0);
+
+    if (tid < FAST_WARPS * FAST_NSTAGE) mbar_init(smem_u32(fsmem + FastSmem::full) + tid * 8, 1);
+    if (tid < 2 * FAST_WARPS) { wacc[tid] = 0ull; wcnt[tid] = 0u; wflag[tid] = 0u; }
+    if (tid == 0) asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+    __syncthreads();
+
+    const uint32_t first = blockIdx.x * GROUPS + group;
+    const uint32_t stride = gridDim.x * GROUPS;
+    if (first >= p.units_total) return;      // whole groups leave together (no barrier is shared across groups)
+
+    // Hadamard operand of the tensor-core stage: column n of MMA m is output 4*(n/2) + (n%2) + 2m.
+    uint32_t hb[2][2];
+#pragma unroll
+    for (int m = 0; m < 2; ++m) {
+        const int col = 4 * (g >> 1) + (g & 1) + 2 * m;
+        hb[m][0] = hadamard_bf16(2 * q, col) | (hadamard_bf16(2 * q + 1, col) << 16);
+        hb[m][1] = hadamard_bf16(2 * q + 8, col) | (hadamard_bf16(2 * q + 9, col) << 16);
+    }
+    // ldmatrix source offset of tile 0: lane l feeds row (l & 7) of matrix (l >> 3); slot 2t + (mi & 1)
+    // of lane group r8 comes from chunk r8*8 + (slot ^ f), halves swapped when r8 & 4.  Tile t is at
+    // this offset XOR (t << 6).
+    uint32_t lm0;
+    {
+        const int r8 = lane & 7, mi = lane >> 3;
+        const int f = r8 & 3, fh = (r8 >> 2) & 1;
+        lm0 = (uint32_t)((r8 * 8 + ((mi & 1) ^ f)) * 32 + (((mi >> 1) ^ fh) * 16));
+    }
+    const int f_g = g & 3;
+    // byte offset of this lane's 16-bit code piece of slot 0 inside the segment's 512 code bytes;
+    // slot s is at this offset XOR (s * 8)
+    const uint32_t code_lane = (uint32_t)((g * 8 + (f_g & ~PM)) * 8 + 2 * q);
+    // sign of the held value relative to the true output, per (s & 3 & PM): folded into multipliers
+    const float half_sign = ((g & 4) && q >= 2) ? -1.0f : 1.0f;
+    float sgn[NCLS];
+#pragma unroll
+    for (int k = 0; k < NCLS; ++k) sgn[k] = (__popc(k & f_g & PM) & 1) ? -half_sign : half_sign;
+
+    const uint16_t *xin = p.x + (size_t)w_in_g * 0;   // unit u starts at xin + u * G * SEG_ELEMS
+    // prologue: fill the ring
+    if (leader) {
+#pragma unroll
+        for (int s = 0; s < FAST_NSTAGE; ++s) {
+            const uint32_t u = first + (uint32_t)s * stride;
+            if (u < p.units_total) {
+                mbar_expect_tx(full_base + s * 8, UNIT_BYTES);
+                bulk_load(stage_base + s * UNIT_BYTES, xin + (size_t)u * (G * SEG_ELEMS), UNIT_BYTES, full_base + s * 8);
+            }
+        }
+    }
+
+    uint32_t it = 0;
+    for (uint32_t unit = first; unit < p.units_total; unit += stride, ++it) {
+        const uint32_t stage = it % FAST_NSTAGE;
+        const uint32_t parity = (it / FAST_NSTAGE) & 1u;
+        const uint32_t par2 = it & 1u;
+        if (!mbar_wait(full_base + stage * 8, parity)) {
+            if (lane == 0) atomicOr(&g_perq_device_error, 1u);
+            return;
+        }
+        const uint32_t seg_addr = stage_base + stage * UNIT_BYTES + (uint32_t)w_in_g * SEG_BYTES;
+        const uint16_t *seg = reinterpret_cast<const uint16_t *>(fsmem + FastSmem::stages) +
+                              ((size_t)group * FAST_NSTAGE + stage) * (G * SEG_ELEMS) + (size_t)w_in_g * SEG_ELEMS;
+        const size_t seg_index = (size_t)unit * G + w_in_g;
+
+        // ---- H_16 on the tensor cores; v[s][h] = outputs (2h, 2h+1) of this lane's four of slot s
+        f32x2 v[8][2];
+        {
+            const uint32_t a0 = seg_addr + lm0;
+#pragma unroll
+            for (int t = 0; t < 4; ++t) {
+                uint32_t a[4];
+                ldmatrix_x4(a, a0 ^ (uint32_t)(t << 6));
+                float c0[4], c1[4];
+                mma_bf16(c0, a, hb[0][0], hb[0][1]);
+                mma_bf16(c1, a, hb[1][0], hb[1][1]);
+                v[2 * t][0] = pack2(c0[0], c0[1]);
+                v[2 * t][1] = pack2(c1[0], c1[1]);
+                v[2 * t + 1][0] = pack2(c0[2], c0[3]);
+                v[2 * t + 1][1] = pack2(c1[2], c1[3]);
+            }
+        }
+        // refill the stage the previous iteration used (every warp of the group is past it now:
+        // for G == 1 because this warp is, for G > 1 after the named barrier below)
+        auto refill = [&]() {
+            if (leader && it > 0) {
+                const uint32_t u = unit + (FAST_NSTAGE - 1) * stride;
+                if (u < p.units_total && u > unit) {
+                    const uint32_t ps = (it - 1) % FAST_NSTAGE;
+                    mbar_expect_tx(full_base + ps * 8, UNIT_BYTES);
+                    bulk_load(stage_base + ps * UNIT_BYTES, xin + (size_t)u * (G * SEG_ELEMS), UNIT_BYTES,
+                              full_base + ps * 8);
+                }
+            }
+        };
+        if (G == 1) refill();
+
+        // ---- remaining butterfly stages over the slot bits inside a block (packed add/sub)
+#pragma unroll
+        for (int t = 0; t < CB; ++t) {
+#pragma unroll
+            for (int s = 0; s < 8; ++s) {
+                if ((s & (1 << t)) == 0) {
+#pragma unroll
+                    for (int h = 0; h < 2; ++h) {
+                        const f32x2 a = v[s][h], c = v[s | (1 << t)][h];
+                        v[s][h] = add2(a, c);
+                        v[s | (1 << t)][h] = sub2(a, c);
+                    }
+                }
+            }
+        }
+
+        // ---- fp32 maxima per slot
+        float ms[8];
+#pragma unroll
+        for (int s = 0; s < 8; ++s) ms[s] = fmaxf(max3abs(fabsf(v[s][0].x), v[s][0].y, v[s][1].x), fabsf(v[s][1].y));
+
+        const uint32_t code_buf = code_base + par2 * SEG_CODE_BYTES;
+        const uint32_t code_addr0 = code_buf + code_lane;
+        uint8_t *code_gen = fsmem + FastSmem::codes + (size_t)warp * (2 * SEG_CODE_BYTES) + (size_t)par2 * SEG_CODE_BYTES;
+        bulk_store_wait_read<1>();           // the store that last read this staging buffer has drained
+        __syncwarp();
