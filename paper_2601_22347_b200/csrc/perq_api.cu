@@ -98,23 +98,23 @@ int launch_generic(const void *x, const int32_t *perm, int64_t T, int32_t d, int
     return cudaGetLastError() == cudaSuccess ? PERQ_OK : PERQ_ERR_CUDA;
 }
 
-template <int LOG2B, int MODE>
+template <int LOG2B, int MODE, int LOG2G>
 int launch_fast_inst(const perq::FastParams &p, int grid, cudaStream_t st)
 {
-    auto kernel = perq::perq_fast_kernel<LOG2B, MODE>;
+    auto kernel = perq::perq_fast_kernel<LOG2B, MODE, LOG2G>;
     if (int rc = allow_smem(kernel, perq::FastSmem::total)) return rc;
     kernel<<<grid, perq::FAST_THREADS, perq::FastSmem::total, st>>>(p);
     return cudaGetLastError() == cudaSuccess ? PERQ_OK : PERQ_ERR_CUDA;
 }
 
-template <int MODE>
+template <int MODE, int LOG2G>
 int launch_fast_mode(int log2b, const perq::FastParams &p, int grid, cudaStream_t st)
 {
     switch (log2b) {
-    case 4: return launch_fast_inst<4, MODE>(p, grid, st);
-    case 5: return launch_fast_inst<5, MODE>(p, grid, st);
-    case 6: return launch_fast_inst<6, MODE>(p, grid, st);
-    default: return launch_fast_inst<7, MODE>(p, grid, st);
+    case 4: return launch_fast_inst<4, MODE, LOG2G>(p, grid, st);
+    case 5: return launch_fast_inst<5, MODE, LOG2G>(p, grid, st);
+    case 6: return launch_fast_inst<6, MODE, LOG2G>(p, grid, st);
+    default: return launch_fast_inst<7, MODE, LOG2G>(p, grid, st);
     }
 }
 
@@ -136,23 +136,29 @@ int try_launch_fast(const void *x, const int32_t *perm, int64_t T, int32_t d, in
     } else {
         return -1;
     }
+    const long long units = (long long)T * (d / perq::SEG_ELEMS) / G;
+    if (units >= (1ll << 31)) return -1;
     perq::FastParams p;
     p.x = static_cast<const uint16_t *>(x);
     p.out_codes = static_cast<uint8_t *>(out_codes);
     p.out_scales = out_scales;
-    p.G = G;
-    p.units_total = (long long)T * (d / perq::SEG_ELEMS) / G;
+    p.units_total = (uint32_t)units;
     p.sqrt_b = std::sqrt((double)b);
     p.inv_7_sqrt_b = 1.0 / (7.0 * p.sqrt_b);
     const int sms = sm_count();
     if (sms <= 0) return PERQ_ERR_CUDA;
     const int groups_per_cta = perq::FAST_WARPS / G;
-    const long long want = (p.units_total + groups_per_cta - 1) / groups_per_cta;
+    const long long want = (units + groups_per_cta - 1) / groups_per_cta;
     const int grid = (int)std::min<long long>(want, sms);
     const int log2b = ilog2(b);
-    if (mode == perq::MODE_MX) return launch_fast_mode<perq::MODE_MX>(log2b, p, grid, st);
-    if (mode == perq::MODE_G128) return launch_fast_mode<perq::MODE_G128>(log2b, p, grid, st);
-    return launch_fast_mode<perq::MODE_TOKEN>(log2b, p, grid, st);
+    if (mode == perq::MODE_MX) return launch_fast_mode<perq::MODE_MX, 0>(log2b, p, grid, st);
+    if (mode == perq::MODE_G128) return launch_fast_mode<perq::MODE_G128, 0>(log2b, p, grid, st);
+    switch (G) {
+    case 1: return launch_fast_mode<perq::MODE_TOKEN, 0>(log2b, p, grid, st);
+    case 2: return launch_fast_mode<perq::MODE_TOKEN, 1>(log2b, p, grid, st);
+    case 4: return launch_fast_mode<perq::MODE_TOKEN, 2>(log2b, p, grid, st);
+    default: return launch_fast_mode<perq::MODE_TOKEN, 3>(log2b, p, grid, st);
+    }
 }
 
 int launch_any(const void *x, const int32_t *perm, int64_t T, int32_t d, int32_t b, int32_t fmt, int g,

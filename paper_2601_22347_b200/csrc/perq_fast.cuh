@@ -467,3 +467,314 @@ __global__ void __launch_bounds__(FAST_THREADS, 1) perq_fast_kernel(FastParams p
         uint8_t *code_gen = fsmem + FastSmem::codes + (size_t)warp * (2 * SEG_CODE_BYTES) + (size_t)par2 * SEG_CODE_BYTES;
         bulk_store_wait_read<1>();           // the store that last read this staging buffer has drained
         __syncwarp();
+
+        if (MODE == MODE_TOKEN || MODE == MODE_G128) {
+            // lane maximum, then the maximum of the scale range in fp32 (a32); the exact maximum
+            // (a_bits, bit pattern of a double) only where it is known without waiting
+            const float lane_max = fmaxf(fmaxf(fmaxf(ms[0], ms[1]), fmaxf(ms[2], ms[3])),
+                                         fmaxf(fmaxf(ms[4], ms[5]), fmaxf(ms[6], ms[7])));
+            float a32;
+            unsigned long long a_bits = 0ull;
+            bool have_exact = true;          // warp-uniform: a_bits is the range's exact maximum
+            bool is_cand = false;            // per token: this warp holds candidates for the row maximum
+            int ncand = 1;
+            const uint32_t pidx = par2 * FAST_WARPS + group;
+            if (MODE == MODE_G128) {
+                a32 = fmaxf(lane_max, __shfl_xor_sync(0xffffffffu, lane_max, 1));
+                a32 = fmaxf(a32, __shfl_xor_sync(0xffffffffu, a32, 2));
+                const float thr = a32 * (1.0f - 2.0f * err_rel - 2.4e-7f);
+                const bool has_cand = (a32 > 0.0f) && (lane_max >= thr);
+                double a_exact = 0.0;
+                unsigned cq = __ballot_sync(0xffffffffu, has_cand) & qmask;      // candidate lanes of my quad
+                while (cq) {
+                    const int src = __ffs(cq) - 1;
+                    cq &= cq - 1;
+                    uint32_t cm = 0u;
+                    if (lane == src) cm = candidate_mask(v, ms, thr);
+                    cm = __shfl_sync(qmask, cm, src);
+                    while (cm) {
+                        const int e = __ffs(cm) - 1;
+                        cm &= cm - 1;
+                        int blk_elem, i, elem;
+                        locate<LOG2B>(src >> 2, src & 3, e, blk_elem, i, elem);
+                        a_exact = fmax(a_exact, fabs(exact_coord_quad<LOG2B>(seg + blk_elem, i, q, qmask)));
+                    }
+                }
+                if (q == 0)
+                    reinterpret_cast<float *>(p.out_scales)[seg_index * 8 + g] =
+                        (a_exact == 0.0) ? 0.0f : (float)(a_exact * p.inv_7_sqrt_b);
+                a_bits = (unsigned long long)__double_as_longlong(a_exact);
+            } else {
+                const float aw = warp_max_f32(lane_max);
+                unsigned candw;
+                if (G > 1) {
+                    if (lane == 0) wmax[par2 * FAST_WARPS + warp] = aw;
+                    named_barrier(1 + group, G * 32);
+                    const float am = (lane < G) ? wmax[par2 * FAST_WARPS + group * G + lane] : 0.0f;
+                    a32 = warp_max_f32(am);
+                    const float thr_row = a32 * (1.0f - 2.0f * err_rel - 2.4e-7f);
+                    candw = __ballot_sync(0xffffffffu, (lane < G) && (a32 > 0.0f) && (am >= thr_row));
+                    refill();
+                } else {
+                    a32 = aw;
+                    candw = (a32 > 0.0f) ? 1u : 0u;
+                }
+                is_cand = (candw >> w_in_g) & 1u;
+                ncand = __popc(candw);
+                have_exact = (ncand <= 1) && (is_cand || ncand == 0);
+                if (ncand == 0 && leader) reinterpret_cast<float *>(p.out_scales)[unit] = 0.0f;
+            }
+
+            // ---- quantise: packed fp32 multiply-add against the magic constant, with the multiplier
+            // nudged up and down by the error bound; elements whose two codes differ are resolved exactly
+            const float inv = (a32 > 0.0f) ? fminf(__fdividef(7.0f, a32), 3.0e38f) : 0.0f;
+            const float delta = 16.0f * err_rel + 5.0e-7f;
+            f32x2 mul_p[NCLS], mul_m[NCLS];
+#pragma unroll
+            for (int k = 0; k < NCLS; ++k) {
+                const float mp = sgn[k] * inv * (1.0f + delta), mm = sgn[k] * inv * (1.0f - delta);
+                mul_p[k] = pack2(mp, mp);
+                mul_m[k] = pack2(mm, mm);
+            }
+            const f32x2 magic2 = pack2(MAGIC, MAGIC);
+            uint32_t tie_any = 0u;
+#pragma unroll
+            for (int s = 0; s < 8; ++s) {
+                const int k = s & 3 & PM;
+                const f32x2 tp0 = fma2(v[s][0], mul_p[k], magic2), tp1 = fma2(v[s][1], mul_p[k], magic2);
+                const f32x2 tm0 = fma2(v[s][0], mul_m[k], magic2), tm1 = fma2(v[s][1], mul_m[k], magic2);
+                const uint32_t pp = ((__float_as_uint(tp1.y) * 16u + __float_as_uint(tp1.x)) * 16u + __float_as_uint(tp0.y)) * 16u
+                                    + __float_as_uint(tp0.x);
+                const uint32_t pm = ((__float_as_uint(tm1.y) * 16u + __float_as_uint(tm1.x)) * 16u + __float_as_uint(tm0.y)) * 16u
+                                    + __float_as_uint(tm0.x);
+                tie_any |= pp ^ pm;          // low 16 bits: the four codes (offset by 8) under either multiplier
+                sts_u16(code_addr0 ^ (uint32_t)(s * 8), pp ^ 0x8888u);
+            }
+            tie_any &= 0xffffu;
+
+            // ---- per token: the exact row maximum and the stored scale, by the candidate warps only
+            if (MODE == MODE_TOKEN && is_cand) {
+                const float thr_row = a32 * (1.0f - 2.0f * err_rel - 2.4e-7f);
+                const unsigned long long wb = exact_max_of_candidates<LOG2B>(seg, ms, thr_row, lane);
+                if (ncand == 1) {
+                    a_bits = wb;
+                    if (lane == 0) {
+                        reinterpret_cast<float *>(p.out_scales)[unit] =
+                            (wb == 0ull) ? 0.0f : (float)(__longlong_as_double((long long)wb) * p.inv_7_sqrt_b);
+                        if (G > 1) {
+                            wpub[pidx] = wb;
+                            __threadfence_block();
+                            *reinterpret_cast<volatile uint32_t *>(&wflag[pidx]) = it + 1u;
+                        }
+                    }
+                } else if (lane == 0) {
+                    atomicMax(&wacc[pidx], wb);
+                    __threadfence_block();
+                    if (atomicAdd(&wcnt[pidx], 1u) == (uint32_t)(ncand - 1)) {      // last candidate warp of the row
+                        const unsigned long long fin = atomicExch(&wacc[pidx], 0ull);
+                        wcnt[pidx] = 0u;
+                        reinterpret_cast<float *>(p.out_scales)[unit] =
+                            (fin == 0ull) ? 0.0f : (float)(__longlong_as_double((long long)fin) * p.inv_7_sqrt_b);
+                        wpub[pidx] = fin;
+                        __threadfence_block();
+                        *reinterpret_cast<volatile uint32_t *>(&wflag[pidx]) = it + 1u;
+                    }
+                }
+            }
+
+            // ---- exact resolution of near ties (rare)
+            if (__any_sync(0xffffffffu, tie_any != 0u)) {
+                if (!have_exact) {           // the row maximum comes from another warp: wait for its publication
+                    uint32_t spin = 0;
+                    while (ld_volatile_shared_u32(&wflag[pidx]) != it + 1u) {
+                        if (++spin >= WAIT_SPIN_LIMIT) {
+                            if (lane == 0) atomicOr(&g_perq_device_error, 2u);
+                            return;
+                        }
+                    }
+                    __threadfence_block();
+                    a_bits = *reinterpret_cast<volatile unsigned long long *>(&wpub[pidx]);
+                }
+                uint32_t fm = 0u;
+                if (tie_any != 0u) {
+#pragma unroll
+                    for (int s = 0; s < 8; ++s) {
+                        const int k = s & 3 & PM;
+                        const f32x2 tp0 = fma2(v[s][0], mul_p[k], magic2), tp1 = fma2(v[s][1], mul_p[k], magic2);
+                        const f32x2 tm0 = fma2(v[s][0], mul_m[k], magic2), tm1 = fma2(v[s][1], mul_m[k], magic2);
+                        const float t[4] = {tp0.x, tp0.y, tp1.x, tp1.y}, u[4] = {tm0.x, tm0.y, tm1.x, tm1.y};
+#pragma unroll
+                        for (int j = 0; j < 4; ++j) fm |= (t[j] != u[j]) ? (1u << (4 * s + j)) : 0u;
+                    }
+                }
+                __syncwarp();
+                unsigned tl = __ballot_sync(0xffffffffu, fm != 0u);
+                while (tl) {
+                    const int src = __ffs(tl) - 1;
+                    tl &= tl - 1;
+                    uint32_t fs = __shfl_sync(0xffffffffu, fm, src);
+                    // the same sequence of fp64 operations as the definition, so exact ties land on exact halves
+                    const double a_src = __longlong_as_double((long long)__shfl_sync(0xffffffffu, a_bits, src));
+                    const double s_src = (a_src / p.sqrt_b) / 7.0;
+                    while (fs) {
+                        const int e = __ffs(fs) - 1;
+                        fs &= fs - 1;
+                        int blk_elem, i, elem;
+                        locate<LOG2B>(src >> 2, src & 3, e, blk_elem, i, elem);
+                        const double ue = exact_coord_fast<B>(seg + blk_elem, i, lane);
+                        if (lane == 0) {
+                            uint32_t code = 0u;
+                            if (s_src != 0.0) {
+                                double qd = rint((ue / p.sqrt_b) / s_src);
+                                qd = fmin(fmax(qd, -8.0), 7.0);
+                                code = (uint32_t)((int)qd) & 0xFu;
+                            }
+                            uint8_t *bp = code_gen + (elem >> 1);
+                            *bp = (elem & 1) ? (uint8_t)((*bp & 0x0F) | (code << 4)) : (uint8_t)((*bp & 0xF0) | code);
+                        }
+                        __syncwarp();
+                    }
+                }
+            }
+        } else {   // ---------------------------------------------------------------- MXFP4
+            float vf[8][4];
+#pragma unroll
+            for (int s = 0; s < 8; ++s) {
+                vf[s][0] = v[s][0].x; vf[s][1] = v[s][0].y;
+                vf[s][2] = v[s][1].x; vf[s][3] = v[s][1].y;
+            }
+            uint32_t tie_any = 0u;
+            int E_pack = 0;                      // E + 127 of the lane's four groups, one per byte
+            float cp_[4], cm_[4];
+            uint32_t word = 0u;
+#pragma unroll
+            for (int m = 0; m < 4; ++m) {
+                float a32 = fmaxf(ms[2 * m], ms[2 * m + 1]);
+                a32 = fmaxf(a32, __shfl_xor_sync(0xffffffffu, a32, 1));
+                a32 = fmaxf(a32, __shfl_xor_sync(0xffffffffu, a32, 2));
+                // error reference: the largest |u| of the Hadamard block (the group may be smaller than the block)
+                float bref = a32;
+                if (CB >= 2) {
+                    float bm = (CB == 2) ? fmaxf(fmaxf(ms[(2 * m) & 4], ms[((2 * m) & 4) + 1]), fmaxf(ms[((2 * m) & 4) + 2], ms[((2 * m) & 4) + 3]))
+                                         : fmaxf(fmaxf(fmaxf(ms[0], ms[1]), fmaxf(ms[2], ms[3])), fmaxf(fmaxf(ms[4], ms[5]), fmaxf(ms[6], ms[7])));
+                    bm = fmaxf(bm, __shfl_xor_sync(0xffffffffu, bm, 1));
+                    bm = fmaxf(bm, __shfl_xor_sync(0xffffffffu, bm, 2));
+                    bref = bm;
+                }
+                const float ratio = (a32 > 0.0f) ? bref / a32 : 1.0f;
+                const float rho = err_rel * ratio + 2.4e-7f;          // relative uncertainty of a32
+                // E = floor(log2(a / sqrt(b))) - 2 from the bits of a32; exact re-derivation near a boundary
+                const uint32_t bits = __float_as_uint(a32);
+                int eu = (int)(bits >> 23) - 127;
+                const uint32_t mant = bits & 0x7fffffu;
+                const float mrel = __uint_as_float(0x3f800000u | mant);          // [1, 2)
+                bool near;
+                int E;
+                if ((LOG2B & 1) == 0) {
+                    E = eu - LOG2B / 2 - 2;
+                    near = (mrel * (1.0f - rho) < 1.0f) || (mrel * (1.0f + rho) >= 2.0f);
+                } else {
+                    const float SQ2 = 1.41421356237f;
+                    E = eu - (LOG2B + 1) / 2 + (mant >= 0x3504f3u ? 1 : 0) - 2;
+                    near = (mrel * (1.0f - rho) < 1.0f) || (mrel * (1.0f + rho) >= 2.0f) || (fabsf(mrel - SQ2) <= rho * 2.0f);
+                }
+                if (a32 > 0.0f && (near || (bits >> 23) == 0u)) {
+                    // rare: exact maximum of the group from every element that could attain it
+                    const float thr = a32 - 2.0f * err_rel * bref - a32 * 2.4e-7f;
+                    const bool has = fmaxf(ms[2 * m], ms[2 * m + 1]) >= thr;
+                    unsigned cq = __ballot_sync(qmask, has) & qmask;
+                    double best = 0.0;
+                    while (cq) {
+                        const int src = __ffs(cq) - 1;
+                        cq &= cq - 1;
+                        uint32_t cm = 0u;
+                        if (lane == src) {
+#pragma unroll
+                            for (int e = 0; e < 8; ++e) cm |= (fabsf(vf[2 * m + (e >> 2)][e & 3]) >= thr) ? (1u << e) : 0u;
+                        }
+                        cm = __shfl_sync(qmask, cm, src);
+                        while (cm) {
+                            const int e = __ffs(cm) - 1;
+                            cm &= cm - 1;
+                            int blk_elem, i, elem;
+                            locate<LOG2B>(src >> 2, src & 3, 8 * m + e, blk_elem, i, elem);
+                            best = fmax(best, fabs(exact_coord_quad<LOG2B>(seg + blk_elem, i, q, qmask)));
+                        }
+                    }
+                    int ex;
+                    (void)frexp(best / p.sqrt_b, &ex);
+                    E = ex - 3;
+                }
+                E = min(max(E, -127), 127);
+                const uint32_t byte = (a32 > 0.0f) ? (uint32_t)(E + 127) : 0u;
+                E_pack |= (int)(byte << (8 * m));
+                // multiplier 2^-E / sqrt(b)
+                float c;
+                if ((LOG2B & 1) == 0) c = __uint_as_float((uint32_t)min(max(127 - E - LOG2B / 2, 1), 254) << 23);
+                else c = __uint_as_float(0x3fb504f3u + ((uint32_t)(min(max(127 - E - (LOG2B + 1) / 2, 1), 253) - 127) << 23));
+                if (!(a32 > 0.0f)) c = 0.0f;
+                const float delta = 32.0f * err_rel * ratio + 5.0e-7f;
+                cp_[m] = c * (1.0f + delta);
+                cm_[m] = c * (1.0f - delta);
+                // scale byte position: group index inside the lane group's four groups
+                word |= byte << (8 * (m ^ ((f_g & ~PM) >> 1)));
+            }
+            if (q == 0) reinterpret_cast<uint32_t *>(p.out_scales)[seg_index * 8 + g] = word;
+#pragma unroll
+            for (int s = 0; s < 8; ++s) {
+                const float sg = sgn[s & 3 & PM];
+                const float kp = sg * cp_[s >> 1], km = sg * cm_[s >> 1];
+                const uint32_t p0 = cvt_e2m1x2(fmaf(vf[s][0], kp, 0.0f), fmaf(vf[s][1], kp, 0.0f));
+                const uint32_t p1 = cvt_e2m1x2(fmaf(vf[s][2], kp, 0.0f), fmaf(vf[s][3], kp, 0.0f));
+                const uint32_t m0 = cvt_e2m1x2(fmaf(vf[s][0], km, 0.0f), fmaf(vf[s][1], km, 0.0f));
+                const uint32_t m1 = cvt_e2m1x2(fmaf(vf[s][2], km, 0.0f), fmaf(vf[s][3], km, 0.0f));
+                tie_any |= (p0 ^ m0) | (p1 ^ m1);
+                sts_u16(code_addr0 ^ (uint32_t)(s * 8), p0 | (p1 << 8));
+            }
+            if (__any_sync(0xffffffffu, tie_any != 0u)) {
+                __syncwarp();
+                unsigned tl = __ballot_sync(0xffffffffu, tie_any != 0u);
+                while (tl) {
+                    const int src = __ffs(tl) - 1;
+                    tl &= tl - 1;
+                    uint32_t fm = 0u;
+#pragma unroll
+                    for (int e = 0; e < 32; e += 2) {
+                        const int s = e >> 2;
+                        const float sg = sgn[s & 3 & PM];
+                        const float kp = sg * cp_[s >> 1], km = sg * cm_[s >> 1];
+                        const uint32_t pp = cvt_e2m1x2(fmaf(vf[s][e & 3], kp, 0.0f), fmaf(vf[s][(e & 3) + 1], kp, 0.0f));
+                        const uint32_t mm = cvt_e2m1x2(fmaf(vf[s][e & 3], km, 0.0f), fmaf(vf[s][(e & 3) + 1], km, 0.0f));
+                        const uint32_t x = pp ^ mm;
+                        fm |= ((x & 0x0Fu) ? (1u << e) : 0u) | ((x & 0xF0u) ? (2u << e) : 0u);
+                    }
+                    fm = __shfl_sync(0xffffffffu, fm, src);
+                    const int Ep = __shfl_sync(0xffffffffu, E_pack, src);
+                    while (fm) {
+                        const int e = __ffs(fm) - 1;
+                        fm &= fm - 1;
+                        int blk_elem, i, elem;
+                        locate<LOG2B>(src >> 2, src & 3, e, blk_elem, i, elem);
+                        const double ue = exact_coord_fast<B>(seg + blk_elem, i, lane);
+                        if (lane == 0) {
+                            const int E = ((Ep >> (8 * (e >> 3))) & 0xFF) - 127;
+                            const double y = ue / p.sqrt_b;
+                            const uint32_t code = e2m1_code_exact(scalbn(y, -E), signbit(y));
+                            uint8_t *bp = code_gen + (elem >> 1);
+                            *bp = (elem & 1) ? (uint8_t)((*bp & 0x0F) | (code << 4)) : (uint8_t)((*bp & 0xF0) | code);
+                        }
+                        __syncwarp();
+                    }
+                }
+            }
+        }
+
+        // ---- packed codes: shared staging -> global
+        fence_async_smem();
+        __syncwarp();
+        if (lane == 0) bulk_store(p.out_codes + seg_index * SEG_CODE_BYTES, code_buf, SEG_CODE_BYTES);
+    }
+    bulk_store_wait_read<0>();
+}
+
+}  // namespace perq
