@@ -72,7 +72,8 @@ struct FastSmem {
     static constexpr size_t wmax = wpub + (size_t)FAST_WARPS * 2 * 8;               // [2][FAST_WARPS] f32 warp maxima
     static constexpr size_t wcnt = wmax + (size_t)FAST_WARPS * 2 * 4;               // [2][FAST_WARPS] u32 arrival counts
     static constexpr size_t wflag = wcnt + (size_t)FAST_WARPS * 2 * 4;              // [2][FAST_WARPS] u32 publication flags
-    static constexpr size_t used = wflag + (size_t)FAST_WARPS * 2 * 4;
+    static constexpr size_t wreq = wflag + (size_t)FAST_WARPS * 2 * 4;              // [FAST_WARPS][32] u64 deferred scale requests
+    static constexpr size_t used = wreq + (size_t)FAST_WARPS * 32 * 8;
     static constexpr size_t total = used + 1024;                                    // room to align the base
 };
 
@@ -312,6 +313,59 @@ __device__ __forceinline__ unsigned long long exact_max_of_candidates(const uint
     return warp_max_u64((unsigned long long)__double_as_longlong(best));
 }
 
+// ---------------------------------------------------------------- deferred per-token scales
+//
+// A per-token scale needs the exact magnitude of the row's largest rotated value.  In the common
+// case the fp32 pass pins that value down to one slot (four adjacent outputs of one 16-element
+// chunk).  The warp that owns the slot only records (row, position); when 32 records have
+// gathered, each lane of the warp serves one of them on its own: it re-reads the block's b bf16
+// inputs from global memory (64 to 256 bytes, usually still in L2), forms the four outputs in
+// fp64 and stores the scale.  This costs a few instructions per row instead of a cooperative
+// evaluation on the row's critical path.
+//
+// Record: bits 63..32 = row, bits 15..0 = element index in the row of the slot's first output.
+
+template <int LOG2B>
+__device__ __forceinline__ double exact_slot_max_global(const uint16_t *row, uint32_t pos)
+{
+    constexpr int B = 1 << LOG2B;
+    const uint32_t blk = (pos >> LOG2B) << LOG2B;
+    const uint32_t i0 = pos - blk;                       // multiple of 4
+    const uint4 *src = reinterpret_cast<const uint4 *>(row + blk);
+    double S[4] = {0.0, 0.0, 0.0, 0.0};                  // sums of the terms with k & 3 == m, signed by the high bits of i0
+#pragma unroll
+    for (int c = 0; c < B / 8; ++c) {
+        const uint4 w4 = __ldg(src + c);
+        const uint32_t w[4] = {w4.x, w4.y, w4.z, w4.w};
+#pragma unroll
+        for (int h = 0; h < 2; ++h) {
+            const bool neg = __popc(i0 & (uint32_t)(8 * c + 4 * h)) & 1;
+#pragma unroll
+            for (int e = 0; e < 4; ++e) {
+                const uint32_t word = w[2 * h + (e >> 1)];
+                const double val = (double)__uint_as_float((e & 1) ? (word & 0xffff0000u) : (word << 16));
+                S[e] += neg ? -val : val;
+            }
+        }
+    }
+    const double a0 = S[0] + S[1], a1 = S[0] - S[1], a2 = S[2] + S[3], a3 = S[2] - S[3];
+    return fmax(fmax(fabs(a0 + a2), fabs(a1 + a3)), fmax(fabs(a0 - a2), fabs(a1 - a3)));
+}
+
+template <int LOG2B>
+__device__ __forceinline__ void serve_scale_requests(const FastParams &p, const unsigned long long *req, uint32_t n,
+                                                     uint32_t row_elems, int lane)
+{
+    __syncwarp();
+    if ((uint32_t)lane < n) {
+        const unsigned long long r = req[lane];
+        const uint32_t unit = (uint32_t)(r >> 32), pos = (uint32_t)r & 0xffffu;
+        const double a = exact_slot_max_global<LOG2B>(p.x + (size_t)unit * row_elems, pos);
+        reinterpret_cast<float *>(p.out_scales)[unit] = (a == 0.0) ? 0.0f : (float)(a * p.inv_7_sqrt_b);
+    }
+    __syncwarp();
+}
+
 // ---------------------------------------------------------------- the kernel
 
 template <int LOG2B, int MODE, int LOG2G>
@@ -344,6 +398,8 @@ __global__ void __launch_bounds__(FAST_THREADS, 1) perq_fast_kernel(FastParams p
     float *wmax = reinterpret_cast<float *>(fsmem + FastSmem::wmax);
     uint32_t *wcnt = reinterpret_cast<uint32_t *>(fsmem + FastSmem::wcnt);
     uint32_t *wflag = reinterpret_cast<uint32_t *>(fsmem + FastSmem::wflag);
+    unsigned long long *wreq = reinterpret_cast<unsigned long long *>(fsmem + FastSmem::wreq) + warp * 32;
+    uint32_t nreq = 0;                       // records waiting in wreq (the same in every lane)
     const bool leader = (w_in_g == 0) && (lane == 0);
 
     if (tid < FAST_WARPS * FAST_NSTAGE) mbar_init(smem_u32(fsmem + FastSmem::full) + tid * 8, 1);
@@ -521,7 +577,7 @@ __global__ void __launch_bounds__(FAST_THREADS, 1) perq_fast_kernel(FastParams p
                 }
                 is_cand = (candw >> w_in_g) & 1u;
                 ncand = __popc(candw);
-                have_exact = (ncand <= 1) && (is_cand || ncand == 0);
+                have_exact = (ncand == 0);
                 if (ncand == 0 && leader) reinterpret_cast<float *>(p.out_scales)[unit] = 0.0f;
             }
 
@@ -553,47 +609,87 @@ __global__ void __launch_bounds__(FAST_THREADS, 1) perq_fast_kernel(FastParams p
             tie_any &= 0xffffu;
 
             // ---- per token: the exact row maximum and the stored scale, by the candidate warps only
+            uint32_t my_pos = 0xffffffffu;   // simple case: row position of the one candidate slot (this warp's)
             if (MODE == MODE_TOKEN && is_cand) {
                 const float thr_row = a32 * (1.0f - 2.0f * err_rel - 2.4e-7f);
-                const unsigned long long wb = exact_max_of_candidates<LOG2B>(seg, ms, thr_row, lane);
-                if (ncand == 1) {
-                    a_bits = wb;
+                uint32_t slot_mask = 0u;
+#pragma unroll
+                for (int s = 0; s < 8; ++s) slot_mask |= (ms[s] >= thr_row) ? (1u << s) : 0u;
+                const unsigned cl = __ballot_sync(0xffffffffu, slot_mask != 0u);
+                const int src = __ffs(cl) - 1;
+                const uint32_t sm = __shfl_sync(0xffffffffu, slot_mask, src);
+                if (ncand == 1 && (cl & (cl - 1)) == 0u && (sm & (sm - 1)) == 0u) {
+                    // one slot holds the maximum: record it, the scale is stored later
+                    const int sl = __ffs(sm) - 1, sg = src >> 2;
+                    const int pch = sg * 8 + (sl ^ ((sg & 3) & ~PM));
+                    my_pos = (uint32_t)(w_in_g * SEG_ELEMS + pch * 16 + 4 * (src & 3));
                     if (lane == 0) {
-                        reinterpret_cast<float *>(p.out_scales)[unit] =
-                            (wb == 0ull) ? 0.0f : (float)(__longlong_as_double((long long)wb) * p.inv_7_sqrt_b);
+                        wreq[nreq] = ((unsigned long long)unit << 32) | my_pos;
                         if (G > 1) {
-                            wpub[pidx] = wb;
+                            wpub[pidx] = (1ull << 63) | my_pos;
                             __threadfence_block();
                             *reinterpret_cast<volatile uint32_t *>(&wflag[pidx]) = it + 1u;
                         }
                     }
-                } else if (lane == 0) {
-                    atomicMax(&wacc[pidx], wb);
-                    __threadfence_block();
-                    if (atomicAdd(&wcnt[pidx], 1u) == (uint32_t)(ncand - 1)) {      // last candidate warp of the row
-                        const unsigned long long fin = atomicExch(&wacc[pidx], 0ull);
-                        wcnt[pidx] = 0u;
-                        reinterpret_cast<float *>(p.out_scales)[unit] =
-                            (fin == 0ull) ? 0.0f : (float)(__longlong_as_double((long long)fin) * p.inv_7_sqrt_b);
-                        wpub[pidx] = fin;
+                    if (++nreq == 32u) {
+                        serve_scale_requests<LOG2B>(p, wreq, nreq, G * SEG_ELEMS, lane);
+                        nreq = 0;
+                    }
+                } else {
+                    // several candidates: exact values now, combined over the candidate warps
+                    const unsigned long long wb = exact_max_of_candidates<LOG2B>(seg, ms, thr_row, lane);
+                    if (ncand == 1) {
+                        a_bits = wb;
+                        have_exact = true;
+                        if (lane == 0) {
+                            reinterpret_cast<float *>(p.out_scales)[unit] =
+                                (wb == 0ull) ? 0.0f : (float)(__longlong_as_double((long long)wb) * p.inv_7_sqrt_b);
+                            if (G > 1) {
+                                wpub[pidx] = wb;
+                                __threadfence_block();
+                                *reinterpret_cast<volatile uint32_t *>(&wflag[pidx]) = it + 1u;
+                            }
+                        }
+                    } else if (lane == 0) {
+                        atomicMax(&wacc[pidx], wb);
                         __threadfence_block();
-                        *reinterpret_cast<volatile uint32_t *>(&wflag[pidx]) = it + 1u;
+                        if (atomicAdd(&wcnt[pidx], 1u) == (uint32_t)(ncand - 1)) {      // last candidate warp of the row
+                            const unsigned long long fin = atomicExch(&wacc[pidx], 0ull);
+                            wcnt[pidx] = 0u;
+                            reinterpret_cast<float *>(p.out_scales)[unit] =
+                                (fin == 0ull) ? 0.0f : (float)(__longlong_as_double((long long)fin) * p.inv_7_sqrt_b);
+                            wpub[pidx] = fin;
+                            __threadfence_block();
+                            *reinterpret_cast<volatile uint32_t *>(&wflag[pidx]) = it + 1u;
+                        }
                     }
                 }
             }
 
             // ---- exact resolution of near ties (rare)
             if (__any_sync(0xffffffffu, tie_any != 0u)) {
-                if (!have_exact) {           // the row maximum comes from another warp: wait for its publication
-                    uint32_t spin = 0;
-                    while (ld_volatile_shared_u32(&wflag[pidx]) != it + 1u) {
-                        if (++spin >= WAIT_SPIN_LIMIT) {
-                            if (lane == 0) atomicOr(&g_perq_device_error, 2u);
-                            return;
+                if (!have_exact) {
+                    unsigned long long d = (1ull << 63) | my_pos;
+                    if (my_pos == 0xffffffffu) {      // published by a candidate warp of the row: wait for it
+                        uint32_t spin = 0;
+                        while (ld_volatile_shared_u32(&wflag[pidx]) != it + 1u) {
+                            if (++spin >= WAIT_SPIN_LIMIT) {
+                                if (lane == 0) atomicOr(&g_perq_device_error, 2u);
+                                return;
+                            }
                         }
+                        __threadfence_block();
+                        d = *reinterpret_cast<volatile unsigned long long *>(&wpub[pidx]);
                     }
-                    __threadfence_block();
-                    a_bits = *reinterpret_cast<volatile unsigned long long *>(&wpub[pidx]);
+                    if (d >> 63) {                    // a position: evaluate its four outputs from the staged row
+                        const uint32_t pos = (uint32_t)d & 0xffffu;
+                        const uint32_t blk = (pos >> LOG2B) << LOG2B;
+                        const uint16_t *rowp = seg - (size_t)w_in_g * SEG_ELEMS;
+                        const double val = fabs(exact_coord4<B>(rowp + blk, (int)(pos - blk), lane));
+                        a_bits = warp_max_u64((unsigned long long)__double_as_longlong(val));
+                    } else {
+                        a_bits = d;
+                    }
                 }
                 uint32_t fm = 0u;
                 if (tie_any != 0u) {
@@ -774,6 +870,7 @@ __global__ void __launch_bounds__(FAST_THREADS, 1) perq_fast_kernel(FastParams p
         __syncwarp();
         if (lane == 0) bulk_store(p.out_codes + seg_index * SEG_CODE_BYTES, code_buf, SEG_CODE_BYTES);
     }
+    if (MODE == MODE_TOKEN && nreq > 0u) serve_scale_requests<LOG2B>(p, wreq, nreq, G * SEG_ELEMS, lane);
     bulk_store_wait_read<0>();
 }
 
