@@ -733,127 +733,147 @@ __global__ void __launch_bounds__(FAST_THREADS, 1) perq_fast_kernel(FastParams p
                 }
             }
         } else {   // ---------------------------------------------------------------- MXFP4
-            float vf[8][4];
-#pragma unroll
-            for (int s = 0; s < 8; ++s) {
-                vf[s][0] = v[s][0].x; vf[s][1] = v[s][0].y;
-                vf[s][2] = v[s][1].x; vf[s][3] = v[s][1].y;
+            // A group of 32 = slots 2m, 2m+1 of the four lanes of a quad.  Lane q of the quad derives
+            // the shared exponent of slot pair m = q, then the quad exchanges multipliers.
+            float a32, bref;
+            {
+                const float g0 = fmaxf(ms[0], ms[1]), g1 = fmaxf(ms[2], ms[3]);
+                const float g2 = fmaxf(ms[4], ms[5]), g3 = fmaxf(ms[6], ms[7]);
+                const bool q1 = (q & 1) != 0, q2 = (q & 2) != 0;
+                float k0 = q2 ? g2 : g0, k1 = q2 ? g3 : g1;
+                const float s0 = q2 ? g0 : g2, s1 = q2 ? g1 : g3;
+                k0 = fmaxf(k0, __shfl_xor_sync(0xffffffffu, s0, 2));
+                k1 = fmaxf(k1, __shfl_xor_sync(0xffffffffu, s1, 2));
+                const float keep = q1 ? k1 : k0, send = q1 ? k0 : k1;
+                a32 = fmaxf(keep, __shfl_xor_sync(0xffffffffu, send, 1));
+                // error reference: the largest |u| of the Hadamard block (it may span several groups)
+                bref = a32;
+                if (CB >= 2) bref = fmaxf(bref, __shfl_xor_sync(0xffffffffu, bref, 1));
+                if (CB >= 3) bref = fmaxf(bref, __shfl_xor_sync(0xffffffffu, bref, 2));
             }
-            uint32_t tie_any = 0u;
-            int E_pack = 0;                      // E + 127 of the lane's four groups, one per byte
-            float cp_[4], cm_[4];
-            uint32_t word = 0u;
-#pragma unroll
-            for (int m = 0; m < 4; ++m) {
-                float a32 = fmaxf(ms[2 * m], ms[2 * m + 1]);
-                a32 = fmaxf(a32, __shfl_xor_sync(0xffffffffu, a32, 1));
-                a32 = fmaxf(a32, __shfl_xor_sync(0xffffffffu, a32, 2));
-                // error reference: the largest |u| of the Hadamard block (the group may be smaller than the block)
-                float bref = a32;
-                if (CB >= 2) {
-                    float bm = (CB == 2) ? fmaxf(fmaxf(ms[(2 * m) & 4], ms[((2 * m) & 4) + 1]), fmaxf(ms[((2 * m) & 4) + 2], ms[((2 * m) & 4) + 3]))
-                                         : fmaxf(fmaxf(fmaxf(ms[0], ms[1]), fmaxf(ms[2], ms[3])), fmaxf(fmaxf(ms[4], ms[5]), fmaxf(ms[6], ms[7])));
-                    bm = fmaxf(bm, __shfl_xor_sync(0xffffffffu, bm, 1));
-                    bm = fmaxf(bm, __shfl_xor_sync(0xffffffffu, bm, 2));
-                    bref = bm;
-                }
-                const float ratio = (a32 > 0.0f) ? bref / a32 : 1.0f;
-                const float rho = err_rel * ratio + 2.4e-7f;          // relative uncertainty of a32
-                // E = floor(log2(a / sqrt(b))) - 2 from the bits of a32; exact re-derivation near a boundary
-                const uint32_t bits = __float_as_uint(a32);
-                int eu = (int)(bits >> 23) - 127;
+            // E + 127 with E = floor(log2(a / sqrt(b))) - 2, from the bits of a32; near a boundary of
+            // that floor the maximum is re-derived exactly
+            const uint32_t bits = __float_as_uint(a32);
+            const int e8 = (int)(bits >> 23);
+            int Eb;
+            float dist;
+            if ((LOG2B & 1) == 0) {
+                Eb = e8 - LOG2B / 2 - 2;
+                const float lower = __uint_as_float(bits & 0x7f800000u);
+                dist = fminf(a32 - lower, 2.0f * lower - a32);
+            } else {
                 const uint32_t mant = bits & 0x7fffffu;
-                const float mrel = __uint_as_float(0x3f800000u | mant);          // [1, 2)
-                bool near;
-                int E;
-                if ((LOG2B & 1) == 0) {
-                    E = eu - LOG2B / 2 - 2;
-                    near = (mrel * (1.0f - rho) < 1.0f) || (mrel * (1.0f + rho) >= 2.0f);
-                } else {
-                    const float SQ2 = 1.41421356237f;
-                    E = eu - (LOG2B + 1) / 2 + (mant >= 0x3504f3u ? 1 : 0) - 2;
-                    near = (mrel * (1.0f - rho) < 1.0f) || (mrel * (1.0f + rho) >= 2.0f) || (fabsf(mrel - SQ2) <= rho * 2.0f);
-                }
-                if (a32 > 0.0f && (near || (bits >> 23) == 0u)) {
-                    // rare: exact maximum of the group from every element that could attain it
-                    const float thr = a32 - 2.0f * err_rel * bref - a32 * 2.4e-7f;
-                    const bool has = fmaxf(ms[2 * m], ms[2 * m + 1]) >= thr;
-                    unsigned cq = __ballot_sync(qmask, has) & qmask;
-                    double best = 0.0;
-                    while (cq) {
-                        const int src = __ffs(cq) - 1;
-                        cq &= cq - 1;
-                        uint32_t cm = 0u;
-                        if (lane == src) {
+                Eb = e8 - (LOG2B - 1) / 2 - 3 + (mant >= 0x3504f4u ? 1 : 0);
+                dist = fabsf(a32 - __uint_as_float((bits & 0x7f800000u) | 0x3504f3u));
+            }
+            const float tol = 2.0f * err_rel * bref + a32 * 2.4e-7f;
+            const bool near = (a32 > 0.0f) && (dist <= tol || e8 == 0);
+            const unsigned near_w = __ballot_sync(0xffffffffu, near);
+            if (near_w != 0u) {   // rare: exact maximum of the group from every element that could attain it
+                const unsigned nearq = (near_w >> (lane & 28)) & 0xFu;
 #pragma unroll
-                            for (int e = 0; e < 8; ++e) cm |= (fabsf(vf[2 * m + (e >> 2)][e & 3]) >= thr) ? (1u << e) : 0u;
+                for (int m = 0; m < 4; ++m) {
+                    if ((nearq >> m) & 1u) {
+                        const int owner = (lane & 28) | m;
+                        const float a_m = __shfl_sync(qmask, a32, owner), tol_m = __shfl_sync(qmask, tol, owner);
+                        const float thr = a_m - tol_m;
+                        const bool has = fmaxf(ms[2 * m], ms[2 * m + 1]) >= thr;
+                        unsigned cq = __ballot_sync(qmask, has) & qmask;
+                        double best = 0.0;
+                        while (cq) {
+                            const int src = __ffs(cq) - 1;
+                            cq &= cq - 1;
+                            uint32_t cm = 0u;
+                            if (lane == src) {
+                                const float e[8] = {v[2 * m][0].x, v[2 * m][0].y, v[2 * m][1].x, v[2 * m][1].y,
+                                                    v[2 * m + 1][0].x, v[2 * m + 1][0].y, v[2 * m + 1][1].x, v[2 * m + 1][1].y};
+#pragma unroll
+                                for (int k = 0; k < 8; ++k) cm |= (fabsf(e[k]) >= thr) ? (1u << k) : 0u;
+                            }
+                            cm = __shfl_sync(qmask, cm, src);
+                            while (cm) {
+                                const int k = __ffs(cm) - 1;
+                                cm &= cm - 1;
+                                int blk_elem, i, elem;
+                                locate<LOG2B>(src >> 2, src & 3, 8 * m + k, blk_elem, i, elem);
+                                best = fmax(best, fabs(exact_coord_quad<LOG2B>(seg + blk_elem, i, q, qmask)));
+                            }
                         }
-                        cm = __shfl_sync(qmask, cm, src);
-                        while (cm) {
-                            const int e = __ffs(cm) - 1;
-                            cm &= cm - 1;
-                            int blk_elem, i, elem;
-                            locate<LOG2B>(src >> 2, src & 3, 8 * m + e, blk_elem, i, elem);
-                            best = fmax(best, fabs(exact_coord_quad<LOG2B>(seg + blk_elem, i, q, qmask)));
+                        if (q == m) {
+                            int ex;
+                            (void)frexp(best / p.sqrt_b, &ex);
+                            Eb = ex - 3 + 127;
                         }
                     }
-                    int ex;
-                    (void)frexp(best / p.sqrt_b, &ex);
-                    E = ex - 3;
                 }
-                E = min(max(E, -127), 127);
-                const uint32_t byte = (a32 > 0.0f) ? (uint32_t)(E + 127) : 0u;
-                E_pack |= (int)(byte << (8 * m));
-                // multiplier 2^-E / sqrt(b)
-                float c;
-                if ((LOG2B & 1) == 0) c = __uint_as_float((uint32_t)min(max(127 - E - LOG2B / 2, 1), 254) << 23);
-                else c = __uint_as_float(0x3fb504f3u + ((uint32_t)(min(max(127 - E - (LOG2B + 1) / 2, 1), 253) - 127) << 23));
-                if (!(a32 > 0.0f)) c = 0.0f;
-                const float delta = 32.0f * err_rel * ratio + 5.0e-7f;
-                cp_[m] = c * (1.0f + delta);
-                cm_[m] = c * (1.0f - delta);
-                // scale byte position: group index inside the lane group's four groups
-                word |= byte << (8 * (m ^ ((f_g & ~PM) >> 1)));
             }
+            Eb = min(max(Eb, 0), 254);
+            // multiplier 2^-E / sqrt(b) and the additive rounding window, in scaled units
+            float c;
+            if ((LOG2B & 1) == 0) c = __uint_as_float((uint32_t)min(max(254 - Eb - LOG2B / 2, 1), 254) << 23);
+            else c = __uint_as_float((uint32_t)min(max(254 - Eb - (LOG2B - 1) / 2, 1), 254) << 23) * 0.70710678118654752f;
+            uint32_t byte = (uint32_t)Eb;
+            if (!(a32 > 0.0f)) { c = 0.0f; byte = 0u; }
+            const float tau = 2.0f * err_rel * bref * c + 2.0e-6f;
+            // scale bytes of the quad's four groups: slot pair m is chunk pair m ^ (f >> 1)
+            uint32_t word = byte << (8 * (q ^ ((f_g & ~PM) >> 1)));
+            word |= __shfl_xor_sync(0xffffffffu, word, 1);
+            word |= __shfl_xor_sync(0xffffffffu, word, 2);
             if (q == 0) reinterpret_cast<uint32_t *>(p.out_scales)[seg_index * 8 + g] = word;
+
+            uint32_t tie_any = 0u;
+            f32x2 mulc[8], tau2[4];
+#pragma unroll
+            for (int m = 0; m < 4; ++m) {
+                const float c_m = __shfl_sync(0xffffffffu, c, (lane & 28) | m);
+                const float t_m = __shfl_sync(0xffffffffu, tau, (lane & 28) | m);
+                tau2[m] = pack2(t_m, t_m);
+#pragma unroll
+                for (int h = 0; h < 2; ++h) {
+                    const float mc = sgn[(2 * m + h) & 3 & PM] * c_m;
+                    mulc[2 * m + h] = pack2(mc, mc);
+                }
+            }
 #pragma unroll
             for (int s = 0; s < 8; ++s) {
-                const float sg = sgn[s & 3 & PM];
-                const float kp = sg * cp_[s >> 1], km = sg * cm_[s >> 1];
-                const uint32_t p0 = cvt_e2m1x2(fmaf(vf[s][0], kp, 0.0f), fmaf(vf[s][1], kp, 0.0f));
-                const uint32_t p1 = cvt_e2m1x2(fmaf(vf[s][2], kp, 0.0f), fmaf(vf[s][3], kp, 0.0f));
-                const uint32_t m0 = cvt_e2m1x2(fmaf(vf[s][0], km, 0.0f), fmaf(vf[s][1], km, 0.0f));
-                const uint32_t m1 = cvt_e2m1x2(fmaf(vf[s][2], km, 0.0f), fmaf(vf[s][3], km, 0.0f));
+                const f32x2 tneg = pack2(-tau2[s >> 1].x, -tau2[s >> 1].y);
+                const f32x2 up0 = fma2(v[s][0], mulc[s], tau2[s >> 1]), up1 = fma2(v[s][1], mulc[s], tau2[s >> 1]);
+                const f32x2 dn0 = fma2(v[s][0], mulc[s], tneg), dn1 = fma2(v[s][1], mulc[s], tneg);
+                const uint32_t p0 = cvt_e2m1x2(up0.x, up0.y), p1 = cvt_e2m1x2(up1.x, up1.y);
+                const uint32_t m0 = cvt_e2m1x2(dn0.x, dn0.y), m1 = cvt_e2m1x2(dn1.x, dn1.y);
                 tie_any |= (p0 ^ m0) | (p1 ^ m1);
                 sts_u16(code_addr0 ^ (uint32_t)(s * 8), p0 | (p1 << 8));
             }
             if (__any_sync(0xffffffffu, tie_any != 0u)) {
+                uint32_t fm = 0u;
+                if (tie_any != 0u) {
+#pragma unroll
+                    for (int s = 0; s < 8; ++s) {
+                        const f32x2 tneg = pack2(-tau2[s >> 1].x, -tau2[s >> 1].y);
+                        const f32x2 up0 = fma2(v[s][0], mulc[s], tau2[s >> 1]), up1 = fma2(v[s][1], mulc[s], tau2[s >> 1]);
+                        const f32x2 dn0 = fma2(v[s][0], mulc[s], tneg), dn1 = fma2(v[s][1], mulc[s], tneg);
+                        const uint32_t x0 = cvt_e2m1x2(up0.x, up0.y) ^ cvt_e2m1x2(dn0.x, dn0.y);
+                        const uint32_t x1 = cvt_e2m1x2(up1.x, up1.y) ^ cvt_e2m1x2(dn1.x, dn1.y);
+                        fm |= ((x0 & 0x0Fu) ? 1u : 0u) << (4 * s) | ((x0 & 0xF0u) ? 2u : 0u) << (4 * s);
+                        fm |= ((x1 & 0x0Fu) ? 4u : 0u) << (4 * s) | ((x1 & 0xF0u) ? 8u : 0u) << (4 * s);
+                    }
+                }
                 __syncwarp();
-                unsigned tl = __ballot_sync(0xffffffffu, tie_any != 0u);
+                unsigned tl = __ballot_sync(0xffffffffu, fm != 0u);
                 while (tl) {
                     const int src = __ffs(tl) - 1;
                     tl &= tl - 1;
-                    uint32_t fm = 0u;
-#pragma unroll
-                    for (int e = 0; e < 32; e += 2) {
-                        const int s = e >> 2;
-                        const float sg = sgn[s & 3 & PM];
-                        const float kp = sg * cp_[s >> 1], km = sg * cm_[s >> 1];
-                        const uint32_t pp = cvt_e2m1x2(fmaf(vf[s][e & 3], kp, 0.0f), fmaf(vf[s][(e & 3) + 1], kp, 0.0f));
-                        const uint32_t mm = cvt_e2m1x2(fmaf(vf[s][e & 3], km, 0.0f), fmaf(vf[s][(e & 3) + 1], km, 0.0f));
-                        const uint32_t x = pp ^ mm;
-                        fm |= ((x & 0x0Fu) ? (1u << e) : 0u) | ((x & 0xF0u) ? (2u << e) : 0u);
-                    }
-                    fm = __shfl_sync(0xffffffffu, fm, src);
-                    const int Ep = __shfl_sync(0xffffffffu, E_pack, src);
-                    while (fm) {
-                        const int e = __ffs(fm) - 1;
-                        fm &= fm - 1;
+                    uint32_t fs = __shfl_sync(0xffffffffu, fm, src);
+                    const uint32_t wsrc = __shfl_sync(0xffffffffu, word, src);
+                    const int fsrc = (((src >> 2) & 3) & ~PM) >> 1;
+                    while (fs) {
+                        const int e = __ffs(fs) - 1;
+                        fs &= fs - 1;
                         int blk_elem, i, elem;
                         locate<LOG2B>(src >> 2, src & 3, e, blk_elem, i, elem);
                         const double ue = exact_coord_fast<B>(seg + blk_elem, i, lane);
                         if (lane == 0) {
-                            const int E = ((Ep >> (8 * (e >> 3))) & 0xFF) - 127;
+                            const int E = (int)((wsrc >> (8 * ((e >> 3) ^ fsrc))) & 0xFFu) - 127;
                             const double y = ue / p.sqrt_b;
                             const uint32_t code = e2m1_code_exact(scalbn(y, -E), signbit(y));
                             uint8_t *bp = code_gen + (elem >> 1);
