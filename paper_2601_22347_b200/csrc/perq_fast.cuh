@@ -167,6 +167,15 @@ __device__ __forceinline__ unsigned long long warp_max_u64(unsigned long long v)
 }
 __device__ __forceinline__ float max3abs(float acc, float a, float b) { return fmaxf(fmaxf(acc, fabsf(a)), fabsf(b)); }
 
+// Four fp32 values -> 16 bits of four E2M1 codes (first operand in the lowest nibble), RNE, saturating.
+__device__ __forceinline__ uint32_t cvt_e2m1x4(float a, float b, float c, float d)
+{
+    uint32_t r;
+    asm("{ .reg .b8 t0, t1; .reg .b16 h; cvt.rn.satfinite.e2m1x2.f32 t0, %2, %1; cvt.rn.satfinite.e2m1x2.f32 t1, %4, %3; "
+        "mov.b16 h, {t0, t1}; cvt.u32.u16 %0, h; }" : "=r"(r) : "f"(a), "f"(b), "f"(c), "f"(d));
+    return r;
+}
+
 __device__ __forceinline__ uint32_t hadamard_bf16(int k, int n) { return (__popc(k & n) & 1) ? 0xBF80u : 0x3F80u; }
 
 // ---------------------------------------------------------------- exact re-evaluation
@@ -822,12 +831,13 @@ __global__ void __launch_bounds__(FAST_THREADS, 1) perq_fast_kernel(FastParams p
             if (q == 0) reinterpret_cast<uint32_t *>(p.out_scales)[seg_index * 8 + g] = word;
 
             uint32_t tie_any = 0u;
-            f32x2 mulc[8], tau2[4];
+            f32x2 mulc[8], tau_p[4], tau_m[4];
 #pragma unroll
             for (int m = 0; m < 4; ++m) {
                 const float c_m = __shfl_sync(0xffffffffu, c, (lane & 28) | m);
                 const float t_m = __shfl_sync(0xffffffffu, tau, (lane & 28) | m);
-                tau2[m] = pack2(t_m, t_m);
+                tau_p[m] = pack2(t_m, t_m);
+                tau_m[m] = pack2(-t_m, -t_m);
 #pragma unroll
                 for (int h = 0; h < 2; ++h) {
                     const float mc = sgn[(2 * m + h) & 3 & PM] * c_m;
@@ -836,22 +846,20 @@ __global__ void __launch_bounds__(FAST_THREADS, 1) perq_fast_kernel(FastParams p
             }
 #pragma unroll
             for (int s = 0; s < 8; ++s) {
-                const f32x2 tneg = pack2(-tau2[s >> 1].x, -tau2[s >> 1].y);
-                const f32x2 up0 = fma2(v[s][0], mulc[s], tau2[s >> 1]), up1 = fma2(v[s][1], mulc[s], tau2[s >> 1]);
-                const f32x2 dn0 = fma2(v[s][0], mulc[s], tneg), dn1 = fma2(v[s][1], mulc[s], tneg);
-                const uint32_t p0 = cvt_e2m1x2(up0.x, up0.y), p1 = cvt_e2m1x2(up1.x, up1.y);
-                const uint32_t m0 = cvt_e2m1x2(dn0.x, dn0.y), m1 = cvt_e2m1x2(dn1.x, dn1.y);
-                tie_any |= (p0 ^ m0) | (p1 ^ m1);
-                sts_u16(code_addr0 ^ (uint32_t)(s * 8), p0 | (p1 << 8));
+                const f32x2 up0 = fma2(v[s][0], mulc[s], tau_p[s >> 1]), up1 = fma2(v[s][1], mulc[s], tau_p[s >> 1]);
+                const f32x2 dn0 = fma2(v[s][0], mulc[s], tau_m[s >> 1]), dn1 = fma2(v[s][1], mulc[s], tau_m[s >> 1]);
+                const uint32_t pu = cvt_e2m1x4(up0.x, up0.y, up1.x, up1.y);
+                const uint32_t pd = cvt_e2m1x4(dn0.x, dn0.y, dn1.x, dn1.y);
+                tie_any |= pu ^ pd;
+                sts_u16(code_addr0 ^ (uint32_t)(s * 8), pu);
             }
             if (__any_sync(0xffffffffu, tie_any != 0u)) {
                 uint32_t fm = 0u;
                 if (tie_any != 0u) {
 #pragma unroll
                     for (int s = 0; s < 8; ++s) {
-                        const f32x2 tneg = pack2(-tau2[s >> 1].x, -tau2[s >> 1].y);
-                        const f32x2 up0 = fma2(v[s][0], mulc[s], tau2[s >> 1]), up1 = fma2(v[s][1], mulc[s], tau2[s >> 1]);
-                        const f32x2 dn0 = fma2(v[s][0], mulc[s], tneg), dn1 = fma2(v[s][1], mulc[s], tneg);
+                        const f32x2 up0 = fma2(v[s][0], mulc[s], tau_p[s >> 1]), up1 = fma2(v[s][1], mulc[s], tau_p[s >> 1]);
+                        const f32x2 dn0 = fma2(v[s][0], mulc[s], tau_m[s >> 1]), dn1 = fma2(v[s][1], mulc[s], tau_m[s >> 1]);
                         const uint32_t x0 = cvt_e2m1x2(up0.x, up0.y) ^ cvt_e2m1x2(dn0.x, dn0.y);
                         const uint32_t x1 = cvt_e2m1x2(up1.x, up1.y) ^ cvt_e2m1x2(dn1.x, dn1.y);
                         fm |= ((x0 & 0x0Fu) ? 1u : 0u) << (4 * s) | ((x0 & 0xF0u) ? 2u : 0u) << (4 * s);
