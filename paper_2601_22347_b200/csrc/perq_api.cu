@@ -98,51 +98,72 @@ int launch_generic(const void *x, const int32_t *perm, int64_t T, int32_t d, int
     return cudaGetLastError() == cudaSuccess ? PERQ_OK : PERQ_ERR_CUDA;
 }
 
-template <int LOG2B, int MODE, int LOG2G>
+template <int LOG2B, int MODE, int LOG2G, bool PERM>
 int launch_fast_inst(const perq::FastParams &p, int grid, cudaStream_t st)
 {
-    auto kernel = perq::perq_fast_kernel<LOG2B, MODE, LOG2G>;
-    if (int rc = allow_smem(kernel, perq::FastSmem::total)) return rc;
-    kernel<<<grid, perq::FAST_THREADS, perq::FastSmem::total, st>>>(p);
+    auto kernel = perq::perq_fast_kernel<LOG2B, MODE, LOG2G, PERM>;
+    const size_t smem = PERM ? perq::FastSmem::total_perm : perq::FastSmem::total;
+    if (int rc = allow_smem(kernel, smem)) return rc;
+    kernel<<<grid, perq::FAST_THREADS, smem, st>>>(p);
     return cudaGetLastError() == cudaSuccess ? PERQ_OK : PERQ_ERR_CUDA;
 }
 
-template <int MODE, int LOG2G>
-int launch_fast_mode(int log2b, const perq::FastParams &p, int grid, cudaStream_t st)
+template <int MODE, int LOG2G, bool PERM>
+int launch_fast_b(int log2b, const perq::FastParams &p, int grid, cudaStream_t st)
 {
     switch (log2b) {
-    case 4: return launch_fast_inst<4, MODE, LOG2G>(p, grid, st);
-    case 5: return launch_fast_inst<5, MODE, LOG2G>(p, grid, st);
-    case 6: return launch_fast_inst<6, MODE, LOG2G>(p, grid, st);
-    default: return launch_fast_inst<7, MODE, LOG2G>(p, grid, st);
+    case 4: return launch_fast_inst<4, MODE, LOG2G, PERM>(p, grid, st);
+    case 5: return launch_fast_inst<5, MODE, LOG2G, PERM>(p, grid, st);
+    case 6: return launch_fast_inst<6, MODE, LOG2G, PERM>(p, grid, st);
+    default: return launch_fast_inst<7, MODE, LOG2G, PERM>(p, grid, st);
     }
 }
 
-// The fast kernel covers: no permutation, b <= 128, d % 1024 == 0, and scales per token
-// (d / 1024 in {1,2,4,8}), per 128 (INT4) or per 32 (MXFP4).  Returns -1 if it does not apply.
+template <bool PERM>
+int launch_fast_mode(int mode, int G, int log2b, const perq::FastParams &p, int grid, cudaStream_t st)
+{
+    if (mode == perq::MODE_MX) return launch_fast_b<perq::MODE_MX, 0, PERM>(log2b, p, grid, st);
+    if (mode == perq::MODE_G128) return launch_fast_b<perq::MODE_G128, 0, PERM>(log2b, p, grid, st);
+    switch (G) {
+    case 1: return launch_fast_b<perq::MODE_TOKEN, 0, PERM>(log2b, p, grid, st);
+    case 2: return launch_fast_b<perq::MODE_TOKEN, 1, PERM>(log2b, p, grid, st);
+    case 4: return launch_fast_b<perq::MODE_TOKEN, 2, PERM>(log2b, p, grid, st);
+    default: return launch_fast_b<perq::MODE_TOKEN, 3, PERM>(log2b, p, grid, st);
+    }
+}
+
+// The fast kernel covers b <= 128, d % 1024 == 0, and scales per token (d / 1024 in {1,2,4,8}),
+// per 128 (INT4) or per 32 (MXFP4); with a permutation also d <= 16384.  Returns -1 if it does not apply.
 int try_launch_fast(const void *x, const int32_t *perm, int64_t T, int32_t d, int32_t b, int32_t fmt, int g,
                     void *out_codes, void *out_scales, cudaStream_t st)
 {
-    if (perm != nullptr || b > 128 || d % perq::SEG_ELEMS != 0) return -1;
+    if (b > 128 || d % perq::SEG_ELEMS != 0) return -1;
+    const int segs = d / perq::SEG_ELEMS;
+    const bool permuted = perm != nullptr;
+    if (permuted && (d > perq::FastSmem::PERM_MAX_D || segs > perq::FAST_WARPS)) return -1;
     int mode, G = 1;
     if (fmt == PERQ_FMT_MXFP4) {
         mode = perq::MODE_MX;
     } else if (fmt == PERQ_FMT_INT4 && g == 128) {
         mode = perq::MODE_G128;
     } else if (fmt == PERQ_FMT_INT4 && g == d) {
-        G = d / perq::SEG_ELEMS;
+        G = segs;
         if (G != 1 && G != 2 && G != 4 && G != 8) return -1;
         mode = perq::MODE_TOKEN;
     } else {
         return -1;
     }
-    const long long units = (long long)T * (d / perq::SEG_ELEMS) / G;
+    if (permuted) G = segs;          // a permuted unit is a whole row
+    const long long units = (long long)T * segs / G;
     if (units >= (1ll << 31)) return -1;
     perq::FastParams p;
     p.x = static_cast<const uint16_t *>(x);
     p.out_codes = static_cast<uint8_t *>(out_codes);
     p.out_scales = out_scales;
     p.units_total = (uint32_t)units;
+    p.perm = perm;
+    p.G = G;
+    p.d = d;
     p.sqrt_b = std::sqrt((double)b);
     p.inv_7_sqrt_b = 1.0 / (7.0 * p.sqrt_b);
     const int sms = sm_count();
@@ -151,14 +172,8 @@ int try_launch_fast(const void *x, const int32_t *perm, int64_t T, int32_t d, in
     const long long want = (units + groups_per_cta - 1) / groups_per_cta;
     const int grid = (int)std::min<long long>(want, sms);
     const int log2b = ilog2(b);
-    if (mode == perq::MODE_MX) return launch_fast_mode<perq::MODE_MX, 0>(log2b, p, grid, st);
-    if (mode == perq::MODE_G128) return launch_fast_mode<perq::MODE_G128, 0>(log2b, p, grid, st);
-    switch (G) {
-    case 1: return launch_fast_mode<perq::MODE_TOKEN, 0>(log2b, p, grid, st);
-    case 2: return launch_fast_mode<perq::MODE_TOKEN, 1>(log2b, p, grid, st);
-    case 4: return launch_fast_mode<perq::MODE_TOKEN, 2>(log2b, p, grid, st);
-    default: return launch_fast_mode<perq::MODE_TOKEN, 3>(log2b, p, grid, st);
-    }
+    return permuted ? launch_fast_mode<true>(mode, G, log2b, p, grid, st)
+                    : launch_fast_mode<false>(mode, G, log2b, p, grid, st);
 }
 
 int launch_any(const void *x, const int32_t *perm, int64_t T, int32_t d, int32_t b, int32_t fmt, int g,

@@ -54,7 +54,10 @@ struct FastParams {
     const uint16_t *x;
     uint8_t *out_codes;
     void *out_scales;
-    uint32_t units_total;    // units of G = 2^LOG2G segments (fewer than 2^31)
+    uint32_t units_total;    // units of G segments (fewer than 2^31); rows when G = d / 1024
+    const int32_t *perm;     // permuted variants only: perm[d] (device)
+    int G;                   // permuted variants: segments per row
+    int d;
     double sqrt_b;
     double inv_7_sqrt_b;     // 1 / (7 sqrt(b)): INT4 scale = exact |u|max times this
 };
@@ -73,8 +76,15 @@ struct FastSmem {
     static constexpr size_t wcnt = wmax + (size_t)FAST_WARPS * 2 * 4;               // [2][FAST_WARPS] u32 arrival counts
     static constexpr size_t wflag = wcnt + (size_t)FAST_WARPS * 2 * 4;              // [2][FAST_WARPS] u32 publication flags
     static constexpr size_t wreq = wflag + (size_t)FAST_WARPS * 2 * 4;              // [FAST_WARPS][32] u64 deferred scale requests
-    static constexpr size_t used = wreq + (size_t)FAST_WARPS * 32 * 8;
+    static constexpr size_t empty = wreq + (size_t)FAST_WARPS * 32 * 8;             // [FAST_WARPS * FAST_NSTAGE] mbarriers
+    static constexpr size_t used = empty + (size_t)FAST_WARPS * FAST_NSTAGE * 8;
     static constexpr size_t total = used + 1024;                                    // room to align the base
+    // permuted variants: the stage area holds 3 raw-row stages per group (96 KB in all) followed by
+    // one permuted 2 KB segment per warp; the permutation (as 16-bit byte offsets) follows `used`
+    static constexpr size_t pbuf = stages + (size_t)FAST_WARPS * 3 * SEG_BYTES;
+    static constexpr size_t perm_tab = used;
+    static constexpr int PERM_MAX_D = 16384;
+    static constexpr size_t total_perm = used + (size_t)PERM_MAX_D * 2 + 1024;
 };
 
 // ---------------------------------------------------------------- PTX wrappers
@@ -99,6 +109,10 @@ __device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity)
         if (done) return true;
     }
     return false;
+}
+__device__ __forceinline__ void mbar_arrive(uint32_t bar)
+{
+    asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];" ::"r"(bar) : "memory");
 }
 __device__ __forceinline__ void bulk_load(uint32_t dst, const void *src, uint32_t bytes, uint32_t bar)
 {
@@ -136,6 +150,16 @@ __device__ __forceinline__ void named_barrier(int id, int threads)
 __device__ __forceinline__ void sts_u16(uint32_t addr, uint32_t v)
 {
     asm volatile("st.shared.u16 [%0], %1;" ::"r"(addr), "h"((uint16_t)v) : "memory");
+}
+__device__ __forceinline__ uint32_t lds_u16(uint32_t addr)
+{
+    uint16_t v;
+    asm volatile("ld.shared.u16 %0, [%1];" : "=h"(v) : "r"(addr));
+    return v;
+}
+__device__ __forceinline__ void sts_v4(uint32_t addr, uint32_t a, uint32_t b, uint32_t c, uint32_t d)
+{
+    asm volatile("st.shared.v4.b32 [%0], {%1, %2, %3, %4};" ::"r"(addr), "r"(a), "r"(b), "r"(c), "r"(d) : "memory");
 }
 __device__ __forceinline__ uint32_t ld_volatile_shared_u32(const uint32_t *p)
 {
@@ -261,6 +285,31 @@ __device__ __forceinline__ double exact_coord4(const uint16_t *blk, int i0, int 
     return acc;
 }
 
+// The same for a permuted row: term k of the block is raw[off[k] / 2], with off the 16-bit byte
+// offsets of the permutation, already advanced to the block's first position.
+template <int B>
+__device__ __forceinline__ double exact_coord4_perm(const uint16_t *raw, const uint16_t *off, int i0, int lane)
+{
+    double acc = 0.0;
+#pragma unroll
+    for (int k0 = 0; k0 < B; k0 += 32) {
+        const int k = k0 + lane;
+        if (B >= 32 || k < B) {
+            const double v = bf16_bits_to_f64(raw[off[k] >> 1]);
+            acc += (__popc(i0 & k) & 1) ? -v : v;
+        }
+    }
+    acc += __shfl_xor_sync(0xffffffffu, acc, 4);
+    acc += __shfl_xor_sync(0xffffffffu, acc, 8);
+    acc += __shfl_xor_sync(0xffffffffu, acc, 16);
+#pragma unroll
+    for (int bit = 1; bit <= 2; bit <<= 1) {
+        const double other = __shfl_xor_sync(0xffffffffu, acc, bit);
+        acc = (lane & bit) ? other - acc : acc + other;
+    }
+    return acc;
+}
+
 // Element e = s*4 + j of lane (g, q): block start (in elements, segment relative) and index inside the block.
 template <int LOG2B>
 __device__ __forceinline__ void locate(int g, int q, int e, int &blk_elem, int &i, int &elem)
@@ -334,8 +383,8 @@ __device__ __forceinline__ unsigned long long exact_max_of_candidates(const uint
 //
 // Record: bits 63..32 = row, bits 15..0 = element index in the row of the slot's first output.
 
-template <int LOG2B>
-__device__ __forceinline__ double exact_slot_max_global(const uint16_t *row, uint32_t pos)
+template <int LOG2B, bool PERM>
+__device__ __forceinline__ double exact_slot_max_global(const uint16_t *row, uint32_t pos, const int32_t *perm, int d)
 {
     constexpr int B = 1 << LOG2B;
     const uint32_t blk = (pos >> LOG2B) << LOG2B;
@@ -344,8 +393,18 @@ __device__ __forceinline__ double exact_slot_max_global(const uint16_t *row, uin
     double S[4] = {0.0, 0.0, 0.0, 0.0};                  // sums of the terms with k & 3 == m, signed by the high bits of i0
 #pragma unroll
     for (int c = 0; c < B / 8; ++c) {
-        const uint4 w4 = __ldg(src + c);
-        const uint32_t w[4] = {w4.x, w4.y, w4.z, w4.w};
+        uint32_t w[4];
+        if (PERM) {
+#pragma unroll
+            for (int e = 0; e < 4; ++e) {
+                const int s0 = min(max(__ldg(perm + blk + 8 * c + 2 * e), 0), d - 1);
+                const int s1 = min(max(__ldg(perm + blk + 8 * c + 2 * e + 1), 0), d - 1);
+                w[e] = (uint32_t)__ldg(row + s0) | ((uint32_t)__ldg(row + s1) << 16);
+            }
+        } else {
+            const uint4 w4 = __ldg(src + c);
+            w[0] = w4.x; w[1] = w4.y; w[2] = w4.z; w[3] = w4.w;
+        }
 #pragma unroll
         for (int h = 0; h < 2; ++h) {
             const bool neg = __popc(i0 & (uint32_t)(8 * c + 4 * h)) & 1;
@@ -361,7 +420,7 @@ __device__ __forceinline__ double exact_slot_max_global(const uint16_t *row, uin
     return fmax(fmax(fabs(a0 + a2), fabs(a1 + a3)), fmax(fabs(a0 - a2), fabs(a1 - a3)));
 }
 
-template <int LOG2B>
+template <int LOG2B, bool PERM>
 __device__ __forceinline__ void serve_scale_requests(const FastParams &p, const unsigned long long *req, uint32_t n,
                                                      uint32_t row_elems, int lane)
 {
@@ -369,7 +428,7 @@ __device__ __forceinline__ void serve_scale_requests(const FastParams &p, const 
     if ((uint32_t)lane < n) {
         const unsigned long long r = req[lane];
         const uint32_t unit = (uint32_t)(r >> 32), pos = (uint32_t)r & 0xffffu;
-        const double a = exact_slot_max_global<LOG2B>(p.x + (size_t)unit * row_elems, pos);
+        const double a = exact_slot_max_global<LOG2B, PERM>(p.x + (size_t)unit * row_elems, pos, p.perm, p.d);
         reinterpret_cast<float *>(p.out_scales)[unit] = (a == 0.0) ? 0.0f : (float)(a * p.inv_7_sqrt_b);
     }
     __syncwarp();
@@ -377,16 +436,18 @@ __device__ __forceinline__ void serve_scale_requests(const FastParams &p, const 
 
 // ---------------------------------------------------------------- the kernel
 
-template <int LOG2B, int MODE, int LOG2G>
+template <int LOG2B, int MODE, int LOG2G, bool PERM>
 __global__ void __launch_bounds__(FAST_THREADS, 1) perq_fast_kernel(FastParams p)
 {
     constexpr int B = 1 << LOG2B;
     constexpr int CB = LOG2B - 4;                 // butterfly stages left after the tensor-core H_16
     constexpr int PM = (1 << CB) - 1;             // slot bits inside a Hadamard block
     constexpr int NCLS = (PM & 3) + 1;            // sign classes of the slot relabelling
-    constexpr int G = 1 << LOG2G;                 // warps (segments) per unit
-    constexpr int GROUPS = FAST_WARPS / G;
-    constexpr uint32_t UNIT_BYTES = (uint32_t)G * SEG_BYTES;
+    constexpr bool RUNTIME_G = PERM && MODE != MODE_TOKEN;     // a permuted unit is a whole row of any length
+    constexpr int NST = PERM ? 3 : FAST_NSTAGE;
+    const int G = RUNTIME_G ? p.G : (1 << LOG2G);               // warps (segments) per unit
+    const int GROUPS = FAST_WARPS / G;
+    const uint32_t UNIT_BYTES = (uint32_t)G * SEG_BYTES;
     constexpr float MAGIC = 12582920.0f;          // 1.5 * 2^23 + 8: low nibble of the sum = code + 8
     static_assert(MODE == MODE_TOKEN || LOG2G == 0, "only per-token scales couple the warps of a row");
     extern __shared__ __align__(128) unsigned char fsmem_raw[];
@@ -395,11 +456,15 @@ __global__ void __launch_bounds__(FAST_THREADS, 1) perq_fast_kernel(FastParams p
 
     const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
     const int g = lane >> 2, q = lane & 3;
-    const int group = warp >> LOG2G, w_in_g = warp & (G - 1);
+    const int group = RUNTIME_G ? warp / G : warp >> LOG2G;
+    const int w_in_g = warp - group * G;
     const unsigned qmask = 0xFu << (lane & 28);
     const float err_rel = FAST_ERR_K * (float)LOG2B * TWO_M24;
 
-    const uint32_t stage_base = smem_u32(fsmem + FastSmem::stages) + (uint32_t)group * (FAST_NSTAGE * UNIT_BYTES);
+    const uint32_t stage_base = smem_u32(fsmem + FastSmem::stages) + (uint32_t)group * (NST * UNIT_BYTES);
+    const uint32_t empty_base = smem_u32(fsmem + FastSmem::empty) + (uint32_t)group * (FAST_NSTAGE * 8);
+    const uint32_t pbuf_addr = smem_u32(fsmem + FastSmem::pbuf) + (uint32_t)warp * SEG_BYTES;
+    const uint16_t *ptab = reinterpret_cast<const uint16_t *>(fsmem + FastSmem::perm_tab);
     const uint32_t code_base = smem_u32(fsmem + FastSmem::codes) + (uint32_t)warp * (2 * SEG_CODE_BYTES);
     const uint32_t full_base = smem_u32(fsmem + FastSmem::full) + (uint32_t)group * (FAST_NSTAGE * 8);
     unsigned long long *wacc = reinterpret_cast<unsigned long long *>(fsmem + FastSmem::wacc);
@@ -411,14 +476,21 @@ __global__ void __launch_bounds__(FAST_THREADS, 1) perq_fast_kernel(FastParams p
     uint32_t nreq = 0;                       // records waiting in wreq (the same in every lane)
     const bool leader = (w_in_g == 0) && (lane == 0);
 
-    if (tid < FAST_WARPS * FAST_NSTAGE) mbar_init(smem_u32(fsmem + FastSmem::full) + tid * 8, 1);
+    if (tid < FAST_WARPS * FAST_NSTAGE) {
+        mbar_init(smem_u32(fsmem + FastSmem::full) + tid * 8, 1);
+        if (PERM) mbar_init(smem_u32(fsmem + FastSmem::empty) + tid * 8, (uint32_t)G);
+    }
+    if (PERM) {     // the permutation as byte offsets into a staged row; out-of-range entries are clamped
+        uint16_t *pt = reinterpret_cast<uint16_t *>(fsmem + FastSmem::perm_tab);
+        for (int i = tid; i < p.d; i += FAST_THREADS) pt[i] = (uint16_t)(2 * min(max(__ldg(p.perm + i), 0), p.d - 1));
+    }
     if (tid < 2 * FAST_WARPS) { wacc[tid] = 0ull; wcnt[tid] = 0u; wflag[tid] = 0u; }
     if (tid == 0) asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
     __syncthreads();
 
     const uint32_t first = blockIdx.x * GROUPS + group;
     const uint32_t stride = gridDim.x * GROUPS;
-    if (first >= p.units_total) return;      // whole groups leave together (no barrier is shared across groups)
+    if (group >= GROUPS || first >= p.units_total) return;   // whole groups leave together (no barrier is shared across groups)
 
     // Hadamard operand of the tensor-core stage: column n of MMA m is output 4*(n/2) + (n%2) + 2m.
     uint32_t hb[2][2];
@@ -447,11 +519,11 @@ __global__ void __launch_bounds__(FAST_THREADS, 1) perq_fast_kernel(FastParams p
 #pragma unroll
     for (int k = 0; k < NCLS; ++k) sgn[k] = (__popc(k & f_g & PM) & 1) ? -half_sign : half_sign;
 
-    const uint16_t *xin = p.x + (size_t)w_in_g * 0;   // unit u starts at xin + u * G * SEG_ELEMS
+    const uint16_t *xin = p.x;               // unit u starts at xin + u * G * SEG_ELEMS
     // prologue: fill the ring
     if (leader) {
 #pragma unroll
-        for (int s = 0; s < FAST_NSTAGE; ++s) {
+        for (int s = 0; s < NST; ++s) {
             const uint32_t u = first + (uint32_t)s * stride;
             if (u < p.units_total) {
                 mbar_expect_tx(full_base + s * 8, UNIT_BYTES);
@@ -462,16 +534,37 @@ __global__ void __launch_bounds__(FAST_THREADS, 1) perq_fast_kernel(FastParams p
 
     uint32_t it = 0;
     for (uint32_t unit = first; unit < p.units_total; unit += stride, ++it) {
-        const uint32_t stage = it % FAST_NSTAGE;
-        const uint32_t parity = (it / FAST_NSTAGE) & 1u;
+        const uint32_t stage = it % NST;
+        const uint32_t parity = (it / NST) & 1u;
         const uint32_t par2 = it & 1u;
         if (!mbar_wait(full_base + stage * 8, parity)) {
             if (lane == 0) atomicOr(&g_perq_device_error, 1u);
             return;
         }
-        const uint32_t seg_addr = stage_base + stage * UNIT_BYTES + (uint32_t)w_in_g * SEG_BYTES;
-        const uint16_t *seg = reinterpret_cast<const uint16_t *>(fsmem + FastSmem::stages) +
-                              ((size_t)group * FAST_NSTAGE + stage) * (G * SEG_ELEMS) + (size_t)w_in_g * SEG_ELEMS;
+        // the staged row (or, unpermuted, the staged unit) and this warp's 1024 elements of it
+        const uint16_t *raw_row = reinterpret_cast<const uint16_t *>(fsmem + FastSmem::stages) +
+                                  ((size_t)group * NST + stage) * ((size_t)G * SEG_ELEMS);
+        uint32_t seg_addr = stage_base + stage * UNIT_BYTES + (uint32_t)w_in_g * SEG_BYTES;
+        const uint16_t *seg = raw_row + (size_t)w_in_g * SEG_ELEMS;
+        if (PERM) {
+            // gather this warp's segment of the permuted row into its own buffer: lane l takes
+            // positions r*256 + 8l .. +7 in round r (16-byte conflict-free stores)
+            const uint32_t raw_addr = stage_base + stage * UNIT_BYTES;
+            const uint4 *offs = reinterpret_cast<const uint4 *>(ptab + (size_t)w_in_g * SEG_ELEMS) + lane;
+#pragma unroll
+            for (int r = 0; r < 4; ++r) {
+                const uint4 o = offs[r * 32];
+                const uint32_t ow[4] = {o.x, o.y, o.z, o.w};
+                uint32_t wv[4];
+#pragma unroll
+                for (int e = 0; e < 4; ++e)
+                    wv[e] = lds_u16(raw_addr + (ow[e] & 0xffffu)) | (lds_u16(raw_addr + (ow[e] >> 16)) << 16);
+                sts_v4(pbuf_addr + (uint32_t)(r * 512 + lane * 16), wv[0], wv[1], wv[2], wv[3]);
+            }
+            __syncwarp();
+            seg_addr = pbuf_addr;
+            seg = reinterpret_cast<const uint16_t *>(fsmem + FastSmem::pbuf) + (size_t)warp * SEG_ELEMS;
+        }
         const size_t seg_index = (size_t)unit * G + w_in_g;
 
         // ---- H_16 on the tensor cores; v[s][h] = outputs (2h, 2h+1) of this lane's four of slot s
@@ -495,16 +588,18 @@ __global__ void __launch_bounds__(FAST_THREADS, 1) perq_fast_kernel(FastParams p
         // for G == 1 because this warp is, for G > 1 after the named barrier below)
         auto refill = [&]() {
             if (leader && it > 0) {
-                const uint32_t u = unit + (FAST_NSTAGE - 1) * stride;
+                const uint32_t u = unit + (NST - 1) * stride;
                 if (u < p.units_total && u > unit) {
-                    const uint32_t ps = (it - 1) % FAST_NSTAGE;
+                    const uint32_t ps = (it - 1) % NST;
+                    // permuted rows are read until the end of an iteration: wait until every warp is done
+                    if (PERM && !mbar_wait(empty_base + ps * 8, ((it - 1) / NST) & 1u)) atomicOr(&g_perq_device_error, 4u);
                     mbar_expect_tx(full_base + ps * 8, UNIT_BYTES);
                     bulk_load(stage_base + ps * UNIT_BYTES, xin + (size_t)u * (G * SEG_ELEMS), UNIT_BYTES,
                               full_base + ps * 8);
                 }
             }
         };
-        if (G == 1) refill();
+        if (G == 1 || MODE != MODE_TOKEN) refill();
 
         // ---- remaining butterfly stages over the slot bits inside a block (packed add/sub)
 #pragma unroll
@@ -641,7 +736,7 @@ __global__ void __launch_bounds__(FAST_THREADS, 1) perq_fast_kernel(FastParams p
                         }
                     }
                     if (++nreq == 32u) {
-                        serve_scale_requests<LOG2B>(p, wreq, nreq, G * SEG_ELEMS, lane);
+                        serve_scale_requests<LOG2B, PERM>(p, wreq, nreq, G * SEG_ELEMS, lane);
                         nreq = 0;
                     }
                 } else {
@@ -693,8 +788,8 @@ __global__ void __launch_bounds__(FAST_THREADS, 1) perq_fast_kernel(FastParams p
                     if (d >> 63) {                    // a position: evaluate its four outputs from the staged row
                         const uint32_t pos = (uint32_t)d & 0xffffu;
                         const uint32_t blk = (pos >> LOG2B) << LOG2B;
-                        const uint16_t *rowp = seg - (size_t)w_in_g * SEG_ELEMS;
-                        const double val = fabs(exact_coord4<B>(rowp + blk, (int)(pos - blk), lane));
+                        const double val = PERM ? fabs(exact_coord4_perm<B>(raw_row, ptab + blk, (int)(pos - blk), lane))
+                                                : fabs(exact_coord4<B>(raw_row + blk, (int)(pos - blk), lane));
                         a_bits = warp_max_u64((unsigned long long)__double_as_longlong(val));
                     } else {
                         a_bits = d;
@@ -896,9 +991,12 @@ __global__ void __launch_bounds__(FAST_THREADS, 1) perq_fast_kernel(FastParams p
         // ---- packed codes: shared staging -> global
         fence_async_smem();
         __syncwarp();
-        if (lane == 0) bulk_store(p.out_codes + seg_index * SEG_CODE_BYTES, code_buf, SEG_CODE_BYTES);
+        if (lane == 0) {
+            bulk_store(p.out_codes + seg_index * SEG_CODE_BYTES, code_buf, SEG_CODE_BYTES);
+            if (PERM) mbar_arrive(empty_base + stage * 8);     // this warp no longer reads the staged row
+        }
     }
-    if (MODE == MODE_TOKEN && nreq > 0u) serve_scale_requests<LOG2B>(p, wreq, nreq, G * SEG_ELEMS, lane);
+    if (MODE == MODE_TOKEN && nreq > 0u) serve_scale_requests<LOG2B, PERM>(p, wreq, nreq, G * SEG_ELEMS, lane);
     bulk_store_wait_read<0>();
 }
 
