@@ -381,7 +381,9 @@ __device__ __forceinline__ unsigned long long exact_max_of_candidates(const uint
 // fp64 and stores the scale.  This costs a few instructions per row instead of a cooperative
 // evaluation on the row's critical path.
 //
-// Record: bits 63..32 = row, bits 15..0 = element index in the row of the slot's first output.
+// Record: bits 63..32 = index of a 1024-element segment, bits 15..0 = element offset from that
+// segment's start to the slot's first output (per token: first segment of the row, offset in the row).
+// The same scheme serves the per-128 scales, with one record per quad.
 
 template <int LOG2B, bool PERM>
 __device__ __forceinline__ double exact_slot_max_global(const uint16_t *row, uint32_t pos, const int32_t *perm, int d)
@@ -420,16 +422,19 @@ __device__ __forceinline__ double exact_slot_max_global(const uint16_t *row, uin
     return fmax(fmax(fabs(a0 + a2), fabs(a1 + a3)), fmax(fabs(a0 - a2), fabs(a1 - a3)));
 }
 
-template <int LOG2B, bool PERM>
-__device__ __forceinline__ void serve_scale_requests(const FastParams &p, const unsigned long long *req, uint32_t n,
-                                                     uint32_t row_elems, int lane)
+template <int LOG2B, int MODE, bool PERM>
+__device__ __forceinline__ void serve_scale_requests(const FastParams &p, const unsigned long long *req, uint32_t n, int lane)
 {
     __syncwarp();
     if ((uint32_t)lane < n) {
         const unsigned long long r = req[lane];
-        const uint32_t unit = (uint32_t)(r >> 32), pos = (uint32_t)r & 0xffffu;
-        const double a = exact_slot_max_global<LOG2B, PERM>(p.x + (size_t)unit * row_elems, pos, p.perm, p.d);
-        reinterpret_cast<float *>(p.out_scales)[unit] = (a == 0.0) ? 0.0f : (float)(a * p.inv_7_sqrt_b);
+        const uint32_t segi = (uint32_t)(r >> 32), off = (uint32_t)r & 0xffffu;
+        const uint32_t segs = (uint32_t)p.d / SEG_ELEMS;
+        const uint32_t row = segi / segs;
+        const uint32_t pos = (segi - row * segs) * SEG_ELEMS + off;      // position in the row
+        const double a = exact_slot_max_global<LOG2B, PERM>(p.x + (size_t)row * p.d, pos, p.perm, p.d);
+        const size_t si = (MODE == MODE_TOKEN) ? (size_t)row : ((size_t)row * p.d + pos) >> 7;
+        reinterpret_cast<float *>(p.out_scales)[si] = (a == 0.0) ? 0.0f : (float)(a * p.inv_7_sqrt_b);
     }
     __syncwarp();
 }
@@ -637,33 +642,63 @@ __global__ void __launch_bounds__(FAST_THREADS, 1) perq_fast_kernel(FastParams p
             unsigned long long a_bits = 0ull;
             bool have_exact = true;          // warp-uniform: a_bits is the range's exact maximum
             bool is_cand = false;            // per token: this warp holds candidates for the row maximum
+            uint32_t my_pos = 0xffffffffu;   // common case: position of the one slot that holds the range's maximum
             int ncand = 1;
             const uint32_t pidx = par2 * FAST_WARPS + group;
             if (MODE == MODE_G128) {
+                // a scale range is the 128 elements of one quad.  Common case: one slot of one lane
+                // reaches the threshold; its position is recorded and the scale stored later.
                 a32 = fmaxf(lane_max, __shfl_xor_sync(0xffffffffu, lane_max, 1));
                 a32 = fmaxf(a32, __shfl_xor_sync(0xffffffffu, a32, 2));
                 const float thr = a32 * (1.0f - 2.0f * err_rel - 2.4e-7f);
-                const bool has_cand = (a32 > 0.0f) && (lane_max >= thr);
-                double a_exact = 0.0;
-                unsigned cq = __ballot_sync(0xffffffffu, has_cand) & qmask;      // candidate lanes of my quad
-                while (cq) {
-                    const int src = __ffs(cq) - 1;
-                    cq &= cq - 1;
-                    uint32_t cm = 0u;
-                    if (lane == src) cm = candidate_mask(v, ms, thr);
-                    cm = __shfl_sync(qmask, cm, src);
-                    while (cm) {
-                        const int e = __ffs(cm) - 1;
-                        cm &= cm - 1;
-                        int blk_elem, i, elem;
-                        locate<LOG2B>(src >> 2, src & 3, e, blk_elem, i, elem);
-                        a_exact = fmax(a_exact, fabs(exact_coord_quad<LOG2B>(seg + blk_elem, i, q, qmask)));
+                uint32_t slot_mask = 0u;
+#pragma unroll
+                for (int s = 0; s < 8; ++s) slot_mask |= (ms[s] >= thr) ? (1u << s) : 0u;
+                if (!(a32 > 0.0f)) slot_mask = 0u;
+                const unsigned cl4 = (__ballot_sync(0xffffffffu, slot_mask != 0u) >> (lane & 28)) & 0xFu;
+                const int srcq = (lane & 28) | ((__ffs(cl4) - 1) & 3);
+                const uint32_t smq = __shfl_sync(0xffffffffu, slot_mask, srcq);
+                const bool simple = cl4 != 0u && (cl4 & (cl4 - 1)) == 0u && (smq & (smq - 1)) == 0u;
+                if (simple) {
+                    const int sl = __ffs(smq) - 1;
+                    const int pch = g * 8 + (sl ^ (f_g & ~PM));
+                    my_pos = (uint32_t)(pch * 16 + 4 * (srcq & 3));
+                }
+                const unsigned enq = __ballot_sync(0xffffffffu, simple && q == 0);
+                if (simple && q == 0)
+                    wreq[nreq + __popc(enq & ((1u << lane) - 1u))] = ((unsigned long long)seg_index << 32) | my_pos;
+                nreq += __popc(enq);
+                if (!(a32 > 0.0f) && q == 0) reinterpret_cast<float *>(p.out_scales)[seg_index * 8 + g] = 0.0f;
+                // rare: several candidates in a quad are evaluated now, by the quad
+                const bool has_cand = !simple && (a32 > 0.0f) && (lane_max >= thr);
+                unsigned cq = __ballot_sync(0xffffffffu, has_cand) & qmask;
+                if (__any_sync(0xffffffffu, cq != 0u)) {
+                    double a_exact = 0.0;
+                    while (cq) {
+                        const int src = __ffs(cq) - 1;
+                        cq &= cq - 1;
+                        uint32_t cm = 0u;
+                        if (lane == src) cm = candidate_mask(v, ms, thr);
+                        cm = __shfl_sync(qmask, cm, src);
+                        while (cm) {
+                            const int e = __ffs(cm) - 1;
+                            cm &= cm - 1;
+                            int blk_elem, i, elem;
+                            locate<LOG2B>(src >> 2, src & 3, e, blk_elem, i, elem);
+                            a_exact = fmax(a_exact, fabs(exact_coord_quad<LOG2B>(seg + blk_elem, i, q, qmask)));
+                        }
+                    }
+                    if (has_cand || (!simple && (a32 > 0.0f))) {
+                        if (q == 0)
+                            reinterpret_cast<float *>(p.out_scales)[seg_index * 8 + g] =
+                                (a_exact == 0.0) ? 0.0f : (float)(a_exact * p.inv_7_sqrt_b);
+                        a_bits = (unsigned long long)__double_as_longlong(a_exact);
                     }
                 }
-                if (q == 0)
-                    reinterpret_cast<float *>(p.out_scales)[seg_index * 8 + g] =
-                        (a_exact == 0.0) ? 0.0f : (float)(a_exact * p.inv_7_sqrt_b);
-                a_bits = (unsigned long long)__double_as_longlong(a_exact);
+                if (nreq > 24u) {
+                    serve_scale_requests<LOG2B, MODE, PERM>(p, wreq, nreq, lane);
+                    nreq = 0;
+                }
             } else {
                 const float aw = warp_max_f32(lane_max);
                 unsigned candw;
@@ -713,7 +748,6 @@ __global__ void __launch_bounds__(FAST_THREADS, 1) perq_fast_kernel(FastParams p
             tie_any &= 0xffffu;
 
             // ---- per token: the exact row maximum and the stored scale, by the candidate warps only
-            uint32_t my_pos = 0xffffffffu;   // simple case: row position of the one candidate slot (this warp's)
             if (MODE == MODE_TOKEN && is_cand) {
                 const float thr_row = a32 * (1.0f - 2.0f * err_rel - 2.4e-7f);
                 uint32_t slot_mask = 0u;
@@ -728,7 +762,7 @@ __global__ void __launch_bounds__(FAST_THREADS, 1) perq_fast_kernel(FastParams p
                     const int pch = sg * 8 + (sl ^ ((sg & 3) & ~PM));
                     my_pos = (uint32_t)(w_in_g * SEG_ELEMS + pch * 16 + 4 * (src & 3));
                     if (lane == 0) {
-                        wreq[nreq] = ((unsigned long long)unit << 32) | my_pos;
+                        wreq[nreq] = ((unsigned long long)(unit * (uint32_t)G) << 32) | my_pos;
                         if (G > 1) {
                             wpub[pidx] = (1ull << 63) | my_pos;
                             __threadfence_block();
@@ -736,7 +770,7 @@ __global__ void __launch_bounds__(FAST_THREADS, 1) perq_fast_kernel(FastParams p
                         }
                     }
                     if (++nreq == 32u) {
-                        serve_scale_requests<LOG2B, PERM>(p, wreq, nreq, G * SEG_ELEMS, lane);
+                        serve_scale_requests<LOG2B, MODE, PERM>(p, wreq, nreq, lane);
                         nreq = 0;
                     }
                 } else {
@@ -814,7 +848,16 @@ __global__ void __launch_bounds__(FAST_THREADS, 1) perq_fast_kernel(FastParams p
                     tl &= tl - 1;
                     uint32_t fs = __shfl_sync(0xffffffffu, fm, src);
                     // the same sequence of fp64 operations as the definition, so exact ties land on exact halves
-                    const double a_src = __longlong_as_double((long long)__shfl_sync(0xffffffffu, a_bits, src));
+                    unsigned long long ab_src = __shfl_sync(0xffffffffu, a_bits, src);
+                    if (MODE == MODE_G128) {
+                        const uint32_t pos_src = __shfl_sync(0xffffffffu, my_pos, src);
+                        if (pos_src != 0xffffffffu) {
+                            const uint32_t blk = (pos_src >> LOG2B) << LOG2B;
+                            const double val = fabs(exact_coord4<B>(seg + blk, (int)(pos_src - blk), lane));
+                            ab_src = warp_max_u64((unsigned long long)__double_as_longlong(val));
+                        }
+                    }
+                    const double a_src = __longlong_as_double((long long)ab_src);
                     const double s_src = (a_src / p.sqrt_b) / 7.0;
                     while (fs) {
                         const int e = __ffs(fs) - 1;
@@ -996,7 +1039,7 @@ __global__ void __launch_bounds__(FAST_THREADS, 1) perq_fast_kernel(FastParams p
             if (PERM) mbar_arrive(empty_base + stage * 8);     // this warp no longer reads the staged row
         }
     }
-    if (MODE == MODE_TOKEN && nreq > 0u) serve_scale_requests<LOG2B, PERM>(p, wreq, nreq, G * SEG_ELEMS, lane);
+    if (MODE != MODE_MX && nreq > 0u) serve_scale_requests<LOG2B, MODE, PERM>(p, wreq, nreq, lane);
     bulk_store_wait_read<0>();
 }
 
