@@ -658,7 +658,9 @@ __global__ void __launch_bounds__(FAST_THREADS, 1) perq_fast_kernel(FastParams p
                 const unsigned cl4 = (__ballot_sync(0xffffffffu, slot_mask != 0u) >> (lane & 28)) & 0xFu;
                 const int srcq = (lane & 28) | ((__ffs(cl4) - 1) & 3);
                 const uint32_t smq = __shfl_sync(0xffffffffu, slot_mask, srcq);
-                const bool simple = cl4 != 0u && (cl4 & (cl4 - 1)) == 0u && (smq & (smq - 1)) == 0u;
+                // (deferring pays while a block is short and the row can be re-read contiguously)
+                constexpr bool DEFER = !PERM && LOG2B <= 5;
+                const bool simple = DEFER && cl4 != 0u && (cl4 & (cl4 - 1)) == 0u && (smq & (smq - 1)) == 0u;
                 if (simple) {
                     const int sl = __ffs(smq) - 1;
                     const int pch = g * 8 + (sl ^ (f_g & ~PM));
