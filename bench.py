@@ -70,7 +70,7 @@ class ClockSampler:
         out = {"sm_mhz": None, "sm_max_mhz": None, "reasons": [], "samples": 0}
         if self.proc is None:
             return out
-        time.sleep(0.06)
+        time.sleep(0.12)
         self.proc.terminate()
         try:
             text, _ = self.proc.communicate(timeout=5)
@@ -143,7 +143,7 @@ def run_reference(args):
 def main():
     ap = argparse.ArgumentParser()
     ap.add_argument("--gpus", type=int, default=1)
-    ap.add_argument("--steps", type=int, default=200)
+    ap.add_argument("--steps", type=int, default=4000)
     ap.add_argument("--warmup", type=int, default=10)
     ap.add_argument("--impl", default="perq", choices=["perq", "reference"])
     ap.add_argument("--no-sweep", action="store_true", help="skip the per-variant sweep after the timed steps")
@@ -194,7 +194,16 @@ def main():
     barrier()
     sampler = ClockSampler(local_rank)
     if rank == 0:
+        # nvidia-smi needs a moment to start sampling: keep the GPU under the same load meanwhile (untimed)
         sampler.start()
+        t_end = time.perf_counter() + 0.4
+        i = 0
+        while time.perf_counter() < t_end:
+            step(i)
+            i += 1
+            if i % 256 == 0:
+                torch.cuda.synchronize()
+    barrier()
     ev = [torch.cuda.Event(enable_timing=True) for _ in range(args.steps + 1)]
     ev[0].record()
     for i in range(args.steps):

@@ -98,11 +98,11 @@ int launch_generic(const void *x, const int32_t *perm, int64_t T, int32_t d, int
     return cudaGetLastError() == cudaSuccess ? PERQ_OK : PERQ_ERR_CUDA;
 }
 
-template <int LOG2B, int MODE, int LOG2G, bool PERM>
+template <int LOG2B, int MODE, int LOG2G, bool PERM, bool FULLV>
 int launch_fast_inst(const perq::FastParams &p, int grid, cudaStream_t st)
 {
-    auto kernel = perq::perq_fast_kernel<LOG2B, MODE, LOG2G, PERM>;
-    const size_t smem = PERM ? perq::FastSmem::total_perm : perq::FastSmem::total;
+    auto kernel = perq::perq_fast_kernel<LOG2B, MODE, LOG2G, PERM, FULLV>;
+    const size_t smem = PERM ? perq::FastSmem::total_perm : FULLV ? perq::FastSmem::total_full : perq::FastSmem::total;
     if (int rc = allow_smem(kernel, smem)) return rc;
     kernel<<<grid, perq::FAST_THREADS, smem, st>>>(p);
     return cudaGetLastError() == cudaSuccess ? PERQ_OK : PERQ_ERR_CUDA;
@@ -112,10 +112,10 @@ template <int MODE, int LOG2G, bool PERM>
 int launch_fast_b(int log2b, const perq::FastParams &p, int grid, cudaStream_t st)
 {
     switch (log2b) {
-    case 4: return launch_fast_inst<4, MODE, LOG2G, PERM>(p, grid, st);
-    case 5: return launch_fast_inst<5, MODE, LOG2G, PERM>(p, grid, st);
-    case 6: return launch_fast_inst<6, MODE, LOG2G, PERM>(p, grid, st);
-    default: return launch_fast_inst<7, MODE, LOG2G, PERM>(p, grid, st);
+    case 4: return launch_fast_inst<4, MODE, LOG2G, PERM, false>(p, grid, st);
+    case 5: return launch_fast_inst<5, MODE, LOG2G, PERM, false>(p, grid, st);
+    case 6: return launch_fast_inst<6, MODE, LOG2G, PERM, false>(p, grid, st);
+    default: return launch_fast_inst<7, MODE, LOG2G, PERM, false>(p, grid, st);
     }
 }
 
@@ -132,19 +132,35 @@ int launch_fast_mode(int mode, int G, int log2b, const perq::FastParams &p, int 
     }
 }
 
-// The fast kernel covers b <= 128, d % 1024 == 0, and scales per token (d / 1024 in {1,2,4,8}),
-// per 128 (INT4) or per 32 (MXFP4); with a permutation also d <= 16384.  Returns -1 if it does not apply.
+// full-vector block (b == d): unpermuted, per-token INT4 or MXFP4
+template <int MODE>
+int launch_fast_full(int G, const perq::FastParams &p, int grid, cudaStream_t st)
+{
+    switch (G) {
+    case 1: return launch_fast_inst<7, MODE, 0, false, true>(p, grid, st);
+    case 2: return launch_fast_inst<7, MODE, 1, false, true>(p, grid, st);
+    case 4: return launch_fast_inst<7, MODE, 2, false, true>(p, grid, st);
+    default: return launch_fast_inst<7, MODE, 3, false, true>(p, grid, st);
+    }
+}
+
+// The fast kernel covers d % 1024 == 0 with b <= 128 and scales per token (d / 1024 in {1,2,4,8}),
+// per 128 (INT4) or per 32 (MXFP4), with a permutation also d <= 16384; and b == d in {1024 .. 8192}
+// without a permutation, per token or MXFP4.  Returns -1 if it does not apply.
 int try_launch_fast(const void *x, const int32_t *perm, int64_t T, int32_t d, int32_t b, int32_t fmt, int g,
                     void *out_codes, void *out_scales, cudaStream_t st)
 {
-    if (b > 128 || d % perq::SEG_ELEMS != 0) return -1;
+    if (d % perq::SEG_ELEMS != 0) return -1;
     const int segs = d / perq::SEG_ELEMS;
     const bool permuted = perm != nullptr;
+    const bool full = b == d && b > 128;
+    if (!full && b > 128) return -1;
+    if (full && (permuted || (segs != 1 && segs != 2 && segs != 4 && segs != 8))) return -1;
     if (permuted && (d > perq::FastSmem::PERM_MAX_D || segs > perq::FAST_WARPS)) return -1;
     int mode, G = 1;
     if (fmt == PERQ_FMT_MXFP4) {
         mode = perq::MODE_MX;
-    } else if (fmt == PERQ_FMT_INT4 && g == 128) {
+    } else if (fmt == PERQ_FMT_INT4 && g == 128 && !full) {
         mode = perq::MODE_G128;
     } else if (fmt == PERQ_FMT_INT4 && g == d) {
         G = segs;
@@ -153,7 +169,7 @@ int try_launch_fast(const void *x, const int32_t *perm, int64_t T, int32_t d, in
     } else {
         return -1;
     }
-    if (permuted) G = segs;          // a permuted unit is a whole row
+    if (permuted || full) G = segs;          // the unit is a whole row
     const long long units = (long long)T * segs / G;
     if (units >= (1ll << 31)) return -1;
     perq::FastParams p;
@@ -171,6 +187,9 @@ int try_launch_fast(const void *x, const int32_t *perm, int64_t T, int32_t d, in
     const int groups_per_cta = perq::FAST_WARPS / G;
     const long long want = (units + groups_per_cta - 1) / groups_per_cta;
     const int grid = (int)std::min<long long>(want, sms);
+    if (full)
+        return mode == perq::MODE_MX ? launch_fast_full<perq::MODE_MX>(G, p, grid, st)
+                                     : launch_fast_full<perq::MODE_TOKEN>(G, p, grid, st);
     const int log2b = ilog2(b);
     return permuted ? launch_fast_mode<true>(mode, G, log2b, p, grid, st)
                     : launch_fast_mode<false>(mode, G, log2b, p, grid, st);

@@ -85,6 +85,9 @@ struct FastSmem {
     static constexpr size_t perm_tab = used;
     static constexpr int PERM_MAX_D = 16384;
     static constexpr size_t total_perm = used + (size_t)PERM_MAX_D * 2 + 1024;
+    // full-vector variants (unpermuted): 3 stages as well, and 4 KB per warp of fp32 exchange space after `used`
+    static constexpr size_t xbuf = used;
+    static constexpr size_t total_full = used + (size_t)FAST_WARPS * 4096 + 1024;
 };
 
 // ---------------------------------------------------------------- PTX wrappers
@@ -160,6 +163,14 @@ __device__ __forceinline__ uint32_t lds_u16(uint32_t addr)
 __device__ __forceinline__ void sts_v4(uint32_t addr, uint32_t a, uint32_t b, uint32_t c, uint32_t d)
 {
     asm volatile("st.shared.v4.b32 [%0], {%1, %2, %3, %4};" ::"r"(addr), "r"(a), "r"(b), "r"(c), "r"(d) : "memory");
+}
+__device__ __forceinline__ void sts_v4f(uint32_t addr, float a, float b, float c, float d)
+{
+    asm volatile("st.shared.v4.f32 [%0], {%1, %2, %3, %4};" ::"r"(addr), "f"(a), "f"(b), "f"(c), "f"(d) : "memory");
+}
+__device__ __forceinline__ void lds_v4f(uint32_t addr, float &a, float &b, float &c, float &d)
+{
+    asm volatile("ld.shared.v4.f32 {%0, %1, %2, %3}, [%4];" : "=f"(a), "=f"(b), "=f"(c), "=f"(d) : "r"(addr) : "memory");
 }
 __device__ __forceinline__ uint32_t ld_volatile_shared_u32(const uint32_t *p)
 {
@@ -245,7 +256,7 @@ template <int B>
 __device__ __forceinline__ double exact_coord_fast(const uint16_t *blk, int i, int lane)
 {
     double acc = 0.0;
-#pragma unroll
+#pragma unroll(B <= 128 ? 4 : 8)
     for (int k0 = 0; k0 < B; k0 += 32) {
         const int k = k0 + lane;
         if (B >= 32 || k < B) {
@@ -266,7 +277,7 @@ template <int B>
 __device__ __forceinline__ double exact_coord4(const uint16_t *blk, int i0, int lane)
 {
     double acc = 0.0;
-#pragma unroll
+#pragma unroll(B <= 128 ? 4 : 8)
     for (int k0 = 0; k0 < B; k0 += 32) {
         const int k = k0 + lane;
         if (B >= 32 || k < B) {
@@ -343,8 +354,10 @@ __device__ __forceinline__ uint32_t candidate_mask(const f32x2 (&v)[8][2], const
 
 // Exact maximum magnitude (bit pattern of a non-negative double, the same in every lane) over the
 // slots of this warp's segment whose fp32 maximum reaches thr.
-template <int LOG2B>
-__device__ __forceinline__ unsigned long long exact_max_of_candidates(const uint16_t *seg, const float (&ms)[8],
+// FULL_LOG2 == 0: blocks of 2^LOG2B inside the segment at seg.  FULL_LOG2 > 0: one block of 2^FULL_LOG2
+// elements, the whole row at seg, of which this warp's segment starts at seg_off.
+template <int LOG2B, int FULL_LOG2>
+__device__ __forceinline__ unsigned long long exact_max_of_candidates(const uint16_t *seg, int seg_off, const float (&ms)[8],
                                                                       float thr, int lane)
 {
     constexpr int CB = LOG2B - 4;
@@ -363,9 +376,13 @@ __device__ __forceinline__ unsigned long long exact_max_of_candidates(const uint
             const int sl = __ffs(sm) - 1;
             sm &= sm - 1;
             const int pch = sg * 8 + (sl ^ ((sg & 3) & ~PM));      // chunk position in the segment
-            const int blk_elem = (pch >> CB) << LOG2B;
-            const int i0 = pch * 16 - blk_elem + 4 * (src & 3);
-            best = fmax(best, fabs(exact_coord4<(1 << LOG2B)>(seg + blk_elem, i0, lane)));
+            if (FULL_LOG2 > 0) {
+                best = fmax(best, fabs(exact_coord4<(1 << (FULL_LOG2 > 0 ? FULL_LOG2 : 4))>(seg, seg_off + pch * 16 + 4 * (src & 3), lane)));
+            } else {
+                const int blk_elem = (pch >> CB) << LOG2B;
+                const int i0 = pch * 16 - blk_elem + 4 * (src & 3);
+                best = fmax(best, fabs(exact_coord4<(1 << LOG2B)>(seg + blk_elem, i0, lane)));
+            }
         }
     }
     return warp_max_u64((unsigned long long)__double_as_longlong(best));
@@ -393,7 +410,7 @@ __device__ __forceinline__ double exact_slot_max_global(const uint16_t *row, uin
     const uint32_t i0 = pos - blk;                       // multiple of 4
     const uint4 *src = reinterpret_cast<const uint4 *>(row + blk);
     double S[4] = {0.0, 0.0, 0.0, 0.0};                  // sums of the terms with k & 3 == m, signed by the high bits of i0
-#pragma unroll
+#pragma unroll(B <= 128 ? B / 8 : 2)
     for (int c = 0; c < B / 8; ++c) {
         uint32_t w[4];
         if (PERM) {
@@ -441,20 +458,26 @@ __device__ __forceinline__ void serve_scale_requests(const FastParams &p, const 
 
 // ---------------------------------------------------------------- the kernel
 
-template <int LOG2B, int MODE, int LOG2G, bool PERM>
+// FULLV: the Hadamard block is the whole row of 2^LOG2G segments (LOG2B must be 7: the part of the
+// butterfly done inside a warp's registers); the lane-group bits go through shuffles, the warp bits
+// through shared memory.
+template <int LOG2B, int MODE, int LOG2G, bool PERM, bool FULLV>
 __global__ void __launch_bounds__(FAST_THREADS, 1) perq_fast_kernel(FastParams p)
 {
     constexpr int B = 1 << LOG2B;
+    constexpr int LOG2BF = FULLV ? 10 + LOG2G : LOG2B;      // log2 of the Hadamard block
+    constexpr int BF = 1 << LOG2BF;
+    static_assert(!FULLV || (LOG2B == 7 && !PERM && MODE != MODE_G128), "full-vector variant: unpermuted, per token or MX");
     constexpr int CB = LOG2B - 4;                 // butterfly stages left after the tensor-core H_16
     constexpr int PM = (1 << CB) - 1;             // slot bits inside a Hadamard block
     constexpr int NCLS = (PM & 3) + 1;            // sign classes of the slot relabelling
     constexpr bool RUNTIME_G = PERM && MODE != MODE_TOKEN;     // a permuted unit is a whole row of any length
-    constexpr int NST = PERM ? 3 : FAST_NSTAGE;
+    constexpr int NST = (PERM || FULLV) ? 3 : FAST_NSTAGE;
     const int G = RUNTIME_G ? p.G : (1 << LOG2G);               // warps (segments) per unit
     const int GROUPS = FAST_WARPS / G;
     const uint32_t UNIT_BYTES = (uint32_t)G * SEG_BYTES;
     constexpr float MAGIC = 12582920.0f;          // 1.5 * 2^23 + 8: low nibble of the sum = code + 8
-    static_assert(MODE == MODE_TOKEN || LOG2G == 0, "only per-token scales couple the warps of a row");
+    static_assert(MODE == MODE_TOKEN || LOG2G == 0 || FULLV, "only per-token scales or a full-vector block couple the warps of a row");
     extern __shared__ __align__(128) unsigned char fsmem_raw[];
     // 1024-byte aligned base: the ldmatrix and code-store addresses below are formed with XOR
     unsigned char *fsmem = fsmem_raw + ((1024u - (smem_u32(fsmem_raw) & 1023u)) & 1023u);
@@ -464,7 +487,8 @@ __global__ void __launch_bounds__(FAST_THREADS, 1) perq_fast_kernel(FastParams p
     const int group = RUNTIME_G ? warp / G : warp >> LOG2G;
     const int w_in_g = warp - group * G;
     const unsigned qmask = 0xFu << (lane & 28);
-    const float err_rel = FAST_ERR_K * (float)LOG2B * TWO_M24;
+    const float err_rel = FAST_ERR_K * (float)LOG2BF * TWO_M24;
+    const uint32_t xbuf_addr = smem_u32(fsmem + FastSmem::xbuf) + (uint32_t)(group * G) * 4096u;   // FULLV: this row's exchange space
 
     const uint32_t stage_base = smem_u32(fsmem + FastSmem::stages) + (uint32_t)group * (NST * UNIT_BYTES);
     const uint32_t empty_base = smem_u32(fsmem + FastSmem::empty) + (uint32_t)group * (FAST_NSTAGE * 8);
@@ -520,9 +544,11 @@ __global__ void __launch_bounds__(FAST_THREADS, 1) perq_fast_kernel(FastParams p
     const uint32_t code_lane = (uint32_t)((g * 8 + (f_g & ~PM)) * 8 + 2 * q);
     // sign of the held value relative to the true output, per (s & 3 & PM): folded into multipliers
     const float half_sign = ((g & 4) && q >= 2) ? -1.0f : 1.0f;
-    float sgn[NCLS];
+    float sgn[4];
 #pragma unroll
-    for (int k = 0; k < NCLS; ++k) sgn[k] = (__popc(k & f_g & PM) & 1) ? -half_sign : half_sign;
+    for (int k = 0; k < 4; ++k) sgn[k] = (__popc(k & f_g & PM) & 1) ? -half_sign : half_sign;
+    // sign to fold into the quantisation multiplier of class k (none once the true signs are restored)
+    auto qsgn = [&](int k) { return FULLV ? 1.0f : sgn[k]; };
 
     const uint16_t *xin = p.x;               // unit u starts at xin + u * G * SEG_ELEMS
     // prologue: fill the ring
@@ -571,6 +597,18 @@ __global__ void __launch_bounds__(FAST_THREADS, 1) perq_fast_kernel(FastParams p
             seg = reinterpret_cast<const uint16_t *>(fsmem + FastSmem::pbuf) + (size_t)warp * SEG_ELEMS;
         }
         const size_t seg_index = (size_t)unit * G + w_in_g;
+        // Hadamard block of the element at offset e of this warp's segment: its bf16 inputs and the
+        // element's index inside the block
+        auto block_of = [&](int e, const uint16_t *&bp, int &i) {
+            if (FULLV) {
+                bp = raw_row;
+                i = w_in_g * SEG_ELEMS + e;
+            } else {
+                const int be = (e >> LOG2B) << LOG2B;
+                bp = seg + be;
+                i = e - be;
+            }
+        };
 
         // ---- H_16 on the tensor cores; v[s][h] = outputs (2h, 2h+1) of this lane's four of slot s
         f32x2 v[8][2];
@@ -604,7 +642,7 @@ __global__ void __launch_bounds__(FAST_THREADS, 1) perq_fast_kernel(FastParams p
                 }
             }
         };
-        if (G == 1 || MODE != MODE_TOKEN) refill();
+        if (G == 1 || (MODE != MODE_TOKEN && !FULLV)) refill();
 
         // ---- remaining butterfly stages over the slot bits inside a block (packed add/sub)
 #pragma unroll
@@ -617,6 +655,60 @@ __global__ void __launch_bounds__(FAST_THREADS, 1) perq_fast_kernel(FastParams p
                         const f32x2 a = v[s][h], c = v[s | (1 << t)][h];
                         v[s][h] = add2(a, c);
                         v[s | (1 << t)][h] = sub2(a, c);
+                    }
+                }
+            }
+        }
+
+        if (FULLV) {
+            // ---- the rest of a full-vector butterfly.  First the true signs (the relabelling signs
+            // can no longer be folded into a multiplier once values of different lanes are mixed).
+#pragma unroll
+            for (int s = 0; s < 8; ++s) {
+                const f32x2 sg2 = pack2(sgn[s & 3], sgn[s & 3]);
+                v[s][0] = mul2(v[s][0], sg2);
+                v[s][1] = mul2(v[s][1], sg2);
+            }
+            // lane-group bits (chunk index bits 3..5): exchange with lanes 4, 8, 16 away
+#pragma unroll
+            for (int bit = 4; bit <= 16; bit <<= 1) {
+                const float sg = (lane & bit) ? -1.0f : 1.0f;
+                const f32x2 sg2 = pack2(sg, sg);
+#pragma unroll
+                for (int s = 0; s < 8; ++s) {
+#pragma unroll
+                    for (int h = 0; h < 2; ++h) {
+                        const f32x2 o = pack2(__shfl_xor_sync(0xffffffffu, v[s][h].x, bit),
+                                              __shfl_xor_sync(0xffffffffu, v[s][h].y, bit));
+                        v[s][h] = fma2(v[s][h], sg2, o);          // upper partner: other - mine, lower: mine + other
+                    }
+                }
+            }
+            // warp bits (segment index): through shared memory, every warp combines all G copies
+            if (G > 1) {
+                const uint32_t mine = xbuf_addr + (uint32_t)w_in_g * 4096u + (uint32_t)lane * 16u;
+#pragma unroll
+                for (int s = 0; s < 8; ++s) sts_v4f(mine + s * 512, v[s][0].x, v[s][0].y, v[s][1].x, v[s][1].y);
+                named_barrier(1 + group, G * 32);
+                refill();
+                {
+                    const float sg = (__popc(w_in_g) & 1) ? -1.0f : 1.0f;
+                    const f32x2 sg2 = pack2(sg, sg);
+#pragma unroll
+                    for (int s = 0; s < 8; ++s) { v[s][0] = mul2(v[s][0], sg2); v[s][1] = mul2(v[s][1], sg2); }
+                }
+#pragma unroll
+                for (int dw = 1; dw < (1 << LOG2G); ++dw) {
+                    const int wo = w_in_g ^ dw;                   // every other warp of the row once
+                    const float sg = (__popc(w_in_g & wo) & 1) ? -1.0f : 1.0f;
+                    const f32x2 sg2 = pack2(sg, sg);
+                    const uint32_t theirs = xbuf_addr + (uint32_t)wo * 4096u + (uint32_t)lane * 16u;
+#pragma unroll
+                    for (int s = 0; s < 8; ++s) {
+                        float a, b, c, d;
+                        lds_v4f(theirs + s * 512, a, b, c, d);
+                        v[s][0] = fma2(pack2(a, b), sg2, v[s][0]);
+                        v[s][1] = fma2(pack2(c, d), sg2, v[s][1]);
                     }
                 }
             }
@@ -698,7 +790,7 @@ __global__ void __launch_bounds__(FAST_THREADS, 1) perq_fast_kernel(FastParams p
                     }
                 }
                 if (nreq > 24u) {
-                    serve_scale_requests<LOG2B, MODE, PERM>(p, wreq, nreq, lane);
+                    serve_scale_requests<LOG2BF, MODE, PERM>(p, wreq, nreq, lane);
                     nreq = 0;
                 }
             } else {
@@ -711,7 +803,7 @@ __global__ void __launch_bounds__(FAST_THREADS, 1) perq_fast_kernel(FastParams p
                     a32 = warp_max_f32(am);
                     const float thr_row = a32 * (1.0f - 2.0f * err_rel - 2.4e-7f);
                     candw = __ballot_sync(0xffffffffu, (lane < G) && (a32 > 0.0f) && (am >= thr_row));
-                    refill();
+                    if (!FULLV) refill();
                 } else {
                     a32 = aw;
                     candw = (a32 > 0.0f) ? 1u : 0u;
@@ -729,7 +821,7 @@ __global__ void __launch_bounds__(FAST_THREADS, 1) perq_fast_kernel(FastParams p
             f32x2 mul_p[NCLS], mul_m[NCLS];
 #pragma unroll
             for (int k = 0; k < NCLS; ++k) {
-                const float mp = sgn[k] * inv * (1.0f + delta), mm = sgn[k] * inv * (1.0f - delta);
+                const float mp = qsgn(k) * inv * (1.0f + delta), mm = qsgn(k) * inv * (1.0f - delta);
                 mul_p[k] = pack2(mp, mp);
                 mul_m[k] = pack2(mm, mm);
             }
@@ -772,12 +864,14 @@ __global__ void __launch_bounds__(FAST_THREADS, 1) perq_fast_kernel(FastParams p
                         }
                     }
                     if (++nreq == 32u) {
-                        serve_scale_requests<LOG2B, MODE, PERM>(p, wreq, nreq, lane);
+                        serve_scale_requests<LOG2BF, MODE, PERM>(p, wreq, nreq, lane);
                         nreq = 0;
                     }
                 } else {
                     // several candidates: exact values now, combined over the candidate warps
-                    const unsigned long long wb = exact_max_of_candidates<LOG2B>(seg, ms, thr_row, lane);
+                    const unsigned long long wb = FULLV
+                        ? exact_max_of_candidates<LOG2B, FULLV ? LOG2BF : 0>(raw_row, w_in_g * SEG_ELEMS, ms, thr_row, lane)
+                        : exact_max_of_candidates<LOG2B, 0>(seg, 0, ms, thr_row, lane);
                     if (ncand == 1) {
                         a_bits = wb;
                         have_exact = true;
@@ -823,9 +917,9 @@ __global__ void __launch_bounds__(FAST_THREADS, 1) perq_fast_kernel(FastParams p
                     }
                     if (d >> 63) {                    // a position: evaluate its four outputs from the staged row
                         const uint32_t pos = (uint32_t)d & 0xffffu;
-                        const uint32_t blk = (pos >> LOG2B) << LOG2B;
-                        const double val = PERM ? fabs(exact_coord4_perm<B>(raw_row, ptab + blk, (int)(pos - blk), lane))
-                                                : fabs(exact_coord4<B>(raw_row + blk, (int)(pos - blk), lane));
+                        const uint32_t blk = (pos >> LOG2BF) << LOG2BF;
+                        const double val = PERM ? fabs(exact_coord4_perm<BF>(raw_row, ptab + blk, (int)(pos - blk), lane))
+                                                : fabs(exact_coord4<BF>(raw_row + blk, (int)(pos - blk), lane));
                         a_bits = warp_max_u64((unsigned long long)__double_as_longlong(val));
                     } else {
                         a_bits = d;
@@ -866,7 +960,9 @@ __global__ void __launch_bounds__(FAST_THREADS, 1) perq_fast_kernel(FastParams p
                         fs &= fs - 1;
                         int blk_elem, i, elem;
                         locate<LOG2B>(src >> 2, src & 3, e, blk_elem, i, elem);
-                        const double ue = exact_coord_fast<B>(seg + blk_elem, i, lane);
+                        const uint16_t *bp;
+                        block_of(elem, bp, i);
+                        const double ue = exact_coord_fast<BF>(bp, i, lane);
                         if (lane == 0) {
                             uint32_t code = 0u;
                             if (s_src != 0.0) {
@@ -899,6 +995,14 @@ __global__ void __launch_bounds__(FAST_THREADS, 1) perq_fast_kernel(FastParams p
                 bref = a32;
                 if (CB >= 2) bref = fmaxf(bref, __shfl_xor_sync(0xffffffffu, bref, 1));
                 if (CB >= 3) bref = fmaxf(bref, __shfl_xor_sync(0xffffffffu, bref, 2));
+                if (FULLV) {     // the block is the row: maximum over the warp, then over the row's warps
+                    bref = warp_max_f32(bref);
+                    if (G > 1) {
+                        if (lane == 0) wmax[par2 * FAST_WARPS + warp] = bref;
+                        named_barrier(1 + group, G * 32);      // also: every warp has read the exchange space
+                        bref = warp_max_f32((lane < G) ? wmax[par2 * FAST_WARPS + group * G + lane] : 0.0f);
+                    }
+                }
             }
             // E + 127 with E = floor(log2(a / sqrt(b))) - 2, from the bits of a32; near a boundary of
             // that floor the maximum is re-derived exactly
@@ -906,19 +1010,55 @@ __global__ void __launch_bounds__(FAST_THREADS, 1) perq_fast_kernel(FastParams p
             const int e8 = (int)(bits >> 23);
             int Eb;
             float dist;
-            if ((LOG2B & 1) == 0) {
-                Eb = e8 - LOG2B / 2 - 2;
+            if ((LOG2BF & 1) == 0) {
+                Eb = e8 - LOG2BF / 2 - 2;
                 const float lower = __uint_as_float(bits & 0x7f800000u);
                 dist = fminf(a32 - lower, 2.0f * lower - a32);
             } else {
                 const uint32_t mant = bits & 0x7fffffu;
-                Eb = e8 - (LOG2B - 1) / 2 - 3 + (mant >= 0x3504f4u ? 1 : 0);
+                Eb = e8 - (LOG2BF - 1) / 2 - 3 + (mant >= 0x3504f4u ? 1 : 0);
                 dist = fabsf(a32 - __uint_as_float((bits & 0x7f800000u) | 0x3504f3u));
             }
             const float tol = 2.0f * err_rel * bref + a32 * 2.4e-7f;
             const bool near = (a32 > 0.0f) && (dist <= tol || e8 == 0);
             const unsigned near_w = __ballot_sync(0xffffffffu, near);
-            if (near_w != 0u) {   // rare: exact maximum of the group from every element that could attain it
+            if (FULLV && near_w != 0u) {   // rare; whole-row blocks are evaluated by the whole warp, one group at a time
+                unsigned nw = near_w;
+                while (nw) {
+                    const int owner = __ffs(nw) - 1;
+                    nw &= nw - 1;
+                    const int m = owner & 3;
+                    const float thr = __shfl_sync(0xffffffffu, a32 - tol, owner);
+                    uint32_t mymask = 0u;
+                    if ((lane >> 2) == (owner >> 2)) {
+#pragma unroll
+                        for (int mm = 0; mm < 4; ++mm) {
+                            if (mm == m) {
+                                const float e[8] = {v[2 * mm][0].x, v[2 * mm][0].y, v[2 * mm][1].x, v[2 * mm][1].y,
+                                                    v[2 * mm + 1][0].x, v[2 * mm + 1][0].y, v[2 * mm + 1][1].x, v[2 * mm + 1][1].y};
+#pragma unroll
+                                for (int k = 0; k < 8; ++k) mymask |= (fabsf(e[k]) >= thr) ? (1u << k) : 0u;
+                            }
+                        }
+                    }
+                    double best = 0.0;
+                    for (int ql = 0; ql < 4; ++ql) {
+                        uint32_t cm = __shfl_sync(0xffffffffu, mymask, (owner & 28) | ql);
+                        while (cm) {
+                            const int k = __ffs(cm) - 1;
+                            cm &= cm - 1;
+                            int blk_elem, i, elem;
+                            locate<LOG2B>(owner >> 2, ql, 8 * m + k, blk_elem, i, elem);
+                            best = fmax(best, fabs(exact_coord_fast<BF>(raw_row, w_in_g * SEG_ELEMS + elem, lane)));
+                        }
+                    }
+                    if (lane == owner) {
+                        int ex;
+                        (void)frexp(best / p.sqrt_b, &ex);
+                        Eb = ex - 3 + 127;
+                    }
+                }
+            } else if (near_w != 0u) {   // rare: exact maximum of the group from every element that could attain it
                 const unsigned nearq = (near_w >> (lane & 28)) & 0xFu;
 #pragma unroll
                 for (int m = 0; m < 4; ++m) {
@@ -959,8 +1099,8 @@ __global__ void __launch_bounds__(FAST_THREADS, 1) perq_fast_kernel(FastParams p
             Eb = min(max(Eb, 0), 254);
             // multiplier 2^-E / sqrt(b) and the additive rounding window, in scaled units
             float c;
-            if ((LOG2B & 1) == 0) c = __uint_as_float((uint32_t)min(max(254 - Eb - LOG2B / 2, 1), 254) << 23);
-            else c = __uint_as_float((uint32_t)min(max(254 - Eb - (LOG2B - 1) / 2, 1), 254) << 23) * 0.70710678118654752f;
+            if ((LOG2BF & 1) == 0) c = __uint_as_float((uint32_t)min(max(254 - Eb - LOG2BF / 2, 1), 254) << 23);
+            else c = __uint_as_float((uint32_t)min(max(254 - Eb - (LOG2BF - 1) / 2, 1), 254) << 23) * 0.70710678118654752f;
             uint32_t byte = (uint32_t)Eb;
             if (!(a32 > 0.0f)) { c = 0.0f; byte = 0u; }
             const float tau = 2.0f * err_rel * bref * c + 2.0e-6f;
@@ -980,7 +1120,7 @@ __global__ void __launch_bounds__(FAST_THREADS, 1) perq_fast_kernel(FastParams p
                 tau_m[m] = pack2(-t_m, -t_m);
 #pragma unroll
                 for (int h = 0; h < 2; ++h) {
-                    const float mc = sgn[(2 * m + h) & 3 & PM] * c_m;
+                    const float mc = qsgn((2 * m + h) & 3 & PM) * c_m;
                     mulc[2 * m + h] = pack2(mc, mc);
                 }
             }
@@ -1019,7 +1159,9 @@ __global__ void __launch_bounds__(FAST_THREADS, 1) perq_fast_kernel(FastParams p
                         fs &= fs - 1;
                         int blk_elem, i, elem;
                         locate<LOG2B>(src >> 2, src & 3, e, blk_elem, i, elem);
-                        const double ue = exact_coord_fast<B>(seg + blk_elem, i, lane);
+                        const uint16_t *bp;
+                        block_of(elem, bp, i);
+                        const double ue = exact_coord_fast<BF>(bp, i, lane);
                         if (lane == 0) {
                             const int E = (int)((wsrc >> (8 * ((e >> 3) ^ fsrc))) & 0xFFu) - 127;
                             const double y = ue / p.sqrt_b;
@@ -1041,7 +1183,7 @@ __global__ void __launch_bounds__(FAST_THREADS, 1) perq_fast_kernel(FastParams p
             if (PERM) mbar_arrive(empty_base + stage * 8);     // this warp no longer reads the staged row
         }
     }
-    if (MODE != MODE_MX && nreq > 0u) serve_scale_requests<LOG2B, MODE, PERM>(p, wreq, nreq, lane);
+    if (MODE != MODE_MX && nreq > 0u) serve_scale_requests<LOG2BF, MODE, PERM>(p, wreq, nreq, lane);
     bulk_store_wait_read<0>();
 }
 
