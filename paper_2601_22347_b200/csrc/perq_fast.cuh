@@ -45,7 +45,8 @@ constexpr int FAST_NSTAGE = 4;
 constexpr int SEG_ELEMS = 1024;
 constexpr int SEG_BYTES = 2048;
 constexpr int SEG_CODE_BYTES = 512;
-constexpr float FAST_ERR_K = 4.0f;
+constexpr float FAST_ERR_K = 4.0f;          // fp32 error model: |u32 - u| <= K * log2(b) * 2^-24 * max|u32| of the block
+constexpr float FAST_ERR_K_FULL = 1.0f;     // whole-row blocks: 4096 outputs share the rounding errors of 12 stages
 constexpr uint32_t WAIT_SPIN_LIMIT = 1u << 22;
 
 enum FastMode { MODE_TOKEN = 0, MODE_G128 = 1, MODE_MX = 2 };
@@ -443,6 +444,26 @@ template <int LOG2B, int MODE, bool PERM>
 __device__ __forceinline__ void serve_scale_requests(const FastParams &p, const unsigned long long *req, uint32_t n, int lane)
 {
     __syncwarp();
+    if (LOG2B >= 10 && !PERM && n < 16u) {
+        // long blocks, few records: the whole warp evaluates one record at a time (coalesced reads)
+        for (uint32_t j = 0; j < n; ++j) {
+            const unsigned long long r = req[j];
+            const uint32_t segi = (uint32_t)(r >> 32), off = (uint32_t)r & 0xffffu;
+            const uint32_t segs = (uint32_t)p.d / SEG_ELEMS;
+            const uint32_t row = segi / segs;
+            const uint32_t pos = (segi - row * segs) * SEG_ELEMS + off;
+            const uint32_t blk = (pos >> LOG2B) << LOG2B;
+            const double val = fabs(exact_coord4<(1 << LOG2B)>(p.x + (size_t)row * p.d + blk, (int)(pos - blk), lane));
+            const unsigned long long ab = warp_max_u64((unsigned long long)__double_as_longlong(val));
+            if (lane == 0) {
+                const size_t si = (MODE == MODE_TOKEN) ? (size_t)row : ((size_t)row * p.d + pos) >> 7;
+                reinterpret_cast<float *>(p.out_scales)[si] =
+                    (ab == 0ull) ? 0.0f : (float)(__longlong_as_double((long long)ab) * p.inv_7_sqrt_b);
+            }
+        }
+        __syncwarp();
+        return;
+    }
     if ((uint32_t)lane < n) {
         const unsigned long long r = req[lane];
         const uint32_t segi = (uint32_t)(r >> 32), off = (uint32_t)r & 0xffffu;
@@ -487,7 +508,7 @@ __global__ void __launch_bounds__(FAST_THREADS, 1) perq_fast_kernel(FastParams p
     const int group = RUNTIME_G ? warp / G : warp >> LOG2G;
     const int w_in_g = warp - group * G;
     const unsigned qmask = 0xFu << (lane & 28);
-    const float err_rel = FAST_ERR_K * (float)LOG2BF * TWO_M24;
+    const float err_rel = (FULLV ? FAST_ERR_K_FULL : FAST_ERR_K) * (float)LOG2BF * TWO_M24;
     const uint32_t xbuf_addr = smem_u32(fsmem + FastSmem::xbuf) + (uint32_t)(group * G) * 4096u;   // FULLV: this row's exchange space
 
     const uint32_t stage_base = smem_u32(fsmem + FastSmem::stages) + (uint32_t)group * (NST * UNIT_BYTES);
