@@ -208,7 +208,11 @@ struct StatsPlan {
     int rows_per_cta;
     size_t smem;
     size_t ws_bytes;
+    int kc;            // 16-byte chunks of a row per thread
 };
+
+template <int KC>
+int launch_stats_partial(const perq::StatsParams &p, const struct StatsPlan &plan, cudaStream_t st);
 
 int plan_stats(int64_t T, int32_t d, int32_t b, StatsPlan *plan)
 {
@@ -220,7 +224,9 @@ int plan_stats(int64_t T, int32_t d, int32_t b, StatsPlan *plan)
     const long long rows = std::max<long long>(1, (T + max_cta - 1) / max_cta);
     plan->rows_per_cta = (int)std::min<long long>(rows, 1 << 30);
     plan->n_cta = (int)std::max<long long>(1, (T + rows - 1) / rows);
-    plan->smem = (size_t)d * 4 + (size_t)(d / 8) * 4 + 32 * 4;
+    plan->kc = d <= 4096 ? 1 : d <= 8192 ? 2 : d <= 16384 ? 4 : 8;
+    const size_t rif = 8 / plan->kc;      // rows in flight per CTA
+    plan->smem = (rif + 1) * (size_t)d * 2 + rif * (size_t)(d / 8) * 4 + rif * 16 * 4;
     plan->ws_bytes = (size_t)plan->n_cta * ((size_t)d + (size_t)(d / b)) * sizeof(float);
     return PERQ_OK;
 }
@@ -232,6 +238,14 @@ constexpr int kMaxDevices = 64;
 static __device__ __align__(256) float g_stats_scratch[PERQ_STATS_STATIC_MAX_FLOATS];
 float *g_stats_scratch_addr[kMaxDevices] = {};   // device address of the array, per device ordinal
 std::mutex g_stats_scratch_mutex;
+
+template <int KC>
+int launch_stats_partial(const perq::StatsParams &p, const StatsPlan &plan, cudaStream_t st)
+{
+    if (int rc = allow_smem(perq::perq_stats_partial_kernel<KC>, plan.smem)) return rc;
+    perq::perq_stats_partial_kernel<KC><<<plan.n_cta, perq::ST_THREADS, plan.smem, st>>>(p);
+    return cudaGetLastError() == cudaSuccess ? PERQ_OK : PERQ_ERR_CUDA;
+}
 
 }  // namespace
 
@@ -361,9 +375,14 @@ int perq_block_l1_stats(const void *x, const int32_t *perm, int64_t T, int32_t d
     p.ws_chan = chan_abs_sum ? ws : nullptr;
     p.ws_block = block_l1_mean ? ws + (size_t)plan.n_cta * d : nullptr;
     p.token_max = token_max_block_l1;
-    if (int rc = allow_smem(perq::perq_stats_partial_kernel, plan.smem)) return rc;
-    perq::perq_stats_partial_kernel<<<plan.n_cta, perq::ST_THREADS, plan.smem, st>>>(p);
-    if (cudaGetLastError() != cudaSuccess) return PERQ_ERR_CUDA;
+    int rc = PERQ_OK;
+    switch (plan.kc) {
+    case 1: rc = launch_stats_partial<1>(p, plan, st); break;
+    case 2: rc = launch_stats_partial<2>(p, plan, st); break;
+    case 4: rc = launch_stats_partial<4>(p, plan, st); break;
+    default: rc = launch_stats_partial<8>(p, plan, st); break;
+    }
+    if (rc != PERQ_OK) return rc;
     if (chan_abs_sum || block_l1_mean) {
         const int threads = 256;
         perq::perq_stats_reduce_kernel<<<(d + threads - 1) / threads, threads, 0, st>>>(

@@ -1,9 +1,11 @@
 // Calibration statistic kernels: per-channel sum of |x|, per-block mean l1 norm and
 // per-token max block l1 norm under an optional permutation.
 //
-// Phase 1: each CTA walks a contiguous slab of rows with the whole row in shared memory,
-// keeps per-channel and per-block partial sums in registers (every thread owns fixed
-// columns / blocks), and writes them to its own slice of the workspace.
+// Phase 1: each CTA walks a contiguous slab of rows, a few rows at a time (64 KB of loads in
+// flight per CTA, the next batch being fetched while the current one is reduced), keeps
+// per-channel and per-block partial sums in registers (every thread owns fixed columns /
+// blocks), and writes them to its own slice of the workspace.  Rows go through shared memory
+// only when a block statistic needs the gather through the permutation.
 // Phase 2: one thread per output adds the CTA slices in CTA order.  All additions happen
 // in a fixed order, so the results are bit-identical from run to run.
 #pragma once
@@ -29,24 +31,28 @@ struct StatsParams {
 
 __device__ __forceinline__ float abs_bf16(uint16_t h) { return __uint_as_float(((uint32_t)h & 0x7fffu) << 16); }
 
+// KC = 16-byte chunks of a row per thread (d <= KC * 4096); R = rows in flight per CTA, chosen so
+// that every thread always has 8 loads of 16 bytes outstanding (64 KB per CTA).
+template <int KC>
 __global__ void __launch_bounds__(ST_THREADS) perq_stats_partial_kernel(StatsParams p)
 {
+    constexpr int R = 8 / KC;
     extern __shared__ __align__(16) unsigned char smem[];
     const int d = p.d, L = p.log2b, nb = d >> L, nchunks = d >> 3;
-    uint16_t *raw = (uint16_t *)smem;                         // [d] one row, original order
-    uint16_t *sperm = raw + d;                                // [d] permutation (d <= 32768 fits 16 bits)
-    float *cs = (float *)(smem + (size_t)d * 4);              // [d/8] per-chunk l1 of the permuted row
-    float *red = cs + nchunks;                                // [32]
+    uint16_t *sperm = (uint16_t *)smem;                                  // [d] permutation (d <= 32768 fits 16 bits)
+    uint16_t *raw = sperm + d;                                           // [R][d] rows, original order
+    float *cs = (float *)(smem + (size_t)(R + 1) * d * 2);               // [R][d/8] per-chunk l1 of the permuted rows
+    float *red = cs + (size_t)R * nchunks;                               // [R][16]
     const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
 
     for (int i = tid; i < d; i += ST_THREADS) {
         int q = p.perm ? __ldg(p.perm + i) : i;
         sperm[i] = (uint16_t)min(max(q, 0), d - 1);
     }
-    float csum[ST_MAX_CHUNKS][8];
-    float bsum[ST_MAX_CHUNKS];
+    float csum[KC][8];
+    float bsum[KC];
 #pragma unroll
-    for (int k = 0; k < ST_MAX_CHUNKS; ++k) {
+    for (int k = 0; k < KC; ++k) {
         bsum[k] = 0.0f;
 #pragma unroll
         for (int e = 0; e < 8; ++e) csum[k][e] = 0.0f;
@@ -54,28 +60,48 @@ __global__ void __launch_bounds__(ST_THREADS) perq_stats_partial_kernel(StatsPar
     const long long t0 = (long long)blockIdx.x * p.rows_per_cta;
     const long long t1 = min(p.T, t0 + p.rows_per_cta);
     const bool want_blocks = (p.ws_block != nullptr) || (p.token_max != nullptr);
+    const uint4 zero4 = make_uint4(0u, 0u, 0u, 0u);
+
+    uint4 w[R][KC];
+    auto load_batch = [&](long long t) {
+#pragma unroll
+        for (int r = 0; r < R; ++r) {
+            const uint4 *src = (const uint4 *)(p.x + (size_t)(t + r) * d);
+#pragma unroll
+            for (int k = 0; k < KC; ++k) {
+                const int c = tid + k * ST_THREADS;
+                w[r][k] = (t + r < t1 && c < nchunks) ? __ldcs(src + c) : zero4;
+            }
+        }
+    };
+    if (t0 < t1) load_batch(t0);
     __syncthreads();
 
-    for (long long t = t0; t < t1; ++t) {
-        const uint4 *src = (const uint4 *)(p.x + (size_t)t * d);
+    for (long long t = t0; t < t1; t += R) {
+        // ---- channel sums from the registers; rows to shared memory for the gather
 #pragma unroll
-        for (int k = 0; k < ST_MAX_CHUNKS; ++k) {
-            const int c = tid + k * ST_THREADS;
-            if (c < nchunks) {
-                const uint4 w = __ldcs(src + c);
-                ((uint4 *)raw)[c] = w;
-                const uint32_t ww[4] = {w.x, w.y, w.z, w.w};
+        for (int r = 0; r < R; ++r) {
+#pragma unroll
+            for (int k = 0; k < KC; ++k) {
+                const uint32_t ww[4] = {w[r][k].x, w[r][k].y, w[r][k].z, w[r][k].w};
 #pragma unroll
                 for (int e = 0; e < 4; ++e) {
                     csum[k][2 * e] += __uint_as_float((ww[e] << 16) & 0x7fffffffu);
                     csum[k][2 * e + 1] += __uint_as_float(ww[e] & 0x7fff0000u);
                 }
+                const int c = tid + k * ST_THREADS;
+                if (want_blocks && c < nchunks) ((uint4 *)(raw + (size_t)r * d))[c] = w[r][k];
             }
         }
-        if (want_blocks) {
-            __syncthreads();
+        // ---- next batch: loads in flight while this one is reduced
+        if (t + R < t1) load_batch(t + R);
+        if (!want_blocks) continue;
+        __syncthreads();
 #pragma unroll
-            for (int k = 0; k < ST_MAX_CHUNKS; ++k) {
+        for (int r = 0; r < R; ++r) {
+            const uint16_t *row = raw + (size_t)r * d;
+#pragma unroll
+            for (int k = 0; k < KC; ++k) {
                 const int c = tid + k * ST_THREADS;
                 if (c < nchunks) {
                     const uint4 pi = ((const uint4 *)sperm)[c];
@@ -83,46 +109,52 @@ __global__ void __launch_bounds__(ST_THREADS) perq_stats_partial_kernel(StatsPar
                     float s = 0.0f;
 #pragma unroll
                     for (int e = 0; e < 4; ++e) {
-                        s += abs_bf16(raw[pp[e] & 0xffffu]);
-                        s += abs_bf16(raw[pp[e] >> 16]);
+                        s += abs_bf16(row[pp[e] & 0xffffu]);
+                        s += abs_bf16(row[pp[e] >> 16]);
                     }
-                    cs[c] = s;
+                    cs[(size_t)r * nchunks + c] = s;
                 }
             }
-            __syncthreads();
-            float mx = 0.0f;
-            const int cpb = 1 << (L - 3);          // chunks per block
-#pragma unroll
-            for (int k = 0; k < ST_MAX_CHUNKS; ++k) {
-                const int j = tid + k * ST_THREADS;
-                if (j < nb) {
-                    float s = 0.0f;
-                    for (int c = 0; c < cpb; ++c) s += cs[j * cpb + c];
-                    bsum[k] += s;
-                    mx = fmaxf(mx, s);
-                }
-            }
-            if (p.token_max) {
-#pragma unroll
-                for (int o = 16; o > 0; o >>= 1) mx = fmaxf(mx, __shfl_xor_sync(0xffffffffu, mx, o));
-                if (lane == 0) red[warp] = mx;
-                __syncthreads();
-                if (tid == 0) {
-                    float m = red[0];
-                    for (int w = 1; w < ST_THREADS / 32; ++w) m = fmaxf(m, red[w]);
-                    p.token_max[t] = m;
-                }
-            }
-            __syncthreads();
-        } else {
-            __syncthreads();
         }
+        __syncthreads();
+        const int cpb = 1 << (L - 3);          // chunks per block
+        float mx[R];
+#pragma unroll
+        for (int r = 0; r < R; ++r) {
+            mx[r] = 0.0f;
+            const bool live = t + r < t1;
+#pragma unroll
+            for (int k = 0; k < KC; ++k) {
+                const int j = tid + k * ST_THREADS;
+                if (j < nb && live) {
+                    float s = 0.0f;
+                    for (int c = 0; c < cpb; ++c) s += cs[(size_t)r * nchunks + j * cpb + c];
+                    bsum[k] += s;
+                    mx[r] = fmaxf(mx[r], s);
+                }
+            }
+        }
+        if (p.token_max) {
+#pragma unroll
+            for (int r = 0; r < R; ++r) {
+#pragma unroll
+                for (int o = 16; o > 0; o >>= 1) mx[r] = fmaxf(mx[r], __shfl_xor_sync(0xffffffffu, mx[r], o));
+                if (lane == 0) red[r * 16 + warp] = mx[r];
+            }
+            __syncthreads();
+            if (tid < R && t + tid < t1) {
+                float m = red[tid * 16];
+                for (int wv = 1; wv < ST_THREADS / 32; ++wv) m = fmaxf(m, red[tid * 16 + wv]);
+                p.token_max[t + tid] = m;
+            }
+        }
+        __syncthreads();
     }
 
     if (p.ws_chan) {
         float4 *dst = (float4 *)(p.ws_chan + (size_t)blockIdx.x * d);
 #pragma unroll
-        for (int k = 0; k < ST_MAX_CHUNKS; ++k) {
+        for (int k = 0; k < KC; ++k) {
             const int c = tid + k * ST_THREADS;
             if (c < nchunks) {
                 dst[2 * c] = make_float4(csum[k][0], csum[k][1], csum[k][2], csum[k][3]);
@@ -132,7 +164,7 @@ __global__ void __launch_bounds__(ST_THREADS) perq_stats_partial_kernel(StatsPar
     }
     if (p.ws_block) {
 #pragma unroll
-        for (int k = 0; k < ST_MAX_CHUNKS; ++k) {
+        for (int k = 0; k < KC; ++k) {
             const int j = tid + k * ST_THREADS;
             if (j < nb) p.ws_block[(size_t)blockIdx.x * nb + j] = bsum[k];
         }
