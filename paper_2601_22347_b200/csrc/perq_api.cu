@@ -384,8 +384,7 @@ int perq_block_l1_stats(const void *x, const int32_t *perm, int64_t T, int32_t d
     }
     if (rc != PERQ_OK) return rc;
     if (chan_abs_sum || block_l1_mean) {
-        const int threads = 256;
-        perq::perq_stats_reduce_kernel<<<(d + threads - 1) / threads, threads, 0, st>>>(
+        perq::perq_stats_reduce_kernel<<<(d + 63) / 64, 256, 0, st>>>(
             p.ws_chan, p.ws_block, plan.n_cta, d, d / b, (float)(1.0 / (double)T), chan_abs_sum, block_l1_mean);
         if (cudaGetLastError() != cudaSuccess) return PERQ_ERR_CUDA;
     }

@@ -62,8 +62,10 @@ __global__ void __launch_bounds__(ST_THREADS) perq_stats_partial_kernel(StatsPar
     const bool want_blocks = (p.ws_block != nullptr) || (p.token_max != nullptr);
     const uint4 zero4 = make_uint4(0u, 0u, 0u, 0u);
 
-    uint4 w[R][KC];
-    auto load_batch = [&](long long t) {
+    // two batches of rows in flight in registers: while one is reduced the other is still arriving
+    constexpr int NBUF = KC >= 8 ? 1 : 2;      // (the widest rows leave registers for one batch only)
+    uint4 wbuf[NBUF][R][KC];
+    auto load_batch = [&](uint4 (&w)[R][KC], long long t) {
 #pragma unroll
         for (int r = 0; r < R; ++r) {
             const uint4 *src = (const uint4 *)(p.x + (size_t)(t + r) * d);
@@ -74,10 +76,11 @@ __global__ void __launch_bounds__(ST_THREADS) perq_stats_partial_kernel(StatsPar
             }
         }
     };
-    if (t0 < t1) load_batch(t0);
+    load_batch(wbuf[0], t0);
+    if (NBUF == 2) load_batch(wbuf[NBUF - 1], t0 + R);
     __syncthreads();
 
-    for (long long t = t0; t < t1; t += R) {
+    auto process = [&](uint4 (&w)[R][KC], long long t) {
         // ---- channel sums from the registers; rows to shared memory for the gather
 #pragma unroll
         for (int r = 0; r < R; ++r) {
@@ -90,15 +93,28 @@ __global__ void __launch_bounds__(ST_THREADS) perq_stats_partial_kernel(StatsPar
                     csum[k][2 * e + 1] += __uint_as_float(ww[e] & 0x7fff0000u);
                 }
                 const int c = tid + k * ST_THREADS;
-                if (want_blocks && c < nchunks) ((uint4 *)(raw + (size_t)r * d))[c] = w[r][k];
+                if (want_blocks && c < nchunks) {
+                    if (p.perm) {
+                        ((uint4 *)(raw + (size_t)r * d))[c] = w[r][k];
+                    } else {      // identity: the chunk's l1 norm is this thread's own eight values
+                        float s = 0.0f;
+#pragma unroll
+                        for (int e = 0; e < 4; ++e) {
+                            s += __uint_as_float((ww[e] << 16) & 0x7fffffffu);
+                            s += __uint_as_float(ww[e] & 0x7fff0000u);
+                        }
+                        cs[(size_t)r * nchunks + c] = s;
+                    }
+                }
             }
         }
-        // ---- next batch: loads in flight while this one is reduced
-        if (t + R < t1) load_batch(t + R);
-        if (!want_blocks) continue;
+        // ---- refill these registers with the batch after next
+        load_batch(w, t + NBUF * R);
+        if (!want_blocks) return;
         __syncthreads();
 #pragma unroll
         for (int r = 0; r < R; ++r) {
+            if (!p.perm) break;
             const uint16_t *row = raw + (size_t)r * d;
 #pragma unroll
             for (int k = 0; k < KC; ++k) {
@@ -116,7 +132,7 @@ __global__ void __launch_bounds__(ST_THREADS) perq_stats_partial_kernel(StatsPar
                 }
             }
         }
-        __syncthreads();
+        if (p.perm) __syncthreads();
         const int cpb = 1 << (L - 3);          // chunks per block
         float mx[R];
 #pragma unroll
@@ -149,6 +165,10 @@ __global__ void __launch_bounds__(ST_THREADS) perq_stats_partial_kernel(StatsPar
             }
         }
         __syncthreads();
+    };
+    for (long long t = t0; t < t1; t += NBUF * R) {
+        process(wbuf[0], t);
+        if (NBUF == 2 && t + R < t1) process(wbuf[NBUF - 1], t + R);
     }
 
     if (p.ws_chan) {
@@ -171,19 +191,43 @@ __global__ void __launch_bounds__(ST_THREADS) perq_stats_partial_kernel(StatsPar
     }
 }
 
-__global__ void perq_stats_reduce_kernel(const float *ws_chan, const float *ws_block, int n_cta, int d, int nb,
-                                         float inv_T, float *chan_abs_sum, float *block_l1_mean)
+// 256 threads: 64 outputs, each summed by 4 threads over a quarter of the CTA slices, then
+// combined in a fixed order (deterministic).
+__global__ void __launch_bounds__(256) perq_stats_reduce_kernel(const float *ws_chan, const float *ws_block, int n_cta, int d,
+                                                                int nb, float inv_T, float *chan_abs_sum, float *block_l1_mean)
 {
-    const int i = blockIdx.x * blockDim.x + threadIdx.x;
+    __shared__ float part[2][4][64];
+    const int o = threadIdx.x & 63, quarter = threadIdx.x >> 6;
+    const int i = blockIdx.x * 64 + o;
+    const int per = (n_cta + 3) / 4;
+    const int c0 = quarter * per, c1 = min(n_cta, c0 + per);
+    float sc = 0.0f, sb = 0.0f;
+    // eight independent loads at a time, added in slice order (x + 0 is exact, so padding is harmless)
     if (chan_abs_sum && i < d) {
-        float s = 0.0f;
-        for (int c = 0; c < n_cta; ++c) s += ws_chan[(size_t)c * d + i];
-        chan_abs_sum[i] = s;
+        for (int c = c0; c < c1; c += 8) {
+            float v[8];
+#pragma unroll
+            for (int j = 0; j < 8; ++j) v[j] = (c + j < c1) ? ws_chan[(size_t)(c + j) * d + i] : 0.0f;
+#pragma unroll
+            for (int j = 0; j < 8; ++j) sc += v[j];
+        }
     }
     if (block_l1_mean && i < nb) {
-        float s = 0.0f;
-        for (int c = 0; c < n_cta; ++c) s += ws_block[(size_t)c * nb + i];
-        block_l1_mean[i] = s * inv_T;
+        for (int c = c0; c < c1; c += 8) {
+            float v[8];
+#pragma unroll
+            for (int j = 0; j < 8; ++j) v[j] = (c + j < c1) ? ws_block[(size_t)(c + j) * nb + i] : 0.0f;
+#pragma unroll
+            for (int j = 0; j < 8; ++j) sb += v[j];
+        }
+    }
+    part[0][quarter][o] = sc;
+    part[1][quarter][o] = sb;
+    __syncthreads();
+    if (quarter == 0) {
+        if (chan_abs_sum && i < d) chan_abs_sum[i] = ((part[0][0][o] + part[0][1][o]) + part[0][2][o]) + part[0][3][o];
+        if (block_l1_mean && i < nb)
+            block_l1_mean[i] = (((part[1][0][o] + part[1][1][o]) + part[1][2][o]) + part[1][3][o]) * inv_T;
     }
 }
 
