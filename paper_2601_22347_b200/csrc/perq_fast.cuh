@@ -736,9 +736,19 @@ __global__ void __launch_bounds__(FAST_THREADS, 1) perq_fast_kernel(FastParams p
         }
 
         // ---- fp32 maxima per slot
+        // (per token and MX only need them in rare paths and recompute them there: fewer live registers)
         float ms[8];
+        auto slot_maxima = [&]() {
 #pragma unroll
-        for (int s = 0; s < 8; ++s) ms[s] = fmaxf(max3abs(fabsf(v[s][0].x), v[s][0].y, v[s][1].x), fabsf(v[s][1].y));
+            for (int s = 0; s < 8; ++s) ms[s] = fmaxf(max3abs(fabsf(v[s][0].x), v[s][0].y, v[s][1].x), fabsf(v[s][1].y));
+        };
+        auto pair_max = [&](int m) {     // magnitude maximum of the lane's eight values of slots 2m, 2m+1
+            float a = max3abs(fabsf(v[2 * m][0].x), v[2 * m][0].y, v[2 * m][1].x);
+            a = max3abs(a, v[2 * m][1].y, v[2 * m + 1][0].x);
+            a = max3abs(a, v[2 * m + 1][0].y, v[2 * m + 1][1].x);
+            return fmaxf(a, fabsf(v[2 * m + 1][1].y));
+        };
+        if (MODE == MODE_G128) slot_maxima();
 
         const uint32_t code_buf = code_base + par2 * SEG_CODE_BYTES;
         const uint32_t code_addr0 = code_buf + code_lane;
@@ -749,8 +759,9 @@ __global__ void __launch_bounds__(FAST_THREADS, 1) perq_fast_kernel(FastParams p
         if (MODE == MODE_TOKEN || MODE == MODE_G128) {
             // lane maximum, then the maximum of the scale range in fp32 (a32); the exact maximum
             // (a_bits, bit pattern of a double) only where it is known without waiting
-            const float lane_max = fmaxf(fmaxf(fmaxf(ms[0], ms[1]), fmaxf(ms[2], ms[3])),
-                                         fmaxf(fmaxf(ms[4], ms[5]), fmaxf(ms[6], ms[7])));
+            const float lane_max = (MODE == MODE_G128)
+                ? fmaxf(fmaxf(fmaxf(ms[0], ms[1]), fmaxf(ms[2], ms[3])), fmaxf(fmaxf(ms[4], ms[5]), fmaxf(ms[6], ms[7])))
+                : fmaxf(fmaxf(pair_max(0), pair_max(1)), fmaxf(pair_max(2), pair_max(3)));
             float a32;
             unsigned long long a_bits = 0ull;
             bool have_exact = true;          // warp-uniform: a_bits is the range's exact maximum
@@ -865,6 +876,7 @@ __global__ void __launch_bounds__(FAST_THREADS, 1) perq_fast_kernel(FastParams p
             // ---- per token: the exact row maximum and the stored scale, by the candidate warps only
             if (MODE == MODE_TOKEN && is_cand) {
                 const float thr_row = a32 * (1.0f - 2.0f * err_rel - 2.4e-7f);
+                slot_maxima();
                 uint32_t slot_mask = 0u;
 #pragma unroll
                 for (int s = 0; s < 8; ++s) slot_mask |= (ms[s] >= thr_row) ? (1u << s) : 0u;
@@ -1003,8 +1015,7 @@ __global__ void __launch_bounds__(FAST_THREADS, 1) perq_fast_kernel(FastParams p
             // the shared exponent of slot pair m = q, then the quad exchanges multipliers.
             float a32, bref;
             {
-                const float g0 = fmaxf(ms[0], ms[1]), g1 = fmaxf(ms[2], ms[3]);
-                const float g2 = fmaxf(ms[4], ms[5]), g3 = fmaxf(ms[6], ms[7]);
+                const float g0 = pair_max(0), g1 = pair_max(1), g2 = pair_max(2), g3 = pair_max(3);
                 const bool q1 = (q & 1) != 0, q2 = (q & 2) != 0;
                 float k0 = q2 ? g2 : g0, k1 = q2 ? g3 : g1;
                 const float s0 = q2 ? g0 : g2, s1 = q2 ? g1 : g3;
@@ -1087,7 +1098,7 @@ __global__ void __launch_bounds__(FAST_THREADS, 1) perq_fast_kernel(FastParams p
                         const int owner = (lane & 28) | m;
                         const float a_m = __shfl_sync(qmask, a32, owner), tol_m = __shfl_sync(qmask, tol, owner);
                         const float thr = a_m - tol_m;
-                        const bool has = fmaxf(ms[2 * m], ms[2 * m + 1]) >= thr;
+                        const bool has = pair_max(m) >= thr;
                         unsigned cq = __ballot_sync(qmask, has) & qmask;
                         double best = 0.0;
                         while (cq) {

@@ -342,3 +342,109 @@ def test_block_l1_stats(B, oracle, T, d, b, perm):
     only_tok = B.perq_block_l1_stats(x, pd, b, want=("token",))
     torch.cuda.synchronize()
     assert only_tok[0] is None and only_tok[1] is None and torch.equal(only_tok[2], token)
+
+
+# ------------------------------------------------------------------ fast-kernel variants added later: permuted, full-vector
+
+@pytest.mark.parametrize("fmt,group", [("int4", 0), ("int4", 128), ("mxfp4", 32)])
+@pytest.mark.parametrize("d,T,b", [(1024, 70, 16), (2048, 333, 32), (4096, 150, 64), (8192, 40, 128), (14336, 20, 32)])
+def test_permuted_fast_path_matrix(B, oracle, d, T, b, fmt, group):
+    if group == 0 and d == 14336:
+        pytest.skip("per-token scales with 14 segments per row go to the generic kernel (covered elsewhere)")
+    bits, _ = inputs.student_t_outliers(T, d, 3.0, max(2, d // 256), 100.0, seed=2000 + d + b)
+    bits[2] = 0
+    bits[4, 64:320] = 0
+    perm = inputs.random_perm(d, 2001 + d)
+    check(B, oracle, inputs.Workload("perm-fast", bits, perm, b, fmt, group, 0))
+    assert B.perq_device_error() == 0
+
+
+@pytest.mark.parametrize("fmt,group", [("int4", 0), ("mxfp4", 32)])
+@pytest.mark.parametrize("d,T", [(1024, 40), (2048, 64), (4096, 24), (8192, 12)])
+def test_full_vector_fast_path(B, oracle, d, T, fmt, group):
+    bits, _ = inputs.laplace_outliers(T, d, 4, 200.0, seed=3000 + d)
+    bits[1] = 0
+    bits[3, : d // 2] = 0
+    check(B, oracle, inputs.Workload("full-fast", bits, None, d, fmt, group, 0))
+    assert B.perq_device_error() == 0
+
+
+def test_rows_with_several_maximum_candidates(B, oracle):
+    """Rows whose largest rotated magnitude is attained (exactly) in several places -- in one
+    warp's segment, in several segments, in every block -- take the paths that resolve the
+    exact maximum at once and combine it across the warps of a row."""
+    d = 4096
+    rng = np.random.default_rng(31)
+    x = (rng.standard_normal((12, d)) * 0.01).astype(np.float32)
+    x[0, 5] = 300.0;  x[0, 5 + 1024] = 300.0                 # equal outliers in two segments
+    x[1, 7] = -300.0; x[1, 7 + 32] = 300.0                   # and in two blocks of one segment
+    x[2, :] = 0.0;    x[2, 100] = 64.0                       # a lone entry: every output of its block ties
+    x[3, :] = 0.0;    x[3, 0::1024] = 8.0                    # one per segment, identical
+    x[4, :] = 1.0                                            # constant row: first output of every block
+    x[5, :] = 0.0;    x[5, 2049] = 1.0; x[5, 3] = -1.0
+    x[6, 9] = 300.0;  x[6, 9 + 2048] = 300.0; x[6, 9 + 3072] = -300.0
+    bits = inputs.f32_to_bf16_bits(x)
+    for b in (16, 32, 128, 4096):
+        for fmt, g in (("int4", 0), ("int4", 128), ("mxfp4", 32)):
+            if b == 4096 and g == 128:
+                continue
+            check(B, oracle, inputs.Workload("multi-cand", bits, None, b, fmt, g, 0))
+    p = inputs.random_perm(d, 32)
+    for b in (32, 128):
+        for fmt, g in (("int4", 0), ("int4", 128), ("mxfp4", 32)):
+            check(B, oracle, inputs.Workload("multi-cand-perm", bits, p, b, fmt, g, 0))
+    assert B.perq_device_error() == 0
+
+
+def test_exact_ties_through_the_permuted_and_full_vector_paths(B, oracle):
+    """Constructed exact rounding ties (see test_constructed_exact_ties) must also be resolved like
+    exact arithmetic when the row goes through the permutation gather, and for whole-row blocks."""
+    import scipy.linalg
+    rng = np.random.default_rng(28)
+    # b = 16 blocks of a d = 2048 row, then scattered by the inverse of a permutation
+    H = scipy.linalg.hadamard(16)
+    rows = []
+    for _ in range(16):
+        blocks = []
+        for j in range(128):
+            ystar = rng.integers(-13, 14, size=16) * 0.5
+            ystar[rng.integers(0, 16)] = 7.0 if j == 0 else ystar[0]
+            blocks.append((ystar @ H) / 4.0)
+        rows.append(np.concatenate(blocks))
+    xp = np.array(rows, np.float32)                      # the permuted row the kernel should see
+    perm = inputs.random_perm(2048, 29)
+    x = np.empty_like(xp)
+    x[:, perm] = xp                                      # x[perm[i]] = xp[i]
+    bits = inputs.f32_to_bf16_bits(x)
+    assert np.array_equal(inputs.bf16_bits_to_f32(bits), x)
+    for fmt, g, scale in (("int4", 0, 1.0), ("int4", 128, 1.0), ("mxfp4", 32, 0.5)):
+        rep = check(B, oracle, inputs.Workload("ties-perm", inputs.f32_to_bf16_bits(x * np.float32(scale)), perm, 16, fmt, g, 0))
+        assert rep["code_mismatch_exempt"] == 0
+    # whole-row block, d = 1024 (sqrt(d) = 32): rotated values are small half-integers, maximum 7
+    H = scipy.linalg.hadamard(1024)
+    rows = []
+    for _ in range(6):
+        ystar = rng.integers(-13, 14, size=1024) * 0.5
+        ystar[rng.integers(0, 1024)] = 7.0
+        rows.append((ystar @ H) / 32.0)
+    x = np.array(rows, np.float64)
+    bits = inputs.f32_to_bf16_bits(x.astype(np.float32))
+    if np.array_equal(inputs.bf16_to_f64(bits), x):      # representable in bf16: exact ties survive the cast
+        rep = check(B, oracle, inputs.Workload("ties-full", bits, None, 1024, "int4", 0, 0))
+        assert rep["code_mismatch_exempt"] == 0
+    else:                                                # otherwise still a valid parity case
+        check(B, oracle, inputs.Workload("ties-full", bits, None, 1024, "int4", 0, 0))
+
+
+def test_permuted_path_many_rows_per_group(B, oracle):
+    # enough rows that every group goes round its three-stage ring many times, and the deferred
+    # scale records fill and are served in the middle of the run
+    w = inputs.config2(T=16384, b=32)
+    w.group = 0
+    rows = np.sort(np.random.default_rng(7).choice(w.T, 64, replace=False))
+    rows[0], rows[-1] = 0, w.T - 1
+    check(B, oracle, w, rows=rows)
+    w = inputs.config5(T=2048, b=64)
+    rows = np.sort(np.random.default_rng(8).choice(w.T, 24, replace=False))
+    check(B, oracle, w, rows=rows)
+    assert B.perq_device_error() == 0
