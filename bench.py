@@ -155,7 +155,7 @@ def main():
 
     import numpy as np
     import torch
-    from paper_2601_22347_b200 import binding as B, inputs
+    from paper_2601_22347_b200 import binding as B, inputs, sharding
 
     world = int(os.environ.get("WORLD_SIZE", "1"))
     rank = int(os.environ.get("RANK", "0"))
@@ -213,10 +213,7 @@ def main():
     clocks = sampler.stop() if rank == 0 else None
     total_ms = ev[0].elapsed_time(ev[-1])
     per_launch_ms = [ev[i].elapsed_time(ev[i + 1]) for i in range(args.steps)]
-    t = torch.tensor([total_ms], dtype=torch.float64, device="cuda")
-    if dist is not None:
-        dist.all_reduce(t, op=dist.ReduceOp.MAX)
-    total_ms = float(t.item())
+    total_ms = sharding.max_over_ranks(total_ms, device="cuda")
     ms_per_step = total_ms / args.steps
     value = world * bytes_per_step / (ms_per_step * 1e-3) / 1e9
 
@@ -233,10 +230,7 @@ def main():
     for _ in range(e2e_steps):
         B.perq_rotate_quantize_host(xh, None, B_HEAD, fmt, GROUP_HEAD, ch, sh, ws)   # synchronises its stream
     e2e_s = (time.perf_counter() - t0) / e2e_steps
-    t = torch.tensor([e2e_s], dtype=torch.float64, device="cuda")
-    if dist is not None:
-        dist.all_reduce(t, op=dist.ReduceOp.MAX)
-    e2e_s = float(t.item())
+    e2e_s = sharding.max_over_ranks(e2e_s, device="cuda")
     e2e = {"value": world * bytes_per_step / e2e_s / 1e9, "unit": UNIT,
            "h2d_bytes_per_step": int(xh.numel() * 2), "d2h_bytes_per_step": int(ch.numel() + sh.numel() * 4),
            "ms_per_step": e2e_s * 1e3, "api": "perq_rotate_quantize_host"}
@@ -292,6 +286,36 @@ def main():
         by = 4096 * 8192 * 2
         sweep.append({"call": "perq_block_l1_stats", "T": 4096, "d": 8192, "b": 32, "ms": ms,
                       "GB/s": by / (ms * 1e-3) / 1e9, "frac_of_" + peak_kind: by / (ms * 1e-3) / 1e9 / peak})
+        del xs, outs, base
+
+        # the other workloads, with their permutations (cold inputs: rings larger than L2)
+        def time_workload(name, bits, perm, b, f, grp):
+            T, d = bits.shape
+            fcode = B.FMT_BY_NAME[f]
+            ring = max(2, int(300e6 // max(1, T * d * 2)) + 1)
+            ring = min(ring, 64)
+            x0 = torch.from_numpy(bits.view(np.int16).copy()).cuda().view(torch.bfloat16)
+            xr = [x0] + [torch.roll(x0, shifts=3 * (i + 1), dims=0).contiguous() if T > 1 else x0.clone()
+                         for i in range(ring - 1)]
+            orr = [B.alloc_outputs(T, d, fcode, grp, x0.device) for _ in range(ring)]
+            pd = None if perm is None else torch.from_numpy(perm).cuda()
+            ms = time_calls(lambda i: B.perq_rotate_quantize(xr[i % ring], pd, b, fcode, grp,
+                                                             out_codes=orr[i % ring][0], out_scales=orr[i % ring][1]))
+            by = bytes_per_token(d, f, grp) * T
+            gbs = by / (ms * 1e-3) / 1e9
+            sweep.append({"call": "perq_rotate_quantize", "workload": name, "T": T, "d": d, "b": b, "fmt": f, "group": grp,
+                          "perm": perm is not None, "us": ms * 1e3, "GB/s": gbs, "frac_of_" + peak_kind: gbs / peak,
+                          "Mtokens/s": T / ms / 1e3})
+
+        w2 = inputs.config2(T=4096, b=32)
+        time_workload("cfg2", w2.x, w2.perm, 32, "int4", 128)
+        chan, _, _ = B.perq_block_l1_stats(x3[0], None, 32, want=("chan",), workspace=wsb)
+        torch.cuda.synchronize()
+        time_workload("cfg3 (MassDiff permutation)", w3.x, B.perq_massdiff_perm(chan.cpu().numpy(), 32), 32, "mxfp4", 32)
+        del x3
+        for T5 in (1, 16, 128, 1024, 16384):
+            w5 = inputs.config5(T=T5, b=32)
+            time_workload("cfg5", w5.x, w5.perm, 32, "int4", 128)
 
     cpu_baseline = None
     if not args.no_cpu_baseline:
