@@ -209,6 +209,7 @@ struct StatsPlan {
     size_t smem;
     size_t ws_bytes;
     int kc;            // 16-byte chunks of a row per thread
+    int n_stages;      // stages of the row ring in shared memory
 };
 
 template <int KC>
@@ -225,8 +226,12 @@ int plan_stats(int64_t T, int32_t d, int32_t b, StatsPlan *plan)
     plan->rows_per_cta = (int)std::min<long long>(rows, 1 << 30);
     plan->n_cta = (int)std::max<long long>(1, (T + rows - 1) / rows);
     plan->kc = d <= 4096 ? 1 : d <= 8192 ? 2 : d <= 16384 ? 4 : 8;
-    const size_t rif = 8 / plan->kc;      // rows in flight per CTA
-    plan->smem = (rif + 1) * (size_t)d * 2 + rif * (size_t)(d / 8) * 4 + rif * 16 * 4;
+    const size_t rpb = 8 / plan->kc;      // rows per batch
+    auto smem_for = [&](size_t nst) {
+        return nst * rpb * (size_t)d * 2 + (size_t)d * 2 + rpb * (size_t)(d / 8) * 4 + rpb * 16 * 4 + nst * 8 + 128;
+    };
+    plan->n_stages = smem_for(3) <= 220 * 1024 ? 3 : 2;
+    plan->smem = smem_for((size_t)plan->n_stages);
     plan->ws_bytes = (size_t)plan->n_cta * ((size_t)d + (size_t)(d / b)) * sizeof(float);
     return PERQ_OK;
 }
@@ -371,6 +376,7 @@ int perq_block_l1_stats(const void *x, const int32_t *perm, int64_t T, int32_t d
     p.d = d;
     p.log2b = ilog2(b);
     p.rows_per_cta = plan.rows_per_cta;
+    p.n_stages = plan.n_stages;
     float *ws = static_cast<float *>(workspace);
     p.ws_chan = chan_abs_sum ? ws : nullptr;
     p.ws_block = block_l1_mean ? ws + (size_t)plan.n_cta * d : nullptr;

@@ -1,8 +1,8 @@
 // Calibration statistic kernels: per-channel sum of |x|, per-block mean l1 norm and
 // per-token max block l1 norm under an optional permutation.
 //
-// Phase 1: each CTA walks a contiguous slab of rows, a few rows at a time (64 KB of loads in
-// flight per CTA, the next batch being fetched while the current one is reduced), keeps
+// Phase 1: each CTA walks a contiguous slab of rows, 64 KB of rows at a time through a ring of
+// bulk-copied shared-memory stages, keeps
 // per-channel and per-block partial sums in registers (every thread owns fixed columns /
 // blocks), and writes them to its own slice of the workspace.  Rows go through shared memory
 // only when a block statistic needs the gather through the permutation.
@@ -11,6 +11,8 @@
 #pragma once
 #include <cuda_runtime.h>
 #include <stdint.h>
+
+#include "perq_fast.cuh"   // mbarrier / bulk-copy wrappers, device error word
 
 namespace perq {
 
@@ -27,22 +29,28 @@ struct StatsParams {
     float *ws_chan;      // [n_cta, d]
     float *ws_block;     // [n_cta, d/b]
     float *token_max;    // [T] or null
+    int n_stages;        // shared-memory stages of the row ring
 };
 
 __device__ __forceinline__ float abs_bf16(uint16_t h) { return __uint_as_float(((uint32_t)h & 0x7fffu) << 16); }
 
-// KC = 16-byte chunks of a row per thread (d <= KC * 4096); R = rows in flight per CTA, chosen so
-// that every thread always has 8 loads of 16 bytes outstanding (64 KB per CTA).
+// KC = 16-byte chunks of a row per thread (d <= KC * 4096); R = rows per batch (64 KB).  Batches of
+// consecutive rows are contiguous in global memory: one elected thread fetches each with a single
+// cp.async.bulk into a ring of shared-memory stages (bulk copies are not limited by the load
+// queue of the SM the way per-thread loads are), everybody reads its columns from there.
 template <int KC>
 __global__ void __launch_bounds__(ST_THREADS) perq_stats_partial_kernel(StatsParams p)
 {
     constexpr int R = 8 / KC;
-    extern __shared__ __align__(16) unsigned char smem[];
+    const int NST = p.n_stages;                   // 3, or 2 where 3 stages would not fit
+    extern __shared__ __align__(128) unsigned char smem[];
     const int d = p.d, L = p.log2b, nb = d >> L, nchunks = d >> 3;
-    uint16_t *sperm = (uint16_t *)smem;                                  // [d] permutation (d <= 32768 fits 16 bits)
-    uint16_t *raw = sperm + d;                                           // [R][d] rows, original order
-    float *cs = (float *)(smem + (size_t)(R + 1) * d * 2);               // [R][d/8] per-chunk l1 of the permuted rows
+    const size_t stage_bytes = (size_t)R * d * 2;
+    uint16_t *stages = (uint16_t *)smem;                                 // [NST][R][d] rows, original order
+    uint16_t *sperm = (uint16_t *)(smem + NST * stage_bytes);            // [d] permutation (d <= 32768 fits 16 bits)
+    float *cs = (float *)(smem + NST * stage_bytes + (size_t)d * 2);     // [R][d/8] per-chunk l1 of the permuted rows
     float *red = cs + (size_t)R * nchunks;                               // [R][16]
+    uint64_t *full = (uint64_t *)(red + R * 16);                         // [NST] mbarriers
     const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
 
     for (int i = tid; i < d; i += ST_THREADS) {
@@ -60,79 +68,70 @@ __global__ void __launch_bounds__(ST_THREADS) perq_stats_partial_kernel(StatsPar
     const long long t0 = (long long)blockIdx.x * p.rows_per_cta;
     const long long t1 = min(p.T, t0 + p.rows_per_cta);
     const bool want_blocks = (p.ws_block != nullptr) || (p.token_max != nullptr);
-    const uint4 zero4 = make_uint4(0u, 0u, 0u, 0u);
 
-    // two batches of rows in flight in registers: while one is reduced the other is still arriving
-    constexpr int NBUF = KC >= 8 ? 1 : 2;      // (the widest rows leave registers for one batch only)
-    uint4 wbuf[NBUF][R][KC];
-    auto load_batch = [&](uint4 (&w)[R][KC], long long t) {
-#pragma unroll
-        for (int r = 0; r < R; ++r) {
-            const uint4 *src = (const uint4 *)(p.x + (size_t)(t + r) * d);
-#pragma unroll
-            for (int k = 0; k < KC; ++k) {
-                const int c = tid + k * ST_THREADS;
-                w[r][k] = (t + r < t1 && c < nchunks) ? __ldcs(src + c) : zero4;
-            }
+    auto fetch = [&](int stage, long long t) {      // one thread: rows t .. t+R-1 (those below t1) into a stage
+        if (t < t1) {
+            const uint32_t bytes = (uint32_t)(min((long long)R, t1 - t) * d * 2);
+            mbar_expect_tx(smem_u32(&full[stage]), bytes);
+            bulk_load(smem_u32(stages + (size_t)stage * R * d), p.x + (size_t)t * d, bytes, smem_u32(&full[stage]));
         }
     };
-    load_batch(wbuf[0], t0);
-    if (NBUF == 2) load_batch(wbuf[NBUF - 1], t0 + R);
+    if (tid == 0) {
+        for (int s = 0; s < NST; ++s) mbar_init(smem_u32(&full[s]), 1);
+        asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+        for (int s = 0; s < NST; ++s) fetch(s, t0 + (long long)s * R);
+    }
     __syncthreads();
 
-    auto process = [&](uint4 (&w)[R][KC], long long t) {
-        // ---- channel sums from the registers; rows to shared memory for the gather
+    uint32_t it = 0;
+    for (long long t = t0; t < t1; t += R, ++it) {
+        const int stage = (int)(it % NST);
+        if (!mbar_wait(smem_u32(&full[stage]), (it / NST) & 1u)) {
+            if (tid == 0) atomicOr(&g_perq_device_error, 8u);
+            return;
+        }
+        const uint16_t *rows = stages + (size_t)stage * R * d;
+        // ---- channel sums; chunk l1 norms (directly, or through the permutation gather)
 #pragma unroll
         for (int r = 0; r < R; ++r) {
+            if (t + r < t1) {
 #pragma unroll
-            for (int k = 0; k < KC; ++k) {
-                const uint32_t ww[4] = {w[r][k].x, w[r][k].y, w[r][k].z, w[r][k].w};
-#pragma unroll
-                for (int e = 0; e < 4; ++e) {
-                    csum[k][2 * e] += __uint_as_float((ww[e] << 16) & 0x7fffffffu);
-                    csum[k][2 * e + 1] += __uint_as_float(ww[e] & 0x7fff0000u);
-                }
-                const int c = tid + k * ST_THREADS;
-                if (want_blocks && c < nchunks) {
-                    if (p.perm) {
-                        ((uint4 *)(raw + (size_t)r * d))[c] = w[r][k];
-                    } else {      // identity: the chunk's l1 norm is this thread's own eight values
+                for (int k = 0; k < KC; ++k) {
+                    const int c = tid + k * ST_THREADS;
+                    if (c < nchunks) {
+                        const uint4 w = ((const uint4 *)(rows + (size_t)r * d))[c];
+                        const uint32_t ww[4] = {w.x, w.y, w.z, w.w};
                         float s = 0.0f;
 #pragma unroll
                         for (int e = 0; e < 4; ++e) {
-                            s += __uint_as_float((ww[e] << 16) & 0x7fffffffu);
-                            s += __uint_as_float(ww[e] & 0x7fff0000u);
+                            const float lo = __uint_as_float((ww[e] << 16) & 0x7fffffffu);
+                            const float hi = __uint_as_float(ww[e] & 0x7fff0000u);
+                            csum[k][2 * e] += lo;
+                            csum[k][2 * e + 1] += hi;
+                            s += lo;
+                            s += hi;
                         }
-                        cs[(size_t)r * nchunks + c] = s;
+                        if (want_blocks) {
+                            if (p.perm) {
+                                const uint4 pi = ((const uint4 *)sperm)[c];
+                                const uint32_t pp[4] = {pi.x, pi.y, pi.z, pi.w};
+                                const uint16_t *row = rows + (size_t)r * d;
+                                s = 0.0f;
+#pragma unroll
+                                for (int e = 0; e < 4; ++e) {
+                                    s += abs_bf16(row[pp[e] & 0xffffu]);
+                                    s += abs_bf16(row[pp[e] >> 16]);
+                                }
+                            }
+                            cs[(size_t)r * nchunks + c] = s;
+                        }
                     }
                 }
             }
         }
-        // ---- refill these registers with the batch after next
-        load_batch(w, t + NBUF * R);
-        if (!want_blocks) return;
-        __syncthreads();
-#pragma unroll
-        for (int r = 0; r < R; ++r) {
-            if (!p.perm) break;
-            const uint16_t *row = raw + (size_t)r * d;
-#pragma unroll
-            for (int k = 0; k < KC; ++k) {
-                const int c = tid + k * ST_THREADS;
-                if (c < nchunks) {
-                    const uint4 pi = ((const uint4 *)sperm)[c];
-                    const uint32_t pp[4] = {pi.x, pi.y, pi.z, pi.w};
-                    float s = 0.0f;
-#pragma unroll
-                    for (int e = 0; e < 4; ++e) {
-                        s += abs_bf16(row[pp[e] & 0xffffu]);
-                        s += abs_bf16(row[pp[e] >> 16]);
-                    }
-                    cs[(size_t)r * nchunks + c] = s;
-                }
-            }
-        }
-        if (p.perm) __syncthreads();
+        __syncthreads();                                 // every thread is done with the stage; cs is complete
+        if (tid == 0) fetch(stage, t + (long long)NST * R);
+        if (!want_blocks) continue;
         const int cpb = 1 << (L - 3);          // chunks per block
         float mx[R];
 #pragma unroll
@@ -164,11 +163,7 @@ __global__ void __launch_bounds__(ST_THREADS) perq_stats_partial_kernel(StatsPar
                 p.token_max[t + tid] = m;
             }
         }
-        __syncthreads();
-    };
-    for (long long t = t0; t < t1; t += NBUF * R) {
-        process(wbuf[0], t);
-        if (NBUF == 2 && t + R < t1) process(wbuf[NBUF - 1], t + R);
+        __syncthreads();                                 // cs and red may be overwritten by the next batch
     }
 
     if (p.ws_chan) {
