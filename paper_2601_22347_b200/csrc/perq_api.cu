@@ -228,7 +228,7 @@ int plan_stats(int64_t T, int32_t d, int32_t b, StatsPlan *plan)
     plan->kc = d <= 4096 ? 1 : d <= 8192 ? 2 : d <= 16384 ? 4 : 8;
     const size_t rpb = 8 / plan->kc;      // rows per batch
     auto smem_for = [&](size_t nst) {
-        return nst * rpb * (size_t)d * 2 + (size_t)d * 2 + rpb * (size_t)(d / 8) * 4 + rpb * 16 * 4 + nst * 8 + 128;
+        return nst * rpb * (size_t)d * 2 + (size_t)d * 2 + rpb * (size_t)(d / 8) * 4 + 2 * rpb * 16 * 4 + nst * 8 + 128;
     };
     plan->n_stages = smem_for(3) <= 220 * 1024 ? 3 : 2;
     plan->smem = smem_for((size_t)plan->n_stages);

@@ -49,25 +49,27 @@ __global__ void __launch_bounds__(ST_THREADS) perq_stats_partial_kernel(StatsPar
     uint16_t *stages = (uint16_t *)smem;                                 // [NST][R][d] rows, original order
     uint16_t *sperm = (uint16_t *)(smem + NST * stage_bytes);            // [d] permutation (d <= 32768 fits 16 bits)
     float *cs = (float *)(smem + NST * stage_bytes + (size_t)d * 2);     // [R][d/8] per-chunk l1 of the permuted rows
-    float *red = cs + (size_t)R * nchunks;                               // [R][16]
-    uint64_t *full = (uint64_t *)(red + R * 16);                         // [NST] mbarriers
+    float *red = cs + (size_t)R * nchunks;                               // [2][R][16]
+    uint64_t *full = (uint64_t *)(red + 2 * R * 16);                     // [NST] mbarriers
     const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
 
     for (int i = tid; i < d; i += ST_THREADS) {
         int q = p.perm ? __ldg(p.perm + i) : i;
         sperm[i] = (uint16_t)min(max(q, 0), d - 1);
     }
-    float csum[KC][8];
+    float2 csum[KC][4];      // per-channel sums of |x|, as pairs for the packed fp32 add
     float bsum[KC];
 #pragma unroll
     for (int k = 0; k < KC; ++k) {
         bsum[k] = 0.0f;
 #pragma unroll
-        for (int e = 0; e < 8; ++e) csum[k][e] = 0.0f;
+        for (int e = 0; e < 4; ++e) csum[k][e] = make_float2(0.0f, 0.0f);
     }
     const long long t0 = (long long)blockIdx.x * p.rows_per_cta;
     const long long t1 = min(p.T, t0 + p.rows_per_cta);
     const bool want_blocks = (p.ws_block != nullptr) || (p.token_max != nullptr);
+    const int cpb = 1 << (L - 3);                 // 16-byte chunks per block
+    const bool shuffle_blocks = cpb <= 32;        // a block's chunks sit in adjacent lanes of one warp
 
     auto fetch = [&](int stage, long long t) {      // one thread: rows t .. t+R-1 (those below t1) into a stage
         if (t < t1) {
@@ -91,49 +93,75 @@ __global__ void __launch_bounds__(ST_THREADS) perq_stats_partial_kernel(StatsPar
             return;
         }
         const uint16_t *rows = stages + (size_t)stage * R * d;
-        // ---- channel sums; chunk l1 norms (directly, or through the permutation gather)
+        // ---- channel sums; chunk l1 norms (directly, or through the permutation gather); blocks of up
+        // to 256 channels are summed with shuffles over the adjacent lanes that hold their chunks
+        float mx[R];
 #pragma unroll
         for (int r = 0; r < R; ++r) {
-            if (t + r < t1) {
+            mx[r] = 0.0f;
+            const bool live = t + r < t1;
 #pragma unroll
-                for (int k = 0; k < KC; ++k) {
-                    const int c = tid + k * ST_THREADS;
-                    if (c < nchunks) {
-                        const uint4 w = ((const uint4 *)(rows + (size_t)r * d))[c];
-                        const uint32_t ww[4] = {w.x, w.y, w.z, w.w};
-                        float s = 0.0f;
+            for (int k = 0; k < KC; ++k) {
+                const int c = tid + k * ST_THREADS;
+                float s = 0.0f;
+                if (live && c < nchunks) {
+                    const uint4 w = ((const uint4 *)(rows + (size_t)r * d))[c];
+                    const uint32_t ww[4] = {w.x, w.y, w.z, w.w};
+                    float2 m[4];
 #pragma unroll
-                        for (int e = 0; e < 4; ++e) {
-                            const float lo = __uint_as_float((ww[e] << 16) & 0x7fffffffu);
-                            const float hi = __uint_as_float(ww[e] & 0x7fff0000u);
-                            csum[k][2 * e] += lo;
-                            csum[k][2 * e + 1] += hi;
-                            s += lo;
-                            s += hi;
-                        }
-                        if (want_blocks) {
-                            if (p.perm) {
-                                const uint4 pi = ((const uint4 *)sperm)[c];
-                                const uint32_t pp[4] = {pi.x, pi.y, pi.z, pi.w};
-                                const uint16_t *row = rows + (size_t)r * d;
-                                s = 0.0f;
+                    for (int e = 0; e < 4; ++e) {
+                        const uint32_t a = ww[e] & 0x7fff7fffu;                 // |.| of both halves
+                        m[e] = make_float2(__uint_as_float(a << 16), __uint_as_float(a & 0xffff0000u));
+                        csum[k][e] = __fadd2_rn(csum[k][e], m[e]);
+                    }
+                    if (want_blocks) {
+                        if (p.perm) {
+                            const uint4 pi = ((const uint4 *)sperm)[c];
+                            const uint32_t pp[4] = {pi.x, pi.y, pi.z, pi.w};
+                            const uint16_t *row = rows + (size_t)r * d;
 #pragma unroll
-                                for (int e = 0; e < 4; ++e) {
-                                    s += abs_bf16(row[pp[e] & 0xffffu]);
-                                    s += abs_bf16(row[pp[e] >> 16]);
-                                }
+                            for (int e = 0; e < 4; ++e) {
+                                s += abs_bf16(row[pp[e] & 0xffffu]);
+                                s += abs_bf16(row[pp[e] >> 16]);
                             }
-                            cs[(size_t)r * nchunks + c] = s;
+                        } else {
+                            const float2 h = __fadd2_rn(__fadd2_rn(m[0], m[1]), __fadd2_rn(m[2], m[3]));
+                            s = h.x + h.y;
                         }
+                    }
+                }
+                if (want_blocks) {
+                    if (shuffle_blocks) {
+                        for (int o = 1; o < cpb; o <<= 1) s += __shfl_xor_sync(0xffffffffu, s, o);
+                        if ((c & (cpb - 1)) == 0) bsum[k] += s;       // the block's first chunk keeps its sum
+                        mx[r] = fmaxf(mx[r], s);
+                    } else if (live && c < nchunks) {
+                        cs[(size_t)r * nchunks + c] = s;
                     }
                 }
             }
         }
-        __syncthreads();                                 // every thread is done with the stage; cs is complete
+        float *redp = red + (it & 1u) * (R * 16);        // double-buffered: one barrier per batch suffices
+        if (shuffle_blocks && p.token_max) {
+#pragma unroll
+            for (int r = 0; r < R; ++r) {
+#pragma unroll
+                for (int o = 16; o > 0; o >>= 1) mx[r] = fmaxf(mx[r], __shfl_xor_sync(0xffffffffu, mx[r], o));
+                if (lane == 0) redp[r * 16 + warp] = mx[r];
+            }
+        }
+        __syncthreads();                                 // every thread is done with the stage; cs / red are complete
         if (tid == 0) fetch(stage, t + (long long)NST * R);
         if (!want_blocks) continue;
-        const int cpb = 1 << (L - 3);          // chunks per block
-        float mx[R];
+        if (shuffle_blocks) {
+            if (p.token_max && tid < R && t + tid < t1) {
+                float m = redp[tid * 16];
+                for (int wv = 1; wv < ST_THREADS / 32; ++wv) m = fmaxf(m, redp[tid * 16 + wv]);
+                p.token_max[t + tid] = m;
+            }
+            continue;
+        }
+        // ---- long blocks (more than 256 channels): per-chunk sums through shared memory
 #pragma unroll
         for (int r = 0; r < R; ++r) {
             mx[r] = 0.0f;
@@ -142,10 +170,10 @@ __global__ void __launch_bounds__(ST_THREADS) perq_stats_partial_kernel(StatsPar
             for (int k = 0; k < KC; ++k) {
                 const int j = tid + k * ST_THREADS;
                 if (j < nb && live) {
-                    float s = 0.0f;
-                    for (int c = 0; c < cpb; ++c) s += cs[(size_t)r * nchunks + j * cpb + c];
-                    bsum[k] += s;
-                    mx[r] = fmaxf(mx[r], s);
+                    float sb = 0.0f;
+                    for (int c = 0; c < cpb; ++c) sb += cs[(size_t)r * nchunks + j * cpb + c];
+                    bsum[k] += sb;
+                    mx[r] = fmaxf(mx[r], sb);
                 }
             }
         }
@@ -154,16 +182,16 @@ __global__ void __launch_bounds__(ST_THREADS) perq_stats_partial_kernel(StatsPar
             for (int r = 0; r < R; ++r) {
 #pragma unroll
                 for (int o = 16; o > 0; o >>= 1) mx[r] = fmaxf(mx[r], __shfl_xor_sync(0xffffffffu, mx[r], o));
-                if (lane == 0) red[r * 16 + warp] = mx[r];
+                if (lane == 0) redp[r * 16 + warp] = mx[r];
             }
             __syncthreads();
             if (tid < R && t + tid < t1) {
-                float m = red[tid * 16];
-                for (int wv = 1; wv < ST_THREADS / 32; ++wv) m = fmaxf(m, red[tid * 16 + wv]);
+                float m = redp[tid * 16];
+                for (int wv = 1; wv < ST_THREADS / 32; ++wv) m = fmaxf(m, redp[tid * 16 + wv]);
                 p.token_max[t + tid] = m;
             }
         }
-        __syncthreads();                                 // cs and red may be overwritten by the next batch
+        __syncthreads();                                 // cs may be overwritten by the next batch
     }
 
     if (p.ws_chan) {
@@ -172,16 +200,20 @@ __global__ void __launch_bounds__(ST_THREADS) perq_stats_partial_kernel(StatsPar
         for (int k = 0; k < KC; ++k) {
             const int c = tid + k * ST_THREADS;
             if (c < nchunks) {
-                dst[2 * c] = make_float4(csum[k][0], csum[k][1], csum[k][2], csum[k][3]);
-                dst[2 * c + 1] = make_float4(csum[k][4], csum[k][5], csum[k][6], csum[k][7]);
+                dst[2 * c] = make_float4(csum[k][0].x, csum[k][0].y, csum[k][1].x, csum[k][1].y);
+                dst[2 * c + 1] = make_float4(csum[k][2].x, csum[k][2].y, csum[k][3].x, csum[k][3].y);
             }
         }
     }
     if (p.ws_block) {
 #pragma unroll
         for (int k = 0; k < KC; ++k) {
-            const int j = tid + k * ST_THREADS;
-            if (j < nb) p.ws_block[(size_t)blockIdx.x * nb + j] = bsum[k];
+            const int c = tid + k * ST_THREADS;
+            if (shuffle_blocks) {      // the thread of a block's first chunk holds its sum
+                if (c < nchunks && (c & (cpb - 1)) == 0) p.ws_block[(size_t)blockIdx.x * nb + (c >> (L - 3))] = bsum[k];
+            } else if (c < nb) {
+                p.ws_block[(size_t)blockIdx.x * nb + c] = bsum[k];
+            }
         }
     }
 }
