@@ -110,9 +110,15 @@ def run_reference(args):
     from oracle import perq_oracle
     from paper_2601_22347_b200 import inputs
     perq_oracle.build()
-    rows = 2048
-    w = inputs.config4(T=rows, b=B_HEAD, fmt=FMT_HEAD)
     fmt = perq_oracle.FMT_INT4
+    w = inputs.config4(T=2048, b=B_HEAD, fmt=FMT_HEAD)
+    # bounded sample: as many rows per step (16 .. 2048) as keep the K steps within about a minute
+    perq_oracle.rotate_quantize(w.x[:256], None, w.b, fmt, w.group)
+    t0 = time.perf_counter()
+    perq_oracle.rotate_quantize(w.x[:256], None, w.b, fmt, w.group)
+    per_row = (time.perf_counter() - t0) / 256
+    rows = int(min(2048, max(16, 60.0 / (max(1, args.steps) * per_row))))
+    w.x = np.ascontiguousarray(w.x[:rows])
     for _ in range(max(1, min(args.warmup, 2))):
         perq_oracle.rotate_quantize(w.x, None, w.b, fmt, w.group)
     t0 = time.perf_counter()
