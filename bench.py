@@ -36,7 +36,7 @@ T_HEAD, D_HEAD, B_HEAD, FMT_HEAD, GROUP_HEAD = 16384, 4096, 32, "int4", 0
 
 # DRAM traffic per token (dram__bytes_read.sum + dram__bytes_write.sum) / T of the headline
 # kernel from an ncu capture; None until a capture of the current kernel exists.  See profiles/.
-NCU_TRAFFIC_BYTES_PER_TOKEN = (135.27e6 + 17.65e6) / 16384   # profiles/perq_fast_kernel_cfg4_b32_int4.md
+NCU_TRAFFIC_BYTES_PER_TOKEN = (135.28e6 + 17.03e6) / 16384   # profiles/perq_fast_kernel_cfg4_b32_int4.md
 
 
 def measured_peak():
