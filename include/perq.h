@@ -42,7 +42,7 @@ typedef enum {
     PERQ_OK = 0,
     PERQ_ERR_NULL = 1,   /* a required pointer is NULL */
     PERQ_ERR_SHAPE = 2,  /* T < 0, d <= 0, d % 32 != 0 or d > PERQ_MAX_D */
-    PERQ_ERR_BLOCK = 3,  /* b is not one of 16/32/64/128 dividing d, nor b == d with d a power of two */
+    PERQ_ERR_BLOCK = 3,  /* b is not a power of two in [16, d] that divides d */
     PERQ_ERR_GROUP = 4,  /* INT4: group not 0 and (d % group != 0 or group % 8 != 0); MXFP4: group not 0/32 */
     PERQ_ERR_FMT = 5,    /* unknown format */
     PERQ_ERR_ALIGN = 6,  /* a device pointer is not 16-byte aligned */
@@ -80,7 +80,8 @@ typedef enum {
  *            perq_validate_perm to check a permutation beforehand.
  * T, d       rows and channels.  T == 0 is a no-op (pointers are then not looked at).
  *            d % 32 == 0, d <= PERQ_MAX_D.
- * b          16, 32, 64 or 128 with d % b == 0; or b == d when d is a power of two.
+ * b          a power of two, 16 <= b <= d, with d % b == 0 (b == d is the full-vector rotation and
+ *            needs d itself to be a power of two).  b <= 128 and b == d have the fastest kernels.
  * fmt        perq_fmt_t.
  * group      INT4: 0 (per token) or a multiple of 8 dividing d.  MXFP4: 0 or 32 (always 32).
  *            Scale ranges are consecutive coordinates of the ROTATED row, independent of b.

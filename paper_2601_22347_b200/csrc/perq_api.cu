@@ -30,9 +30,7 @@ int check_shape(int64_t T, int32_t d, int32_t b, int32_t fmt, int32_t group, int
 {
     if (T < 0 || d <= 0 || d % 32 != 0 || d > PERQ_MAX_D) return PERQ_ERR_SHAPE;
     if (fmt != PERQ_FMT_INT4 && fmt != PERQ_FMT_MXFP4 && fmt != PERQ_FMT_F32_DEBUG) return PERQ_ERR_FMT;
-    const bool small_block = (b == 16 || b == 32 || b == 64 || b == 128) && d % b == 0;
-    const bool full_vector = (b == d) && is_pow2(d);
-    if (!small_block && !full_vector) return PERQ_ERR_BLOCK;
+    if (!is_pow2(b) || b < 16 || b > d || d % b != 0) return PERQ_ERR_BLOCK;
     int g = d;
     if (fmt == PERQ_FMT_INT4) {
         if (group < 0) return PERQ_ERR_GROUP;
@@ -264,7 +262,7 @@ const char *perq_status_string(int status)
     case PERQ_OK: return "ok";
     case PERQ_ERR_NULL: return "a required pointer is NULL";
     case PERQ_ERR_SHAPE: return "bad shape: need T >= 0, 0 < d <= 32768, d % 32 == 0 (and the row must fit in shared memory)";
-    case PERQ_ERR_BLOCK: return "bad block size: need b in {16,32,64,128} dividing d, or b == d with d a power of two";
+    case PERQ_ERR_BLOCK: return "bad block size: need a power of two b, 16 <= b <= d, dividing d";
     case PERQ_ERR_GROUP: return "bad group: INT4 needs 0 or a multiple of 8 dividing d; MXFP4 needs 0 or 32";
     case PERQ_ERR_FMT: return "unknown format";
     case PERQ_ERR_ALIGN: return "device pointers must be 16-byte aligned";

@@ -66,7 +66,9 @@ def test_argument_validation_happens_before_any_launch(lib):
     assert call(p, None, 4, 4100, 32, 0, 0, p, p) == 2           # d % 32
     assert call(p, None, 4, 65536, 32, 0, 0, p, p) == 2          # d too large
     assert call(p, None, 4, 4096, 8, 0, 0, p, p) == 3            # b not allowed
-    assert call(p, None, 4, 4096, 256, 0, 0, p, p) == 3          # b neither small nor d
+    assert call(p, None, 4, 4096, 24, 0, 0, p, p) == 3           # b not a power of two
+    assert call(p, None, 4, 4096, 8192, 0, 0, p, p) == 3         # b larger than d
+    assert call(p, None, 4, 12288, 8192, 0, 0, p, p) == 3        # b does not divide d
     assert call(p, None, 4, 14336, 14336, 0, 0, p, p) == 3       # full vector needs a power of two
     assert call(p, None, 4, 4096, 32, 0, 12, p, p) == 4          # group % 8
     assert call(p, None, 4, 4096, 32, 0, 24, p, p) == 4          # group does not divide d

@@ -448,3 +448,13 @@ def test_permuted_path_many_rows_per_group(B, oracle):
     rows = np.sort(np.random.default_rng(8).choice(w.T, 24, replace=False))
     check(B, oracle, w, rows=rows)
     assert B.perq_device_error() == 0
+
+
+@pytest.mark.parametrize("d,b,T,perm", [(4096, 256, 40, False), (8192, 512, 24, True), (8192, 2048, 16, False),
+                                        (4096, 1024, 24, True), (14336, 2048, 6, True)])
+def test_intermediate_block_sizes(B, oracle, d, b, T, perm):
+    """Block sizes between 128 and d (the paper's block-size sweep goes 16 ... 2048 at d = 8192)."""
+    bits, _ = inputs.gaussian_outliers(T, d, 8, 50.0, seed=4000 + d + b)
+    p = inputs.random_perm(d, 4001) if perm else None
+    for fmt, g in (("int4", 0), ("int4", 128), ("mxfp4", 32)):
+        check(B, oracle, inputs.Workload("mid-b", bits, p, b, fmt, g, 0))
