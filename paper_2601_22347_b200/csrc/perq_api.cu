@@ -96,11 +96,11 @@ int launch_generic(const void *x, const int32_t *perm, int64_t T, int32_t d, int
     return cudaGetLastError() == cudaSuccess ? PERQ_OK : PERQ_ERR_CUDA;
 }
 
-template <int LOG2B, int MODE, int LOG2G, bool PERM, bool FULLV>
+template <int LOG2B, int MODE, int LOG2G, bool PERM, int XB>
 int launch_fast_inst(const perq::FastParams &p, int grid, cudaStream_t st)
 {
-    auto kernel = perq::perq_fast_kernel<LOG2B, MODE, LOG2G, PERM, FULLV>;
-    const size_t smem = PERM ? perq::FastSmem::total_perm : FULLV ? perq::FastSmem::total_full : perq::FastSmem::total;
+    auto kernel = perq::perq_fast_kernel<LOG2B, MODE, LOG2G, PERM, XB>;
+    const size_t smem = PERM ? perq::FastSmem::total_perm : XB > 3 ? perq::FastSmem::total_full : perq::FastSmem::total;
     if (int rc = allow_smem(kernel, smem)) return rc;
     kernel<<<grid, perq::FAST_THREADS, smem, st>>>(p);
     return cudaGetLastError() == cudaSuccess ? PERQ_OK : PERQ_ERR_CUDA;
@@ -110,10 +110,10 @@ template <int MODE, int LOG2G, bool PERM>
 int launch_fast_b(int log2b, const perq::FastParams &p, int grid, cudaStream_t st)
 {
     switch (log2b) {
-    case 4: return launch_fast_inst<4, MODE, LOG2G, PERM, false>(p, grid, st);
-    case 5: return launch_fast_inst<5, MODE, LOG2G, PERM, false>(p, grid, st);
-    case 6: return launch_fast_inst<6, MODE, LOG2G, PERM, false>(p, grid, st);
-    default: return launch_fast_inst<7, MODE, LOG2G, PERM, false>(p, grid, st);
+    case 4: return launch_fast_inst<4, MODE, LOG2G, PERM, 0>(p, grid, st);
+    case 5: return launch_fast_inst<5, MODE, LOG2G, PERM, 0>(p, grid, st);
+    case 6: return launch_fast_inst<6, MODE, LOG2G, PERM, 0>(p, grid, st);
+    default: return launch_fast_inst<7, MODE, LOG2G, PERM, 0>(p, grid, st);
     }
 }
 
@@ -135,10 +135,33 @@ template <int MODE>
 int launch_fast_full(int G, const perq::FastParams &p, int grid, cudaStream_t st)
 {
     switch (G) {
-    case 1: return launch_fast_inst<7, MODE, 0, false, true>(p, grid, st);
-    case 2: return launch_fast_inst<7, MODE, 1, false, true>(p, grid, st);
-    case 4: return launch_fast_inst<7, MODE, 2, false, true>(p, grid, st);
-    default: return launch_fast_inst<7, MODE, 3, false, true>(p, grid, st);
+    case 1: return launch_fast_inst<7, MODE, 0, false, 3>(p, grid, st);
+    case 2: return launch_fast_inst<7, MODE, 1, false, 4>(p, grid, st);
+    case 4: return launch_fast_inst<7, MODE, 2, false, 5>(p, grid, st);
+    default: return launch_fast_inst<7, MODE, 3, false, 6>(p, grid, st);
+    }
+}
+
+// blocks of 256, 512 or 1024 inside a longer row: unpermuted, per-token INT4 or MXFP4
+template <int MODE, int XB>
+int launch_fast_long_g(int G, const perq::FastParams &p, int grid, cudaStream_t st)
+{
+    if (MODE != perq::MODE_TOKEN) return launch_fast_inst<7, MODE, 0, false, XB>(p, grid, st);
+    switch (G) {
+    case 1: return launch_fast_inst<7, perq::MODE_TOKEN, 0, false, XB>(p, grid, st);
+    case 2: return launch_fast_inst<7, perq::MODE_TOKEN, 1, false, XB>(p, grid, st);
+    case 4: return launch_fast_inst<7, perq::MODE_TOKEN, 2, false, XB>(p, grid, st);
+    default: return launch_fast_inst<7, perq::MODE_TOKEN, 3, false, XB>(p, grid, st);
+    }
+}
+
+template <int MODE>
+int launch_fast_long(int xb, int G, const perq::FastParams &p, int grid, cudaStream_t st)
+{
+    switch (xb) {
+    case 1: return launch_fast_long_g<MODE, 1>(G, p, grid, st);
+    case 2: return launch_fast_long_g<MODE, 2>(G, p, grid, st);
+    default: return launch_fast_long_g<MODE, 3>(G, p, grid, st);
     }
 }
 
@@ -152,13 +175,14 @@ int try_launch_fast(const void *x, const int32_t *perm, int64_t T, int32_t d, in
     const int segs = d / perq::SEG_ELEMS;
     const bool permuted = perm != nullptr;
     const bool full = b == d && b > 128;
-    if (!full && b > 128) return -1;
+    const bool longb = !full && b > 128;                  // 256, 512 or 1024 inside a longer row
+    if (longb && (b > perq::SEG_ELEMS || permuted)) return -1;
     if (full && (permuted || (segs != 1 && segs != 2 && segs != 4 && segs != 8))) return -1;
     if (permuted && (d > perq::FastSmem::PERM_MAX_D || segs > perq::FAST_WARPS)) return -1;
     int mode, G = 1;
     if (fmt == PERQ_FMT_MXFP4) {
         mode = perq::MODE_MX;
-    } else if (fmt == PERQ_FMT_INT4 && g == 128 && !full) {
+    } else if (fmt == PERQ_FMT_INT4 && g == 128 && !full && !longb) {
         mode = perq::MODE_G128;
     } else if (fmt == PERQ_FMT_INT4 && g == d) {
         G = segs;
@@ -188,6 +212,9 @@ int try_launch_fast(const void *x, const int32_t *perm, int64_t T, int32_t d, in
     if (full)
         return mode == perq::MODE_MX ? launch_fast_full<perq::MODE_MX>(G, p, grid, st)
                                      : launch_fast_full<perq::MODE_TOKEN>(G, p, grid, st);
+    if (longb)
+        return mode == perq::MODE_MX ? launch_fast_long<perq::MODE_MX>(ilog2(b) - 7, G, p, grid, st)
+                                     : launch_fast_long<perq::MODE_TOKEN>(ilog2(b) - 7, G, p, grid, st);
     const int log2b = ilog2(b);
     return permuted ? launch_fast_mode<true>(mode, G, log2b, p, grid, st)
                     : launch_fast_mode<false>(mode, G, log2b, p, grid, st);

@@ -46,6 +46,7 @@ constexpr int SEG_ELEMS = 1024;
 constexpr int SEG_BYTES = 2048;
 constexpr int SEG_CODE_BYTES = 512;
 constexpr float FAST_ERR_K = 4.0f;          // fp32 error model: |u32 - u| <= K * log2(b) * 2^-24 * max|u32| of the block
+constexpr float FAST_ERR_K_LONG = 2.0f;     // blocks of 256 and 512
 constexpr float FAST_ERR_K_FULL = 1.0f;     // whole-row blocks: 4096 outputs share the rounding errors of 12 stages
 constexpr uint32_t WAIT_SPIN_LIMIT = 1u << 22;
 
@@ -355,8 +356,8 @@ __device__ __forceinline__ uint32_t candidate_mask(const f32x2 (&v)[8][2], const
 
 // Exact maximum magnitude (bit pattern of a non-negative double, the same in every lane) over the
 // slots of this warp's segment whose fp32 maximum reaches thr.
-// FULL_LOG2 == 0: blocks of 2^LOG2B inside the segment at seg.  FULL_LOG2 > 0: one block of 2^FULL_LOG2
-// elements, the whole row at seg, of which this warp's segment starts at seg_off.
+// FULL_LOG2 == 0: blocks of 2^LOG2B inside the segment at seg.  FULL_LOG2 > 0: blocks of 2^FULL_LOG2
+// elements of the unit (row or segment) at seg, of which this warp's segment starts at seg_off.
 template <int LOG2B, int FULL_LOG2>
 __device__ __forceinline__ unsigned long long exact_max_of_candidates(const uint16_t *seg, int seg_off, const float (&ms)[8],
                                                                       float thr, int lane)
@@ -378,7 +379,8 @@ __device__ __forceinline__ unsigned long long exact_max_of_candidates(const uint
             sm &= sm - 1;
             const int pch = sg * 8 + (sl ^ ((sg & 3) & ~PM));      // chunk position in the segment
             if (FULL_LOG2 > 0) {
-                best = fmax(best, fabs(exact_coord4<(1 << (FULL_LOG2 > 0 ? FULL_LOG2 : 4))>(seg, seg_off + pch * 16 + 4 * (src & 3), lane)));
+                const int pr = seg_off + pch * 16 + 4 * (src & 3), be = (pr >> FULL_LOG2) << FULL_LOG2;
+                best = fmax(best, fabs(exact_coord4<(1 << (FULL_LOG2 > 0 ? FULL_LOG2 : 4))>(seg + be, pr - be, lane)));
             } else {
                 const int blk_elem = (pch >> CB) << LOG2B;
                 const int i0 = pch * 16 - blk_elem + 4 * (src & 3);
@@ -479,26 +481,31 @@ __device__ __forceinline__ void serve_scale_requests(const FastParams &p, const 
 
 // ---------------------------------------------------------------- the kernel
 
-// FULLV: the Hadamard block is the whole row of 2^LOG2G segments (LOG2B must be 7: the part of the
+// XB > 0: the Hadamard block has 2^(7 + XB) elements (LOG2B must be 7: the part of the
 // butterfly done inside a warp's registers); the lane-group bits go through shuffles, the warp bits
 // through shared memory.
-template <int LOG2B, int MODE, int LOG2G, bool PERM, bool FULLV>
+// XB = 1..3 keeps the block inside a warp's segment; XB = 3 + LOG2G is the whole row.
+template <int LOG2B, int MODE, int LOG2G, bool PERM, int XB>
 __global__ void __launch_bounds__(FAST_THREADS, 1) perq_fast_kernel(FastParams p)
 {
     constexpr int B = 1 << LOG2B;
-    constexpr int LOG2BF = FULLV ? 10 + LOG2G : LOG2B;      // log2 of the Hadamard block
+    constexpr bool FULLV = XB > 0;                           // a block longer than the in-register part
+    constexpr int WBITS = XB > 3 ? XB - 3 : 0;               // index bits that span the warps of a row
+    constexpr int LBITS = XB > 3 ? 3 : XB;                   // index bits that span the lane groups of a warp
+    constexpr int LOG2BF = FULLV ? 7 + XB : LOG2B;           // log2 of the Hadamard block
+    static_assert(WBITS == 0 || WBITS == LOG2G, "blocks that span warps are whole rows");
     constexpr int BF = 1 << LOG2BF;
     static_assert(!FULLV || (LOG2B == 7 && !PERM && MODE != MODE_G128), "full-vector variant: unpermuted, per token or MX");
     constexpr int CB = LOG2B - 4;                 // butterfly stages left after the tensor-core H_16
     constexpr int PM = (1 << CB) - 1;             // slot bits inside a Hadamard block
     constexpr int NCLS = (PM & 3) + 1;            // sign classes of the slot relabelling
     constexpr bool RUNTIME_G = PERM && MODE != MODE_TOKEN;     // a permuted unit is a whole row of any length
-    constexpr int NST = (PERM || FULLV) ? 3 : FAST_NSTAGE;
+    constexpr int NST = (PERM || WBITS > 0) ? 3 : FAST_NSTAGE;
     const int G = RUNTIME_G ? p.G : (1 << LOG2G);               // warps (segments) per unit
     const int GROUPS = FAST_WARPS / G;
     const uint32_t UNIT_BYTES = (uint32_t)G * SEG_BYTES;
     constexpr float MAGIC = 12582920.0f;          // 1.5 * 2^23 + 8: low nibble of the sum = code + 8
-    static_assert(MODE == MODE_TOKEN || LOG2G == 0 || FULLV, "only per-token scales or a full-vector block couple the warps of a row");
+    static_assert(MODE == MODE_TOKEN || LOG2G == 0 || WBITS > 0, "only per-token scales or a full-vector block couple the warps of a row");
     extern __shared__ __align__(128) unsigned char fsmem_raw[];
     // 1024-byte aligned base: the ldmatrix and code-store addresses below are formed with XOR
     unsigned char *fsmem = fsmem_raw + ((1024u - (smem_u32(fsmem_raw) & 1023u)) & 1023u);
@@ -508,7 +515,7 @@ __global__ void __launch_bounds__(FAST_THREADS, 1) perq_fast_kernel(FastParams p
     const int group = RUNTIME_G ? warp / G : warp >> LOG2G;
     const int w_in_g = warp - group * G;
     const unsigned qmask = 0xFu << (lane & 28);
-    const float err_rel = (FULLV ? FAST_ERR_K_FULL : FAST_ERR_K) * (float)LOG2BF * TWO_M24;
+    const float err_rel = (!FULLV ? FAST_ERR_K : LOG2BF >= 10 ? FAST_ERR_K_FULL : FAST_ERR_K_LONG) * (float)LOG2BF * TWO_M24;
     const uint32_t xbuf_addr = smem_u32(fsmem + FastSmem::xbuf) + (uint32_t)(group * G) * 4096u;   // FULLV: this row's exchange space
 
     const uint32_t stage_base = smem_u32(fsmem + FastSmem::stages) + (uint32_t)group * (NST * UNIT_BYTES);
@@ -622,8 +629,9 @@ __global__ void __launch_bounds__(FAST_THREADS, 1) perq_fast_kernel(FastParams p
         // element's index inside the block
         auto block_of = [&](int e, const uint16_t *&bp, int &i) {
             if (FULLV) {
-                bp = raw_row;
-                i = w_in_g * SEG_ELEMS + e;
+                const int er = w_in_g * SEG_ELEMS + e, be = (er >> LOG2BF) << LOG2BF;
+                bp = raw_row + be;
+                i = er - be;
             } else {
                 const int be = (e >> LOG2B) << LOG2B;
                 bp = seg + be;
@@ -663,7 +671,7 @@ __global__ void __launch_bounds__(FAST_THREADS, 1) perq_fast_kernel(FastParams p
                 }
             }
         };
-        if (G == 1 || (MODE != MODE_TOKEN && !FULLV)) refill();
+        if (G == 1 || (MODE != MODE_TOKEN && WBITS == 0)) refill();
 
         // ---- remaining butterfly stages over the slot bits inside a block (packed add/sub)
 #pragma unroll
@@ -692,7 +700,7 @@ __global__ void __launch_bounds__(FAST_THREADS, 1) perq_fast_kernel(FastParams p
             }
             // lane-group bits (chunk index bits 3..5): exchange with lanes 4, 8, 16 away
 #pragma unroll
-            for (int bit = 4; bit <= 16; bit <<= 1) {
+            for (int bit = 4; bit < (4 << LBITS); bit <<= 1) {
                 const float sg = (lane & bit) ? -1.0f : 1.0f;
                 const f32x2 sg2 = pack2(sg, sg);
 #pragma unroll
@@ -706,7 +714,7 @@ __global__ void __launch_bounds__(FAST_THREADS, 1) perq_fast_kernel(FastParams p
                 }
             }
             // warp bits (segment index): through shared memory, every warp combines all G copies
-            if (G > 1) {
+            if (WBITS > 0) {
                 const uint32_t mine = xbuf_addr + (uint32_t)w_in_g * 4096u + (uint32_t)lane * 16u;
 #pragma unroll
                 for (int s = 0; s < 8; ++s) sts_v4f(mine + s * 512, v[s][0].x, v[s][0].y, v[s][1].x, v[s][1].y);
@@ -835,7 +843,7 @@ __global__ void __launch_bounds__(FAST_THREADS, 1) perq_fast_kernel(FastParams p
                     a32 = warp_max_f32(am);
                     const float thr_row = a32 * (1.0f - 2.0f * err_rel - 2.4e-7f);
                     candw = __ballot_sync(0xffffffffu, (lane < G) && (a32 > 0.0f) && (am >= thr_row));
-                    if (!FULLV) refill();
+                    if (WBITS == 0) refill();
                 } else {
                     a32 = aw;
                     candw = (a32 > 0.0f) ? 1u : 0u;
@@ -1027,9 +1035,10 @@ __global__ void __launch_bounds__(FAST_THREADS, 1) perq_fast_kernel(FastParams p
                 bref = a32;
                 if (CB >= 2) bref = fmaxf(bref, __shfl_xor_sync(0xffffffffu, bref, 1));
                 if (CB >= 3) bref = fmaxf(bref, __shfl_xor_sync(0xffffffffu, bref, 2));
-                if (FULLV) {     // the block is the row: maximum over the warp, then over the row's warps
-                    bref = warp_max_f32(bref);
-                    if (G > 1) {
+                if (FULLV) {     // longer blocks: over their lane groups, then (whole rows) over the row's warps
+#pragma unroll
+                    for (int bit = 4; bit < (4 << LBITS); bit <<= 1) bref = fmaxf(bref, __shfl_xor_sync(0xffffffffu, bref, bit));
+                    if (WBITS > 0) {
                         if (lane == 0) wmax[par2 * FAST_WARPS + warp] = bref;
                         named_barrier(1 + group, G * 32);      // also: every warp has read the exchange space
                         bref = warp_max_f32((lane < G) ? wmax[par2 * FAST_WARPS + group * G + lane] : 0.0f);
@@ -1081,7 +1090,9 @@ __global__ void __launch_bounds__(FAST_THREADS, 1) perq_fast_kernel(FastParams p
                             cm &= cm - 1;
                             int blk_elem, i, elem;
                             locate<LOG2B>(owner >> 2, ql, 8 * m + k, blk_elem, i, elem);
-                            best = fmax(best, fabs(exact_coord_fast<BF>(raw_row, w_in_g * SEG_ELEMS + elem, lane)));
+                            const uint16_t *bp;
+                            block_of(elem, bp, i);
+                            best = fmax(best, fabs(exact_coord_fast<BF>(bp, i, lane)));
                         }
                     }
                     if (lane == owner) {

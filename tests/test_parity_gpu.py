@@ -384,7 +384,7 @@ def test_rows_with_several_maximum_candidates(B, oracle):
     x[5, :] = 0.0;    x[5, 2049] = 1.0; x[5, 3] = -1.0
     x[6, 9] = 300.0;  x[6, 9 + 2048] = 300.0; x[6, 9 + 3072] = -300.0
     bits = inputs.f32_to_bf16_bits(x)
-    for b in (16, 32, 128, 4096):
+    for b in (16, 32, 128, 256, 1024, 4096):
         for fmt, g in (("int4", 0), ("int4", 128), ("mxfp4", 32)):
             if b == 4096 and g == 128:
                 continue
@@ -451,7 +451,8 @@ def test_permuted_path_many_rows_per_group(B, oracle):
 
 
 @pytest.mark.parametrize("d,b,T,perm", [(4096, 256, 40, False), (8192, 512, 24, True), (8192, 2048, 16, False),
-                                        (4096, 1024, 24, True), (14336, 2048, 6, True)])
+                                        (4096, 1024, 24, True), (14336, 2048, 6, True), (8192, 512, 150, False),
+                                        (4096, 1024, 70, False), (2048, 1024, 301, False), (1024, 256, 67, False)])
 def test_intermediate_block_sizes(B, oracle, d, b, T, perm):
     """Block sizes between 128 and d (the paper's block-size sweep goes 16 ... 2048 at d = 8192)."""
     bits, _ = inputs.gaussian_outliers(T, d, 8, 50.0, seed=4000 + d + b)
