@@ -81,7 +81,9 @@ typedef enum {
  * T, d       rows and channels.  T == 0 is a no-op (pointers are then not looked at).
  *            d % 32 == 0, d <= PERQ_MAX_D.
  * b          a power of two, 16 <= b <= d, with d % b == 0 (b == d is the full-vector rotation and
- *            needs d itself to be a power of two).  b <= 128 and b == d have the fastest kernels.
+ *            needs d itself to be a power of two).  The tensor-core kernels cover d % 1024 == 0 with
+ *            b <= 128 (any scale mode, with or without perm) and, unpermuted with per-token or MX
+ *            scales, b <= 1024 and b == d <= 8192; everything else runs on a slower general kernel.
  * fmt        perq_fmt_t.
  * group      INT4: 0 (per token) or a multiple of 8 dividing d.  MXFP4: 0 or 32 (always 32).
  *            Scale ranges are consecutive coordinates of the ROTATED row, independent of b.
