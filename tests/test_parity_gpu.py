@@ -459,3 +459,33 @@ def test_intermediate_block_sizes(B, oracle, d, b, T, perm):
     p = inputs.random_perm(d, 4001) if perm else None
     for fmt, g in (("int4", 0), ("int4", 128), ("mxfp4", 32)):
         check(B, oracle, inputs.Workload("mid-b", bits, p, b, fmt, g, 0))
+
+
+def test_randomised_shapes_and_modes(B, oracle):
+    """A seeded sweep over shapes, block sizes, formats, groups, permutations and value
+    distributions (including rows scaled far up and down), every case held to the oracle."""
+    rng = np.random.default_rng(2601)
+    ds = [256, 1024, 1536, 2048, 3072, 4096, 6144, 8192, 14336]
+    n_cases = 40
+    for case in range(n_cases):
+        d = int(rng.choice(ds))
+        bs = [b for b in (16, 32, 64, 128, 256, 512, 1024, 2048, 4096, 8192) if b <= d and d % b == 0]
+        b = int(rng.choice(bs))
+        fmt, g = [("int4", 0), ("int4", 128), ("int4", 32), ("mxfp4", 32)][int(rng.integers(0, 4))]
+        if fmt == "int4" and g and d % g:
+            g = 0
+        T = int(rng.integers(1, 40))
+        kind = int(rng.integers(0, 3))
+        seed = 5000 + case
+        if kind == 0:
+            bits, _ = inputs.gaussian_outliers(T, d, int(rng.integers(0, 9)), 50.0, seed)
+        elif kind == 1:
+            bits, _ = inputs.student_t_outliers(T, d, 3.0, int(rng.integers(0, 17)), 100.0, seed)
+        else:
+            bits, _ = inputs.laplace_outliers(T, d, int(rng.integers(0, 5)), 200.0, seed)
+        # rows at very different magnitudes (exact powers of two keep the values bf16)
+        scale = np.exp2(rng.integers(-30, 31, size=(T, 1))).astype(np.float32)
+        bits = inputs.f32_to_bf16_bits(inputs.bf16_bits_to_f32(bits) * scale)
+        perm = inputs.random_perm(d, seed + 1) if rng.random() < 0.5 else None
+        check(B, oracle, inputs.Workload("fuzz%d" % case, bits, perm, b, fmt, g, seed))
+    assert B.perq_device_error() == 0
