@@ -126,7 +126,8 @@ int launch_fast_mode(int mode, int G, int log2b, const perq::FastParams &p, int 
     case 1: return launch_fast_b<perq::MODE_TOKEN, 0, PERM>(log2b, p, grid, st);
     case 2: return launch_fast_b<perq::MODE_TOKEN, 1, PERM>(log2b, p, grid, st);
     case 4: return launch_fast_b<perq::MODE_TOKEN, 2, PERM>(log2b, p, grid, st);
-    default: return launch_fast_b<perq::MODE_TOKEN, 3, PERM>(log2b, p, grid, st);
+    case 8: return launch_fast_b<perq::MODE_TOKEN, 3, PERM>(log2b, p, grid, st);
+    default: return launch_fast_b<perq::MODE_TOKEN, -1, PERM>(log2b, p, grid, st);   // any other row length: G at run time
     }
 }
 
@@ -186,7 +187,8 @@ int try_launch_fast(const void *x, const int32_t *perm, int64_t T, int32_t d, in
         mode = perq::MODE_G128;
     } else if (fmt == PERQ_FMT_INT4 && g == d) {
         G = segs;
-        if (G != 1 && G != 2 && G != 4 && G != 8) return -1;
+        if (G > perq::FAST_WARPS - 1) return -1;          // named barriers 1..15: one per group of G warps
+        if ((full || longb) && G != 1 && G != 2 && G != 4 && G != 8) return -1;
         mode = perq::MODE_TOKEN;
     } else {
         return -1;

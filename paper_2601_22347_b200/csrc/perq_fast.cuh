@@ -499,9 +499,10 @@ __global__ void __launch_bounds__(FAST_THREADS, 1) perq_fast_kernel(FastParams p
     constexpr int CB = LOG2B - 4;                 // butterfly stages left after the tensor-core H_16
     constexpr int PM = (1 << CB) - 1;             // slot bits inside a Hadamard block
     constexpr int NCLS = (PM & 3) + 1;            // sign classes of the slot relabelling
-    constexpr bool RUNTIME_G = PERM && MODE != MODE_TOKEN;     // a permuted unit is a whole row of any length
+    // G is a template constant 2^LOG2G, or (LOG2G < 0, and permuted rows without per-token scales) p.G
+    constexpr bool RUNTIME_G = (PERM && MODE != MODE_TOKEN) || LOG2G < 0;
     constexpr int NST = (PERM || WBITS > 0) ? 3 : FAST_NSTAGE;
-    const int G = RUNTIME_G ? p.G : (1 << LOG2G);               // warps (segments) per unit
+    const int G = RUNTIME_G ? p.G : (1 << (LOG2G < 0 ? 0 : LOG2G));   // warps (segments) per unit
     const int GROUPS = FAST_WARPS / G;
     const uint32_t UNIT_BYTES = (uint32_t)G * SEG_BYTES;
     constexpr float MAGIC = 12582920.0f;          // 1.5 * 2^23 + 8: low nibble of the sum = code + 8
@@ -512,7 +513,7 @@ __global__ void __launch_bounds__(FAST_THREADS, 1) perq_fast_kernel(FastParams p
 
     const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
     const int g = lane >> 2, q = lane & 3;
-    const int group = RUNTIME_G ? warp / G : warp >> LOG2G;
+    const int group = RUNTIME_G ? warp / G : warp >> (LOG2G < 0 ? 0 : LOG2G);
     const int w_in_g = warp - group * G;
     const unsigned qmask = 0xFu << (lane & 28);
     const float err_rel = (!FULLV ? FAST_ERR_K : LOG2BF >= 10 ? FAST_ERR_K_FULL : FAST_ERR_K_LONG) * (float)LOG2BF * TWO_M24;
@@ -727,7 +728,7 @@ __global__ void __launch_bounds__(FAST_THREADS, 1) perq_fast_kernel(FastParams p
                     for (int s = 0; s < 8; ++s) { v[s][0] = mul2(v[s][0], sg2); v[s][1] = mul2(v[s][1], sg2); }
                 }
 #pragma unroll
-                for (int dw = 1; dw < (1 << LOG2G); ++dw) {
+                for (int dw = 1; dw < (1 << WBITS); ++dw) {
                     const int wo = w_in_g ^ dw;                   // every other warp of the row once
                     const float sg = (__popc(w_in_g & wo) & 1) ? -1.0f : 1.0f;
                     const f32x2 sg2 = pack2(sg, sg);

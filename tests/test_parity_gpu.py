@@ -349,8 +349,6 @@ def test_block_l1_stats(B, oracle, T, d, b, perm):
 @pytest.mark.parametrize("fmt,group", [("int4", 0), ("int4", 128), ("mxfp4", 32)])
 @pytest.mark.parametrize("d,T,b", [(1024, 70, 16), (2048, 333, 32), (4096, 150, 64), (8192, 40, 128), (14336, 20, 32)])
 def test_permuted_fast_path_matrix(B, oracle, d, T, b, fmt, group):
-    if group == 0 and d == 14336:
-        pytest.skip("per-token scales with 14 segments per row go to the generic kernel (covered elsewhere)")
     bits, _ = inputs.student_t_outliers(T, d, 3.0, max(2, d // 256), 100.0, seed=2000 + d + b)
     bits[2] = 0
     bits[4, 64:320] = 0
@@ -488,4 +486,14 @@ def test_randomised_shapes_and_modes(B, oracle):
         bits = inputs.f32_to_bf16_bits(inputs.bf16_bits_to_f32(bits) * scale)
         perm = inputs.random_perm(d, seed + 1) if rng.random() < 0.5 else None
         check(B, oracle, inputs.Workload("fuzz%d" % case, bits, perm, b, fmt, g, seed))
+    assert B.perq_device_error() == 0
+
+
+@pytest.mark.parametrize("d,T", [(3072, 90), (6144, 70), (12288, 30), (14336, 33)])
+def test_per_token_scales_for_rows_of_any_number_of_segments(B, oracle, d, T):
+    bits, _ = inputs.laplace_outliers(T, d, 6, 200.0, seed=6000 + d)
+    bits[5] = 0
+    for b in (16, 128):
+        check(B, oracle, inputs.Workload("token-anyG", bits, None, b, "int4", 0, 0))
+    check(B, oracle, inputs.Workload("token-anyG-perm", bits, inputs.random_perm(d, 6001), 32, "int4", 0, 0))
     assert B.perq_device_error() == 0
