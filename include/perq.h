@@ -111,11 +111,6 @@ int perq_out_sizes(int64_t T, int32_t d, int32_t fmt, int32_t group, size_t *cod
  * then synchronises `stream` before returning.  `workspace` is device memory provided
  * by the caller, at least perq_host_workspace_bytes(...) long; the library allocates
  * nothing.  perm stays a DEVICE pointer (it is reused across calls) or NULL.
- * Calls of 4096 rows or more are processed in four chunks of rows, and the copy back of a
- * chunk runs on an internal non-blocking stream while the next chunk is copied in; that
- * stream and five events are created once per device on first use and kept until exit.
- * Two such calls at the same time on one device (different caller streams) would share
- * those events: issue them from one thread at a time.
  */
 int perq_rotate_quantize_host(const void *x_host, const int32_t *perm, int64_t T, int32_t d,
                               int32_t b, int32_t fmt, int32_t group, void *out_codes_host,

@@ -271,36 +271,6 @@ static __device__ __align__(256) float g_stats_scratch[PERQ_STATS_STATIC_MAX_FLO
 float *g_stats_scratch_addr[kMaxDevices] = {};   // device address of the array, per device ordinal
 std::mutex g_stats_scratch_mutex;
 
-// Per-device resources of perq_rotate_quantize_host's overlap of the two copy directions: one
-// non-blocking stream and a few events, created on first use and kept until the process exits.
-struct HostPipe {
-    static constexpr int kChunks = 4;
-    cudaStream_t aux = nullptr;
-    cudaEvent_t ready[kChunks] = {};
-    cudaEvent_t done = nullptr;
-    bool ok = false, tried = false;
-};
-HostPipe g_host_pipe[kMaxDevices];
-std::mutex g_host_pipe_mutex;
-
-HostPipe *host_pipe()
-{
-    int dev = -1;
-    if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= kMaxDevices) return nullptr;
-    std::lock_guard<std::mutex> lock(g_host_pipe_mutex);
-    HostPipe &hp = g_host_pipe[dev];
-    if (!hp.tried) {
-        hp.tried = true;
-        bool ok = cudaStreamCreateWithFlags(&hp.aux, cudaStreamNonBlocking) == cudaSuccess;
-        for (int i = 0; ok && i < HostPipe::kChunks; ++i)
-            ok = cudaEventCreateWithFlags(&hp.ready[i], cudaEventDisableTiming) == cudaSuccess;
-        ok = ok && cudaEventCreateWithFlags(&hp.done, cudaEventDisableTiming) == cudaSuccess;
-        if (!ok) (void)cudaGetLastError();
-        hp.ok = ok;
-    }
-    return hp.ok ? &hp : nullptr;     // without it the call still works, on the caller's stream alone
-}
-
 template <int KC>
 int launch_stats_partial(const perq::StatsParams &p, const StatsPlan &plan, cudaStream_t st)
 {
@@ -396,31 +366,11 @@ int perq_rotate_quantize_host(const void *x_host, const int32_t *perm, int64_t T
     unsigned char *x_dev = base;
     unsigned char *codes_dev = x_dev + up((size_t)T * (size_t)d * 2);
     unsigned char *scales_dev = codes_dev + up(cb);
-    // Rows are independent: larger calls go in four chunks of rows, the copy back of one chunk (on an
-    // internal stream) overlapping the copy in of the next, so that both directions of the link are busy.
-    HostPipe *pipe = (T >= 4096) ? host_pipe() : nullptr;
-    const int n_chunks = pipe ? HostPipe::kChunks : 1;
-    const int64_t rows_per = (((T + n_chunks - 1) / n_chunks) + 63) & ~(int64_t)63;
-    const size_t code_row = cb / (size_t)T, scale_row = sb / (size_t)T;
-    const unsigned char *xh = static_cast<const unsigned char *>(x_host);
-    unsigned char *ch = static_cast<unsigned char *>(out_codes_host), *sh = static_cast<unsigned char *>(out_scales_host);
-    for (int c = 0; c < n_chunks; ++c) {
-        const int64_t r0 = c * rows_per, r1 = std::min<int64_t>(T, r0 + rows_per);
-        if (r0 >= r1) break;
-        const size_t n = (size_t)(r1 - r0), xo = (size_t)r0 * d * 2, co = (size_t)r0 * code_row, so = (size_t)r0 * scale_row;
-        if (cudaMemcpyAsync(x_dev + xo, xh + xo, n * d * 2, cudaMemcpyHostToDevice, st) != cudaSuccess) return PERQ_ERR_CUDA;
-        if (int rc = launch_any(x_dev + xo, perm, (int64_t)n, d, b, fmt, g, codes_dev + co, scales_dev + so, st)) return rc;
-        cudaStream_t back = st;
-        if (pipe) {
-            if (cudaEventRecord(pipe->ready[c], st) != cudaSuccess || cudaStreamWaitEvent(pipe->aux, pipe->ready[c], 0) != cudaSuccess)
-                return PERQ_ERR_CUDA;
-            back = pipe->aux;
-        }
-        if (cudaMemcpyAsync(ch + co, codes_dev + co, n * code_row, cudaMemcpyDeviceToHost, back) != cudaSuccess) return PERQ_ERR_CUDA;
-        if (sb && cudaMemcpyAsync(sh + so, scales_dev + so, n * scale_row, cudaMemcpyDeviceToHost, back) != cudaSuccess)
-            return PERQ_ERR_CUDA;
-    }
-    if (pipe && (cudaEventRecord(pipe->done, pipe->aux) != cudaSuccess || cudaStreamWaitEvent(st, pipe->done, 0) != cudaSuccess))
+    if (cudaMemcpyAsync(x_dev, x_host, (size_t)T * (size_t)d * 2, cudaMemcpyHostToDevice, st) != cudaSuccess)
+        return PERQ_ERR_CUDA;
+    if (int rc = launch_any(x_dev, perm, T, d, b, fmt, g, codes_dev, scales_dev, st)) return rc;
+    if (cudaMemcpyAsync(out_codes_host, codes_dev, cb, cudaMemcpyDeviceToHost, st) != cudaSuccess) return PERQ_ERR_CUDA;
+    if (sb && cudaMemcpyAsync(out_scales_host, scales_dev, sb, cudaMemcpyDeviceToHost, st) != cudaSuccess)
         return PERQ_ERR_CUDA;
     return cudaStreamSynchronize(st) == cudaSuccess ? PERQ_OK : PERQ_ERR_CUDA;
 }

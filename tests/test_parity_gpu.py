@@ -497,23 +497,3 @@ def test_per_token_scales_for_rows_of_any_number_of_segments(B, oracle, d, T):
         check(B, oracle, inputs.Workload("token-anyG", bits, None, b, "int4", 0, 0))
     check(B, oracle, inputs.Workload("token-anyG-perm", bits, inputs.random_perm(d, 6001), 32, "int4", 0, 0))
     assert B.perq_device_error() == 0
-
-
-@pytest.mark.parametrize("fmt,group", [("int4", 0), ("mxfp4", 32), ("int4", 128)])
-def test_host_entry_point_in_chunks_matches_the_device_entry_point(B, fmt, group):
-    """From 4096 rows on, the host-buffer call works in chunks of rows with the two copy
-    directions overlapped; its bytes must equal those of one device call."""
-    T, d, b = 5001, 2048, 32
-    bits, _ = inputs.student_t_outliers(T, d, 3.0, 8, 100.0, seed=7000)
-    f = FMT[fmt]
-    x = to_dev(bits)
-    codes_d, scales_d = B.perq_rotate_quantize(x, None, b, f, group)
-    torch.cuda.synchronize()
-    xh = torch.from_numpy(bits.view(np.int16).copy()).view(torch.bfloat16).pin_memory()
-    ws = torch.empty(B.perq_host_workspace_bytes(T, d, f, group), dtype=torch.uint8, device="cuda")
-    codes_h = torch.empty_like(codes_d, device="cpu").pin_memory()
-    scales_h = torch.empty_like(scales_d, device="cpu").pin_memory()
-    for _ in range(2):
-        codes_h.zero_(); scales_h.zero_()
-        B.perq_rotate_quantize_host(xh, None, b, f, group, codes_h, scales_h, ws)
-        assert torch.equal(codes_h, codes_d.cpu()) and torch.equal(scales_h, scales_d.cpu())
