@@ -251,8 +251,49 @@ int perq_oracle_quantize_mxfp4(const double *y, int64_t T, int32_t d, uint8_t *c
     return 0;
 }
 
+/* ---------------------------------------------------------------- FP4 with a per-token scale
+ * Appendix B, "(MX)FP4 Quantization": "For FP4 activations, scaling factor
+ * s = ||X||_inf / (2^{q-1} - 1) is defined dynamically per-token", elements E2M1 as above.
+ * With q = 4 the step is the row maximum over 7 (the same scale as the INT4 quantiser of
+ * Sec. 3), so the largest element maps to 7 and saturates to 6, like the (6, 8) band of MXFP4.
+ * Elements: v = y / s in double, magnitude to the nearest of {0, .5, 1, 1.5, 2, 3, 4, 6}, ties to
+ * the even code, |v| > 6 saturates; the sign bit of y is kept.  A zero row stores scale 0 and
+ * sign-only codes.
+ *
+ * codes: packed [T, d/2]; scales: float [T]; v_pre (optional): y_i / s, [T, d]. */
+int perq_oracle_quantize_fp4(const double *y, int64_t T, int32_t d, uint8_t *codes, float *scales,
+                             double *v_pre)
+{
+    if (!y || !codes || !scales || T < 0 || d <= 0 || d % 2 != 0) return 1;
+#pragma omp parallel
+    {
+        uint8_t *c = (uint8_t *)malloc((size_t)d);
+#pragma omp for schedule(static)
+        for (int64_t t = 0; t < T; ++t) {
+            const double *yr = y + (size_t)t * d;
+            double a = 0.0;
+            for (int32_t i = 0; i < d; ++i) {
+                const double m = fabs(yr[i]);
+                if (m > a) a = m;
+            }
+            const double s = a / 7.0;
+            scales[t] = (a == 0.0) ? 0.0f : (float)s;
+            for (int32_t i = 0; i < d; ++i) {
+                const double v = (a == 0.0) ? 0.0 : yr[i] / s;
+                if (v_pre) v_pre[(size_t)t * d + i] = v;
+                const int k = e2m1_nearest_index(fabs(v));
+                c[i] = (uint8_t)((signbit(yr[i]) ? 8 : 0) | k);
+            }
+            pack_row(c, d, codes + (size_t)t * (d / 2));
+        }
+        free(c);
+    }
+    return 0;
+}
+
 /* ---------------------------------------------------------------- whole path
- * (X P) R~ then Q(.), Fig. "perq-pipeline" / Sec. 4 overview.  fmt: 0 = INT4, 1 = MXFP4.
+ * (X P) R~ then Q(.), Fig. "perq-pipeline" / Sec. 4 overview.  fmt: 0 = INT4, 1 = MXFP4,
+ * 3 = FP4 with a per-token scale (2 is not a quantiser).
  * y_out (optional) receives the rotated row, v_pre (optional) the pre-rounding values. */
 int perq_oracle_rotate_quantize(const uint16_t *x, const int32_t *perm, int64_t T, int32_t d,
                                 int32_t b, int32_t fmt, int32_t group, uint8_t *codes,
@@ -265,6 +306,7 @@ int perq_oracle_rotate_quantize(const uint16_t *x, const int32_t *perm, int64_t 
     if (rc == 0) {
         if (fmt == 0) rc = perq_oracle_quantize_int4(y, T, d, group, codes, (float *)scales, v_pre);
         else if (fmt == 1) rc = perq_oracle_quantize_mxfp4(y, T, d, codes, (uint8_t *)scales, v_pre);
+        else if (fmt == 3) rc = perq_oracle_quantize_fp4(y, T, d, codes, (float *)scales, v_pre);
         else rc = 1;
     }
     if (!y_out) free(y);

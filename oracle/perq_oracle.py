@@ -20,6 +20,7 @@ _lib = None
 
 FMT_INT4 = 0
 FMT_MXFP4 = 1
+FMT_FP4 = 3
 
 
 def build(force: bool = False) -> str:
@@ -103,6 +104,18 @@ def quantize_mxfp4(y, want_pre: bool = False):
     return (codes, e8m0, pre) if want_pre else (codes, e8m0)
 
 
+def quantize_fp4(y, want_pre: bool = False):
+    """E2M1 elements with one fp32 scale per token (row maximum over 7)."""
+    y = np.ascontiguousarray(y, dtype=np.float64)
+    T, d = y.shape
+    codes = np.empty((T, d // 2), np.uint8)
+    scales = np.empty((T, 1), np.float32)
+    pre = np.empty((T, d), np.float64) if want_pre else None
+    _check(_load().perq_oracle_quantize_fp4(_p(y), C.c_int64(T), C.c_int32(d), _p(codes), _p(scales), _p(pre)),
+           "quantize_fp4")
+    return (codes, scales, pre) if want_pre else (codes, scales)
+
+
 def rotate_quantize(x, perm, b: int, fmt: int, group: int, want_y: bool = False, want_pre: bool = False):
     """The whole path.  Returns dict(codes, scales[, y][, pre])."""
     x = _x(x); perm = _perm(perm)
@@ -110,6 +123,8 @@ def rotate_quantize(x, perm, b: int, fmt: int, group: int, want_y: bool = False,
     codes = np.empty((T, d // 2), np.uint8)
     if fmt == FMT_INT4:
         scales = np.empty((T, 1 if group == 0 else d // group), np.float32)
+    elif fmt == FMT_FP4:
+        scales = np.empty((T, 1), np.float32)
     else:
         scales = np.empty((T, d // 32), np.uint8)
     y = np.empty((T, d), np.float64) if want_y else None

@@ -218,3 +218,68 @@ def test_constructed_ties_through_the_rotation(oracle):
     assert np.array_equal(r["y"][0, :16], ystar)
     q = int4_value(unpack(r["codes"]))[0, :16]
     assert list(q) == [7, 0, 2, 2, -4, 4, -6, 6, 0, 1, -2, 3, 0, -2, 0, 1]
+
+
+# ------------------------------------------------------------------ FP4 with a per-token scale
+
+E2M1_VALUES = np.array([0.0, 0.5, 1.0, 1.5, 2.0, 3.0, 4.0, 6.0])
+
+
+def _fp4_unpack(codes):
+    lo, hi = codes & 0xF, codes >> 4
+    return np.stack([lo, hi], axis=-1).reshape(codes.shape[0], -1)
+
+
+def test_fp4_per_token_scale_is_row_max_over_seven_and_values_sit_on_the_grid(oracle):
+    rng = np.random.default_rng(71)
+    y = rng.standard_normal((40, 256)) * np.exp2(rng.integers(-20, 20, size=(40, 1)))
+    y[3] = 0.0
+    codes, scales, pre = oracle.quantize_fp4(y, want_pre=True)
+    a = np.abs(y).max(axis=1)
+    assert np.array_equal(scales[:, 0], (a / 7.0).astype(np.float32))
+    nib = _fp4_unpack(codes)
+    mag = E2M1_VALUES[nib & 7]
+    s = (a / 7.0)[:, None]
+    # the element that attains the maximum maps to 7 and saturates to the largest magnitude
+    assert np.all(mag[np.arange(40), np.abs(y).argmax(axis=1)][a > 0] == 6.0)
+    # every element: nearest grid value, error at most half the local spacing (a full step in the 6..7 band)
+    v = np.abs(pre)
+    err = np.abs(v - mag)
+    spacing = np.where(v < 2, 0.5, np.where(v < 4, 1.0, 2.0))
+    assert np.all(err[v <= 6] <= spacing[v <= 6] / 2 + 1e-12)
+    assert np.all(err[v > 6] <= 1.0 + 1e-12)
+    # signs are the input's, also for zeros
+    assert np.array_equal((nib >> 3).astype(bool), np.signbit(y))
+    assert scales[3, 0] == 0.0 and not (nib[3] & 7).any()
+    del s
+
+
+def test_fp4_midpoints_go_to_the_even_code(oracle):
+    # s = 1 when the row maximum is 7: the midpoints themselves are the scaled values
+    y = np.array([[7.0, 0.25, 0.75, 1.25, 1.75, 2.5, 3.5, 5.0, -0.25, -0.75, -1.25, -1.75, -2.5, -3.5, -5.0, 6.5]])
+    codes, scales = oracle.quantize_fp4(y)
+    nib = _fp4_unpack(codes)[0]
+    assert scales[0, 0] == 1.0
+    assert (nib & 7).tolist() == [7, 0, 2, 2, 4, 4, 6, 6, 0, 2, 2, 4, 4, 6, 6, 7]
+    assert (nib >> 3).tolist() == [0] * 8 + [1] * 7 + [0]
+
+
+def test_fp4_agrees_with_the_mx_quantiser_when_the_scale_is_a_power_of_two(oracle):
+    # a row of 32 whose maximum is 7 * 2^k has step 2^k under both quantisers (E = floor(log2(7 * 2^k)) - 2 = k)
+    rng = np.random.default_rng(72)
+    for k in (-9, 0, 5):
+        y = rng.uniform(-6.9, 6.9, size=(25, 32)) * 2.0 ** k
+        y[:, 0] = 7.0 * 2.0 ** k
+        c4, s4 = oracle.quantize_fp4(y)
+        cm, em = oracle.quantize_mxfp4(y)
+        assert np.array_equal(c4, cm)
+        assert np.all(s4 == np.float32(2.0 ** k)) and np.all(em.astype(int) - 127 == k)
+
+
+def test_fp4_whole_path_is_rotation_then_quantiser(oracle):
+    from paper_2601_22347_b200 import inputs
+    bits, _ = inputs.gaussian_outliers(9, 256, 2, 50.0, seed=73)
+    perm = inputs.random_perm(256, 74)
+    out = oracle.rotate_quantize(bits, perm, 32, oracle.FMT_FP4, 0, want_y=True)
+    c, s = oracle.quantize_fp4(out["y"])
+    assert np.array_equal(out["codes"], c) and np.array_equal(out["scales"], s)
