@@ -35,7 +35,8 @@ extern "C" {
 typedef enum {
     PERQ_FMT_INT4 = 0,      /* symmetric INT4, absmax scale (fp32) per token or per group */
     PERQ_FMT_MXFP4 = 1,     /* E2M1 elements, one E8M0 scale per 32 elements */
-    PERQ_FMT_F32_DEBUG = 2  /* no quantisation: the rotated row as fp32 (test hook) */
+    PERQ_FMT_F32_DEBUG = 2, /* no quantisation: the rotated row as fp32 (test hook) */
+    PERQ_FMT_FP4 = 3        /* E2M1 elements, one fp32 scale per token (Appendix B, FP4 activations) */
 } perq_fmt_t;
 
 typedef enum {
@@ -43,7 +44,7 @@ typedef enum {
     PERQ_ERR_NULL = 1,   /* a required pointer is NULL */
     PERQ_ERR_SHAPE = 2,  /* T < 0, d <= 0, d % 32 != 0 or d > PERQ_MAX_D */
     PERQ_ERR_BLOCK = 3,  /* b is not a power of two in [16, d] that divides d */
-    PERQ_ERR_GROUP = 4,  /* INT4: group not 0 and (d % group != 0 or group % 8 != 0); MXFP4: group not 0/32 */
+    PERQ_ERR_GROUP = 4,  /* INT4: group not 0 and (d % group != 0 or group % 8 != 0); MXFP4: group not 0/32; FP4: not 0 */
     PERQ_ERR_FMT = 5,    /* unknown format */
     PERQ_ERR_ALIGN = 6,  /* a device pointer is not 16-byte aligned */
     PERQ_ERR_CUDA = 7,   /* the CUDA runtime reported an error (launch, copy, attribute) */
@@ -72,6 +73,9 @@ typedef enum {
  *             [-127, 127], stored scale byte = E + 127 (0 if a == 0); element code =
  *             sign(y_i) << 3 | index of the nearest of {0, .5, 1, 1.5, 2, 3, 4, 6} to
  *             |y_i| * 2^-E, ties to the even index, saturating at 6.
+ *      FP4:   per token: a = max |y|, s = a / 7 (the step the paper gives for FP4 activations), stored as
+ *             fp32; element code = sign(y_i) << 3 | index of the nearest of {0, .5, 1, 1.5, 2, 3, 4, 6} to
+ *             |y_i| / s, ties to the even index, saturating at 6 (so the row maximum itself saturates).
  *   4. byte k of the output row = code[2k] | code[2k+1] << 4  (INT4 nibbles are two's complement).
  *
  * x          device, bf16 [T, d] row-major.
@@ -85,10 +89,11 @@ typedef enum {
  *            b <= 128 (any scale mode, with or without perm) and, unpermuted with per-token or MX
  *            scales, b <= 1024 and b == d <= 8192; everything else runs on a slower general kernel.
  * fmt        perq_fmt_t.
- * group      INT4: 0 (per token) or a multiple of 8 dividing d.  MXFP4: 0 or 32 (always 32).
+ * group      INT4: 0 (per token) or a multiple of 8 dividing d.  MXFP4: 0 or 32 (always 32).  FP4: 0.
  *            Scale ranges are consecutive coordinates of the ROTATED row, independent of b.
  * out_codes  device.  INT4/MXFP4: uint8 [T, d/2].  F32_DEBUG: float [T, d] (the rotated row y).
- * out_scales device.  INT4: float [T] or [T, d/group].  MXFP4: uint8 [T, d/32].  F32_DEBUG: unused, may be NULL.
+ * out_scales device.  INT4: float [T] or [T, d/group].  MXFP4: uint8 [T, d/32].  FP4: float [T].
+ *            F32_DEBUG: unused, may be NULL.
  *
  * Codes and scales are deterministic (bit-identical from run to run).
  */

@@ -19,7 +19,8 @@ from . import build as _build
 PERQ_FMT_INT4 = 0
 PERQ_FMT_MXFP4 = 1
 PERQ_FMT_F32_DEBUG = 2
-FMT_BY_NAME = {"int4": PERQ_FMT_INT4, "mxfp4": PERQ_FMT_MXFP4, "f32": PERQ_FMT_F32_DEBUG}
+PERQ_FMT_FP4 = 3
+FMT_BY_NAME = {"int4": PERQ_FMT_INT4, "mxfp4": PERQ_FMT_MXFP4, "f32": PERQ_FMT_F32_DEBUG, "fp4": PERQ_FMT_FP4}
 
 PERQ_OK = 0
 
@@ -99,7 +100,9 @@ def alloc_outputs(T: int, d: int, fmt: int, group: int, device):
     if fmt == PERQ_FMT_F32_DEBUG:
         return torch.empty((T, d), dtype=torch.float32, device=device), None
     codes = torch.empty((T, d // 2), dtype=torch.uint8, device=device)
-    if fmt == PERQ_FMT_INT4:
+    if fmt == PERQ_FMT_FP4:
+        scales = torch.empty((T, 1), dtype=torch.float32, device=device)
+    elif fmt == PERQ_FMT_INT4:
         scales = torch.empty((T, 1 if group == 0 else d // group), dtype=torch.float32, device=device)
     else:
         scales = torch.empty((T, d // 32), dtype=torch.uint8, device=device)

@@ -29,7 +29,7 @@ inline bool aligned16(const void *p) { return (reinterpret_cast<uintptr_t>(p) & 
 int check_shape(int64_t T, int32_t d, int32_t b, int32_t fmt, int32_t group, int *g_out)
 {
     if (T < 0 || d <= 0 || d % 32 != 0 || d > PERQ_MAX_D) return PERQ_ERR_SHAPE;
-    if (fmt != PERQ_FMT_INT4 && fmt != PERQ_FMT_MXFP4 && fmt != PERQ_FMT_F32_DEBUG) return PERQ_ERR_FMT;
+    if (fmt != PERQ_FMT_INT4 && fmt != PERQ_FMT_MXFP4 && fmt != PERQ_FMT_F32_DEBUG && fmt != PERQ_FMT_FP4) return PERQ_ERR_FMT;
     if (!is_pow2(b) || b < 16 || b > d || d % b != 0) return PERQ_ERR_BLOCK;
     int g = d;
     if (fmt == PERQ_FMT_INT4) {
@@ -41,6 +41,8 @@ int check_shape(int64_t T, int32_t d, int32_t b, int32_t fmt, int32_t group, int
     } else if (fmt == PERQ_FMT_MXFP4) {
         if (group != 0 && group != 32) return PERQ_ERR_GROUP;
         g = 32;
+    } else if (fmt == PERQ_FMT_FP4) {
+        if (group != 0) return PERQ_ERR_GROUP;      // one scale per token
     }
     if (g_out) *g_out = g;
     return PERQ_OK;
@@ -122,6 +124,15 @@ int launch_fast_mode(int mode, int G, int log2b, const perq::FastParams &p, int 
 {
     if (mode == perq::MODE_MX) return launch_fast_b<perq::MODE_MX, 0, PERM>(log2b, p, grid, st);
     if (mode == perq::MODE_G128) return launch_fast_b<perq::MODE_G128, 0, PERM>(log2b, p, grid, st);
+    if (mode == perq::MODE_FP4) {
+        switch (G) {
+        case 1: return launch_fast_b<perq::MODE_FP4, 0, PERM>(log2b, p, grid, st);
+        case 2: return launch_fast_b<perq::MODE_FP4, 1, PERM>(log2b, p, grid, st);
+        case 4: return launch_fast_b<perq::MODE_FP4, 2, PERM>(log2b, p, grid, st);
+        case 8: return launch_fast_b<perq::MODE_FP4, 3, PERM>(log2b, p, grid, st);
+        default: return launch_fast_b<perq::MODE_FP4, -1, PERM>(log2b, p, grid, st);
+        }
+    }
     switch (G) {
     case 1: return launch_fast_b<perq::MODE_TOKEN, 0, PERM>(log2b, p, grid, st);
     case 2: return launch_fast_b<perq::MODE_TOKEN, 1, PERM>(log2b, p, grid, st);
@@ -185,6 +196,10 @@ int try_launch_fast(const void *x, const int32_t *perm, int64_t T, int32_t d, in
         mode = perq::MODE_MX;
     } else if (fmt == PERQ_FMT_INT4 && g == 128 && !full && !longb) {
         mode = perq::MODE_G128;
+    } else if (fmt == PERQ_FMT_FP4) {
+        G = segs;
+        if (G > perq::FAST_WARPS - 1 || full || longb) return -1;
+        mode = perq::MODE_FP4;
     } else if (fmt == PERQ_FMT_INT4 && g == d) {
         G = segs;
         if (G > perq::FAST_WARPS - 1) return -1;          // named barriers 1..15: one per group of G warps
@@ -292,7 +307,7 @@ const char *perq_status_string(int status)
     case PERQ_ERR_NULL: return "a required pointer is NULL";
     case PERQ_ERR_SHAPE: return "bad shape: need T >= 0, 0 < d <= 32768, d % 32 == 0 (and the row must fit in shared memory)";
     case PERQ_ERR_BLOCK: return "bad block size: need a power of two b, 16 <= b <= d, dividing d";
-    case PERQ_ERR_GROUP: return "bad group: INT4 needs 0 or a multiple of 8 dividing d; MXFP4 needs 0 or 32";
+    case PERQ_ERR_GROUP: return "bad group: INT4 needs 0 or a multiple of 8 dividing d; MXFP4 needs 0 or 32; FP4 needs 0";
     case PERQ_ERR_FMT: return "unknown format";
     case PERQ_ERR_ALIGN: return "device pointers must be 16-byte aligned";
     case PERQ_ERR_CUDA: return "CUDA runtime error";
@@ -314,6 +329,10 @@ int perq_out_sizes(int64_t T, int32_t d, int32_t fmt, int32_t group, size_t *cod
         if (group != 0 && group != 32) return PERQ_ERR_GROUP;
         cb = (size_t)T * (size_t)(d / 2);
         sb = (size_t)T * (size_t)(d / 32);
+    } else if (fmt == PERQ_FMT_FP4) {
+        if (group != 0) return PERQ_ERR_GROUP;
+        cb = (size_t)T * (size_t)(d / 2);
+        sb = (size_t)T * sizeof(float);
     } else if (fmt == PERQ_FMT_F32_DEBUG) {
         cb = (size_t)T * (size_t)d * sizeof(float);
         sb = 0;

@@ -50,7 +50,10 @@ constexpr float FAST_ERR_K_LONG = 2.0f;     // blocks of 256 and 512
 constexpr float FAST_ERR_K_FULL = 1.0f;     // whole-row blocks: 4096 outputs share the rounding errors of 12 stages
 constexpr uint32_t WAIT_SPIN_LIMIT = 1u << 22;
 
-enum FastMode { MODE_TOKEN = 0, MODE_G128 = 1, MODE_MX = 2 };
+// per-token INT4, INT4 per 128, MXFP4, and E2M1 with a per-token fp32 scale (the scale logic of MODE_TOKEN
+// with the element conversion of MODE_MX)
+enum FastMode { MODE_TOKEN = 0, MODE_G128 = 1, MODE_MX = 2, MODE_FP4 = 3 };
+__host__ __device__ constexpr bool per_token_mode(int mode) { return mode == MODE_TOKEN || mode == MODE_FP4; }
 
 struct FastParams {
     const uint16_t *x;
@@ -458,7 +461,7 @@ __device__ __forceinline__ void serve_scale_requests(const FastParams &p, const 
             const double val = fabs(exact_coord4<(1 << LOG2B)>(p.x + (size_t)row * p.d + blk, (int)(pos - blk), lane));
             const unsigned long long ab = warp_max_u64((unsigned long long)__double_as_longlong(val));
             if (lane == 0) {
-                const size_t si = (MODE == MODE_TOKEN) ? (size_t)row : ((size_t)row * p.d + pos) >> 7;
+                const size_t si = per_token_mode(MODE) ? (size_t)row : ((size_t)row * p.d + pos) >> 7;
                 reinterpret_cast<float *>(p.out_scales)[si] =
                     (ab == 0ull) ? 0.0f : (float)(__longlong_as_double((long long)ab) * p.inv_7_sqrt_b);
             }
@@ -473,7 +476,7 @@ __device__ __forceinline__ void serve_scale_requests(const FastParams &p, const 
         const uint32_t row = segi / segs;
         const uint32_t pos = (segi - row * segs) * SEG_ELEMS + off;      // position in the row
         const double a = exact_slot_max_global<LOG2B, PERM>(p.x + (size_t)row * p.d, pos, p.perm, p.d);
-        const size_t si = (MODE == MODE_TOKEN) ? (size_t)row : ((size_t)row * p.d + pos) >> 7;
+        const size_t si = per_token_mode(MODE) ? (size_t)row : ((size_t)row * p.d + pos) >> 7;
         reinterpret_cast<float *>(p.out_scales)[si] = (a == 0.0) ? 0.0f : (float)(a * p.inv_7_sqrt_b);
     }
     __syncwarp();
@@ -500,13 +503,14 @@ __global__ void __launch_bounds__(FAST_THREADS, 1) perq_fast_kernel(FastParams p
     constexpr int PM = (1 << CB) - 1;             // slot bits inside a Hadamard block
     constexpr int NCLS = (PM & 3) + 1;            // sign classes of the slot relabelling
     // G is a template constant 2^LOG2G, or (LOG2G < 0, and permuted rows without per-token scales) p.G
-    constexpr bool RUNTIME_G = (PERM && MODE != MODE_TOKEN) || LOG2G < 0;
+    constexpr bool TOK = per_token_mode(MODE);
+    constexpr bool RUNTIME_G = (PERM && !TOK) || LOG2G < 0;
     constexpr int NST = (PERM || WBITS > 0) ? 3 : FAST_NSTAGE;
     const int G = RUNTIME_G ? p.G : (1 << (LOG2G < 0 ? 0 : LOG2G));   // warps (segments) per unit
     const int GROUPS = FAST_WARPS / G;
     const uint32_t UNIT_BYTES = (uint32_t)G * SEG_BYTES;
     constexpr float MAGIC = 12582920.0f;          // 1.5 * 2^23 + 8: low nibble of the sum = code + 8
-    static_assert(MODE == MODE_TOKEN || LOG2G == 0 || WBITS > 0, "only per-token scales or a full-vector block couple the warps of a row");
+    static_assert(TOK || LOG2G == 0 || WBITS > 0, "only per-token scales or a full-vector block couple the warps of a row");
     extern __shared__ __align__(128) unsigned char fsmem_raw[];
     // 1024-byte aligned base: the ldmatrix and code-store addresses below are formed with XOR
     unsigned char *fsmem = fsmem_raw + ((1024u - (smem_u32(fsmem_raw) & 1023u)) & 1023u);
@@ -672,7 +676,7 @@ __global__ void __launch_bounds__(FAST_THREADS, 1) perq_fast_kernel(FastParams p
                 }
             }
         };
-        if (G == 1 || (MODE != MODE_TOKEN && WBITS == 0)) refill();
+        if (G == 1 || (!TOK && WBITS == 0)) refill();
 
         // ---- remaining butterfly stages over the slot bits inside a block (packed add/sub)
 #pragma unroll
@@ -765,7 +769,7 @@ __global__ void __launch_bounds__(FAST_THREADS, 1) perq_fast_kernel(FastParams p
         bulk_store_wait_read<1>();           // the store that last read this staging buffer has drained
         __syncwarp();
 
-        if (MODE == MODE_TOKEN || MODE == MODE_G128) {
+        if (MODE != MODE_MX) {
             // lane maximum, then the maximum of the scale range in fp32 (a32); the exact maximum
             // (a_bits, bit pattern of a double) only where it is known without waiting
             const float lane_max = (MODE == MODE_G128)
@@ -868,9 +872,24 @@ __global__ void __launch_bounds__(FAST_THREADS, 1) perq_fast_kernel(FastParams p
             }
             const f32x2 magic2 = pack2(MAGIC, MAGIC);
             uint32_t tie_any = 0u;
+            // E2M1 elements: the value scaled to [-7, 7] plus / minus an additive window, converted twice
+            const float tau = (a32 > 0.0f) ? 8.0f * err_rel + 4.0e-6f : 0.0f;
+            const f32x2 tau_p2 = pack2(tau, tau), tau_m2 = pack2(-tau, -tau);
+            f32x2 mul_c[NCLS];
+#pragma unroll
+            for (int k = 0; k < NCLS; ++k) mul_c[k] = pack2(qsgn(k) * inv, qsgn(k) * inv);
 #pragma unroll
             for (int s = 0; s < 8; ++s) {
                 const int k = s & 3 & PM;
+                if (MODE == MODE_FP4) {
+                    const f32x2 up0 = fma2(v[s][0], mul_c[k], tau_p2), up1 = fma2(v[s][1], mul_c[k], tau_p2);
+                    const f32x2 dn0 = fma2(v[s][0], mul_c[k], tau_m2), dn1 = fma2(v[s][1], mul_c[k], tau_m2);
+                    const uint32_t pu = cvt_e2m1x4(up0.x, up0.y, up1.x, up1.y);
+                    const uint32_t pd = cvt_e2m1x4(dn0.x, dn0.y, dn1.x, dn1.y);
+                    tie_any |= pu ^ pd;
+                    sts_u16(code_addr0 ^ (uint32_t)(s * 8), pu);
+                    continue;
+                }
                 const f32x2 tp0 = fma2(v[s][0], mul_p[k], magic2), tp1 = fma2(v[s][1], mul_p[k], magic2);
                 const f32x2 tm0 = fma2(v[s][0], mul_m[k], magic2), tm1 = fma2(v[s][1], mul_m[k], magic2);
                 const uint32_t pp = ((__float_as_uint(tp1.y) * 16u + __float_as_uint(tp1.x)) * 16u + __float_as_uint(tp0.y)) * 16u
@@ -883,7 +902,7 @@ __global__ void __launch_bounds__(FAST_THREADS, 1) perq_fast_kernel(FastParams p
             tie_any &= 0xffffu;
 
             // ---- per token: the exact row maximum and the stored scale, by the candidate warps only
-            if (MODE == MODE_TOKEN && is_cand) {
+            if (TOK && is_cand) {
                 const float thr_row = a32 * (1.0f - 2.0f * err_rel - 2.4e-7f);
                 slot_maxima();
                 uint32_t slot_mask = 0u;
@@ -972,6 +991,14 @@ __global__ void __launch_bounds__(FAST_THREADS, 1) perq_fast_kernel(FastParams p
 #pragma unroll
                     for (int s = 0; s < 8; ++s) {
                         const int k = s & 3 & PM;
+                        if (MODE == MODE_FP4) {
+                            const f32x2 up0 = fma2(v[s][0], mul_c[k], tau_p2), up1 = fma2(v[s][1], mul_c[k], tau_p2);
+                            const f32x2 dn0 = fma2(v[s][0], mul_c[k], tau_m2), dn1 = fma2(v[s][1], mul_c[k], tau_m2);
+                            const uint32_t x = cvt_e2m1x4(up0.x, up0.y, up1.x, up1.y) ^ cvt_e2m1x4(dn0.x, dn0.y, dn1.x, dn1.y);
+#pragma unroll
+                            for (int j = 0; j < 4; ++j) fm |= ((x >> (4 * j)) & 0xFu) ? (1u << (4 * s + j)) : 0u;
+                            continue;
+                        }
                         const f32x2 tp0 = fma2(v[s][0], mul_p[k], magic2), tp1 = fma2(v[s][1], mul_p[k], magic2);
                         const f32x2 tm0 = fma2(v[s][0], mul_m[k], magic2), tm1 = fma2(v[s][1], mul_m[k], magic2);
                         const float t[4] = {tp0.x, tp0.y, tp1.x, tp1.y}, u[4] = {tm0.x, tm0.y, tm1.x, tm1.y};
@@ -1007,7 +1034,10 @@ __global__ void __launch_bounds__(FAST_THREADS, 1) perq_fast_kernel(FastParams p
                         const double ue = exact_coord_fast<BF>(bp, i, lane);
                         if (lane == 0) {
                             uint32_t code = 0u;
-                            if (s_src != 0.0) {
+                            if (MODE == MODE_FP4) {
+                                const double y = ue / p.sqrt_b;
+                                code = e2m1_code_exact((s_src != 0.0) ? y / s_src : 0.0, signbit(y));
+                            } else if (s_src != 0.0) {
                                 double qd = rint((ue / p.sqrt_b) / s_src);
                                 qd = fmin(fmax(qd, -8.0), 7.0);
                                 code = (uint32_t)((int)qd) & 0xFu;

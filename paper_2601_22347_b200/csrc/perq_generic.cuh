@@ -32,7 +32,7 @@ struct GenParams {
     long long T;
     int d;
     int log2b;
-    int fmt;          // 0 INT4, 1 MXFP4, 2 F32 debug
+    int fmt;          // 0 INT4, 1 MXFP4, 2 F32 debug, 3 E2M1 with a per-token fp32 scale
     int g;            // effective scale-range length (d for per-token, 32 for MX)
     void *out_codes;
     void *out_scales;
@@ -173,6 +173,7 @@ __device__ __forceinline__ uint32_t exact_code(const GenParams &p, double u, dou
         q = fmin(fmax(q, -8.0), 7.0);
         return (uint32_t)((int)q) & 0xFu;
     }
+    if (p.fmt == 3) return e2m1_code_exact((s64 == 0.0) ? 0.0 : y / s64, signbit(y));
     return e2m1_code_exact(scalbn(y, -E), signbit(y));
 }
 
@@ -302,7 +303,7 @@ __global__ void __launch_bounds__(GEN_THREADS) perq_generic_kernel(GenParams p)
             const bool exact = r_thr[r] < __int_as_float(0x7f800000);
             const double au = exact ? __longlong_as_double((long long)r_aux[r]) : (double)rm;
             const double yd = au / p.sqrt_b;
-            if (p.fmt == 0) {
+            if (p.fmt != 1) {
                 const double s = yd / 7.0;
                 ((float *)p.out_scales)[(size_t)row * nr + r] = (au == 0.0) ? 0.0f : (float)s;
                 r_mul[r] = (au == 0.0) ? 0.0f : fminf((float)(7.0 / au), 3.0e38f);
@@ -342,8 +343,9 @@ __global__ void __launch_bounds__(GEN_THREADS) perq_generic_kernel(GenParams p)
                 for (int k = 0; k < 8; k += 2) {
                     const float v0 = fmaf(u[k], mul, 0.0f), v1 = fmaf(u[k + 1], mul, 0.0f);
                     word |= cvt_e2m1x2(v0, v1) << (4 * k);
-                    if (e2m1_tie_distance(fabsf(v0)) < tau_abs + fabsf(v0) * 1.0e-6f) flags |= 1u << k;
-                    if (e2m1_tie_distance(fabsf(v1)) < tau_abs + fabsf(v1) * 1.0e-6f) flags |= 2u << k;
+                    // (a value within the error bound of zero may have the wrong sign bit: flagged too)
+                    if (fminf(e2m1_tie_distance(fabsf(v0)), fabsf(v0)) < tau_abs + fabsf(v0) * 1.0e-6f) flags |= 1u << k;
+                    if (fminf(e2m1_tie_distance(fabsf(v1)), fabsf(v1)) < tau_abs + fabsf(v1) * 1.0e-6f) flags |= 2u << k;
                 }
             }
             while (flags) {

@@ -41,10 +41,10 @@ def compare_quantized(fmt: str, gpu_codes, gpu_scales, ora: dict) -> dict:
     gpu_scales = np.asarray(gpu_scales).reshape(ora["scales"].shape)
     assert gpu_codes.shape == ora["codes"].shape
     report = {"elements": int(gpu_codes.size) * 2, "code_mismatch_exempt": 0, "scale_ulp_max": 0}
-    if fmt == "int4":
+    if fmt in ("int4", "fp4"):
         ulp = ulp_distance_f32(gpu_scales, ora["scales"])
         report["scale_ulp_max"] = int(ulp.max()) if ulp.size else 0
-        assert report["scale_ulp_max"] <= 1, "INT4 scale differs by %d ulp" % report["scale_ulp_max"]
+        assert report["scale_ulp_max"] <= 1, "%s scale differs by %d ulp" % (fmt, report["scale_ulp_max"])
     else:
         bad = np.flatnonzero(gpu_scales.ravel() != ora["scales"].ravel())
         assert bad.size == 0, "E8M0 mismatch at %s: gpu %s oracle %s" % (

@@ -54,6 +54,7 @@ def test_out_sizes(lib):
     assert B.perq_out_sizes(4096, 8192, B.PERQ_FMT_MXFP4, 32) == (4096 * 4096, 4096 * 256)
     assert B.perq_out_sizes(3, 64, B.PERQ_FMT_F32_DEBUG, 0) == (3 * 64 * 4, 0)
     assert B.perq_out_sizes(0, 64, B.PERQ_FMT_INT4, 0) == (0, 0)
+    assert B.perq_out_sizes(16384, 4096, B.PERQ_FMT_FP4, 0) == (16384 * 2048, 16384 * 4)
 
 
 def test_argument_validation_happens_before_any_launch(lib):
@@ -74,6 +75,7 @@ def test_argument_validation_happens_before_any_launch(lib):
     assert call(p, None, 4, 4096, 32, 0, 24, p, p) == 4          # group does not divide d
     assert call(p, None, 4, 4096, 32, 1, 64, p, p) == 4          # MX group must be 32
     assert call(p, None, 4, 4096, 32, 7, 0, p, p) == 5           # format
+    assert call(p, None, 4, 4096, 32, 3, 128, p, p) == 4         # FP4 has one scale per token
     assert call(None, None, 4, 4096, 32, 0, 0, p, p) == 1        # null x
     assert call(p, None, 4, 4096, 32, 0, 0, p, None) == 1        # null scales
     assert call(C.c_void_p(0x1004), None, 4, 4096, 32, 0, 0, p, p) == 6   # misaligned

@@ -9,7 +9,7 @@ from parity import compare_quantized, compare_rotated, unpack_nibbles, int4_valu
 
 pytestmark = pytest.mark.gpu
 
-FMT = {"int4": 0, "mxfp4": 1}
+FMT = {"int4": 0, "mxfp4": 1, "fp4": 3}
 
 
 @pytest.fixture(scope="module")
@@ -497,3 +497,41 @@ def test_per_token_scales_for_rows_of_any_number_of_segments(B, oracle, d, T):
         check(B, oracle, inputs.Workload("token-anyG", bits, None, b, "int4", 0, 0))
     check(B, oracle, inputs.Workload("token-anyG-perm", bits, inputs.random_perm(d, 6001), 32, "int4", 0, 0))
     assert B.perq_device_error() == 0
+
+
+# ------------------------------------------------------------------ E2M1 with a per-token scale
+
+@pytest.mark.parametrize("perm", [False, True])
+@pytest.mark.parametrize("d,T,b", [(1024, 67, 16), (2048, 301, 32), (4096, 130, 64), (8192, 45, 128), (6144, 40, 32),
+                                   (1536, 33, 32), (4096, 20, 4096), (4096, 24, 512)])
+def test_fp4_per_token(B, oracle, d, T, b, perm):
+    bits, _ = inputs.student_t_outliers(T, d, 3.0, max(2, d // 256), 100.0, seed=8000 + d + b)
+    bits[3] = 0
+    bits[5, 128:384] = 0
+    p = inputs.random_perm(d, 8001) if perm else None
+    check(B, oracle, inputs.Workload("fp4", bits, p, b, "fp4", 0, 0))
+    assert B.perq_device_error() == 0
+
+
+def test_fp4_exact_midpoints_and_saturation(B, oracle):
+    import scipy.linalg
+    H = scipy.linalg.hadamard(16)
+    rng = np.random.default_rng(88)
+    rows = []
+    for _ in range(24):
+        blocks = []
+        for j in range(64):
+            ystar = rng.integers(-26, 27, size=16) * 0.25          # quarters in [-6.5, 6.5]: every midpoint occurs
+            ystar[rng.integers(0, 16)] = 7.0 if j == 0 else ystar[0]
+            blocks.append((ystar @ H) / 4.0)
+        rows.append(np.concatenate(blocks))
+    x = np.array(rows, np.float32)
+    bits = inputs.f32_to_bf16_bits(x)
+    assert np.array_equal(inputs.bf16_bits_to_f32(bits), x)
+    rep = check(B, oracle, inputs.Workload("fp4-ties", bits, None, 16, "fp4", 0, 0))
+    assert rep["code_mismatch_exempt"] == 0
+    rep = check(B, oracle, inputs.Workload("fp4-ties-perm", bits, inputs.random_perm(1024, 89), 16, "fp4", 0, 0))
+    w = inputs.config4(T=16384, b=32, fmt="fp4")
+    w.group = 0
+    rows_ = np.sort(np.random.default_rng(9).choice(w.T, 64, replace=False))
+    check(B, oracle, w, rows=rows_)
