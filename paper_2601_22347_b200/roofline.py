@@ -18,6 +18,8 @@ def scale_bytes_per_token(d: int, fmt: str, group: int) -> int:
         return 4 * (1 if group == 0 else d // group)
     if fmt == "mxfp4":
         return d // 32
+    if fmt == "fp4":
+        return 4
     raise ValueError(fmt)
 
 
