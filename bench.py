@@ -33,6 +33,7 @@ FALLBACK_HBM_GBS = 6650.0
 
 # headline workload
 T_HEAD, D_HEAD, B_HEAD, FMT_HEAD, GROUP_HEAD = 16384, 4096, 32, "int4", 0
+ORACLE_FMT = {"int4": 0, "mxfp4": 1, "fp4": 3}     # format numbers of oracle/perq_oracle.c
 
 # DRAM traffic per token (dram__bytes_read.sum + dram__bytes_write.sum) / T of the headline
 # kernel from an ncu capture; None until a capture of the current kernel exists.  See profiles/.
@@ -110,7 +111,7 @@ def run_reference(args):
     from oracle import perq_oracle
     from paper_2601_22347_b200 import inputs
     perq_oracle.build()
-    fmt = perq_oracle.FMT_INT4
+    fmt = ORACLE_FMT[FMT_HEAD]
     w = inputs.config4(T=2048, b=B_HEAD, fmt=FMT_HEAD)
     # bounded sample: as many rows per step (16 .. 2048) as keep the K steps within about a minute
     perq_oracle.rotate_quantize(w.x[:256], None, w.b, fmt, w.group)
@@ -132,8 +133,8 @@ def run_reference(args):
         "impl": "reference", "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": args.gpus,
         "steps": args.steps, "warmup": args.warmup, "ms_per_step": dt * 1e3, "higher_is_better": True,
         "scaling": "weak", "vs_baseline": None, "dtype": "f64", "data": "synthetic",
-        "config": {"workload": "cfg4 Llama-3-8B hidden: T=%d d=%d bf16 Laplace+4 outlier channels, b=%d, INT4 per-token"
-                               % (T_HEAD, D_HEAD, B_HEAD), "sample": sample},
+        "config": {"workload": "cfg4 Llama-3-8B hidden: T=%d d=%d bf16 Laplace+4 outlier channels, b=%d, %s"
+                               % (T_HEAD, D_HEAD, B_HEAD, FMT_HEAD), "sample": sample},
         "mtokens_per_s": rows / dt / 1e6,
         "cpu_baseline": {"value": value, "unit": UNIT, "cores": perq_oracle.num_threads(), "kind": "oracle",
                          "sample": sample},
@@ -147,6 +148,7 @@ def run_reference(args):
 # ------------------------------------------------------------------------------ CUDA arm
 
 def main():
+    global FMT_HEAD, GROUP_HEAD
     ap = argparse.ArgumentParser()
     ap.add_argument("--gpus", type=int, default=1)
     ap.add_argument("--steps", type=int, default=4000)
@@ -154,8 +156,11 @@ def main():
     ap.add_argument("--impl", default="perq", choices=["perq", "reference"])
     ap.add_argument("--no-sweep", action="store_true", help="skip the per-variant sweep after the timed steps")
     ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--fmt", default=FMT_HEAD, choices=["int4", "mxfp4", "fp4"],
+                    help="format of the timed step (default: the headline, INT4 with a per-token scale)")
     args = ap.parse_args()
     args.warmup = max(args.warmup, 3)
+    FMT_HEAD, GROUP_HEAD = args.fmt, (32 if args.fmt == "mxfp4" else 0)
     if args.impl == "reference":
         return run_reference(args)
 
@@ -226,7 +231,8 @@ def main():
     # ---- end to end through the host-buffer entry point (pinned host memory, copies inside the timed region)
     xh = torch.from_numpy(w.x.view(np.int16).copy()).view(torch.bfloat16).pin_memory()
     ch = torch.empty((T_HEAD, D_HEAD // 2), dtype=torch.uint8).pin_memory()
-    sh = torch.empty((T_HEAD, 1), dtype=torch.float32).pin_memory()
+    sh = (torch.empty((T_HEAD, D_HEAD // 32), dtype=torch.uint8) if FMT_HEAD == "mxfp4"
+          else torch.empty((T_HEAD, 1), dtype=torch.float32)).pin_memory()
     ws = torch.empty(B.perq_host_workspace_bytes(T_HEAD, D_HEAD, fmt, GROUP_HEAD), dtype=torch.uint8, device="cuda")
     e2e_steps = max(3, min(args.steps, 20))
     for _ in range(3):
@@ -238,7 +244,7 @@ def main():
     e2e_s = (time.perf_counter() - t0) / e2e_steps
     e2e_s = sharding.max_over_ranks(e2e_s, device="cuda")
     e2e = {"value": world * bytes_per_step / e2e_s / 1e9, "unit": UNIT,
-           "h2d_bytes_per_step": int(xh.numel() * 2), "d2h_bytes_per_step": int(ch.numel() + sh.numel() * 4),
+           "h2d_bytes_per_step": int(xh.numel() * 2), "d2h_bytes_per_step": int(ch.numel() + sh.numel() * sh.element_size()),
            "ms_per_step": e2e_s * 1e3, "api": "perq_rotate_quantize_host"}
     del ws
 
@@ -329,11 +335,11 @@ def main():
         perq_oracle.build()
         rows = 4096
         wb = inputs.config4(T=rows, b=B_HEAD, fmt=FMT_HEAD)
-        perq_oracle.rotate_quantize(wb.x[:256], None, B_HEAD, perq_oracle.FMT_INT4, GROUP_HEAD)
+        perq_oracle.rotate_quantize(wb.x[:256], None, B_HEAD, ORACLE_FMT[FMT_HEAD], GROUP_HEAD)
         t0 = time.perf_counter()
         reps = 0
         while time.perf_counter() - t0 < 10.0:
-            perq_oracle.rotate_quantize(wb.x, None, B_HEAD, perq_oracle.FMT_INT4, GROUP_HEAD)
+            perq_oracle.rotate_quantize(wb.x, None, B_HEAD, ORACLE_FMT[FMT_HEAD], GROUP_HEAD)
             reps += 1
         dt = (time.perf_counter() - t0) / reps
         cpu_baseline = {"value": rows * bpt / dt / 1e9, "unit": UNIT, "cores": perq_oracle.num_threads(),
@@ -345,7 +351,8 @@ def main():
         "ms_per_step": ms_per_step, "higher_is_better": True, "scaling": "weak", "vs_baseline": None,
         "dtype": "f32", "data": "synthetic",
         "config": {"workload": "cfg4 Llama-3-8B hidden: T=%d d=%d bf16 Laplace(0,1)+4 outlier channels x200, no perm, "
-                               "block Hadamard b=%d, INT4 per-token absmax scale" % (T_HEAD, D_HEAD, B_HEAD),
+                               "block Hadamard b=%d, %s" % (T_HEAD, D_HEAD, B_HEAD, {"int4": "INT4 per-token absmax scale",
+                               "mxfp4": "MXFP4 (E2M1 + E8M0 per 32)", "fp4": "FP4 (E2M1) per-token scale"}[FMT_HEAD]),
                    "per_gpu_tokens": T_HEAD, "l2": "ring of %d input sets, each 134 MB > 126 MB L2" % RING},
         "mtokens_per_s": world * T_HEAD / ms_per_step / 1e3,
         "pct_of_nominal_8TBs": 100.0 * value / world / NOMINAL_HBM_GBS,

@@ -1,5 +1,9 @@
-// Fast rotate+quantize kernel for the common cases: no permutation, b in {16,32,64,128},
-// d a multiple of 1024, scales per token (d/1024 in {1,2,4,8}), per 128 (INT4) or per 32 (MXFP4).
+// Fast rotate+quantize kernel: rows of d = G * 1024 channels.
+//   b <= 128              every scale mode (INT4 per token / per 128, MXFP4, FP4 per token), with or
+//                         without a permutation (permuted: d <= 16384);
+//   b in {256, 512, 1024} unpermuted, INT4 per token or MXFP4;
+//   b == d <= 8192        unpermuted, INT4 per token or MXFP4 (full-vector rotation).
+// Per-token scales need G <= 15 (one named barrier per group of G warps).
 //
 // Data path (HBM-bound, one pass):
 //   global --cp.async.bulk + mbarrier--> shared memory ring (bf16 rows, as stored)
@@ -28,9 +32,16 @@
 //
 // Per-token scales: the G = d/1024 warps of a row exchange their fp32 maxima through one
 // named barrier.  Only the warps whose maximum is within the error bound of the row's
-// (normally one) derive exact values; with one such warp it stores the scale itself, with
-// several the last one to add its value to a shared accumulator does.  Warps that need the
-// exact maximum for a tie fix-up (rare) wait for it on a flag, with a bounded spin.
+// (normally one) look for the exact value.  Normally one slot holds it: its position is
+// recorded and the scale is stored later, 32 records at a time, one per lane (see "deferred
+// per-token scales" below).  Otherwise the exact values are derived at once; with one such
+// warp it stores the scale itself, with several the last one to add its value to a shared
+// accumulator does.  Warps that need the exact maximum for a tie fix-up (rare) wait for its
+// publication (a value, or the position to evaluate) on a flag, with a bounded spin.
+//
+// Permuted rows are staged raw and gathered by every warp into its own 2 KB buffer; blocks
+// longer than 128 continue the butterfly across lane groups (shuffles) and, for b == d,
+// across the warps of the row (shared-memory exchange).
 #pragma once
 #include <cuda_runtime.h>
 #include <stdint.h>
