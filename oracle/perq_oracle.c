@@ -251,6 +251,56 @@ int perq_oracle_quantize_mxfp4(const double *y, int64_t T, int32_t d, uint8_t *c
     return 0;
 }
 
+/* ---------------------------------------------------------------- asymmetric INT4, per token
+ * Appendix B: activations use "the standard asymmetric activation quantizer, where zero point
+ * z = min(X) / s and scaling factor s = (max(X) - min(X)) / (2^q - 1) are dynamically defined
+ * per-token", in Q(X) = s * (clip(round(X / s) - z, min A, max A) + z)  (the printed equation
+ * adds z outside the product with s; it belongs inside).  The codes have to be integers of the
+ * alphabet {0..15}, so z is read as the integer round(min(X) / s), ties to even like every
+ * rounding here.  q = 4:
+ *     s = (mx - mn) / 15,  z = rne(mn / s),  c_i = clip(rne(y_i / s) - z, 0, 15),  Q = s * (c_i + z).
+ * A constant row (mx == mn, including all-zero) stores s = 0, z = 0 and codes 0.
+ *
+ * codes: packed [T, d/2] (unsigned nibbles); scale_zero: float [T, 2] = (s, z);
+ * v_pre (optional): y_i / s, [T, d]. */
+int perq_oracle_quantize_int4_asym(const double *y, int64_t T, int32_t d, uint8_t *codes,
+                                   float *scale_zero, double *v_pre)
+{
+    if (!y || !codes || !scale_zero || T < 0 || d <= 0 || d % 2 != 0) return 1;
+    if (fegetround() != FE_TONEAREST) return 4;
+#pragma omp parallel
+    {
+        uint8_t *c = (uint8_t *)malloc((size_t)d);
+#pragma omp for schedule(static)
+        for (int64_t t = 0; t < T; ++t) {
+            const double *yr = y + (size_t)t * d;
+            double mx = yr[0], mn = yr[0];
+            for (int32_t i = 1; i < d; ++i) {
+                if (yr[i] > mx) mx = yr[i];
+                if (yr[i] < mn) mn = yr[i];
+            }
+            const double s = (mx - mn) / 15.0;
+            const double z = (s == 0.0) ? 0.0 : nearbyint(mn / s);
+            scale_zero[2 * t] = (float)s;
+            scale_zero[2 * t + 1] = (float)z;
+            for (int32_t i = 0; i < d; ++i) {
+                double v = 0.0, q = 0.0;
+                if (s != 0.0) {
+                    v = yr[i] / s;
+                    q = nearbyint(v) - z;
+                    if (q > 15.0) q = 15.0;
+                    if (q < 0.0) q = 0.0;
+                }
+                if (v_pre) v_pre[(size_t)t * d + i] = v;
+                c[i] = (uint8_t)q;
+            }
+            pack_row(c, d, codes + (size_t)t * (d / 2));
+        }
+        free(c);
+    }
+    return 0;
+}
+
 /* ---------------------------------------------------------------- FP4 with a per-token scale
  * Appendix B, "(MX)FP4 Quantization": "For FP4 activations, scaling factor
  * s = ||X||_inf / (2^{q-1} - 1) is defined dynamically per-token", elements E2M1 as above.
@@ -293,7 +343,7 @@ int perq_oracle_quantize_fp4(const double *y, int64_t T, int32_t d, uint8_t *cod
 
 /* ---------------------------------------------------------------- whole path
  * (X P) R~ then Q(.), Fig. "perq-pipeline" / Sec. 4 overview.  fmt: 0 = INT4, 1 = MXFP4,
- * 3 = FP4 with a per-token scale (2 is not a quantiser).
+ * 3 = FP4 with a per-token scale, 4 = asymmetric INT4 per token (2 is not a quantiser).
  * y_out (optional) receives the rotated row, v_pre (optional) the pre-rounding values. */
 int perq_oracle_rotate_quantize(const uint16_t *x, const int32_t *perm, int64_t T, int32_t d,
                                 int32_t b, int32_t fmt, int32_t group, uint8_t *codes,
@@ -307,6 +357,7 @@ int perq_oracle_rotate_quantize(const uint16_t *x, const int32_t *perm, int64_t 
         if (fmt == 0) rc = perq_oracle_quantize_int4(y, T, d, group, codes, (float *)scales, v_pre);
         else if (fmt == 1) rc = perq_oracle_quantize_mxfp4(y, T, d, codes, (uint8_t *)scales, v_pre);
         else if (fmt == 3) rc = perq_oracle_quantize_fp4(y, T, d, codes, (float *)scales, v_pre);
+        else if (fmt == 4) rc = perq_oracle_quantize_int4_asym(y, T, d, codes, (float *)scales, v_pre);
         else rc = 1;
     }
     if (!y_out) free(y);

@@ -21,6 +21,7 @@ _lib = None
 FMT_INT4 = 0
 FMT_MXFP4 = 1
 FMT_FP4 = 3
+FMT_INT4_ASYM = 4
 
 
 def build(force: bool = False) -> str:
@@ -116,6 +117,18 @@ def quantize_fp4(y, want_pre: bool = False):
     return (codes, scales, pre) if want_pre else (codes, scales)
 
 
+def quantize_int4_asym(y, want_pre: bool = False):
+    """Asymmetric per-token INT4: codes 0..15, (scale, integer zero point) per token."""
+    y = np.ascontiguousarray(y, dtype=np.float64)
+    T, d = y.shape
+    codes = np.empty((T, d // 2), np.uint8)
+    sz = np.empty((T, 2), np.float32)
+    pre = np.empty((T, d), np.float64) if want_pre else None
+    _check(_load().perq_oracle_quantize_int4_asym(_p(y), C.c_int64(T), C.c_int32(d), _p(codes), _p(sz), _p(pre)),
+           "quantize_int4_asym")
+    return (codes, sz, pre) if want_pre else (codes, sz)
+
+
 def rotate_quantize(x, perm, b: int, fmt: int, group: int, want_y: bool = False, want_pre: bool = False):
     """The whole path.  Returns dict(codes, scales[, y][, pre])."""
     x = _x(x); perm = _perm(perm)
@@ -125,6 +138,8 @@ def rotate_quantize(x, perm, b: int, fmt: int, group: int, want_y: bool = False,
         scales = np.empty((T, 1 if group == 0 else d // group), np.float32)
     elif fmt == FMT_FP4:
         scales = np.empty((T, 1), np.float32)
+    elif fmt == FMT_INT4_ASYM:
+        scales = np.empty((T, 2), np.float32)
     else:
         scales = np.empty((T, d // 32), np.uint8)
     y = np.empty((T, d), np.float64) if want_y else None

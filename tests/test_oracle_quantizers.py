@@ -283,3 +283,52 @@ def test_fp4_whole_path_is_rotation_then_quantiser(oracle):
     out = oracle.rotate_quantize(bits, perm, 32, oracle.FMT_FP4, 0, want_y=True)
     c, s = oracle.quantize_fp4(out["y"])
     assert np.array_equal(out["codes"], c) and np.array_equal(out["scales"], s)
+
+
+# ------------------------------------------------------------------ asymmetric INT4, per token
+
+def test_asym_int4_range_extremes_and_round_trip(oracle):
+    rng = np.random.default_rng(81)
+    y = rng.standard_normal((60, 512)) * np.exp2(rng.integers(-12, 12, size=(60, 1))) + rng.standard_normal((60, 1)) * 3
+    y[4] = 2.5            # constant row
+    y[5] = 0.0
+    codes, sz, pre = oracle.quantize_int4_asym(y, want_pre=True)
+    nib = _fp4_unpack(codes).astype(np.int64)
+    mx, mn = y.max(axis=1), y.min(axis=1)
+    s = (mx - mn) / 15.0
+    assert np.array_equal(sz[:, 0], s.astype(np.float32))
+    assert nib.min() >= 0 and nib.max() <= 15
+    live = s > 0
+    rows = np.arange(60)
+    assert np.all(nib[rows, y.argmin(axis=1)][live] == 0)            # the minimum is the first level
+    assert np.all(nib[rows, y.argmax(axis=1)][live] >= 14)           # the maximum the last (15, or 14 at a tie)
+    z = sz[:, 1].astype(np.float64)
+    assert np.all(z == np.rint(z))
+    deq = s[:, None] * (nib + z[:, None])
+    assert np.all(np.abs(y - deq)[live] <= s[live][:, None] * (0.5 + 1e-9))   # half a step, as in Sec. 3
+    assert not nib[4].any() and not nib[5].any() and sz[4, 0] == 0 and sz[5, 1] == 0
+    order = np.argsort(y, axis=1)                                    # codes are monotone in the value
+    assert np.all(np.diff(np.take_along_axis(nib, order, axis=1), axis=1) >= 0)
+
+
+def test_asym_int4_is_equivariant_under_power_of_two_scaling_and_even_step_shifts(oracle):
+    rng = np.random.default_rng(82)
+    base = rng.integers(-40, 41, size=(20, 64)).astype(np.float64)     # small integers: exact in every step below
+    base[:, 0], base[:, 1] = -44.0, 46.0                               # range 90 -> s = 6, min / s = -7.33 (no tie)
+    c0, sz0 = oracle.quantize_int4_asym(base)
+    assert np.all(sz0[:, 0] == 6.0) and np.all(sz0[:, 1] == -7.0)
+    for k in (-7, 3):
+        c, sz = oracle.quantize_int4_asym(base * 2.0 ** k)
+        assert np.array_equal(c, c0) and np.all(sz[:, 0] == np.float32(6.0 * 2.0 ** k)) and np.array_equal(sz[:, 1], sz0[:, 1])
+    for shift in (-4, 2):                       # whole even numbers of steps keep every tie's parity: only z moves
+        c, sz = oracle.quantize_int4_asym(base + 6.0 * shift)
+        assert np.array_equal(c, c0) and np.array_equal(sz[:, 1], sz0[:, 1] + shift)
+
+
+def test_asym_int4_rounds_half_to_even(oracle):
+    # s = 1: min 0, max 15; values k + 1/2 go to the even integer
+    y = np.array([[0.0, 15.0, 0.5, 1.5, 2.5, 3.5, 13.5, 14.5, 7.49, 7.51, 4.0, 4.0, 4.0, 4.0, 4.0, 4.0]])
+    c, sz = oracle.quantize_int4_asym(y)
+    nib = _fp4_unpack(c)[0].tolist()
+    assert sz[0].tolist() == [1.0, 0.0]
+    assert nib[:10] == [0, 15, 0, 2, 2, 4, 14, 14, 7, 8]
