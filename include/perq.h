@@ -36,7 +36,8 @@ typedef enum {
     PERQ_FMT_INT4 = 0,      /* symmetric INT4, absmax scale (fp32) per token or per group */
     PERQ_FMT_MXFP4 = 1,     /* E2M1 elements, one E8M0 scale per 32 elements */
     PERQ_FMT_F32_DEBUG = 2, /* no quantisation: the rotated row as fp32 (test hook) */
-    PERQ_FMT_FP4 = 3        /* E2M1 elements, one fp32 scale per token (Appendix B, FP4 activations) */
+    PERQ_FMT_FP4 = 3,       /* E2M1 elements, one fp32 scale per token (Appendix B, FP4 activations) */
+    PERQ_FMT_INT4_ASYM = 4  /* asymmetric INT4, (scale, zero point) per token (Appendix B, INT4 activations) */
 } perq_fmt_t;
 
 typedef enum {
@@ -76,6 +77,9 @@ typedef enum {
  *      FP4:   per token: a = max |y|, s = a / 7 (the step the paper gives for FP4 activations), stored as
  *             fp32; element code = sign(y_i) << 3 | index of the nearest of {0, .5, 1, 1.5, 2, 3, 4, 6} to
  *             |y_i| / s, ties to the even index, saturating at 6 (so the row maximum itself saturates).
+ *      INT4_ASYM: per token: s = (max y - min y) / 15, z = rne(min y / s),
+ *             code_i = clip(rne(y_i / s) - z, 0, 15) (unsigned nibble); the value is s * (code_i + z).
+ *             Stored: (s, z) as two fp32.  A constant row gives s = 0, z = 0, codes 0.
  *   4. byte k of the output row = code[2k] | code[2k+1] << 4  (INT4 nibbles are two's complement).
  *
  * x          device, bf16 [T, d] row-major.
@@ -89,10 +93,10 @@ typedef enum {
  *            b <= 128 (any scale mode, with or without perm) and, unpermuted with per-token or MX
  *            scales, b <= 1024 and b == d <= 8192; everything else runs on a slower general kernel.
  * fmt        perq_fmt_t.
- * group      INT4: 0 (per token) or a multiple of 8 dividing d.  MXFP4: 0 or 32 (always 32).  FP4: 0.
+ * group      INT4: 0 (per token) or a multiple of 8 dividing d.  MXFP4: 0 or 32 (always 32).  FP4, INT4_ASYM: 0.
  *            Scale ranges are consecutive coordinates of the ROTATED row, independent of b.
  * out_codes  device.  INT4/MXFP4: uint8 [T, d/2].  F32_DEBUG: float [T, d] (the rotated row y).
- * out_scales device.  INT4: float [T] or [T, d/group].  MXFP4: uint8 [T, d/32].  FP4: float [T].
+ * out_scales device.  INT4: float [T] or [T, d/group].  MXFP4: uint8 [T, d/32].  FP4: float [T].  INT4_ASYM: float [T, 2].
  *            F32_DEBUG: unused, may be NULL.
  *
  * Codes and scales are deterministic (bit-identical from run to run).

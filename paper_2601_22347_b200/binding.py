@@ -20,7 +20,9 @@ PERQ_FMT_INT4 = 0
 PERQ_FMT_MXFP4 = 1
 PERQ_FMT_F32_DEBUG = 2
 PERQ_FMT_FP4 = 3
-FMT_BY_NAME = {"int4": PERQ_FMT_INT4, "mxfp4": PERQ_FMT_MXFP4, "f32": PERQ_FMT_F32_DEBUG, "fp4": PERQ_FMT_FP4}
+PERQ_FMT_INT4_ASYM = 4
+FMT_BY_NAME = {"int4": PERQ_FMT_INT4, "mxfp4": PERQ_FMT_MXFP4, "f32": PERQ_FMT_F32_DEBUG, "fp4": PERQ_FMT_FP4,
+               "int4_asym": PERQ_FMT_INT4_ASYM}
 
 PERQ_OK = 0
 
@@ -102,6 +104,8 @@ def alloc_outputs(T: int, d: int, fmt: int, group: int, device):
     codes = torch.empty((T, d // 2), dtype=torch.uint8, device=device)
     if fmt == PERQ_FMT_FP4:
         scales = torch.empty((T, 1), dtype=torch.float32, device=device)
+    elif fmt == PERQ_FMT_INT4_ASYM:
+        scales = torch.empty((T, 2), dtype=torch.float32, device=device)
     elif fmt == PERQ_FMT_INT4:
         scales = torch.empty((T, 1 if group == 0 else d // group), dtype=torch.float32, device=device)
     else:

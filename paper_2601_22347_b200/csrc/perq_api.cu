@@ -29,7 +29,9 @@ inline bool aligned16(const void *p) { return (reinterpret_cast<uintptr_t>(p) & 
 int check_shape(int64_t T, int32_t d, int32_t b, int32_t fmt, int32_t group, int *g_out)
 {
     if (T < 0 || d <= 0 || d % 32 != 0 || d > PERQ_MAX_D) return PERQ_ERR_SHAPE;
-    if (fmt != PERQ_FMT_INT4 && fmt != PERQ_FMT_MXFP4 && fmt != PERQ_FMT_F32_DEBUG && fmt != PERQ_FMT_FP4) return PERQ_ERR_FMT;
+    if (fmt != PERQ_FMT_INT4 && fmt != PERQ_FMT_MXFP4 && fmt != PERQ_FMT_F32_DEBUG && fmt != PERQ_FMT_FP4 &&
+        fmt != PERQ_FMT_INT4_ASYM)
+        return PERQ_ERR_FMT;
     if (!is_pow2(b) || b < 16 || b > d || d % b != 0) return PERQ_ERR_BLOCK;
     int g = d;
     if (fmt == PERQ_FMT_INT4) {
@@ -41,7 +43,7 @@ int check_shape(int64_t T, int32_t d, int32_t b, int32_t fmt, int32_t group, int
     } else if (fmt == PERQ_FMT_MXFP4) {
         if (group != 0 && group != 32) return PERQ_ERR_GROUP;
         g = 32;
-    } else if (fmt == PERQ_FMT_FP4) {
+    } else if (fmt == PERQ_FMT_FP4 || fmt == PERQ_FMT_INT4_ASYM) {
         if (group != 0) return PERQ_ERR_GROUP;      // one scale per token
     }
     if (g_out) *g_out = g;
@@ -183,7 +185,7 @@ int launch_fast_long(int xb, int G, const perq::FastParams &p, int grid, cudaStr
 int try_launch_fast(const void *x, const int32_t *perm, int64_t T, int32_t d, int32_t b, int32_t fmt, int g,
                     void *out_codes, void *out_scales, cudaStream_t st)
 {
-    if (d % perq::SEG_ELEMS != 0) return -1;
+    if (d % perq::SEG_ELEMS != 0 || fmt == PERQ_FMT_INT4_ASYM) return -1;
     const int segs = d / perq::SEG_ELEMS;
     const bool permuted = perm != nullptr;
     const bool full = b == d && b > 128;
@@ -307,7 +309,7 @@ const char *perq_status_string(int status)
     case PERQ_ERR_NULL: return "a required pointer is NULL";
     case PERQ_ERR_SHAPE: return "bad shape: need T >= 0, 0 < d <= 32768, d % 32 == 0 (and the row must fit in shared memory)";
     case PERQ_ERR_BLOCK: return "bad block size: need a power of two b, 16 <= b <= d, dividing d";
-    case PERQ_ERR_GROUP: return "bad group: INT4 needs 0 or a multiple of 8 dividing d; MXFP4 needs 0 or 32; FP4 needs 0";
+    case PERQ_ERR_GROUP: return "bad group: INT4 needs 0 or a multiple of 8 dividing d; MXFP4 needs 0 or 32; FP4 and asymmetric INT4 need 0";
     case PERQ_ERR_FMT: return "unknown format";
     case PERQ_ERR_ALIGN: return "device pointers must be 16-byte aligned";
     case PERQ_ERR_CUDA: return "CUDA runtime error";
@@ -329,10 +331,10 @@ int perq_out_sizes(int64_t T, int32_t d, int32_t fmt, int32_t group, size_t *cod
         if (group != 0 && group != 32) return PERQ_ERR_GROUP;
         cb = (size_t)T * (size_t)(d / 2);
         sb = (size_t)T * (size_t)(d / 32);
-    } else if (fmt == PERQ_FMT_FP4) {
+    } else if (fmt == PERQ_FMT_FP4 || fmt == PERQ_FMT_INT4_ASYM) {
         if (group != 0) return PERQ_ERR_GROUP;
         cb = (size_t)T * (size_t)(d / 2);
-        sb = (size_t)T * sizeof(float);
+        sb = (size_t)T * sizeof(float) * (fmt == PERQ_FMT_INT4_ASYM ? 2 : 1);
     } else if (fmt == PERQ_FMT_F32_DEBUG) {
         cb = (size_t)T * (size_t)d * sizeof(float);
         sb = 0;

@@ -32,7 +32,7 @@ struct GenParams {
     long long T;
     int d;
     int log2b;
-    int fmt;          // 0 INT4, 1 MXFP4, 2 F32 debug, 3 E2M1 with a per-token fp32 scale
+    int fmt;          // 0 INT4, 1 MXFP4, 2 F32 debug, 3 E2M1 with a per-token fp32 scale, 4 asymmetric INT4 per token
     int g;            // effective scale-range length (d for per-token, 32 for MX)
     void *out_codes;
     void *out_scales;
@@ -42,7 +42,7 @@ struct GenParams {
 
 // Shared-memory carve-up, computed identically on host (for the launch) and device.
 struct GenSmem {
-    size_t xs, ub, codes, r_max, r_thr, r_mul, r_aux, r_E, b_max, ties, total;
+    size_t xs, ub, codes, r_max, r_thr, r_mul, r_aux, r_E, b_max, ties, asym, total;
     __host__ __device__ GenSmem(int d, int g, int log2b)
     {
         const size_t nr = (size_t)(d / g), nb = (size_t)(d >> log2b);
@@ -58,6 +58,7 @@ struct GenSmem {
         r_E = o;   o += nr * 4;
         b_max = o; o += nb * 4;
         ties = o;  o += (size_t)TIE_CAP * 4 + 16;
+        asym = o;  o += 4 * 8;      // asymmetric INT4: exact max, exact min (order-preserving codes), step, zero point
         total = o;
     }
 };
@@ -65,6 +66,26 @@ struct GenSmem {
 __device__ __forceinline__ float bf16lo(uint32_t w) { return __uint_as_float(w << 16); }
 __device__ __forceinline__ float bf16hi(uint32_t w) { return __uint_as_float(w & 0xffff0000u); }
 __device__ __forceinline__ double bf16_to_f64(uint16_t h) { return (double)__uint_as_float((uint32_t)h << 16); }
+
+// Order-preserving unsigned codes of signed floating-point values (for atomicMax / atomicMin).
+__device__ __forceinline__ uint32_t ord32(float f)
+{
+    const uint32_t u = __float_as_uint(f);
+    return (u & 0x80000000u) ? ~u : (u | 0x80000000u);
+}
+__device__ __forceinline__ float unord32(uint32_t c)
+{
+    return __uint_as_float((c & 0x80000000u) ? (c & 0x7fffffffu) : ~c);
+}
+__device__ __forceinline__ unsigned long long ord64(double f)
+{
+    const unsigned long long u = (unsigned long long)__double_as_longlong(f);
+    return (u >> 63) ? ~u : (u | 0x8000000000000000ull);
+}
+__device__ __forceinline__ double unord64(unsigned long long c)
+{
+    return __longlong_as_double((long long)((c >> 63) ? (c & 0x7fffffffffffffffull) : ~c));
+}
 
 // In-register butterfly over the low `R` index bits of v[0..2^R).
 template <int R>
@@ -164,9 +185,14 @@ __device__ __forceinline__ uint32_t cvt_e2m1x2(float lo, float hi)
 }
 
 // Exact code of element i (row-relative index) from its exact unnormalised value u.
-__device__ __forceinline__ uint32_t exact_code(const GenParams &p, double u, double s64, int E)
+__device__ __forceinline__ uint32_t exact_code(const GenParams &p, double u, double s64, int E, double z64 = 0.0)
 {
     const double y = u / p.sqrt_b;
+    if (p.fmt == 4) {
+        if (s64 == 0.0) return 0u;
+        const double q = fmin(fmax(rint(y / s64) - z64, 0.0), 15.0);
+        return (uint32_t)((int)q);
+    }
     if (p.fmt == 0) {
         if (s64 == 0.0) return 0u;
         double q = rint(y / s64);
@@ -247,8 +273,49 @@ __global__ void __launch_bounds__(GEN_THREADS) perq_generic_kernel(GenParams p)
             continue;
         }
 
+        unsigned long long *asym = (unsigned long long *)(smem + lay.asym);
+        if (p.fmt == 4) {
+            // ---- C'-E'. asymmetric INT4 (one range: the row): signed fp32 extremes, their exact values, step and zero point
+            uint32_t *cmin = (uint32_t *)r_thr;     // (the threshold slot is free in this mode)
+            if (tid == 0) { r_max[0] = 0u; cmin[0] = 0xffffffffu; asym[0] = 0ull; asym[1] = ~0ull; }
+            __syncthreads();
+            for (int c = tid; c < nchunks; c += GEN_THREADS) {
+                const float4 a = ((const float4 *)ub)[2 * c], e = ((const float4 *)ub)[2 * c + 1];
+                const float hi = fmaxf(fmaxf(fmaxf(a.x, a.y), fmaxf(a.z, a.w)), fmaxf(fmaxf(e.x, e.y), fmaxf(e.z, e.w)));
+                const float lo = fminf(fminf(fminf(a.x, a.y), fminf(a.z, a.w)), fminf(fminf(e.x, e.y), fminf(e.z, e.w)));
+                atomicMax(&r_max[0], ord32(hi));
+                atomicMin(&cmin[0], ord32(lo));
+                atomicMax(&b_max[(c * 8) >> L], __float_as_uint(fmaxf(fabsf(hi), fabsf(lo))));
+            }
+            __syncthreads();
+            const float mx32 = unord32(r_max[0]), mn32 = unord32(cmin[0]);
+            const float err_row = err_rel * fmaxf(fabsf(mx32), fabsf(mn32));     // every block maximum is below this
+            const float thr_hi = mx32 - 2.0f * err_row, thr_lo = mn32 + 2.0f * err_row;
+            for (int i0 = warp * 32; i0 < d; i0 += GEN_THREADS) {
+                const float ui = ub[i0 + lane];
+                unsigned m = __ballot_sync(0xffffffffu, ui >= thr_hi || ui <= thr_lo);
+                while (m) {
+                    const int ic = i0 + (__ffs(m) - 1);
+                    m &= m - 1;
+                    const double u = exact_coord_warp(xs, (ic >> L) << L, b, ic & (b - 1), lane);
+                    if (lane == 0) { atomicMax(&asym[0], ord64(u)); atomicMin(&asym[1], ord64(u)); }
+                }
+            }
+            __syncthreads();
+            if (tid == 0) {
+                const double mxy = unord64(asym[0]) / p.sqrt_b, mny = unord64(asym[1]) / p.sqrt_b;
+                const double s = (mxy - mny) / 15.0;
+                const double z = (s == 0.0) ? 0.0 : rint(mny / s);
+                ((float *)p.out_scales)[(size_t)row * 2] = (float)s;
+                ((float *)p.out_scales)[(size_t)row * 2 + 1] = (float)z;
+                r_mul[0] = (s == 0.0) ? 0.0f : fminf((float)(1.0 / (s * p.sqrt_b)), 3.0e38f);
+                asym[2] = (unsigned long long)__double_as_longlong(s);
+                asym[3] = (unsigned long long)__double_as_longlong(z);
+            }
+            __syncthreads();
+        }
         // ---- C. fp32 absmax per scale range and per Hadamard block
-        for (int c = tid; c < nchunks; c += GEN_THREADS) {
+        for (int c = tid; p.fmt != 4 && c < nchunks; c += GEN_THREADS) {
             const float4 a = ((const float4 *)ub)[2 * c], e = ((const float4 *)ub)[2 * c + 1];
             const float m = fmaxf(fmaxf(fmaxf(fabsf(a.x), fabsf(a.y)), fmaxf(fabsf(a.z), fabsf(a.w))),
                                   fmaxf(fmaxf(fabsf(e.x), fabsf(e.y)), fmaxf(fabsf(e.z), fabsf(e.w))));
@@ -258,7 +325,7 @@ __global__ void __launch_bounds__(GEN_THREADS) perq_generic_kernel(GenParams p)
         __syncthreads();
 
         // ---- D. which ranges need their absmax re-derived exactly, and from which elements
-        for (int r = tid; r < nr; r += GEN_THREADS) {
+        for (int r = tid; p.fmt != 4 && r < nr; r += GEN_THREADS) {
             const float rm = __uint_as_float(r_max[r]);
             const float bm = (g >= b) ? rm : __uint_as_float(b_max[(r * g) >> L]);
             const float err = err_rel * bm;
@@ -276,7 +343,7 @@ __global__ void __launch_bounds__(GEN_THREADS) perq_generic_kernel(GenParams p)
         {
             const int parts = (g + 255) >> 8;
             const int units = nr * parts;
-            for (int unit = warp; unit < units; unit += GEN_WARPS) {
+            for (int unit = warp; p.fmt != 4 && unit < units; unit += GEN_WARPS) {
                 const int r = unit / parts, part = unit - r * parts;
                 const float thr = r_thr[r];
                 if (!(thr < __int_as_float(0x7f800000))) continue;
@@ -298,7 +365,7 @@ __global__ void __launch_bounds__(GEN_THREADS) perq_generic_kernel(GenParams p)
         __syncthreads();
 
         // ---- E. scales
-        for (int r = tid; r < nr; r += GEN_THREADS) {
+        for (int r = tid; p.fmt != 4 && r < nr; r += GEN_THREADS) {
             const float rm = __uint_as_float(r_max[r]);
             const bool exact = r_thr[r] < __int_as_float(0x7f800000);
             const double au = exact ? __longlong_as_double((long long)r_aux[r]) : (double)rm;
@@ -330,7 +397,16 @@ __global__ void __launch_bounds__(GEN_THREADS) perq_generic_kernel(GenParams p)
             const float4 a = ((const float4 *)ub)[2 * c], e = ((const float4 *)ub)[2 * c + 1];
             const float u[8] = {a.x, a.y, a.z, a.w, e.x, e.y, e.z, e.w};
             uint32_t word = 0u, flags = 0u;
-            if (p.fmt == 0) {
+            if (p.fmt == 4) {
+                const float zf = (float)__longlong_as_double((long long)asym[3]);
+#pragma unroll
+                for (int k = 0; k < 8; ++k) {
+                    const float v = u[k] * mul;
+                    const float rq = rintf(v);
+                    if (fabsf(v - rq) > 0.5f - (tau_abs + (fabsf(v) + 8.0f) * 5.0e-7f)) flags |= 1u << k;
+                    word |= (uint32_t)((int)fminf(fmaxf(rq - zf, 0.0f), 15.0f)) << (4 * k);
+                }
+            } else if (p.fmt == 0) {
 #pragma unroll
                 for (int k = 0; k < 8; ++k) {
                     const float v = u[k] * mul;
@@ -357,7 +433,9 @@ __global__ void __launch_bounds__(GEN_THREADS) perq_generic_kernel(GenParams p)
                 } else {   // list full: resolve here, single-threaded
                     const int i = i0 + k;
                     const double ue = exact_coord_thread(xs, (i >> L) << L, b, i & (b - 1));
-                    const uint32_t code = exact_code(p, ue, __longlong_as_double((long long)r_aux[r]), r_E[r]);
+                    const uint32_t code = (p.fmt == 4)
+                        ? exact_code(p, ue, __longlong_as_double((long long)asym[2]), 0, __longlong_as_double((long long)asym[3]))
+                        : exact_code(p, ue, __longlong_as_double((long long)r_aux[r]), r_E[r]);
                     word = (word & ~(0xFu << (4 * k))) | (code << (4 * k));
                 }
             }
@@ -372,7 +450,9 @@ __global__ void __launch_bounds__(GEN_THREADS) perq_generic_kernel(GenParams p)
                 const int i = tie_list[t], r = i / g;
                 const double ue = exact_coord_warp(xs, (i >> L) << L, b, i & (b - 1), lane);
                 if (lane == 0) {
-                    const uint32_t code = exact_code(p, ue, __longlong_as_double((long long)r_aux[r]), r_E[r]);
+                    const uint32_t code = (p.fmt == 4)
+                        ? exact_code(p, ue, __longlong_as_double((long long)asym[2]), 0, __longlong_as_double((long long)asym[3]))
+                        : exact_code(p, ue, __longlong_as_double((long long)r_aux[r]), r_E[r]);
                     const int sh = 4 * (i & 7);
                     atomicAnd(&codes[i >> 3], ~(0xFu << sh));
                     atomicOr(&codes[i >> 3], code << sh);

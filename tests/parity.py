@@ -41,7 +41,12 @@ def compare_quantized(fmt: str, gpu_codes, gpu_scales, ora: dict) -> dict:
     gpu_scales = np.asarray(gpu_scales).reshape(ora["scales"].shape)
     assert gpu_codes.shape == ora["codes"].shape
     report = {"elements": int(gpu_codes.size) * 2, "code_mismatch_exempt": 0, "scale_ulp_max": 0}
-    if fmt in ("int4", "fp4"):
+    if fmt == "int4_asym":
+        ulp = ulp_distance_f32(np.abs(gpu_scales[:, 0]), np.abs(ora["scales"][:, 0]))
+        report["scale_ulp_max"] = int(ulp.max()) if ulp.size else 0
+        assert report["scale_ulp_max"] <= 1, "asymmetric INT4 step differs by %d ulp" % report["scale_ulp_max"]
+        assert np.array_equal(gpu_scales[:, 1], ora["scales"][:, 1]), "zero points differ"
+    elif fmt in ("int4", "fp4"):
         ulp = ulp_distance_f32(gpu_scales, ora["scales"])
         report["scale_ulp_max"] = int(ulp.max()) if ulp.size else 0
         assert report["scale_ulp_max"] <= 1, "%s scale differs by %d ulp" % (fmt, report["scale_ulp_max"])
@@ -55,7 +60,10 @@ def compare_quantized(fmt: str, gpu_codes, gpu_scales, ora: dict) -> dict:
         o = unpack_nibbles(ora["codes"])
         idx = np.nonzero(g != o)
         pre = ora["pre"][idx]
-        if fmt == "int4":
+        if fmt == "int4_asym":
+            step = np.abs(g[idx].astype(np.int64) - o[idx].astype(np.int64))
+            near = np.abs(np.abs(pre - np.floor(pre)) - 0.5) < TIE_WINDOW * np.maximum(1.0, np.abs(pre) / 8.0)
+        elif fmt == "int4":
             step = np.abs(int4_values(g[idx]) - int4_values(o[idx]))
             near = np.abs(np.abs(pre - np.floor(pre)) - 0.5) < TIE_WINDOW
         else:

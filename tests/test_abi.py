@@ -55,6 +55,7 @@ def test_out_sizes(lib):
     assert B.perq_out_sizes(3, 64, B.PERQ_FMT_F32_DEBUG, 0) == (3 * 64 * 4, 0)
     assert B.perq_out_sizes(0, 64, B.PERQ_FMT_INT4, 0) == (0, 0)
     assert B.perq_out_sizes(16384, 4096, B.PERQ_FMT_FP4, 0) == (16384 * 2048, 16384 * 4)
+    assert B.perq_out_sizes(16384, 4096, B.PERQ_FMT_INT4_ASYM, 0) == (16384 * 2048, 16384 * 8)
 
 
 def test_argument_validation_happens_before_any_launch(lib):

@@ -9,7 +9,7 @@ from parity import compare_quantized, compare_rotated, unpack_nibbles, int4_valu
 
 pytestmark = pytest.mark.gpu
 
-FMT = {"int4": 0, "mxfp4": 1, "fp4": 3}
+FMT = {"int4": 0, "mxfp4": 1, "fp4": 3, "int4_asym": 4}
 
 
 @pytest.fixture(scope="module")
@@ -535,3 +535,39 @@ def test_fp4_exact_midpoints_and_saturation(B, oracle):
     w.group = 0
     rows_ = np.sort(np.random.default_rng(9).choice(w.T, 64, replace=False))
     check(B, oracle, w, rows=rows_)
+
+
+# ------------------------------------------------------------------ asymmetric INT4 per token
+
+@pytest.mark.parametrize("perm", [False, True])
+@pytest.mark.parametrize("d,T,b", [(1024, 40, 16), (2048, 100, 32), (4096, 60, 128), (8192, 20, 64), (1536, 33, 32),
+                                   (2048, 12, 2048), (14336, 9, 32)])
+def test_asymmetric_int4_per_token(B, oracle, d, T, b, perm):
+    bits, _ = inputs.student_t_outliers(T, d, 3.0, max(2, d // 256), 100.0, seed=9000 + d + b)
+    x = inputs.bf16_bits_to_f32(bits)
+    x[1] += 3.0                      # a row whose range is far from symmetric
+    x[2] = 0.0                       # constant rows: step 0
+    x[3] = 1.5
+    bits = inputs.f32_to_bf16_bits(x)
+    p = inputs.random_perm(d, 9001) if perm else None
+    check(B, oracle, inputs.Workload("asym", bits, p, b, "int4_asym", 0, 0))
+
+
+def test_asymmetric_int4_exact_ties(B, oracle):
+    import scipy.linalg
+    H = scipy.linalg.hadamard(16)
+    rng = np.random.default_rng(98)
+    rows = []
+    for _ in range(16):
+        blocks = []
+        for j in range(64):
+            ystar = rng.integers(-13, 17, size=16) * 0.5           # halves in [-6.5, 8]
+            if j == 0:
+                ystar[0], ystar[1] = -7.0, 8.0                     # range 15 -> step 1, zero point -7
+            blocks.append((ystar @ H) / 4.0)
+        rows.append(np.concatenate(blocks))
+    x = np.array(rows, np.float32)
+    bits = inputs.f32_to_bf16_bits(x)
+    assert np.array_equal(inputs.bf16_bits_to_f32(bits), x)
+    rep = check(B, oracle, inputs.Workload("asym-ties", bits, None, 16, "int4_asym", 0, 0))
+    assert rep["code_mismatch_exempt"] == 0
