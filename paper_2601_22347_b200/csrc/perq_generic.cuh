@@ -58,6 +58,7 @@ struct GenSmem {
         r_E = o;   o += nr * 4;
         b_max = o; o += nb * 4;
         ties = o;  o += (size_t)TIE_CAP * 4 + 16;
+        o = (o + 7) & ~(size_t)7;   // 64-bit atomics below
         asym = o;  o += 4 * 8;      // asymmetric INT4: exact max, exact min (order-preserving codes), step, zero point
         total = o;
     }
