@@ -337,6 +337,40 @@ __device__ __forceinline__ double exact_coord4_perm(const uint16_t *raw, const u
     return acc;
 }
 
+// Long blocks: the whole warp evaluates one record.  Lane l takes the 8 consecutive inputs
+// 256 r + 8 l .. + 7 of every 256 (coalesced 16-byte loads), keeps the four partial sums by k & 3,
+// and the lanes are summed before the 4-point butterfly.  Returns the largest magnitude of the
+// four outputs i0 .. i0 + 3 (the same in every lane).
+template <int B, bool GLOBAL>
+__device__ __forceinline__ double exact_slot_max_wide(const uint16_t *blk, uint32_t i0, int lane)
+{
+    static_assert(B >= 256, "one 16-byte load per lane covers 256 inputs");
+    double S[4] = {0.0, 0.0, 0.0, 0.0};
+    const uint4 *src = reinterpret_cast<const uint4 *>(blk) + lane;
+#pragma unroll(B / 256 < 16 ? B / 256 : 16)
+    for (int r = 0; r < B / 256; ++r) {
+        const uint4 w4 = GLOBAL ? __ldg(src + r * 32) : src[r * 32];
+        const uint32_t w[4] = {w4.x, w4.y, w4.z, w4.w};
+        const uint32_t k0 = (uint32_t)(r * 256 + lane * 8);
+#pragma unroll
+        for (int h = 0; h < 2; ++h) {
+            const uint32_t flip = (__popc(i0 & (k0 + 4u * h)) & 1) ? 0x80008000u : 0u;
+#pragma unroll
+            for (int e = 0; e < 4; ++e) {
+                const uint32_t word = w[2 * h + (e >> 1)] ^ flip;
+                S[e] += bf16_bits_to_f64((e & 1) ? (word >> 16) : word);
+            }
+        }
+    }
+#pragma unroll
+    for (int m = 0; m < 4; ++m) {
+#pragma unroll
+        for (int o = 16; o > 0; o >>= 1) S[m] += __shfl_xor_sync(0xffffffffu, S[m], o);
+    }
+    const double a0 = S[0] + S[1], a1 = S[0] - S[1], a2 = S[2] + S[3], a3 = S[2] - S[3];
+    return fmax(fmax(fabs(a0 + a2), fabs(a1 + a3)), fmax(fabs(a0 - a2), fabs(a1 - a3)));
+}
+
 // Element e = s*4 + j of lane (g, q): block start (in elements, segment relative) and index inside the block.
 template <int LOG2B>
 __device__ __forceinline__ void locate(int g, int q, int e, int &blk_elem, int &i, int &elem)
@@ -394,7 +428,10 @@ __device__ __forceinline__ unsigned long long exact_max_of_candidates(const uint
             const int pch = sg * 8 + (sl ^ ((sg & 3) & ~PM));      // chunk position in the segment
             if (FULL_LOG2 > 0) {
                 const int pr = seg_off + pch * 16 + 4 * (src & 3), be = (pr >> FULL_LOG2) << FULL_LOG2;
-                best = fmax(best, fabs(exact_coord4<(1 << (FULL_LOG2 > 0 ? FULL_LOG2 : 4))>(seg + be, pr - be, lane)));
+                if (FULL_LOG2 >= 8)
+                    best = fmax(best, exact_slot_max_wide<(1 << (FULL_LOG2 >= 8 ? FULL_LOG2 : 8)), false>(seg + be, (uint32_t)(pr - be), lane));
+                else
+                    best = fmax(best, fabs(exact_coord4<(1 << (FULL_LOG2 > 0 ? FULL_LOG2 : 4))>(seg + be, pr - be, lane)));
             } else {
                 const int blk_elem = (pch >> CB) << LOG2B;
                 const int i0 = pch * 16 - blk_elem + 4 * (src & 3);
@@ -418,6 +455,8 @@ __device__ __forceinline__ unsigned long long exact_max_of_candidates(const uint
 // Record: bits 63..32 = index of a 1024-element segment, bits 15..0 = element offset from that
 // segment's start to the slot's first output (per token: first segment of the row, offset in the row).
 // The same scheme serves the per-128 scales, with one record per quad.
+
+constexpr int WIDE_LOG2B = 10;      // blocks from this length on are served by the whole warp
 
 template <int LOG2B, bool PERM>
 __device__ __forceinline__ double exact_slot_max_global(const uint16_t *row, uint32_t pos, const int32_t *perm, int d)
@@ -460,8 +499,8 @@ template <int LOG2B, int MODE, bool PERM>
 __device__ __forceinline__ void serve_scale_requests(const FastParams &p, const unsigned long long *req, uint32_t n, int lane)
 {
     __syncwarp();
-    if (LOG2B >= 10 && !PERM && n < 16u) {
-        // long blocks, few records: the whole warp evaluates one record at a time (coalesced reads)
+    if (LOG2B >= WIDE_LOG2B && !PERM) {
+        // long blocks: the whole warp evaluates one record at a time (coalesced reads)
         for (uint32_t j = 0; j < n; ++j) {
             const unsigned long long r = req[j];
             const uint32_t segi = (uint32_t)(r >> 32), off = (uint32_t)r & 0xffffu;
@@ -469,12 +508,10 @@ __device__ __forceinline__ void serve_scale_requests(const FastParams &p, const 
             const uint32_t row = segi / segs;
             const uint32_t pos = (segi - row * segs) * SEG_ELEMS + off;
             const uint32_t blk = (pos >> LOG2B) << LOG2B;
-            const double val = fabs(exact_coord4<(1 << LOG2B)>(p.x + (size_t)row * p.d + blk, (int)(pos - blk), lane));
-            const unsigned long long ab = warp_max_u64((unsigned long long)__double_as_longlong(val));
+            const double a = exact_slot_max_wide<(1 << (LOG2B >= 8 ? LOG2B : 8)), true>(p.x + (size_t)row * p.d + blk, pos - blk, lane);
             if (lane == 0) {
                 const size_t si = per_token_mode(MODE) ? (size_t)row : ((size_t)row * p.d + pos) >> 7;
-                reinterpret_cast<float *>(p.out_scales)[si] =
-                    (ab == 0ull) ? 0.0f : (float)(__longlong_as_double((long long)ab) * p.inv_7_sqrt_b);
+                reinterpret_cast<float *>(p.out_scales)[si] = (a == 0.0) ? 0.0f : (float)(a * p.inv_7_sqrt_b);
             }
         }
         __syncwarp();
