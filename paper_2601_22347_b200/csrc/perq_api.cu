@@ -126,6 +126,13 @@ int launch_fast_mode(int mode, int G, int log2b, const perq::FastParams &p, int 
 {
     if (mode == perq::MODE_MX) return launch_fast_b<perq::MODE_MX, 0, PERM>(log2b, p, grid, st);
     if (mode == perq::MODE_G128) return launch_fast_b<perq::MODE_G128, 0, PERM>(log2b, p, grid, st);
+    if (mode == perq::MODE_ASYM) {
+        switch (G) {
+        case 4: return launch_fast_b<perq::MODE_ASYM, 2, PERM>(log2b, p, grid, st);
+        case 8: return launch_fast_b<perq::MODE_ASYM, 3, PERM>(log2b, p, grid, st);
+        default: return launch_fast_b<perq::MODE_ASYM, -1, PERM>(log2b, p, grid, st);    // G at run time
+        }
+    }
     if (mode == perq::MODE_FP4) {
         switch (G) {
         case 1: return launch_fast_b<perq::MODE_FP4, 0, PERM>(log2b, p, grid, st);
@@ -185,7 +192,7 @@ int launch_fast_long(int xb, int G, const perq::FastParams &p, int grid, cudaStr
 int try_launch_fast(const void *x, const int32_t *perm, int64_t T, int32_t d, int32_t b, int32_t fmt, int g,
                     void *out_codes, void *out_scales, cudaStream_t st)
 {
-    if (d % perq::SEG_ELEMS != 0 || fmt == PERQ_FMT_INT4_ASYM) return -1;
+    if (d % perq::SEG_ELEMS != 0) return -1;
     const int segs = d / perq::SEG_ELEMS;
     const bool permuted = perm != nullptr;
     const bool full = b == d && b > 128;
@@ -202,6 +209,10 @@ int try_launch_fast(const void *x, const int32_t *perm, int64_t T, int32_t d, in
         G = segs;
         if (G > perq::FAST_WARPS - 1 || full || longb) return -1;
         mode = perq::MODE_FP4;
+    } else if (fmt == PERQ_FMT_INT4_ASYM) {
+        G = segs;
+        if (G > perq::FAST_WARPS - 1 || full || longb) return -1;
+        mode = perq::MODE_ASYM;
     } else if (fmt == PERQ_FMT_INT4 && g == d) {
         G = segs;
         if (G > perq::FAST_WARPS - 1) return -1;          // named barriers 1..15: one per group of G warps

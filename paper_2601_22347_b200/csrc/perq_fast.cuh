@@ -63,8 +63,9 @@ constexpr uint32_t WAIT_SPIN_LIMIT = 1u << 22;
 
 // per-token INT4, INT4 per 128, MXFP4, and E2M1 with a per-token fp32 scale (the scale logic of MODE_TOKEN
 // with the element conversion of MODE_MX)
-enum FastMode { MODE_TOKEN = 0, MODE_G128 = 1, MODE_MX = 2, MODE_FP4 = 3 };
-__host__ __device__ constexpr bool per_token_mode(int mode) { return mode == MODE_TOKEN || mode == MODE_FP4; }
+// MODE_ASYM: asymmetric INT4 per token (step and integer zero point from the row's signed extremes)
+enum FastMode { MODE_TOKEN = 0, MODE_G128 = 1, MODE_MX = 2, MODE_FP4 = 3, MODE_ASYM = 4 };
+__host__ __device__ constexpr bool per_token_mode(int mode) { return mode == MODE_TOKEN || mode == MODE_FP4 || mode == MODE_ASYM; }
 
 struct FastParams {
     const uint16_t *x;
@@ -88,11 +89,16 @@ struct FastSmem {
     static constexpr size_t full = codes + (size_t)FAST_WARPS * 2 * SEG_CODE_BYTES;
     static constexpr size_t wacc = full + (size_t)FAST_WARPS * FAST_NSTAGE * 8;     // [2][FAST_WARPS] u64 accumulators
     static constexpr size_t wpub = wacc + (size_t)FAST_WARPS * 2 * 8;               // [2][FAST_WARPS] u64 published row maxima
-    static constexpr size_t wmax = wpub + (size_t)FAST_WARPS * 2 * 8;               // [2][FAST_WARPS] f32 warp maxima
-    static constexpr size_t wcnt = wmax + (size_t)FAST_WARPS * 2 * 4;               // [2][FAST_WARPS] u32 arrival counts
+    static constexpr size_t wacc2 = wpub + (size_t)FAST_WARPS * 2 * 8;              // asymmetric: the same two for the row minimum
+    static constexpr size_t wpub2 = wacc2 + (size_t)FAST_WARPS * 2 * 8;             //   (and the published zero point)
+    static constexpr size_t wmax = wpub2 + (size_t)FAST_WARPS * 2 * 8;              // [2][FAST_WARPS] f32 warp maxima
+    static constexpr size_t wmin = wmax + (size_t)FAST_WARPS * 2 * 4;               // [2][FAST_WARPS] f32 warp minima (asymmetric)
+    static constexpr size_t wcnt = wmin + (size_t)FAST_WARPS * 2 * 4;               // [2][FAST_WARPS] u32 arrival counts
     static constexpr size_t wflag = wcnt + (size_t)FAST_WARPS * 2 * 4;              // [2][FAST_WARPS] u32 publication flags
     static constexpr size_t wreq = wflag + (size_t)FAST_WARPS * 2 * 4;              // [FAST_WARPS][32] u64 deferred scale requests
-    static constexpr size_t empty = wreq + (size_t)FAST_WARPS * 32 * 8;             // [FAST_WARPS * FAST_NSTAGE] mbarriers
+    static constexpr size_t wreq2 = wreq + (size_t)FAST_WARPS * 32 * 8;             // asymmetric: [FAST_WARPS][32] u64 second key of a record
+    static constexpr size_t wrequ = wreq2 + (size_t)FAST_WARPS * 32 * 8;            //   and [FAST_WARPS][32] u32 its row
+    static constexpr size_t empty = wrequ + (size_t)FAST_WARPS * 32 * 4;            // [FAST_WARPS * FAST_NSTAGE] mbarriers
     static constexpr size_t used = empty + (size_t)FAST_WARPS * FAST_NSTAGE * 8;
     static constexpr size_t total = used + 1024;                                    // room to align the base
     // permuted variants: the stage area holds 3 raw-row stages per group (96 KB in all) followed by
@@ -209,7 +215,23 @@ __device__ __forceinline__ float warp_max_f32(float v)
     asm volatile("redux.sync.max.f32 %0, %1, 0xffffffff;" : "=f"(r) : "f"(v));
     return r;
 }
-// max over the warp of a non-negative double, on its bit pattern
+__device__ __forceinline__ float warp_min_f32(float v)
+{
+    float r;
+    asm volatile("redux.sync.min.f32 %0, %1, 0xffffffff;" : "=f"(r) : "f"(v));
+    return r;
+}
+// double <-> 64-bit key with the same order (keys of finite values are never 0 or all ones)
+__device__ __forceinline__ unsigned long long order_key(double f)
+{
+    const unsigned long long u = (unsigned long long)__double_as_longlong(f);
+    return (u >> 63) ? ~u : (u | 0x8000000000000000ull);
+}
+__device__ __forceinline__ double order_value(unsigned long long k)
+{
+    return __longlong_as_double((long long)((k >> 63) ? (k & 0x7fffffffffffffffull) : ~k));
+}
+// max over the warp of a non-negative double, on its bit pattern (or of any 64-bit key)
 __device__ __forceinline__ unsigned long long warp_max_u64(unsigned long long v)
 {
     const uint32_t hi = __reduce_max_sync(0xffffffffu, (uint32_t)(v >> 32));
@@ -530,6 +552,30 @@ __device__ __forceinline__ void serve_scale_requests(const FastParams &p, const 
     __syncwarp();
 }
 
+// Asymmetric INT4: step and zero point from the order keys of the exact unnormalised extremes, in the
+// operation order of the definition (y = u / sqrt(b); s = (max y - min y) / 15; z = rne(min y / s)).
+__device__ __forceinline__ void asym_step_zero(unsigned long long khi, unsigned long long klo, double sqrt_b, double &s64, double &z64)
+{
+    const double mxy = order_value(khi) / sqrt_b, mny = order_value(klo) / sqrt_b;
+    s64 = (mxy - mny) / 15.0;
+    z64 = (s64 == 0.0) ? 0.0 : rint(mny / s64);
+}
+
+// Deferred (s, z) of up to 32 rows, one per lane: the divisions above cost a few hundred instructions,
+// which a lane per row amortises over the warp.
+__device__ __forceinline__ void serve_asym_requests(const FastParams &p, const unsigned long long *khi, const unsigned long long *klo,
+                                                    const uint32_t *rows, uint32_t n, int lane)
+{
+    __syncwarp();
+    if ((uint32_t)lane < n) {
+        double s64, z64;
+        asym_step_zero(khi[lane], klo[lane], p.sqrt_b, s64, z64);
+        float2 *dst = reinterpret_cast<float2 *>(p.out_scales) + rows[lane];
+        *dst = make_float2((float)s64, (float)z64);
+    }
+    __syncwarp();
+}
+
 // ---------------------------------------------------------------- the kernel
 
 // XB > 0: the Hadamard block has 2^(7 + XB) elements (LOG2B must be 7: the part of the
@@ -580,9 +626,14 @@ __global__ void __launch_bounds__(FAST_THREADS, 1) perq_fast_kernel(FastParams p
     unsigned long long *wacc = reinterpret_cast<unsigned long long *>(fsmem + FastSmem::wacc);
     unsigned long long *wpub = reinterpret_cast<unsigned long long *>(fsmem + FastSmem::wpub);
     float *wmax = reinterpret_cast<float *>(fsmem + FastSmem::wmax);
+    float *wmin = reinterpret_cast<float *>(fsmem + FastSmem::wmin);
+    unsigned long long *wacc2 = reinterpret_cast<unsigned long long *>(fsmem + FastSmem::wacc2);
+    unsigned long long *wpub2 = reinterpret_cast<unsigned long long *>(fsmem + FastSmem::wpub2);
     uint32_t *wcnt = reinterpret_cast<uint32_t *>(fsmem + FastSmem::wcnt);
     uint32_t *wflag = reinterpret_cast<uint32_t *>(fsmem + FastSmem::wflag);
     unsigned long long *wreq = reinterpret_cast<unsigned long long *>(fsmem + FastSmem::wreq) + warp * 32;
+    unsigned long long *wreq2 = reinterpret_cast<unsigned long long *>(fsmem + FastSmem::wreq2) + warp * 32;
+    uint32_t *wrequ = reinterpret_cast<uint32_t *>(fsmem + FastSmem::wrequ) + warp * 32;
     uint32_t nreq = 0;                       // records waiting in wreq (the same in every lane)
     const bool leader = (w_in_g == 0) && (lane == 0);
 
@@ -594,7 +645,7 @@ __global__ void __launch_bounds__(FAST_THREADS, 1) perq_fast_kernel(FastParams p
         uint16_t *pt = reinterpret_cast<uint16_t *>(fsmem + FastSmem::perm_tab);
         for (int i = tid; i < p.d; i += FAST_THREADS) pt[i] = (uint16_t)(2 * min(max(__ldg(p.perm + i), 0), p.d - 1));
     }
-    if (tid < 2 * FAST_WARPS) { wacc[tid] = 0ull; wcnt[tid] = 0u; wflag[tid] = 0u; }
+    if (tid < 2 * FAST_WARPS) { wacc[tid] = 0ull; wacc2[tid] = ~0ull; wcnt[tid] = 0u; wflag[tid] = 0u; }
     if (tid == 0) asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
     __syncthreads();
 
@@ -817,7 +868,225 @@ __global__ void __launch_bounds__(FAST_THREADS, 1) perq_fast_kernel(FastParams p
         bulk_store_wait_read<1>();           // the store that last read this staging buffer has drained
         __syncwarp();
 
-        if (MODE != MODE_MX) {
+        if (MODE == MODE_ASYM) {
+            // ---------------------------------------------------------------- asymmetric INT4 per token
+            // step s = (max y - min y) / 15, zero point z = rne(min y / s), code = clip(rne(y / s) - z, 0, 15).
+            // A held value is sgn[class of its slot] times the true output.
+            constexpr int CB_ = LOG2B - 4;
+            const float INF = __int_as_float(0x7f800000);
+            float chi[NCLS], clo[NCLS];
+#pragma unroll
+            for (int k = 0; k < NCLS; ++k) { chi[k] = -INF; clo[k] = INF; }
+#pragma unroll
+            for (int s = 0; s < 8; ++s) {
+                const int k = s & 3 & PM;
+                chi[k] = fmaxf(fmaxf(chi[k], v[s][0].x), v[s][0].y);
+                chi[k] = fmaxf(fmaxf(chi[k], v[s][1].x), v[s][1].y);
+                clo[k] = fminf(fminf(clo[k], v[s][0].x), v[s][0].y);
+                clo[k] = fminf(fminf(clo[k], v[s][1].x), v[s][1].y);
+            }
+            float lane_hi = -INF, lane_lo = INF;
+#pragma unroll
+            for (int k = 0; k < NCLS; ++k) {
+                const bool pos = sgn[k] > 0.0f;
+                lane_hi = fmaxf(lane_hi, pos ? chi[k] : -clo[k]);
+                lane_lo = fminf(lane_lo, pos ? clo[k] : -chi[k]);
+            }
+            const float hw = warp_max_f32(lane_hi), lw = warp_min_f32(lane_lo);
+            const uint32_t pidx = par2 * FAST_WARPS + group;
+            float hi_row, lo_row, hm = hw, lm = lw;
+            if (G > 1) {
+                if (lane == 0) { wmax[par2 * FAST_WARPS + warp] = hw; wmin[par2 * FAST_WARPS + warp] = lw; }
+                named_barrier(1 + group, G * 32);
+                hm = (lane < G) ? wmax[par2 * FAST_WARPS + group * G + lane] : -INF;
+                lm = (lane < G) ? wmin[par2 * FAST_WARPS + group * G + lane] : INF;
+                hi_row = warp_max_f32(hm);
+                lo_row = warp_min_f32(lm);
+                refill();
+            } else {
+                hi_row = hw;
+                lo_row = lw;
+            }
+            const float amax = fmaxf(fabsf(hi_row), fabsf(lo_row));
+            const bool live = hi_row > lo_row;               // else: every rotated value is the same (a zero row)
+            const float e_abs = 2.0f * err_rel * amax + amax * 2.4e-7f;
+            const float thr_hi = hi_row - e_abs, thr_lo = lo_row + e_abs;
+            const unsigned candw = (G > 1) ? __ballot_sync(0xffffffffu, live && (lane < G) && (hm >= thr_hi || lm <= thr_lo))
+                                           : (live ? 1u : 0u);
+            const bool is_cand = (candw >> w_in_g) & 1u;
+            const int ncand = __popc(candw);
+            if (!live && leader) {
+                reinterpret_cast<float *>(p.out_scales)[2 * (size_t)unit] = 0.0f;
+                reinterpret_cast<float *>(p.out_scales)[2 * (size_t)unit + 1] = 0.0f;
+            }
+
+            // ---- the exact extremes, by the warps that hold candidates; the last of them derives (s, z)
+            if (is_cand) {
+                uint32_t slot_mask = 0u;
+#pragma unroll
+                for (int s = 0; s < 8; ++s) {
+                    const int k = s & 3 & PM;
+                    const float hs = fmaxf(fmaxf(v[s][0].x, v[s][0].y), fmaxf(v[s][1].x, v[s][1].y));
+                    const float ls = fminf(fminf(v[s][0].x, v[s][0].y), fminf(v[s][1].x, v[s][1].y));
+                    const bool pos = sgn[k] > 0.0f;
+                    const float th = pos ? hs : -ls, tl = pos ? ls : -hs;
+                    slot_mask |= (th >= thr_hi || tl <= thr_lo) ? (1u << s) : 0u;
+                }
+                double bhi = -1.7976931348623157e308, blo = 1.7976931348623157e308;
+                unsigned cw = __ballot_sync(0xffffffffu, slot_mask != 0u);
+                while (cw) {
+                    const int src = __ffs(cw) - 1;
+                    cw &= cw - 1;
+                    uint32_t sm = __shfl_sync(0xffffffffu, slot_mask, src);
+                    const int sg = src >> 2;
+                    while (sm) {
+                        const int sl = __ffs(sm) - 1;
+                        sm &= sm - 1;
+                        const int pch = sg * 8 + (sl ^ ((sg & 3) & ~PM));      // chunk position in the segment
+                        const int blk_elem = (pch >> CB_) << LOG2B;
+                        const int i0 = pch * 16 - blk_elem + 4 * (src & 3);
+                        const double val = exact_coord4<B>(seg + blk_elem, i0, lane);   // outputs i0 .. i0+3, one per lane & 3
+                        bhi = fmax(bhi, val);
+                        blo = fmin(blo, val);
+                    }
+                }
+                const unsigned long long khi = warp_max_u64(order_key(bhi));
+                const unsigned long long klo = ~warp_max_u64(~order_key(blo));
+                uint32_t last = 0u;
+                if (lane == 0) {
+                    atomicMax(&wacc[pidx], khi);
+                    atomicMin(&wacc2[pidx], klo);
+                    __threadfence_block();
+                    if (atomicAdd(&wcnt[pidx], 1u) == (uint32_t)(ncand - 1)) {      // last candidate warp of the row
+                        const unsigned long long fhi = atomicExch(&wacc[pidx], 0ull);
+                        const unsigned long long flo = atomicExch(&wacc2[pidx], ~0ull);
+                        wcnt[pidx] = 0u;
+                        // the keys are published now; (s, z) go to global memory later, 32 rows at a time
+                        wpub[pidx] = fhi;
+                        wpub2[pidx] = flo;
+                        __threadfence_block();
+                        *reinterpret_cast<volatile uint32_t *>(&wflag[pidx]) = it + 1u;
+                        wreq[nreq] = fhi;
+                        wreq2[nreq] = flo;
+                        wrequ[nreq] = unit;
+                        last = 1u;
+                    }
+                }
+                nreq += __shfl_sync(0xffffffffu, last, 0);
+                if (nreq == 32u) {
+                    serve_asym_requests(p, wreq, wreq2, wrequ, nreq, lane);
+                    nreq = 0;
+                }
+            }
+
+            // ---- fp32 step and zero point; where rounding the zero point is a close call, the exact one
+            const float rng = hi_row - lo_row;
+            const float inv = live ? fminf(__fdividef(15.0f, rng), 3.0e38f) : 0.0f;
+            const float ar = live ? fminf(amax * inv * (1.0f / 15.0f), 3.0e38f) : 0.0f;     // |y|max / range >= 1/2
+            const float vmin = lo_row * inv;
+            float z32 = live ? rintf(vmin) : 0.0f;
+            const float wz = 30.0f * err_rel * ar * (1.0f + 2.0f * fabsf(lo_row) * inv * (1.0f / 15.0f)) + (fabsf(vmin) + 1.0f) * 1.0e-6f;
+            bool have_exact = false;
+            double s_ex = 0.0, z_ex = 0.0;
+            auto fetch_exact = [&]() -> bool {            // the row's published (s, z); bounded wait
+                uint32_t spin = 0;
+                while (ld_volatile_shared_u32(&wflag[pidx]) != it + 1u) {
+                    if (++spin >= WAIT_SPIN_LIMIT) return false;
+                }
+                __threadfence_block();
+                asym_step_zero(*reinterpret_cast<volatile unsigned long long *>(&wpub[pidx]),
+                               *reinterpret_cast<volatile unsigned long long *>(&wpub2[pidx]), p.sqrt_b, s_ex, z_ex);
+                have_exact = true;
+                return true;
+            };
+            if (live && !(fabsf(vmin - z32) <= 0.5f - wz)) {
+                if (!fetch_exact()) {
+                    if (lane == 0) atomicOr(&g_perq_device_error, 2u);
+                    return;
+                }
+                z32 = (float)z_ex;
+            }
+
+            // ---- quantise: the magic constant carries -z, so the low nibble of the sum is the code
+            const float delta = 36.0f * err_rel * ar + 6.0e-7f;
+            f32x2 mul_p[NCLS], mul_m[NCLS];
+#pragma unroll
+            for (int k = 0; k < NCLS; ++k) {
+                const float mp = sgn[k] * inv * (1.0f + delta), mm = sgn[k] * inv * (1.0f - delta);
+                mul_p[k] = pack2(mp, mp);
+                mul_m[k] = pack2(mm, mm);
+            }
+            const float magic_z = 12582912.0f - z32;          // 1.5 * 2^23 - z
+            const f32x2 magic2 = pack2(magic_z, magic_z);
+            uint32_t tie_any = 0u;
+#pragma unroll
+            for (int s = 0; s < 8; ++s) {
+                const int k = s & 3 & PM;
+                const f32x2 tp0 = fma2(v[s][0], mul_p[k], magic2), tp1 = fma2(v[s][1], mul_p[k], magic2);
+                const f32x2 tm0 = fma2(v[s][0], mul_m[k], magic2), tm1 = fma2(v[s][1], mul_m[k], magic2);
+                const uint32_t pp = ((__float_as_uint(tp1.y) * 16u + __float_as_uint(tp1.x)) * 16u + __float_as_uint(tp0.y)) * 16u
+                                    + __float_as_uint(tp0.x);
+                const uint32_t pm = ((__float_as_uint(tm1.y) * 16u + __float_as_uint(tm1.x)) * 16u + __float_as_uint(tm0.y)) * 16u
+                                    + __float_as_uint(tm0.x);
+                tie_any |= (pp ^ pm) ? (1u << s) : 0u;       // (the whole sums: a code outside 0..15 carries upwards)
+                sts_u16(code_addr0 ^ (uint32_t)(s * 8), pp);
+            }
+
+            // ---- slots whose two sums differ: all four codes exactly (a carry may have reached a neighbour)
+            if (__any_sync(0xffffffffu, tie_any != 0u)) {
+                if (!have_exact && !fetch_exact()) {
+                    if (lane == 0) atomicOr(&g_perq_device_error, 2u);
+                    return;
+                }
+                // elements whose two sums differ; all four of a slot in which a sum left 0..15 (its carry
+                // may have reached a neighbour)
+                uint32_t fm = 0u;
+                if (tie_any != 0u) {
+                    const float t_lo = 12582912.0f, t_hi = 12582927.0f;
+#pragma unroll
+                    for (int s = 0; s < 8; ++s) {
+                        const int k = s & 3 & PM;
+                        const f32x2 tp0 = fma2(v[s][0], mul_p[k], magic2), tp1 = fma2(v[s][1], mul_p[k], magic2);
+                        const f32x2 tm0 = fma2(v[s][0], mul_m[k], magic2), tm1 = fma2(v[s][1], mul_m[k], magic2);
+                        const float t[4] = {tp0.x, tp0.y, tp1.x, tp1.y}, u[4] = {tm0.x, tm0.y, tm1.x, tm1.y};
+                        uint32_t bits = 0u;
+                        bool outside = false;
+#pragma unroll
+                        for (int j = 0; j < 4; ++j) {
+                            bits |= (t[j] != u[j]) ? (1u << j) : 0u;
+                            outside = outside || t[j] < t_lo || t[j] > t_hi || u[j] < t_lo || u[j] > t_hi;
+                        }
+                        fm |= (outside ? 0xFu : bits) << (4 * s);
+                    }
+                }
+                __syncwarp();
+                unsigned tl = __ballot_sync(0xffffffffu, fm != 0u);
+                while (tl) {
+                    const int src = __ffs(tl) - 1;
+                    tl &= tl - 1;
+                    uint32_t fs = __shfl_sync(0xffffffffu, fm, src);
+                    while (fs) {
+                        const int e = __ffs(fs) - 1;
+                        fs &= fs - 1;
+                        int blk_elem, i, elem;
+                        locate<LOG2B>(src >> 2, src & 3, e, blk_elem, i, elem);
+                        const uint16_t *bp;
+                        block_of(elem, bp, i);
+                        const double ue = exact_coord_fast<BF>(bp, i, lane);
+                        if (lane == 0) {
+                            uint32_t code = 0u;
+                            if (s_ex != 0.0) {
+                                const double qd = rint((ue / p.sqrt_b) / s_ex) - z_ex;
+                                code = (uint32_t)((int)fmin(fmax(qd, 0.0), 15.0));
+                            }
+                            uint8_t *cp = code_gen + (elem >> 1);
+                            *cp = (elem & 1) ? (uint8_t)((*cp & 0x0F) | (code << 4)) : (uint8_t)((*cp & 0xF0) | code);
+                        }
+                        __syncwarp();
+                    }
+                }
+            }
+        } else if (MODE != MODE_MX) {
             // lane maximum, then the maximum of the scale range in fp32 (a32); the exact maximum
             // (a_bits, bit pattern of a double) only where it is known without waiting
             const float lane_max = (MODE == MODE_G128)
@@ -1305,7 +1574,11 @@ __global__ void __launch_bounds__(FAST_THREADS, 1) perq_fast_kernel(FastParams p
             if (PERM) mbar_arrive(empty_base + stage * 8);     // this warp no longer reads the staged row
         }
     }
-    if (MODE != MODE_MX && nreq > 0u) serve_scale_requests<LOG2BF, MODE, PERM>(p, wreq, nreq, lane);
+    if (MODE == MODE_ASYM) {
+        if (nreq > 0u) serve_asym_requests(p, wreq, wreq2, wrequ, nreq, lane);
+    } else if (MODE != MODE_MX && nreq > 0u) {
+        serve_scale_requests<LOG2BF, MODE, PERM>(p, wreq, nreq, lane);
+    }
     bulk_store_wait_read<0>();
 }
 

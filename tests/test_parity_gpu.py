@@ -571,3 +571,76 @@ def test_asymmetric_int4_exact_ties(B, oracle):
     assert np.array_equal(inputs.bf16_bits_to_f32(bits), x)
     rep = check(B, oracle, inputs.Workload("asym-ties", bits, None, 16, "int4_asym", 0, 0))
     assert rep["code_mismatch_exempt"] == 0
+
+
+def _asym_constructed_rows():
+    """Rows built in the rotated domain (H_16 is an involution up to the factor 16), every input exactly a
+    bf16 value: blocks are redrawn until they are."""
+    import scipy.linalg
+    H = scipy.linalg.hadamard(16)
+    rng = np.random.default_rng(99)
+    nblk = 256
+
+    def representable(xb):
+        xb = xb.astype(np.float32)
+        return np.array_equal(inputs.bf16_bits_to_f32(inputs.f32_to_bf16_bits(xb)), xb)
+
+    def block(draw, fix=None):
+        for _ in range(1000):
+            yb = draw().astype(np.float64)
+            if fix:
+                for pos, val in fix.items():
+                    yb[pos] = val
+            xb = (yb @ H) / 4.0
+            if representable(xb):
+                return xb
+        raise AssertionError("no representable block found")
+
+    def row(draw, fixes):
+        return np.concatenate([block(draw, fixes.get(j)) for j in range(nblk)])
+
+    rows = []
+    # (a) even integers, min -26, max 34: step 4, min / step = -6.5 is a tie (zero point -6), v = y / 4 in halves
+    rows.append(row(lambda: rng.integers(-12, 17, size=16) * 2.0, {3: {5: -26.0}, 200: {9: 34.0}}))
+    # (b) all positive: multiples of 4 in [4, 64]: step 4, zero point 1
+    rows.append(row(lambda: rng.integers(1, 17, size=16) * 4.0, {0: {0: 4.0}, 255: {15: 64.0}}))
+    # (c) the same extremes in every 1024-element segment (64 blocks each), twice in one slot
+    fixes = {}
+    for seg in range(4):
+        fixes[64 * seg + 7] = {2: 24.0, 3: 24.0}
+        fixes[64 * seg + 40] = {12: -36.0}
+        fixes[64 * seg + 41] = {1: -36.0}
+    rows.append(row(lambda: rng.integers(-10, 11, size=16) * 1.0, fixes))
+    # (d) constant rotated row
+    rows.append(row(lambda: np.full(16, 2.0), {}))
+    # (e) random even integers: codes in halves of the step whenever the range is 60
+    for _ in range(4):
+        rows.append(row(lambda: rng.integers(-15, 16, size=16) * 2.0, {1: {0: -30.0}, 2: {0: 30.0}}))
+    x = np.array(rows, np.float32)
+    bits = inputs.f32_to_bf16_bits(x)
+    assert np.array_equal(inputs.bf16_bits_to_f32(bits), x)
+    return bits
+
+
+def test_asymmetric_int4_constructed_rows(B, oracle):
+    """A zero point that is an exact tie, an all-positive row, extremes repeated in every segment, a constant
+    rotated row, and rows full of exact rounding ties; also through a permutation."""
+    bits = _asym_constructed_rows()
+    d = bits.shape[1]
+    for perm in (None, inputs.random_perm(d, 991)):
+        pb = bits
+        if perm is not None:      # so that the gathered row is the constructed one: pb[:, perm[i]] = bits[:, i]
+            pb = np.empty_like(bits)
+            pb[:, perm] = bits
+        rep = check(B, oracle, inputs.Workload("asym-constructed", pb, perm, 16, "int4_asym", 0, 0))
+        assert rep["code_mismatch_exempt"] == 0
+
+
+@pytest.mark.parametrize("d,b", [(1024, 32), (2048, 64), (4096, 32), (8192, 128), (6144, 16), (14336, 64), (15360, 32)])
+def test_asymmetric_int4_persistent_kernel_shapes(B, oracle, d, b):
+    bits, _ = inputs.laplace_outliers(150, d, max(1, d // 1024), 200.0, seed=9100 + d)
+    x = inputs.bf16_bits_to_f32(bits)
+    x[5] = np.abs(x[5]) + 0.5            # an all-positive row
+    x[6] = 0.0
+    bits = inputs.f32_to_bf16_bits(x)
+    check(B, oracle, inputs.Workload("asym-shapes", bits, None, b, "int4_asym", 0, 0))
