@@ -276,11 +276,11 @@ def main():
             torch.cuda.synchronize()
             return a.elapsed_time(b_) / n
 
-        for f in ("int4", "mxfp4", "fp4"):
+        for f in ("int4", "mxfp4", "fp4", "int4_asym"):
             fcode = B.FMT_BY_NAME[f]
             grp = 32 if f == "mxfp4" else 0
             o = [B.alloc_outputs(T_HEAD, D_HEAD, fcode, grp, base.device) for _ in range(RING)]
-            for bb in ((16, 32, 128, 4096) if f != "fp4" else (32,)):
+            for bb in ((16, 32, 128, 4096) if f in ("int4", "mxfp4") else (32,)):
                 ms = time_calls(lambda i: B.perq_rotate_quantize(xs[i % RING], None, bb, fcode, grp,
                                                                  out_codes=o[i % RING][0], out_scales=o[i % RING][1]))
                 by = bytes_per_token(D_HEAD, f, grp) * T_HEAD

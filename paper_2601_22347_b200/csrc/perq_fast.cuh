@@ -1,6 +1,6 @@
 // Fast rotate+quantize kernel: rows of d = G * 1024 channels.
-//   b <= 128              every scale mode (INT4 per token / per 128, MXFP4, FP4 per token), with or
-//                         without a permutation (permuted: d <= 16384);
+//   b <= 128              every scale mode (INT4 per token / per 128, MXFP4, FP4 per token, asymmetric
+//                         INT4 per token), with or without a permutation (permuted: d <= 16384);
 //   b in {256, 512, 1024} unpermuted, INT4 per token or MXFP4;
 //   b == d <= 8192        unpermuted, INT4 per token or MXFP4 (full-vector rotation).
 // Per-token scales need G <= 15 (one named barrier per group of G warps).
@@ -38,6 +38,14 @@
 // warp it stores the scale itself, with several the last one to add its value to a shared
 // accumulator does.  Warps that need the exact maximum for a tie fix-up (rare) wait for its
 // publication (a value, or the position to evaluate) on a flag, with a bounded spin.
+//
+// Asymmetric INT4 per token: the warps exchange signed maxima and minima; the warps that hold a
+// candidate for either extreme derive the exact values at once and combine them through two
+// shared accumulators; the last of them publishes the pair.  The step and the zero point (three
+// fp64 divisions) are computed 32 rows at a time, one per lane, and by any warp that needs them
+// for a fix-up.  The zero point is subtracted inside the magic constant of the rounding trick, so
+// the low nibble of the sum is the unsigned code; where rounding min / step in fp32 is a close
+// call the row waits for the exact pair before it quantises.
 //
 // Permuted rows are staged raw and gathered by every warp into its own 2 KB buffer; blocks
 // longer than 128 continue the butterfly across lane groups (shuffles) and, for b == d,

@@ -20,6 +20,8 @@ def scale_bytes_per_token(d: int, fmt: str, group: int) -> int:
         return d // 32
     if fmt == "fp4":
         return 4
+    if fmt == "int4_asym":
+        return 8           # step and zero point, fp32 each
     raise ValueError(fmt)
 
 
