@@ -169,6 +169,12 @@ __device__ __forceinline__ void ldmatrix_x4(uint32_t (&r)[4], uint32_t addr)
     asm volatile("ldmatrix.sync.aligned.m8n8.x4.shared.b16 {%0,%1,%2,%3}, [%4];"
                  : "=r"(r[0]), "=r"(r[1]), "=r"(r[2]), "=r"(r[3]) : "r"(addr));
 }
+template <int OFF>
+__device__ __forceinline__ void ldmatrix_x4_at(uint32_t (&r)[4], uint32_t addr)
+{
+    asm volatile("ldmatrix.sync.aligned.m8n8.x4.shared.b16 {%0,%1,%2,%3}, [%4+%5];"
+                 : "=r"(r[0]), "=r"(r[1]), "=r"(r[2]), "=r"(r[3]) : "r"(addr), "n"(OFF));
+}
 // c = a * b with a zero accumulator input (no registers are cleared for it)
 __device__ __forceinline__ void mma_bf16(float (&c)[4], const uint32_t (&a)[4], uint32_t b0, uint32_t b1)
 {
@@ -183,6 +189,29 @@ __device__ __forceinline__ void named_barrier(int id, int threads)
 __device__ __forceinline__ void sts_u16(uint32_t addr, uint32_t v)
 {
     asm volatile("st.shared.u16 [%0], %1;" ::"r"(addr), "h"((uint16_t)v) : "memory");
+}
+template <int OFF>
+__device__ __forceinline__ void sts_u16_at(uint32_t addr, uint32_t v)
+{
+    asm volatile("st.shared.u16 [%0+%2], %1;" ::"r"(addr), "h"((uint16_t)v), "n"(OFF) : "memory");
+}
+// Store of the 16-bit code piece of slot s (a constant once the slot loop is unrolled) at base ^ (s * 8),
+// for a base whose offset bits 3..5 lie inside XV: the slot bits in XV are XORed into the address, the
+// others are added as an immediate offset (no instruction).
+template <int XV>
+__device__ __forceinline__ void sts_code(uint32_t base, int s, uint32_t v)
+{
+    const uint32_t a = base ^ (uint32_t)((s & XV) * 8);
+    switch (s & ~XV & 7) {
+    case 0: sts_u16_at<0>(a, v); break;
+    case 1: sts_u16_at<8>(a, v); break;
+    case 2: sts_u16_at<16>(a, v); break;
+    case 3: sts_u16_at<24>(a, v); break;
+    case 4: sts_u16_at<32>(a, v); break;
+    case 5: sts_u16_at<40>(a, v); break;
+    case 6: sts_u16_at<48>(a, v); break;
+    default: sts_u16_at<56>(a, v); break;
+    }
 }
 __device__ __forceinline__ uint32_t lds_u16(uint32_t addr)
 {
@@ -758,7 +787,9 @@ __global__ void __launch_bounds__(FAST_THREADS, 1) perq_fast_kernel(FastParams p
 #pragma unroll
             for (int t = 0; t < 4; ++t) {
                 uint32_t a[4];
-                ldmatrix_x4(a, a0 ^ (uint32_t)(t << 6));
+                // (bit 7 of the lane's offset is clear: tile bit 1 is an immediate offset, tile bit 0 an XOR)
+                if (t & 2) ldmatrix_x4_at<128>(a, a0 ^ (uint32_t)((t & 1) << 6));
+                else ldmatrix_x4_at<0>(a, a0 ^ (uint32_t)((t & 1) << 6));
                 float c0[4], c1[4];
                 mma_bf16(c0, a, hb[0][0], hb[0][1]);
                 mma_bf16(c1, a, hb[1][0], hb[1][1]);
@@ -1037,7 +1068,7 @@ __global__ void __launch_bounds__(FAST_THREADS, 1) perq_fast_kernel(FastParams p
                 const uint32_t pm = ((__float_as_uint(tm1.y) * 16u + __float_as_uint(tm1.x)) * 16u + __float_as_uint(tm0.y)) * 16u
                                     + __float_as_uint(tm0.x);
                 tie_any |= (pp ^ pm) ? (1u << s) : 0u;       // (the whole sums: a code outside 0..15 carries upwards)
-                sts_u16(code_addr0 ^ (uint32_t)(s * 8), pp);
+                sts_code<(3 & ~PM)>(code_addr0, s, pp);
             }
 
             // ---- slots whose two sums differ: all four codes exactly (a carry may have reached a neighbour)
@@ -1212,7 +1243,7 @@ __global__ void __launch_bounds__(FAST_THREADS, 1) perq_fast_kernel(FastParams p
                     const uint32_t pu = cvt_e2m1x4(up0.x, up0.y, up1.x, up1.y);
                     const uint32_t pd = cvt_e2m1x4(dn0.x, dn0.y, dn1.x, dn1.y);
                     tie_any |= pu ^ pd;
-                    sts_u16(code_addr0 ^ (uint32_t)(s * 8), pu);
+                    sts_code<(3 & ~PM)>(code_addr0, s, pu);
                     continue;
                 }
                 const f32x2 tp0 = fma2(v[s][0], mul_p[k], magic2), tp1 = fma2(v[s][1], mul_p[k], magic2);
@@ -1222,7 +1253,7 @@ __global__ void __launch_bounds__(FAST_THREADS, 1) perq_fast_kernel(FastParams p
                 const uint32_t pm = ((__float_as_uint(tm1.y) * 16u + __float_as_uint(tm1.x)) * 16u + __float_as_uint(tm0.y)) * 16u
                                     + __float_as_uint(tm0.x);
                 tie_any |= pp ^ pm;          // low 16 bits: the four codes (offset by 8) under either multiplier
-                sts_u16(code_addr0 ^ (uint32_t)(s * 8), pp ^ 0x8888u);
+                sts_code<(3 & ~PM)>(code_addr0, s, pp ^ 0x8888u);
             }
             tie_any &= 0xffffu;
 
@@ -1530,7 +1561,7 @@ __global__ void __launch_bounds__(FAST_THREADS, 1) perq_fast_kernel(FastParams p
                 const uint32_t pu = cvt_e2m1x4(up0.x, up0.y, up1.x, up1.y);
                 const uint32_t pd = cvt_e2m1x4(dn0.x, dn0.y, dn1.x, dn1.y);
                 tie_any |= pu ^ pd;
-                sts_u16(code_addr0 ^ (uint32_t)(s * 8), pu);
+                sts_code<(3 & ~PM)>(code_addr0, s, pu);
             }
             if (__any_sync(0xffffffffu, tie_any != 0u)) {
                 uint32_t fm = 0u;
