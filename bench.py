@@ -151,7 +151,7 @@ def main():
     global FMT_HEAD, GROUP_HEAD
     ap = argparse.ArgumentParser()
     ap.add_argument("--gpus", type=int, default=1)
-    ap.add_argument("--steps", type=int, default=4000)
+    ap.add_argument("--steps", type=int, default=20000)
     ap.add_argument("--warmup", type=int, default=10)
     ap.add_argument("--impl", default="perq", choices=["perq", "reference"])
     ap.add_argument("--no-sweep", action="store_true", help="skip the per-variant sweep after the timed steps")
@@ -215,15 +215,21 @@ def main():
             if i % 256 == 0:
                 torch.cuda.synchronize()
     barrier()
-    ev = [torch.cuda.Event(enable_timing=True) for _ in range(args.steps + 1)]
+    # One event before the K steps and one after them (the step is a single kernel, so the average launch
+    # duration is their distance over K), plus a few in between to show the spread.  An event after every
+    # launch would itself add a few microseconds to each 40 us step.
+    marks = sorted(set([0, args.steps] + [args.steps * k // 8 for k in range(1, 8)]))
+    ev = {m: torch.cuda.Event(enable_timing=True) for m in marks}
     ev[0].record()
     for i in range(args.steps):
         step(i)
-        ev[i + 1].record()
+        if i + 1 in ev:
+            ev[i + 1].record()
     barrier()
     clocks = sampler.stop() if rank == 0 else None
-    total_ms = ev[0].elapsed_time(ev[-1])
-    per_launch_ms = [ev[i].elapsed_time(ev[i + 1]) for i in range(args.steps)]
+    total_ms = ev[0].elapsed_time(ev[args.steps])
+    local_ms = total_ms
+    per_launch_ms = [ev[a].elapsed_time(ev[b]) / (b - a) for a, b in zip(marks[:-1], marks[1:])]
     total_ms = sharding.max_over_ranks(total_ms, device="cuda")
     ms_per_step = total_ms / args.steps
     value = world * bytes_per_step / (ms_per_step * 1e-3) / 1e9
@@ -255,12 +261,13 @@ def main():
         return 0
 
     peak, peak_kind = measured_peak()
-    launch_ms = statistics.fmean(per_launch_ms)
+    launch_ms = local_ms / args.steps          # this rank's K launches between its two events
     achieved = bytes_per_step / (launch_ms * 1e-3) / 1e9
     roofline = {"bound": "hbm", "achieved": achieved, "peak": peak, "unit": "GB/s", "frac": achieved / peak,
                 "peak_kind": "of " + peak_kind, "frac_of_nominal_8TBs": achieved / NOMINAL_HBM_GBS,
                 "traffic": None if NCU_TRAFFIC_BYTES_PER_TOKEN is None else NCU_TRAFFIC_BYTES_PER_TOKEN * T_HEAD,
-                "algorithmic_bytes_per_launch": bytes_per_step, "kernel_ms": launch_ms}
+                "algorithmic_bytes_per_launch": bytes_per_step, "kernel_ms": launch_ms,
+                "kernel_ms_by_eighth_of_the_run": [round(v, 5) for v in per_launch_ms]}
 
     sweep = []
     if not args.no_sweep:
