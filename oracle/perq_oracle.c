@@ -405,6 +405,65 @@ int perq_oracle_block_l1_stats(const uint16_t *x, const int32_t *perm, int64_t T
     return 0;
 }
 
+/* ---------------------------------------------------------------- per-token diagnostics
+ * The quantities the paper plots per token (the figures on delta, on the block bound versus the
+ * block size, and on the bound versus the quantization error), before their normalisation by
+ * ||X||_inf.  With x' = gather(x, perm), blocks of b, y = x' R~ (block Hadamard) and Q the 4-bit
+ * symmetric quantiser of Sec. 3 with one step per token (s = ||y||_inf / 7, round to nearest even):
+ *
+ *   out[t][0] = ||x||_inf                       out[t][1] = ||x||_1
+ *   out[t][2] = max_j ||x'_{j}||_1              (b * max_j delta_{j} ||x'_{j}||_inf, block proposition)
+ *   out[t][3] = ||y||_inf                       out[t][4] = ||y - Q(y)||_2
+ *
+ * so that delta = out1 / (d out0) (full-vector proposition), the normalised block bound is
+ * out2 / (b out0), the outlier suppression ratio out3 / out0 and the normalised error out4 / out0.
+ * A zero row gives five zeros. */
+int perq_oracle_token_diagnostics(const uint16_t *x, const int32_t *perm, int64_t T, int32_t d,
+                                  int32_t b, double *out)
+{
+    if (!x || !out || T < 0 || d <= 0 || b < 1 || (b & (b - 1)) != 0 || d % b != 0) return 1;
+    if (fegetround() != FE_TONEAREST) return 4;
+    double *y = (double *)malloc(sizeof(double) * (size_t)(T > 0 ? T : 1) * (size_t)d);
+    if (!y) return 3;
+    int rc = perq_oracle_rotate(x, perm, T, d, b, y);
+    if (rc) { free(y); return rc; }
+#pragma omp parallel for schedule(static)
+    for (int64_t t = 0; t < T; ++t) {
+        const uint16_t *row = x + (size_t)t * d;
+        const double *yr = y + (size_t)t * d;
+        double xinf = 0.0, x1 = 0.0, bmax = 0.0;
+        for (int32_t i = 0; i < d; ++i) {
+            const double a = fabs(bf16_to_double(row[i]));
+            if (a > xinf) xinf = a;
+            x1 += a;
+        }
+        for (int32_t j = 0; j < d / b; ++j) {
+            double l1 = 0.0;
+            for (int32_t i = 0; i < b; ++i)
+                l1 += fabs(bf16_to_double(row[perm ? perm[(size_t)j * b + i] : (size_t)j * b + i]));
+            if (l1 > bmax) bmax = l1;
+        }
+        double yinf = 0.0;
+        for (int32_t i = 0; i < d; ++i)
+            if (fabs(yr[i]) > yinf) yinf = fabs(yr[i]);
+        double e2 = 0.0;
+        if (yinf > 0.0) {
+            const double s = yinf / 7.0;
+            for (int32_t i = 0; i < d; ++i) {
+                double q = nearbyint(yr[i] / s);
+                if (q > 7.0) q = 7.0;
+                if (q < -8.0) q = -8.0;
+                const double e = yr[i] - s * q;
+                e2 += e * e;
+            }
+        }
+        double *o = out + (size_t)t * 5;
+        o[0] = xinf; o[1] = x1; o[2] = bmax; o[3] = yinf; o[4] = sqrt(e2);
+    }
+    free(y);
+    return 0;
+}
+
 /* ---------------------------------------------------------------- MassDiff (Algorithm 1)
  * Visit coordinates in descending mean magnitude; put each into the not-yet-full block
  * whose running mean l1 norm is smallest; drop a block from the candidates once it holds

@@ -167,6 +167,16 @@ def block_l1_stats(x, perm, b: int):
     return cas, blm, tmx
 
 
+def token_diagnostics(x, perm, b: int) -> np.ndarray:
+    """[T, 5] fp64: ||x||_inf, ||x||_1, max block l1 (under perm), ||y||_inf, ||y - Q(y)||_2 per token."""
+    x = _x(x); perm = _perm(perm)
+    T, d = x.shape
+    out = np.empty((T, 5), np.float64)
+    _check(_load().perq_oracle_token_diagnostics(_p(x), _p(perm), C.c_int64(T), C.c_int32(d), C.c_int32(b), _p(out)),
+           "token_diagnostics")
+    return out
+
+
 def massdiff_perm(chan_abs_sum, b: int) -> np.ndarray:
     a = np.ascontiguousarray(chan_abs_sum, dtype=np.float64)
     d = a.shape[0]
