@@ -179,6 +179,31 @@ int perq_block_l1_stats_static(const void *x, const int32_t *perm, int64_t T, in
                                float *token_max_block_l1, void *stream);
 
 /*
+ * perq_token_diagnostics -- the per-token quantities the paper plots (the figures on the mass
+ * concentration delta, on the block bound versus the block size, and on the bound versus the
+ * quantization error), before their normalisation by ||X||_inf.  With x' = gather(x, perm), blocks of
+ * b channels, y = x' R~ (block Hadamard rotation) and Q the symmetric 4-bit quantiser of Sec. 3 with one
+ * step per token (s = ||y||_inf / 7, round to nearest even), row t of out holds
+ *
+ *   out[t][0] = ||x||_inf                 out[t][1] = ||x||_1
+ *   out[t][2] = max_j ||x'_{j}||_1        (= b max_j delta_{j} ||x'_{j}||_inf, proposition on block rotations)
+ *   out[t][3] = ||y||_inf                 out[t][4] = ||y - Q(y)||_2
+ *
+ * so delta = out1 / (d out0) (proposition on full-vector rotations), the normalised block bound is
+ * out2 / (b out0), the outlier suppression ratio out3 / out0, the normalised error out4 / out0.
+ *
+ *   x, perm, T, d, b   as for perq_rotate_quantize (device pointers; perm may be NULL)
+ *   out                float [T, 5], device, written in full; a zero row gives five zeros
+ *   stream             cudaStream_t (0 = default); the call only enqueues work
+ *
+ * Arithmetic is fp32 (sums in a fixed order: outputs are deterministic); the values agree with their
+ * real-arithmetic definitions to about 1e-5 relative.  The caller owns every buffer; nothing is
+ * allocated.  Errors: as perq_rotate_quantize (NULL, SHAPE, BLOCK, ALIGN, CUDA).
+ */
+int perq_token_diagnostics(const void *x, const int32_t *perm, int64_t T, int32_t d, int32_t b,
+                           float *out, void *stream);
+
+/*
  * perq_validate_perm -- checks on the device that perm[0..d) is a permutation.
  * Writes one int32 to status_dev: 0 = valid, bit 0 = an entry out of range,
  * bit 1 = a duplicate entry.  (Algorithm 1 returns such a permutation; this guards

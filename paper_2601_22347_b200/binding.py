@@ -52,6 +52,7 @@ def load() -> C.CDLL:
         lib.perq_block_l1_stats.argtypes = [vp, vp, i64, i32, i32, vp, vp, vp, vp, sz, vp]
         lib.perq_block_l1_stats_static.argtypes = [vp, vp, i64, i32, i32, vp, vp, vp, vp]
         lib.perq_block_l1_stats_workspace_bytes.argtypes = [i64, i32, i32, C.POINTER(sz)]
+        lib.perq_token_diagnostics.argtypes = [vp, vp, i64, i32, i32, vp, vp]
         lib.perq_validate_perm.argtypes = [vp, i32, vp, vp]
         lib.perq_massdiff_perm.argtypes = [vp, i32, i32, vp]
         lib.perq_device_error.argtypes = [C.POINTER(C.c_uint32)]
@@ -62,7 +63,7 @@ def load() -> C.CDLL:
         for name in ("perq_rotate_quantize", "perq_rotate_quantize_host", "perq_host_workspace_bytes",
                      "perq_out_sizes", "perq_block_l1_stats", "perq_block_l1_stats_static",
                      "perq_block_l1_stats_workspace_bytes",
-                     "perq_validate_perm", "perq_massdiff_perm"):
+                     "perq_token_diagnostics", "perq_validate_perm", "perq_massdiff_perm"):
             getattr(lib, name).restype = C.c_int
         _lib = lib
     return _lib
@@ -184,6 +185,19 @@ def perq_block_l1_stats_static(x: torch.Tensor, perm: Optional[torch.Tensor], b:
                                            _stream(stream))
     _check(rc, "perq_block_l1_stats_static")
     return chan, block, token
+
+
+def perq_token_diagnostics(x: torch.Tensor, perm: Optional[torch.Tensor], b: int, out: Optional[torch.Tensor] = None,
+                           stream=None) -> torch.Tensor:
+    """[T, 5] fp32: ||x||_inf, ||x||_1, largest block l1 under perm, ||y||_inf, ||y - Q(y)||_2 per token."""
+    assert x.is_cuda and x.dtype == torch.bfloat16 and x.dim() == 2 and x.is_contiguous()
+    assert perm is None or (perm.is_cuda and perm.dtype == torch.int32 and perm.is_contiguous())
+    T, d = x.shape
+    if out is None:
+        out = torch.empty((T, 5), dtype=torch.float32, device=x.device)
+    _check(load().perq_token_diagnostics(_ptr(x), _ptr(perm), T, d, b, _ptr(out), _stream(stream)),
+           "perq_token_diagnostics")
+    return out
 
 
 def perq_validate_perm(perm: torch.Tensor, stream=None) -> torch.Tensor:

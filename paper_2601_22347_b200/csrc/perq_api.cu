@@ -15,6 +15,7 @@
 #include "perq_generic.cuh"
 #include "perq_fast.cuh"
 #include "perq_stats.cuh"
+#include "perq_diag.cuh"
 
 namespace {
 
@@ -482,6 +483,33 @@ int perq_block_l1_stats_static(const void *x, const int32_t *perm, int64_t T, in
     }
     return perq_block_l1_stats(x, perm, T, d, b, chan_abs_sum, block_l1_mean, token_max_block_l1, scratch,
                                sizeof(g_stats_scratch), stream);
+}
+
+int perq_token_diagnostics(const void *x, const int32_t *perm, int64_t T, int32_t d, int32_t b, float *out, void *stream)
+{
+    if (!x || !out) return PERQ_ERR_NULL;
+    if (int rc = check_shape(T, d, b, PERQ_FMT_INT4, 0, nullptr)) return rc;
+    if ((reinterpret_cast<uintptr_t>(x) & 15u) != 0 || (reinterpret_cast<uintptr_t>(out) & 3u) != 0 ||
+        (perm && (reinterpret_cast<uintptr_t>(perm) & 3u) != 0))
+        return PERQ_ERR_ALIGN;
+    if (T == 0) return PERQ_OK;
+    perq::DiagParams p;
+    p.x = static_cast<const uint16_t *>(x);
+    p.perm = perm;
+    p.out = out;
+    p.T = T;
+    p.d = d;
+    p.log2b = ilog2(b);
+    p.inv_sqrt_b = (float)(1.0 / std::sqrt((double)b));
+    const perq::DiagSmem lay(d);
+    if (lay.total > kMaxSmem) return PERQ_ERR_SHAPE;
+    if (int rc = allow_smem(perq::perq_diag_kernel, lay.total)) return rc;
+    const int sms = sm_count();
+    if (sms <= 0) return PERQ_ERR_CUDA;
+    const int per_sm = (int)std::max<size_t>(1, std::min<size_t>(2048 / perq::GEN_THREADS, kMaxSmem / lay.total));
+    const long long grid = std::min<long long>(T, (long long)sms * per_sm);
+    perq::perq_diag_kernel<<<(unsigned)grid, perq::GEN_THREADS, lay.total, static_cast<cudaStream_t>(stream)>>>(p);
+    return cudaGetLastError() == cudaSuccess ? PERQ_OK : PERQ_ERR_CUDA;
 }
 
 int perq_validate_perm(const int32_t *perm, int32_t d, int32_t *status_dev, void *stream)

@@ -89,6 +89,18 @@ def test_argument_validation_happens_before_any_launch(lib):
     assert lib.perq_validate_perm(None, 16, p, None) == 1
 
 
+def test_token_diagnostics_validation(lib):
+    f = lib.perq_token_diagnostics
+    f.argtypes = [C.c_void_p, C.c_void_p, C.c_int64, C.c_int32, C.c_int32, C.c_void_p, C.c_void_p]
+    fake = C.c_void_p(0x1000)
+    assert f(None, None, 4, 2048, 32, fake, None) == 1
+    assert f(fake, None, 4, 2048, 32, None, None) == 1
+    assert f(fake, None, 4, 2050, 32, fake, None) == 2
+    assert f(fake, None, 4, 2048, 8, fake, None) == 3          # blocks of at least 16
+    assert f(C.c_void_p(0x1008), None, 4, 2048, 32, fake, None) == 6
+    assert f(fake, None, 0, 2048, 32, fake, None) == 0          # T = 0: nothing to do
+
+
 def test_host_massdiff_matches_oracle(lib, oracle):
     from paper_2601_22347_b200 import binding as B
     rng = np.random.default_rng(41)

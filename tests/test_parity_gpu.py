@@ -644,3 +644,29 @@ def test_asymmetric_int4_persistent_kernel_shapes(B, oracle, d, b):
     x[6] = 0.0
     bits = inputs.f32_to_bf16_bits(x)
     check(B, oracle, inputs.Workload("asym-shapes", bits, None, b, "int4_asym", 0, 0))
+
+
+# ------------------------------------------------------------------ per-token diagnostics
+
+@pytest.mark.parametrize("d,b,perm", [(1024, 16, False), (2048, 32, True), (4096, 128, False), (4096, 4096, False),
+                                      (8192, 32, True), (1536, 64, True), (14336, 128, False)])
+def test_token_diagnostics(B, oracle, d, b, perm):
+    """fp32 on the device against fp64 definitions: 2e-5 relative (the sums run over up to 14336 fp32 terms; a
+    code that flips at a near tie changes the error norm by less than the tie distance)."""
+    T = 70
+    bits, _ = inputs.laplace_outliers(T, d, max(1, d // 1024), 200.0, seed=9300 + d + b)
+    x = inputs.bf16_bits_to_f32(bits)
+    x[3] = 0.0                              # a zero row
+    x[4] = 0.0
+    x[4, 17] = -3.0                         # a one-hot row: no quantization error
+    bits = inputs.f32_to_bf16_bits(x)
+    p = inputs.random_perm(d, 9301) if perm else None
+    ora = oracle.token_diagnostics(bits, p, b)
+    got = B.perq_token_diagnostics(to_dev(bits), None if p is None else torch.from_numpy(p).cuda(), b)
+    torch.cuda.synchronize()
+    got = got.cpu().numpy().astype(np.float64)
+    assert np.array_equal(got[3], np.zeros(5))
+    scale = np.maximum(np.abs(ora[:, 3:4]), 1e-30)
+    assert np.allclose(got[:, :4], ora[:, :4], rtol=2e-5, atol=0)
+    assert np.all(np.abs(got[:, 4] - ora[:, 4]) <= 2e-5 * ora[:, 4] + 1e-6 * scale[:, 0])
+    assert got[4, 4] <= 1e-6 * got[4, 3]
