@@ -330,7 +330,14 @@ def main():
         time_workload("cfg2", w2.x, w2.perm, 32, "int4", 128)
         chan, _, _ = B.perq_block_l1_stats(x3[0], None, 32, want=("chan",), workspace=wsb)
         torch.cuda.synchronize()
-        time_workload("cfg3 (MassDiff permutation)", w3.x, B.perq_massdiff_perm(chan.cpu().numpy(), 32), 32, "mxfp4", 32)
+        # Algorithm 1 on the device (sequential greedy: a latency figure, not a bandwidth one), checked against the host one
+        pws = torch.empty(8192 * 4, dtype=torch.uint8, device="cuda")
+        pdev = torch.empty(8192, dtype=torch.int32, device="cuda")
+        ms = time_calls(lambda i: B.perq_massdiff_perm_device(chan, 32, perm=pdev, workspace=pws), n=5, warm=1)
+        phost = B.perq_massdiff_perm(chan.cpu().numpy(), 32)
+        sweep.append({"call": "perq_massdiff_perm_device", "d": 8192, "b": 32, "ms": ms,
+                      "equals_host_permutation": bool(np.array_equal(pdev.cpu().numpy(), phost))})
+        time_workload("cfg3 (MassDiff permutation)", w3.x, phost, 32, "mxfp4", 32)
         del x3
         for T5 in (1, 16, 128, 1024, 16384):
             w5 = inputs.config5(T=T5, b=32)

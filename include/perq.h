@@ -225,6 +225,23 @@ int perq_validate_perm(const int32_t *perm, int32_t d, int32_t *status_dev, void
 int perq_massdiff_perm(const float *chan_abs_sum_host, int32_t d, int32_t b, int32_t *perm_host);
 
 /*
+ * perq_massdiff_perm_device -- Algorithm 1 (MassDiff) on the device: the same permutation as
+ * perq_massdiff_perm, entry for entry, from a device array, so that a calibration pass (statistic ->
+ * permutation -> permuted rotate+quantize) needs no copy to the host.
+ *
+ *   chan_abs_sum     float [d], device (e.g. the output of perq_block_l1_stats); finite, non-negative
+ *   perm             int32 [d], device, written in full
+ *   workspace        device, at least d * 4 bytes (the channels in visiting order); caller-owned
+ *   stream           cudaStream_t (0 = default); two kernels are enqueued, nothing is synchronised
+ *
+ * b >= 1, d % b == 0, d <= PERQ_MAX_D and at most 4096 blocks (d / b).  The greedy is sequential in the
+ * channels (one warp scans the open blocks d times): about 1-3 ms for d = 8192 ... 14336.
+ * Errors: NULL, SHAPE, BLOCK (also: too many blocks), WORKSPACE, ALIGN, CUDA.
+ */
+int perq_massdiff_perm_device(const float *chan_abs_sum, int32_t d, int32_t b, int32_t *perm,
+                              void *workspace, size_t workspace_bytes, void *stream);
+
+/*
  * perq_device_error -- reads (synchronously, cudaMemcpyFromSymbol) the library's device-side
  * error word on the current device into *flags_host.  0 = no error.  Bit 0 is set when a
  * bounded wait inside a kernel ran out (an asynchronous copy that never completed); the

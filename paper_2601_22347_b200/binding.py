@@ -55,6 +55,7 @@ def load() -> C.CDLL:
         lib.perq_token_diagnostics.argtypes = [vp, vp, i64, i32, i32, vp, vp]
         lib.perq_validate_perm.argtypes = [vp, i32, vp, vp]
         lib.perq_massdiff_perm.argtypes = [vp, i32, i32, vp]
+        lib.perq_massdiff_perm_device.argtypes = [vp, i32, i32, vp, vp, sz, vp]
         lib.perq_device_error.argtypes = [C.POINTER(C.c_uint32)]
         lib.perq_device_error.restype = C.c_int
         lib.perq_status_string.argtypes = [C.c_int]
@@ -63,7 +64,7 @@ def load() -> C.CDLL:
         for name in ("perq_rotate_quantize", "perq_rotate_quantize_host", "perq_host_workspace_bytes",
                      "perq_out_sizes", "perq_block_l1_stats", "perq_block_l1_stats_static",
                      "perq_block_l1_stats_workspace_bytes",
-                     "perq_token_diagnostics", "perq_validate_perm", "perq_massdiff_perm"):
+                     "perq_token_diagnostics", "perq_validate_perm", "perq_massdiff_perm", "perq_massdiff_perm_device"):
             getattr(lib, name).restype = C.c_int
         _lib = lib
     return _lib
@@ -213,6 +214,21 @@ def perq_device_error() -> int:
     v = C.c_uint32(0)
     _check(load().perq_device_error(C.byref(v)), "perq_device_error")
     return int(v.value)
+
+
+def perq_massdiff_perm_device(chan_abs_sum: torch.Tensor, b: int, perm: Optional[torch.Tensor] = None,
+                              workspace: Optional[torch.Tensor] = None, stream=None) -> torch.Tensor:
+    """chan_abs_sum: fp32 CUDA tensor [d]; returns the int32 CUDA permutation [d] (nothing is synchronised)."""
+    assert chan_abs_sum.is_cuda and chan_abs_sum.dtype == torch.float32 and chan_abs_sum.is_contiguous()
+    d = chan_abs_sum.numel()
+    if perm is None:
+        perm = torch.empty(d, dtype=torch.int32, device=chan_abs_sum.device)
+    if workspace is None:
+        workspace = torch.empty(d * 4, dtype=torch.uint8, device=chan_abs_sum.device)
+    _check(load().perq_massdiff_perm_device(_ptr(chan_abs_sum), d, b, _ptr(perm), _ptr(workspace),
+                                            workspace.numel() * workspace.element_size(), _stream(stream)),
+           "perq_massdiff_perm_device")
+    return perm
 
 
 def perq_massdiff_perm(chan_abs_sum_host: np.ndarray, b: int) -> np.ndarray:

@@ -16,6 +16,7 @@
 #include "perq_fast.cuh"
 #include "perq_stats.cuh"
 #include "perq_diag.cuh"
+#include "perq_massdiff.cuh"
 
 namespace {
 
@@ -528,6 +529,24 @@ int perq_device_error(uint32_t *flags_host)
     if (cudaMemcpyFromSymbol(&v, perq::g_perq_device_error, sizeof v) != cudaSuccess) return PERQ_ERR_CUDA;
     *flags_host = v;
     return PERQ_OK;
+}
+
+int perq_massdiff_perm_device(const float *chan_abs_sum, int32_t d, int32_t b, int32_t *perm, void *workspace,
+                              size_t workspace_bytes, void *stream)
+{
+    if (!chan_abs_sum || !perm) return PERQ_ERR_NULL;
+    if (d <= 0 || d > PERQ_MAX_D) return PERQ_ERR_SHAPE;
+    if (b < 1 || d % b != 0 || d / b > perq::MD_MAX_BLOCKS) return PERQ_ERR_BLOCK;
+    if (!workspace || workspace_bytes < (size_t)d * sizeof(int32_t)) return PERQ_ERR_WORKSPACE;
+    if ((reinterpret_cast<uintptr_t>(chan_abs_sum) & 3u) != 0 || (reinterpret_cast<uintptr_t>(perm) & 3u) != 0 ||
+        (reinterpret_cast<uintptr_t>(workspace) & 3u) != 0)
+        return PERQ_ERR_ALIGN;
+    cudaStream_t st = static_cast<cudaStream_t>(stream);
+    int32_t *order = static_cast<int32_t *>(workspace);
+    perq::perq_massdiff_rank_kernel<<<(d + perq::MD_THREADS - 1) / perq::MD_THREADS, perq::MD_THREADS, 0, st>>>(chan_abs_sum, d, order);
+    if (cudaGetLastError() != cudaSuccess) return PERQ_ERR_CUDA;
+    perq::perq_massdiff_greedy_kernel<<<1, 32, 0, st>>>(chan_abs_sum, order, d, b, perm);
+    return cudaGetLastError() == cudaSuccess ? PERQ_OK : PERQ_ERR_CUDA;
 }
 
 int perq_massdiff_perm(const float *chan_abs_sum_host, int32_t d, int32_t b, int32_t *perm_host)

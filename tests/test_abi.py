@@ -101,6 +101,18 @@ def test_token_diagnostics_validation(lib):
     assert f(fake, None, 0, 2048, 32, fake, None) == 0          # T = 0: nothing to do
 
 
+def test_device_massdiff_validation(lib):
+    f = lib.perq_massdiff_perm_device
+    f.argtypes = [C.c_void_p, C.c_int32, C.c_int32, C.c_void_p, C.c_void_p, C.c_size_t, C.c_void_p]
+    fake = C.c_void_p(0x1000)
+    assert f(None, 256, 16, fake, fake, 1024, None) == 1
+    assert f(fake, 0, 16, fake, fake, 1024, None) == 2
+    assert f(fake, 256, 24, fake, fake, 1024, None) == 3
+    assert f(fake, 8192, 1, fake, fake, 32768, None) == 3       # more than 4096 blocks
+    assert f(fake, 256, 16, fake, fake, 1023, None) == 9         # workspace too small
+    assert f(fake, 256, 16, fake, None, 0, None) == 9
+
+
 def test_host_massdiff_matches_oracle(lib, oracle):
     from paper_2601_22347_b200 import binding as B
     rng = np.random.default_rng(41)

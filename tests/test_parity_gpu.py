@@ -670,3 +670,34 @@ def test_token_diagnostics(B, oracle, d, b, perm):
     assert np.allclose(got[:, :4], ora[:, :4], rtol=2e-5, atol=0)
     assert np.all(np.abs(got[:, 4] - ora[:, 4]) <= 2e-5 * ora[:, 4] + 1e-6 * scale[:, 0])
     assert got[4, 4] <= 1e-6 * got[4, 3]
+
+
+# ------------------------------------------------------------------ Algorithm 1 on the device
+
+@pytest.mark.parametrize("d,b", [(256, 16), (2048, 32), (8192, 32), (4096, 4096), (14336, 128), (1000, 8), (96, 1)])
+def test_massdiff_on_the_device_matches_the_oracle(B, oracle, d, b):
+    rng = np.random.default_rng(4100 + d + b)
+    a = (rng.exponential(size=d) * np.where(rng.random(d) < 0.05, 40.0, 1.0)).astype(np.float32)
+    a[rng.integers(0, d, 16)] = a[0]                     # equal masses: the index decides
+    a[rng.integers(0, d, 4)] = 0.0
+    ref = oracle.massdiff_perm(a.astype(np.float64), b)
+    got = B.perq_massdiff_perm_device(torch.from_numpy(a).cuda(), b)
+    torch.cuda.synchronize()
+    assert np.array_equal(got.cpu().numpy(), ref)
+
+
+def test_calibration_pass_stays_on_the_device(B, oracle):
+    """statistic -> permutation -> permuted rotate+quantize without a host copy, against the oracle's chain."""
+    w = inputs.config3(T=96)
+    x = to_dev(w.x)
+    chan, _, _ = B.perq_block_l1_stats(x, None, 32, want=("chan",))
+    perm = B.perq_massdiff_perm_device(chan, 32)
+    codes, scales = B.perq_rotate_quantize(x, perm, 32, FMT["mxfp4"], 32)
+    torch.cuda.synchronize()
+    cas, _, _ = oracle.block_l1_stats(w.x, None, 32)
+    # the device sums are fp32: feed the oracle's greedy the same fp32 masses, then compare everything after it
+    assert np.allclose(chan.cpu().numpy(), cas, rtol=1e-5)
+    ref_perm = oracle.massdiff_perm(chan.cpu().numpy().astype(np.float64), 32)
+    assert np.array_equal(perm.cpu().numpy(), ref_perm)
+    ora = oracle.rotate_quantize(w.x, ref_perm, 32, FMT["mxfp4"], 32, want_pre=True)
+    compare_quantized("mxfp4", codes.cpu().numpy(), scales.cpu().numpy(), ora)
