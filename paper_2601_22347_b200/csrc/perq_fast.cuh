@@ -39,13 +39,15 @@
 // accumulator does.  Warps that need the exact maximum for a tie fix-up (rare) wait for its
 // publication (a value, or the position to evaluate) on a flag, with a bounded spin.
 //
-// Asymmetric INT4 per token: the warps exchange signed maxima and minima; the warps that hold a
-// candidate for either extreme derive the exact values at once and combine them through two
-// shared accumulators; the last of them publishes the pair.  The step and the zero point (three
-// fp64 divisions) are computed 32 rows at a time, one per lane, and by any warp that needs them
-// for a fix-up.  The zero point is subtracted inside the magic constant of the rounding trick, so
-// the low nibble of the sum is the unsigned code; where rounding min / step in fp32 is a close
-// call the row waits for the exact pair before it quantises.
+// Asymmetric INT4 per token: the warps exchange signed maxima and minima.  Normally one warp holds the
+// candidates for the row maximum and one (maybe the same) those for the minimum, each in one slot: the
+// two positions are published and recorded, and the step and the zero point (exact extremes from global
+// memory, three fp64 divisions) are derived 32 rows at a time, one per lane.  A side with several slots
+// publishes its exact value instead of a position; a row with several candidate warps on a side combines
+// exact values through two shared accumulators.  A warp that needs (s, z) for a fix-up evaluates the
+// published pair itself.  The zero point is subtracted inside the magic constant of the rounding trick,
+// so the low nibble of the sum is the unsigned code; where rounding min / step in fp32 is a close call
+// the row waits for the exact pair before it quantises.
 //
 // Permuted rows are staged raw and gathered by every warp into its own 2 KB buffer; blocks
 // longer than 128 continue the butterfly across lane groups (shuffles) and, for b == d,
@@ -598,15 +600,75 @@ __device__ __forceinline__ void asym_step_zero(unsigned long long khi, unsigned 
     z64 = (s64 == 0.0) ? 0.0 : rint(mny / s64);
 }
 
-// Deferred (s, z) of up to 32 rows, one per lane: the divisions above cost a few hundred instructions,
-// which a lane per row amortises over the warp.
-__device__ __forceinline__ void serve_asym_requests(const FastParams &p, const unsigned long long *khi, const unsigned long long *klo,
+// Signed maximum and minimum of the four outputs of one slot (position pos in the row, a multiple of 4),
+// re-derived by one thread from the row in global memory (the signed counterpart of exact_slot_max_global).
+template <int LOG2B, bool PERM>
+__device__ __forceinline__ void exact_slot_extremes_global(const uint16_t *row, uint32_t pos, const int32_t *perm, int d,
+                                                           double &mx, double &mn)
+{
+    constexpr int B = 1 << LOG2B;
+    const uint32_t blk = (pos >> LOG2B) << LOG2B;
+    const uint32_t i0 = pos - blk;
+    const uint4 *src = reinterpret_cast<const uint4 *>(row + blk);
+    double S[4] = {0.0, 0.0, 0.0, 0.0};
+#pragma unroll(B <= 128 ? B / 8 : 2)
+    for (int c = 0; c < B / 8; ++c) {
+        uint32_t w[4];
+        if (PERM) {
+#pragma unroll
+            for (int e = 0; e < 4; ++e) {
+                const int s0 = min(max(__ldg(perm + blk + 8 * c + 2 * e), 0), d - 1);
+                const int s1 = min(max(__ldg(perm + blk + 8 * c + 2 * e + 1), 0), d - 1);
+                w[e] = (uint32_t)__ldg(row + s0) | ((uint32_t)__ldg(row + s1) << 16);
+            }
+        } else {
+            const uint4 w4 = __ldg(src + c);
+            w[0] = w4.x; w[1] = w4.y; w[2] = w4.z; w[3] = w4.w;
+        }
+#pragma unroll
+        for (int h = 0; h < 2; ++h) {
+            const bool neg = __popc(i0 & (uint32_t)(8 * c + 4 * h)) & 1;
+#pragma unroll
+            for (int e = 0; e < 4; ++e) {
+                const uint32_t word = w[2 * h + (e >> 1)];
+                const double val = (double)__uint_as_float((e & 1) ? (word & 0xffff0000u) : (word << 16));
+                S[e] += neg ? -val : val;
+            }
+        }
+    }
+    const double a0 = S[0] + S[1], a1 = S[0] - S[1], a2 = S[2] + S[3], a3 = S[2] - S[3];
+    const double o0 = a0 + a2, o1 = a1 + a3, o2 = a0 - a2, o3 = a1 - a3;
+    mx = fmax(fmax(o0, o1), fmax(o2, o3));
+    mn = fmin(fmin(o0, o1), fmin(o2, o3));
+}
+
+// An entry of an asymmetric record is the order key of an exact extreme (always >= 2^52) or, below 2^32,
+// the position in the row of the one slot that holds it.
+__device__ __forceinline__ bool asym_entry_is_position(unsigned long long e) { return e < (1ull << 32); }
+
+// Deferred (s, z) of up to 32 rows, one per lane: positions are evaluated from global memory, and the three
+// divisions cost a few hundred instructions, which a lane per row amortises over the warp.
+template <int LOG2B, bool PERM>
+__device__ __forceinline__ void serve_asym_requests(const FastParams &p, const unsigned long long *ehi, const unsigned long long *elo,
                                                     const uint32_t *rows, uint32_t n, int lane)
 {
     __syncwarp();
     if ((uint32_t)lane < n) {
+        unsigned long long khi = ehi[lane], klo = elo[lane];
+        const uint16_t *row = p.x + (size_t)rows[lane] * p.d;
+        if (asym_entry_is_position(khi)) {
+            double mx, mn;
+            exact_slot_extremes_global<LOG2B, PERM>(row, (uint32_t)khi, p.perm, p.d, mx, mn);
+            if (asym_entry_is_position(klo) && klo == khi) klo = order_key(mn);
+            khi = order_key(mx);
+        }
+        if (asym_entry_is_position(klo)) {
+            double mx, mn;
+            exact_slot_extremes_global<LOG2B, PERM>(row, (uint32_t)klo, p.perm, p.d, mx, mn);
+            klo = order_key(mn);
+        }
         double s64, z64;
-        asym_step_zero(khi[lane], klo[lane], p.sqrt_b, s64, z64);
+        asym_step_zero(khi, klo, p.sqrt_b, s64, z64);
         float2 *dst = reinterpret_cast<float2 *>(p.out_scales) + rows[lane];
         *dst = make_float2((float)s64, (float)z64);
     }
@@ -950,8 +1012,9 @@ __global__ void __launch_bounds__(FAST_THREADS, 1) perq_fast_kernel(FastParams p
             const bool live = hi_row > lo_row;               // else: every rotated value is the same (a zero row)
             const float e_abs = 2.0f * err_rel * amax + amax * 2.4e-7f;
             const float thr_hi = hi_row - e_abs, thr_lo = lo_row + e_abs;
-            const unsigned candw = (G > 1) ? __ballot_sync(0xffffffffu, live && (lane < G) && (hm >= thr_hi || lm <= thr_lo))
-                                           : (live ? 1u : 0u);
+            const unsigned cand_hi = (G > 1) ? __ballot_sync(0xffffffffu, live && (lane < G) && hm >= thr_hi) : (live ? 1u : 0u);
+            const unsigned cand_lo = (G > 1) ? __ballot_sync(0xffffffffu, live && (lane < G) && lm <= thr_lo) : (live ? 1u : 0u);
+            const unsigned candw = cand_hi | cand_lo;
             const bool is_cand = (candw >> w_in_g) & 1u;
             const int ncand = __popc(candw);
             if (!live && leader) {
@@ -959,61 +1022,104 @@ __global__ void __launch_bounds__(FAST_THREADS, 1) perq_fast_kernel(FastParams p
                 reinterpret_cast<float *>(p.out_scales)[2 * (size_t)unit + 1] = 0.0f;
             }
 
-            // ---- the exact extremes, by the warps that hold candidates; the last of them derives (s, z)
-            if (is_cand) {
+            // ---- the exact extremes.  Common case: one warp holds the row's candidates for the maximum and one
+            // (maybe the same) those for the minimum, each in one slot: the positions are published and
+            // recorded, and (s, z) are derived later, 32 rows at a time.  A side with several slots publishes
+            // its exact value instead; a row with several candidate warps on a side combines exact values of
+            // all of them through the shared accumulators.
+            const bool one_each = __popc(cand_hi) == 1 && __popc(cand_lo) == 1;
+            // an entry for one side from this warp: the position of its one candidate slot, or the exact key
+            auto side_entry = [&](bool hi_side, bool may_be_position) -> unsigned long long {
                 uint32_t slot_mask = 0u;
 #pragma unroll
                 for (int s = 0; s < 8; ++s) {
                     const int k = s & 3 & PM;
-                    const float hs = fmaxf(fmaxf(v[s][0].x, v[s][0].y), fmaxf(v[s][1].x, v[s][1].y));
-                    const float ls = fminf(fminf(v[s][0].x, v[s][0].y), fminf(v[s][1].x, v[s][1].y));
                     const bool pos = sgn[k] > 0.0f;
-                    const float th = pos ? hs : -ls, tl = pos ? ls : -hs;
-                    slot_mask |= (th >= thr_hi || tl <= thr_lo) ? (1u << s) : 0u;
+                    float t;                                  // the slot's true maximum (hi side) or minimum
+                    if (hi_side == pos) {
+                        const float hs = fmaxf(fmaxf(v[s][0].x, v[s][0].y), fmaxf(v[s][1].x, v[s][1].y));
+                        t = hi_side ? hs : -hs;
+                    } else {
+                        const float ls = fminf(fminf(v[s][0].x, v[s][0].y), fminf(v[s][1].x, v[s][1].y));
+                        t = hi_side ? -ls : ls;
+                    }
+                    slot_mask |= (hi_side ? (t >= thr_hi) : (t <= thr_lo)) ? (1u << s) : 0u;
                 }
-                double bhi = -1.7976931348623157e308, blo = 1.7976931348623157e308;
                 unsigned cw = __ballot_sync(0xffffffffu, slot_mask != 0u);
+                const int src0 = (cw != 0u) ? __ffs(cw) - 1 : 0;
+                const uint32_t sm0 = __shfl_sync(0xffffffffu, slot_mask, src0);
+                if (may_be_position && cw != 0u && (cw & (cw - 1)) == 0u && (sm0 & (sm0 - 1)) == 0u) {
+                    const int sl = __ffs(sm0) - 1, lg = src0 >> 2;
+                    const int pch = lg * 8 + (sl ^ ((lg & 3) & ~PM));
+                    return (unsigned long long)(uint32_t)(w_in_g * SEG_ELEMS + pch * 16 + 4 * (src0 & 3));
+                }
+                double best = hi_side ? -1.7976931348623157e308 : 1.7976931348623157e308;
                 while (cw) {
                     const int src = __ffs(cw) - 1;
                     cw &= cw - 1;
                     uint32_t sm = __shfl_sync(0xffffffffu, slot_mask, src);
-                    const int sg = src >> 2;
+                    const int lg = src >> 2;
                     while (sm) {
                         const int sl = __ffs(sm) - 1;
                         sm &= sm - 1;
-                        const int pch = sg * 8 + (sl ^ ((sg & 3) & ~PM));      // chunk position in the segment
+                        const int pch = lg * 8 + (sl ^ ((lg & 3) & ~PM));      // chunk position in the segment
                         const int blk_elem = (pch >> CB_) << LOG2B;
                         const int i0 = pch * 16 - blk_elem + 4 * (src & 3);
                         const double val = exact_coord4<B>(seg + blk_elem, i0, lane);   // outputs i0 .. i0+3, one per lane & 3
-                        bhi = fmax(bhi, val);
-                        blo = fmin(blo, val);
+                        best = hi_side ? fmax(best, val) : fmin(best, val);
                     }
                 }
-                const unsigned long long khi = warp_max_u64(order_key(bhi));
-                const unsigned long long klo = ~warp_max_u64(~order_key(blo));
+                return hi_side ? warp_max_u64(order_key(best)) : ~warp_max_u64(~order_key(best));
+            };
+            if (is_cand) {
                 uint32_t last = 0u;
-                if (lane == 0) {
-                    atomicMax(&wacc[pidx], khi);
-                    atomicMin(&wacc2[pidx], klo);
-                    __threadfence_block();
-                    if (atomicAdd(&wcnt[pidx], 1u) == (uint32_t)(ncand - 1)) {      // last candidate warp of the row
-                        const unsigned long long fhi = atomicExch(&wacc[pidx], 0ull);
-                        const unsigned long long flo = atomicExch(&wacc2[pidx], ~0ull);
-                        wcnt[pidx] = 0u;
-                        // the keys are published now; (s, z) go to global memory later, 32 rows at a time
-                        wpub[pidx] = fhi;
-                        wpub2[pidx] = flo;
+                unsigned long long rec_hi = 0ull, rec_lo = 0ull;
+                const bool mine_hi = (cand_hi >> w_in_g) & 1u, mine_lo = (cand_lo >> w_in_g) & 1u;
+                if (one_each) {
+                    unsigned long long e_hi = 0ull, e_lo = 0ull;
+                    if (mine_hi) e_hi = side_entry(true, true);
+                    if (mine_lo) e_lo = side_entry(false, true);
+                    if (lane == 0) {
+                        if (mine_hi) wpub[pidx] = e_hi;
+                        if (mine_lo) wpub2[pidx] = e_lo;
                         __threadfence_block();
-                        *reinterpret_cast<volatile uint32_t *>(&wflag[pidx]) = it + 1u;
-                        wreq[nreq] = fhi;
-                        wreq2[nreq] = flo;
-                        wrequ[nreq] = unit;
-                        last = 1u;
+                        const uint32_t publishers = (cand_hi == cand_lo) ? 1u : 2u;
+                        if (atomicAdd(&wcnt[pidx], 1u) == publishers - 1u) {         // both sides are published
+                            wcnt[pidx] = 0u;
+                            __threadfence_block();
+                            rec_hi = *reinterpret_cast<volatile unsigned long long *>(&wpub[pidx]);
+                            rec_lo = *reinterpret_cast<volatile unsigned long long *>(&wpub2[pidx]);
+                            *reinterpret_cast<volatile uint32_t *>(&wflag[pidx]) = it + 1u;
+                            last = 1u;
+                        }
                     }
+                } else {
+                    const unsigned long long khi = mine_hi ? side_entry(true, false) : 0ull;
+                    const unsigned long long klo = mine_lo ? side_entry(false, false) : ~0ull;
+                    if (lane == 0) {
+                        atomicMax(&wacc[pidx], khi);
+                        atomicMin(&wacc2[pidx], klo);
+                        __threadfence_block();
+                        if (atomicAdd(&wcnt[pidx], 1u) == (uint32_t)(ncand - 1)) {      // last candidate warp of the row
+                            rec_hi = atomicExch(&wacc[pidx], 0ull);
+                            rec_lo = atomicExch(&wacc2[pidx], ~0ull);
+                            wcnt[pidx] = 0u;
+                            wpub[pidx] = rec_hi;
+                            wpub2[pidx] = rec_lo;
+                            __threadfence_block();
+                            *reinterpret_cast<volatile uint32_t *>(&wflag[pidx]) = it + 1u;
+                            last = 1u;
+                        }
+                    }
+                }
+                if (lane == 0 && last) {
+                    wreq[nreq] = rec_hi;
+                    wreq2[nreq] = rec_lo;
+                    wrequ[nreq] = unit;
                 }
                 nreq += __shfl_sync(0xffffffffu, last, 0);
                 if (nreq == 32u) {
-                    serve_asym_requests(p, wreq, wreq2, wrequ, nreq, lane);
+                    serve_asym_requests<LOG2B, PERM>(p, wreq, wreq2, wrequ, nreq, lane);
                     nreq = 0;
                 }
             }
@@ -1033,8 +1139,21 @@ __global__ void __launch_bounds__(FAST_THREADS, 1) perq_fast_kernel(FastParams p
                     if (++spin >= WAIT_SPIN_LIMIT) return false;
                 }
                 __threadfence_block();
-                asym_step_zero(*reinterpret_cast<volatile unsigned long long *>(&wpub[pidx]),
-                               *reinterpret_cast<volatile unsigned long long *>(&wpub2[pidx]), p.sqrt_b, s_ex, z_ex);
+                unsigned long long khi = *reinterpret_cast<volatile unsigned long long *>(&wpub[pidx]);
+                unsigned long long klo = *reinterpret_cast<volatile unsigned long long *>(&wpub2[pidx]);
+                // a position: the slot's four outputs from the staged row, lane l holding output (l & 3)
+                auto slot_values = [&](uint32_t pos) -> double {
+                    const uint32_t blk = (pos >> LOG2B) << LOG2B;
+                    return PERM ? exact_coord4_perm<B>(raw_row, ptab + blk, (int)(pos - blk), lane)
+                                : exact_coord4<B>(raw_row + blk, (int)(pos - blk), lane);
+                };
+                if (asym_entry_is_position(khi)) {
+                    const double val = slot_values((uint32_t)khi);
+                    if (asym_entry_is_position(klo) && klo == khi) klo = ~warp_max_u64(~order_key(val));
+                    khi = warp_max_u64(order_key(val));
+                }
+                if (asym_entry_is_position(klo)) klo = ~warp_max_u64(~order_key(slot_values((uint32_t)klo)));
+                asym_step_zero(khi, klo, p.sqrt_b, s_ex, z_ex);
                 have_exact = true;
                 return true;
             };
@@ -1614,7 +1733,7 @@ __global__ void __launch_bounds__(FAST_THREADS, 1) perq_fast_kernel(FastParams p
         }
     }
     if (MODE == MODE_ASYM) {
-        if (nreq > 0u) serve_asym_requests(p, wreq, wreq2, wrequ, nreq, lane);
+        if (nreq > 0u) serve_asym_requests<LOG2B, PERM>(p, wreq, wreq2, wrequ, nreq, lane);
     } else if (MODE != MODE_MX && nreq > 0u) {
         serve_scale_requests<LOG2BF, MODE, PERM>(p, wreq, nreq, lane);
     }
