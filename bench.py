@@ -322,10 +322,27 @@ def main():
                                                              out_codes=orr[i % ring][0], out_scales=orr[i % ring][1]))
             by = bytes_per_token(d, f, grp) * T
             gbs = by / (ms * 1e-3) / 1e9
-            sweep.append({"call": "perq_rotate_quantize", "workload": name, "T": T, "d": d, "b": b, "fmt": f, "group": grp,
-                          "perm": perm is not None, "us": ms * 1e3, "GB/s": gbs, "frac_of_" + peak_kind: gbs / peak,
-                          "Mtokens/s": T / ms / 1e3})
+            row = {"call": "perq_rotate_quantize", "workload": name, "T": T, "d": d, "b": b, "fmt": f, "group": grp,
+                   "perm": perm is not None, "us": ms * 1e3, "GB/s": gbs, "frac_of_" + peak_kind: gbs / peak,
+                   "Mtokens/s": T / ms / 1e3}
+            if by < 64e6:
+                # small calls are bound by the host's launch rate when issued one by one from Python: the same
+                # calls replayed from a CUDA graph (50 per graph) give the device-side time per call
+                side = torch.cuda.Stream()
+                side.wait_stream(torch.cuda.current_stream())
+                graph = torch.cuda.CUDAGraph()
+                with torch.cuda.graph(graph, stream=side):
+                    for i in range(50):
+                        B.perq_rotate_quantize(xr[i % ring], pd, b, fcode, grp, out_codes=orr[i % ring][0],
+                                               out_scales=orr[i % ring][1], stream=torch.cuda.current_stream())
+                gms = time_calls(lambda i: graph.replay(), n=10, warm=2) / 50
+                row["us_graph_replay"] = gms * 1e3
+                row["GB/s_graph_replay"] = by / (gms * 1e-3) / 1e9
+                del graph
+            sweep.append(row)
 
+        w1 = inputs.config1()
+        time_workload("cfg1", w1.x, None, 16, "int4", 0)
         w2 = inputs.config2(T=4096, b=32)
         time_workload("cfg2", w2.x, w2.perm, 32, "int4", 128)
         chan, _, _ = B.perq_block_l1_stats(x3[0], None, 32, want=("chan",), workspace=wsb)

@@ -3,6 +3,7 @@
 #include "perq.h"
 
 #include <algorithm>
+#include <map>
 #include <cmath>
 #include <cstdint>
 #include <mutex>
@@ -64,15 +65,27 @@ int sm_count()
     return cached;
 }
 
+// Opt-in to more than 48 KB of dynamic shared memory.  The attribute belongs to (kernel, device): it is set
+// the first time and whenever a launch needs more than was set before (the call costs a microsecond or two,
+// which matters for the small launches).
+std::mutex g_smem_attr_mutex;
+std::map<std::pair<const void *, int>, size_t> g_smem_attr_set;
+
 template <typename K>
 int allow_smem(K kernel, size_t bytes)
 {
-    if (bytes > 48 * 1024) {
-        if (cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)bytes) != cudaSuccess) {
-            (void)cudaGetLastError();
-            return PERQ_ERR_CUDA;
-        }
+    if (bytes <= 48 * 1024) return PERQ_OK;
+    int dev = 0;
+    if (cudaGetDevice(&dev) != cudaSuccess) return PERQ_ERR_CUDA;
+    const void *func = reinterpret_cast<const void *>(kernel);
+    std::lock_guard<std::mutex> lock(g_smem_attr_mutex);
+    size_t &have = g_smem_attr_set[std::make_pair(func, dev)];
+    if (have >= bytes) return PERQ_OK;
+    if (cudaFuncSetAttribute(func, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)bytes) != cudaSuccess) {
+        (void)cudaGetLastError();
+        return PERQ_ERR_CUDA;
     }
+    have = bytes;
     return PERQ_OK;
 }
 

@@ -742,7 +742,18 @@ __global__ void __launch_bounds__(FAST_THREADS, 1) perq_fast_kernel(FastParams p
     }
     if (PERM) {     // the permutation as byte offsets into a staged row; out-of-range entries are clamped
         uint16_t *pt = reinterpret_cast<uint16_t *>(fsmem + FastSmem::perm_tab);
-        for (int i = tid; i < p.d; i += FAST_THREADS) pt[i] = (uint16_t)(2 * min(max(__ldg(p.perm + i), 0), p.d - 1));
+        if ((reinterpret_cast<uintptr_t>(p.perm) & 15u) == 0) {      // four entries per load, all loads independent
+            const int4 *p4 = reinterpret_cast<const int4 *>(p.perm);
+#pragma unroll 8
+            for (int i = tid; i < p.d / 4; i += FAST_THREADS) {
+                const int4 e = __ldg(p4 + i);
+                const uint32_t o0 = (uint32_t)(2 * min(max(e.x, 0), p.d - 1)), o1 = (uint32_t)(2 * min(max(e.y, 0), p.d - 1));
+                const uint32_t o2 = (uint32_t)(2 * min(max(e.z, 0), p.d - 1)), o3 = (uint32_t)(2 * min(max(e.w, 0), p.d - 1));
+                reinterpret_cast<uint2 *>(pt)[i] = make_uint2(o0 | (o1 << 16), o2 | (o3 << 16));
+            }
+        } else {
+            for (int i = tid; i < p.d; i += FAST_THREADS) pt[i] = (uint16_t)(2 * min(max(__ldg(p.perm + i), 0), p.d - 1));
+        }
     }
     if (tid < 2 * FAST_WARPS) { wacc[tid] = 0ull; wacc2[tid] = ~0ull; wcnt[tid] = 0u; wflag[tid] = 0u; }
     if (tid == 0) asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
