@@ -3,6 +3,7 @@
 #include "perq.h"
 
 #include <algorithm>
+#include <atomic>
 #include <map>
 #include <cmath>
 #include <cstdint>
@@ -55,14 +56,15 @@ int check_shape(int64_t T, int32_t d, int32_t b, int32_t fmt, int32_t group, int
 
 int sm_count()
 {
-    static int cached = 0;
-    if (cached == 0) {
-        int dev = 0, n = 0;
-        if (cudaGetDevice(&dev) != cudaSuccess) return 0;
-        if (cudaDeviceGetAttribute(&n, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess) return 0;
-        cached = n;
-    }
-    return cached;
+    static std::atomic<int> cached[64];          // per device ordinal; 0 = not asked yet
+    int dev = 0;
+    if (cudaGetDevice(&dev) != cudaSuccess) return 0;
+    const bool slot = dev >= 0 && dev < 64;
+    if (slot && cached[dev].load() > 0) return cached[dev].load();
+    int n = 0;
+    if (cudaDeviceGetAttribute(&n, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess) return 0;
+    if (slot) cached[dev].store(n);
+    return n;
 }
 
 // Opt-in to more than 48 KB of dynamic shared memory.  The attribute belongs to (kernel, device): it is set
