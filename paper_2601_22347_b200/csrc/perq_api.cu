@@ -316,12 +316,29 @@ static __device__ __align__(256) float g_stats_scratch[PERQ_STATS_STATIC_MAX_FLO
 float *g_stats_scratch_addr[kMaxDevices] = {};   // device address of the array, per device ordinal
 std::mutex g_stats_scratch_mutex;
 
+template <int KC, int CL, bool WB>
+int launch_stats_inst(const perq::StatsParams &p, const StatsPlan &plan, cudaStream_t st)
+{
+    if (int rc = allow_smem(perq::perq_stats_partial_kernel<KC, CL, WB>, plan.smem)) return rc;
+    perq::perq_stats_partial_kernel<KC, CL, WB><<<plan.n_cta, perq::ST_THREADS, plan.smem, st>>>(p);
+    return cudaGetLastError() == cudaSuccess ? PERQ_OK : PERQ_ERR_CUDA;
+}
+
 template <int KC>
 int launch_stats_partial(const perq::StatsParams &p, const StatsPlan &plan, cudaStream_t st)
 {
-    if (int rc = allow_smem(perq::perq_stats_partial_kernel<KC>, plan.smem)) return rc;
-    perq::perq_stats_partial_kernel<KC><<<plan.n_cta, perq::ST_THREADS, plan.smem, st>>>(p);
-    return cudaGetLastError() == cudaSuccess ? PERQ_OK : PERQ_ERR_CUDA;
+    // specialised variants: unpermuted rows of exactly KC * 4096 channels, blocks of 16, 32 or 128
+    if (KC <= 4 && p.perm == nullptr && p.d == KC * 4096) {
+        const bool wb = p.ws_block != nullptr || p.token_max != nullptr;
+        if (!wb) return launch_stats_inst<KC, 2, false>(p, plan, st);
+        switch (p.log2b) {
+        case 4: return launch_stats_inst<KC, 1, true>(p, plan, st);
+        case 5: return launch_stats_inst<KC, 2, true>(p, plan, st);
+        case 7: return launch_stats_inst<KC, 4, true>(p, plan, st);
+        default: break;
+        }
+    }
+    return launch_stats_inst<KC, -1, false>(p, plan, st);
 }
 
 }  // namespace

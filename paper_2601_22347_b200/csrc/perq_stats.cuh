@@ -38,10 +38,15 @@ __device__ __forceinline__ float abs_bf16(uint16_t h) { return __uint_as_float((
 // consecutive rows are contiguous in global memory: one elected thread fetches each with a single
 // cp.async.bulk into a ring of shared-memory stages (bulk copies are not limited by the load
 // queue of the SM the way per-thread loads are), everybody reads its columns from there.
-template <int KC>
+// CL >= 0 selects a specialised variant: rows of exactly KC * 4096 channels, no permutation, blocks of
+// 2^CL chunks (CL <= 5: summed by shuffles), block statistics wanted (WB) or not -- the flags the general
+// variant (CL = -1) tests at run time inside its unrolled loops are constants there.
+template <int KC, int CL, bool WB>
 __global__ void __launch_bounds__(ST_THREADS) perq_stats_partial_kernel(StatsParams p)
 {
     constexpr int R = 8 / KC;
+    constexpr bool FAST = CL >= 0;
+    static_assert(CL <= 5, "shuffle sums need a block inside a warp");
     const int NST = p.n_stages;                   // 3, or 2 where 3 stages would not fit
     extern __shared__ __align__(128) unsigned char smem[];
     const int d = p.d, L = p.log2b, nb = d >> L, nchunks = d >> 3;
@@ -67,9 +72,10 @@ __global__ void __launch_bounds__(ST_THREADS) perq_stats_partial_kernel(StatsPar
     }
     const long long t0 = (long long)blockIdx.x * p.rows_per_cta;
     const long long t1 = min(p.T, t0 + p.rows_per_cta);
-    const bool want_blocks = (p.ws_block != nullptr) || (p.token_max != nullptr);
-    const int cpb = 1 << (L - 3);                 // 16-byte chunks per block
-    const bool shuffle_blocks = cpb <= 32;        // a block's chunks sit in adjacent lanes of one warp
+    const bool want_blocks = FAST ? WB : ((p.ws_block != nullptr) || (p.token_max != nullptr));
+    const bool use_perm = FAST ? false : (p.perm != nullptr);
+    const int cpb = FAST ? (1 << (CL < 0 ? 0 : CL)) : (1 << (L - 3));   // 16-byte chunks per block
+    const bool shuffle_blocks = FAST ? true : cpb <= 32;                // a block's chunks sit in adjacent lanes of one warp
 
     auto fetch = [&](int stage, long long t) {      // one thread: rows t .. t+R-1 (those below t1) into a stage
         if (t < t1) {
@@ -104,7 +110,7 @@ __global__ void __launch_bounds__(ST_THREADS) perq_stats_partial_kernel(StatsPar
             for (int k = 0; k < KC; ++k) {
                 const int c = tid + k * ST_THREADS;
                 float s = 0.0f;
-                if (live && c < nchunks) {
+                if (live && (FAST || c < nchunks)) {
                     const uint4 w = ((const uint4 *)(rows + (size_t)r * d))[c];
                     const uint32_t ww[4] = {w.x, w.y, w.z, w.w};
                     float2 m[4];
@@ -115,7 +121,7 @@ __global__ void __launch_bounds__(ST_THREADS) perq_stats_partial_kernel(StatsPar
                         csum[k][e] = __fadd2_rn(csum[k][e], m[e]);
                     }
                     if (want_blocks) {
-                        if (p.perm) {
+                        if (use_perm) {
                             const uint4 pi = ((const uint4 *)sperm)[c];
                             const uint32_t pp[4] = {pi.x, pi.y, pi.z, pi.w};
                             const uint16_t *row = rows + (size_t)r * d;
@@ -132,6 +138,7 @@ __global__ void __launch_bounds__(ST_THREADS) perq_stats_partial_kernel(StatsPar
                 }
                 if (want_blocks) {
                     if (shuffle_blocks) {
+#pragma unroll
                         for (int o = 1; o < cpb; o <<= 1) s += __shfl_xor_sync(0xffffffffu, s, o);
                         if ((c & (cpb - 1)) == 0) bsum[k] += s;       // the block's first chunk keeps its sum
                         mx[r] = fmaxf(mx[r], s);
