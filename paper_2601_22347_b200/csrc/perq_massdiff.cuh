@@ -5,7 +5,7 @@
 //
 // Two kernels: ranks by counting (every CTA ranks 256 channels against all d: d^2 comparisons spread over the
 // grid), then the greedy itself, which is sequential in the channels: one warp scans the open blocks for the
-// minimum (lanes over blocks, shuffle reduction), d times.
+// minimum (lanes over blocks, integer warp reductions), d times.
 #pragma once
 #include <cuda_runtime.h>
 #include <stdint.h>
@@ -36,16 +36,19 @@ __global__ void __launch_bounds__(MD_THREADS) perq_massdiff_rank_kernel(const fl
     if (i < d) order[rank] = i;
 }
 
-// one warp; n = d / b <= MD_MAX_BLOCKS
+// one warp; n = d / b <= MD_MAX_BLOCKS.  Running sums are non-negative doubles, so their bit patterns order
+// like the values: the minimum over the warp is three integer warp reductions (high word, low word among
+// the lanes that hold the minimal high word, block index among the lanes that hold the minimal sum).  A full
+// block's sum is replaced by +infinity.
 __global__ void __launch_bounds__(32) perq_massdiff_greedy_kernel(const float *a, const int32_t *order, int d, int b,
                                                                   int32_t *perm)
 {
-    __shared__ double sum[MD_MAX_BLOCKS];
+    __shared__ unsigned long long sum[MD_MAX_BLOCKS];      // bit patterns of the doubles
     __shared__ int fill[MD_MAX_BLOCKS];
     const int lane = threadIdx.x, n = d / b;
-    for (int j = lane; j < n; j += 32) { sum[j] = 0.0; fill[j] = 0; }
+    for (int j = lane; j < n; j += 32) { sum[j] = 0ull; fill[j] = 0; }
     __syncwarp();
-    const double INF = __longlong_as_double(0x7ff0000000000000ll);
+    const unsigned long long INF = 0x7ff0000000000000ull;
     for (int s0 = 0; s0 < d; s0 += 32) {
         // the next 32 channels and their masses, one per lane
         const int cl = (s0 + lane < d) ? order[s0 + lane] : 0;
@@ -54,22 +57,23 @@ __global__ void __launch_bounds__(32) perq_massdiff_greedy_kernel(const float *a
         for (int t = 0; t < steps; ++t) {
             const int c = __shfl_sync(0xffffffffu, cl, t);
             const float ac = __shfl_sync(0xffffffffu, al, t);
-            double best = INF;
+            unsigned long long best = ~0ull;
             int bj = 0x7fffffff;
+#pragma unroll 4
             for (int j = lane; j < n; j += 32) {
-                const double v = (fill[j] < b) ? sum[j] : INF;
-                if (v < best || (v == best && j < bj && fill[j] < b)) { best = v; bj = j; }
+                const unsigned long long v = sum[j];
+                if (v < best) { best = v; bj = j; }          // ascending j: equal sums keep the lower block
             }
-#pragma unroll
-            for (int o = 16; o > 0; o >>= 1) {
-                const double ob = __shfl_xor_sync(0xffffffffu, best, o);
-                const int oj = __shfl_xor_sync(0xffffffffu, bj, o);
-                if (ob < best || (ob == best && oj < bj)) { best = ob; bj = oj; }
-            }
+            const uint32_t hi = (uint32_t)(best >> 32), lo = (uint32_t)best;
+            const uint32_t mhi = __reduce_min_sync(0xffffffffu, hi);
+            const uint32_t mlo = __reduce_min_sync(0xffffffffu, hi == mhi ? lo : 0xffffffffu);
+            const int mj = (int)__reduce_min_sync(0xffffffffu, (hi == mhi && lo == mlo) ? (uint32_t)bj : 0x7fffffffu);
             if (lane == 0) {
-                perm[(size_t)bj * b + fill[bj]] = c;
-                fill[bj] += 1;
-                sum[bj] += (double)ac;
+                const int f = fill[mj];
+                perm[(size_t)mj * b + f] = c;
+                fill[mj] = f + 1;
+                const double ns = __longlong_as_double((long long)(((unsigned long long)mhi << 32) | mlo)) + (double)ac;
+                sum[mj] = (f + 1 < b) ? (unsigned long long)__double_as_longlong(ns) : INF;
             }
             __syncwarp();
         }
