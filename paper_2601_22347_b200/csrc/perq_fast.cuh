@@ -1358,6 +1358,7 @@ __global__ void __launch_bounds__(FAST_THREADS, 1) perq_fast_kernel(FastParams p
             }
             const f32x2 magic2 = pack2(MAGIC, MAGIC);
             uint32_t tie_any = 0u;
+            uint32_t xw[MODE == MODE_FP4 ? 8 : 1];     // FP4: per slot, the XOR of the two code words (kept for the fix-up)
             // E2M1 elements: the value scaled to [-7, 7] plus / minus an additive window, converted twice
             const float tau = (a32 > 0.0f) ? 8.0f * err_rel + 4.0e-6f : 0.0f;
             const f32x2 tau_p2 = pack2(tau, tau), tau_m2 = pack2(-tau, -tau);
@@ -1372,6 +1373,7 @@ __global__ void __launch_bounds__(FAST_THREADS, 1) perq_fast_kernel(FastParams p
                     const f32x2 dn0 = fma2(v[s][0], mul_c[k], tau_m2), dn1 = fma2(v[s][1], mul_c[k], tau_m2);
                     const uint32_t pu = cvt_e2m1x4(up0.x, up0.y, up1.x, up1.y);
                     const uint32_t pd = cvt_e2m1x4(dn0.x, dn0.y, dn1.x, dn1.y);
+                    xw[MODE == MODE_FP4 ? s : 0] = pu ^ pd;
                     tie_any |= pu ^ pd;
                     sts_code<(3 & ~PM)>(code_addr0, s, pu);
                     continue;
@@ -1449,7 +1451,33 @@ __global__ void __launch_bounds__(FAST_THREADS, 1) perq_fast_kernel(FastParams p
 
             // ---- exact resolution of near ties (rare)
             if (__any_sync(0xffffffffu, tie_any != 0u)) {
-                if (!have_exact) {
+                // flagged elements; FP4: from the kept difference words, and zm marks those whose two codes differ
+                // in the sign alone (both magnitudes are zero: they need the sign of the exact value, not the scale
+                // and none of its fp64 divisions)
+                uint32_t fm = 0u, zm = 0u;
+                if (tie_any != 0u) {
+#pragma unroll
+                    for (int s = 0; s < 8; ++s) {
+                        const int k = s & 3 & PM;
+                        if (MODE == MODE_FP4) {
+                            const uint32_t x = xw[MODE == MODE_FP4 ? s : 0];
+#pragma unroll
+                            for (int j = 0; j < 4; ++j) {
+                                const uint32_t xn = (x >> (4 * j)) & 0xFu;
+                                fm |= xn ? (1u << (4 * s + j)) : 0u;
+                                zm |= (xn == 8u) ? (1u << (4 * s + j)) : 0u;
+                            }
+                            continue;
+                        }
+                        const f32x2 tp0 = fma2(v[s][0], mul_p[k], magic2), tp1 = fma2(v[s][1], mul_p[k], magic2);
+                        const f32x2 tm0 = fma2(v[s][0], mul_m[k], magic2), tm1 = fma2(v[s][1], mul_m[k], magic2);
+                        const float t[4] = {tp0.x, tp0.y, tp1.x, tp1.y}, u[4] = {tm0.x, tm0.y, tm1.x, tm1.y};
+#pragma unroll
+                        for (int j = 0; j < 4; ++j) fm |= (t[j] != u[j]) ? (1u << (4 * s + j)) : 0u;
+                    }
+                }
+                const bool need_scale = (MODE != MODE_FP4) || __any_sync(0xffffffffu, (fm & ~zm) != 0u);
+                if (!have_exact && need_scale) {
                     unsigned long long d = (1ull << 63) | my_pos;
                     if (my_pos == 0xffffffffu) {      // published by a candidate warp of the row: wait for it
                         uint32_t spin = 0;
@@ -1472,32 +1500,13 @@ __global__ void __launch_bounds__(FAST_THREADS, 1) perq_fast_kernel(FastParams p
                         a_bits = d;
                     }
                 }
-                uint32_t fm = 0u;
-                if (tie_any != 0u) {
-#pragma unroll
-                    for (int s = 0; s < 8; ++s) {
-                        const int k = s & 3 & PM;
-                        if (MODE == MODE_FP4) {
-                            const f32x2 up0 = fma2(v[s][0], mul_c[k], tau_p2), up1 = fma2(v[s][1], mul_c[k], tau_p2);
-                            const f32x2 dn0 = fma2(v[s][0], mul_c[k], tau_m2), dn1 = fma2(v[s][1], mul_c[k], tau_m2);
-                            const uint32_t x = cvt_e2m1x4(up0.x, up0.y, up1.x, up1.y) ^ cvt_e2m1x4(dn0.x, dn0.y, dn1.x, dn1.y);
-#pragma unroll
-                            for (int j = 0; j < 4; ++j) fm |= ((x >> (4 * j)) & 0xFu) ? (1u << (4 * s + j)) : 0u;
-                            continue;
-                        }
-                        const f32x2 tp0 = fma2(v[s][0], mul_p[k], magic2), tp1 = fma2(v[s][1], mul_p[k], magic2);
-                        const f32x2 tm0 = fma2(v[s][0], mul_m[k], magic2), tm1 = fma2(v[s][1], mul_m[k], magic2);
-                        const float t[4] = {tp0.x, tp0.y, tp1.x, tp1.y}, u[4] = {tm0.x, tm0.y, tm1.x, tm1.y};
-#pragma unroll
-                        for (int j = 0; j < 4; ++j) fm |= (t[j] != u[j]) ? (1u << (4 * s + j)) : 0u;
-                    }
-                }
                 __syncwarp();
                 unsigned tl = __ballot_sync(0xffffffffu, fm != 0u);
                 while (tl) {
                     const int src = __ffs(tl) - 1;
                     tl &= tl - 1;
                     uint32_t fs = __shfl_sync(0xffffffffu, fm, src);
+                    const uint32_t zs = __shfl_sync(0xffffffffu, zm, src);
                     // the same sequence of fp64 operations as the definition, so exact ties land on exact halves
                     unsigned long long ab_src = __shfl_sync(0xffffffffu, a_bits, src);
                     if (MODE == MODE_G128) {
@@ -1509,7 +1518,8 @@ __global__ void __launch_bounds__(FAST_THREADS, 1) perq_fast_kernel(FastParams p
                         }
                     }
                     const double a_src = __longlong_as_double((long long)ab_src);
-                    const double s_src = (a_src / p.sqrt_b) / 7.0;
+                    // (sign-only fix-ups do not use the scale: spare them its two fp64 divisions)
+                    const double s_src = (MODE == MODE_FP4 && (fs & ~zs) == 0u) ? 0.0 : (a_src / p.sqrt_b) / 7.0;
                     while (fs) {
                         const int e = __ffs(fs) - 1;
                         fs &= fs - 1;
@@ -1520,7 +1530,9 @@ __global__ void __launch_bounds__(FAST_THREADS, 1) perq_fast_kernel(FastParams p
                         const double ue = exact_coord_fast<BF>(bp, i, lane);
                         if (lane == 0) {
                             uint32_t code = 0u;
-                            if (MODE == MODE_FP4) {
+                            if (MODE == MODE_FP4 && ((zs >> e) & 1u)) {
+                                code = signbit(ue) ? 8u : 0u;          // magnitude zero either way: the sign of y = u / sqrt(b)
+                            } else if (MODE == MODE_FP4) {
                                 const double y = ue / p.sqrt_b;
                                 code = e2m1_code_exact((s_src != 0.0) ? y / s_src : 0.0, signbit(y));
                             } else if (s_src != 0.0) {
