@@ -37,7 +37,7 @@ ORACLE_FMT = {"int4": 0, "mxfp4": 1, "fp4": 3}     # format numbers of oracle/pe
 
 # DRAM traffic per token (dram__bytes_read.sum + dram__bytes_write.sum) / T of the headline
 # kernel from an ncu capture; None until a capture of the current kernel exists.  See profiles/.
-NCU_TRAFFIC_BYTES_PER_TOKEN = (135.28e6 + 18.68e6) / 16384   # mean of the two captured launches   # profiles/perq_fast_kernel_cfg4_b32_int4.md
+NCU_TRAFFIC_BYTES_PER_TOKEN = (135.27e6 + 17.92e6) / 16384   # mean of the two captured launches   # profiles/perq_fast_kernel_cfg4_b32_int4.md
 
 
 def measured_peak():
