@@ -714,6 +714,11 @@ __global__ void __launch_bounds__(FAST_THREADS, 1) perq_fast_kernel(FastParams p
     const int w_in_g = warp - group * G;
     const unsigned qmask = 0xFu << (lane & 28);
     const float err_rel = (!FULLV ? FAST_ERR_K : LOG2BF >= 10 ? FAST_ERR_K_FULL : FAST_ERR_K_LONG) * (float)LOG2BF * TWO_M24;
+    // u / sqrt(b) as the definition computes it.  For an even log2(b) the divisor is a power of two: the
+    // product with its reciprocal is the same double and spares the fix-ups an fp64 division.
+    auto over_sqrt_b = [&](double u) -> double {
+        return (LOG2BF % 2 == 0) ? u * (1.0 / (double)(1 << (LOG2BF / 2))) : u / p.sqrt_b;
+    };
     const uint32_t xbuf_addr = smem_u32(fsmem + FastSmem::xbuf) + (uint32_t)(group * G) * 4096u;   // FULLV: this row's exchange space
 
     const uint32_t stage_base = smem_u32(fsmem + FastSmem::stages) + (uint32_t)group * (NST * UNIT_BYTES);
@@ -1245,7 +1250,7 @@ __global__ void __launch_bounds__(FAST_THREADS, 1) perq_fast_kernel(FastParams p
                         if (lane == 0) {
                             uint32_t code = 0u;
                             if (s_ex != 0.0) {
-                                const double qd = rint((ue / p.sqrt_b) / s_ex) - z_ex;
+                                const double qd = rint(over_sqrt_b(ue) / s_ex) - z_ex;
                                 code = (uint32_t)((int)fmin(fmax(qd, 0.0), 15.0));
                             }
                             uint8_t *cp = code_gen + (elem >> 1);
@@ -1519,7 +1524,7 @@ __global__ void __launch_bounds__(FAST_THREADS, 1) perq_fast_kernel(FastParams p
                     }
                     const double a_src = __longlong_as_double((long long)ab_src);
                     // (sign-only fix-ups do not use the scale: spare them its two fp64 divisions)
-                    const double s_src = (MODE == MODE_FP4 && (fs & ~zs) == 0u) ? 0.0 : (a_src / p.sqrt_b) / 7.0;
+                    const double s_src = (MODE == MODE_FP4 && (fs & ~zs) == 0u) ? 0.0 : over_sqrt_b(a_src) / 7.0;
                     while (fs) {
                         const int e = __ffs(fs) - 1;
                         fs &= fs - 1;
@@ -1533,10 +1538,10 @@ __global__ void __launch_bounds__(FAST_THREADS, 1) perq_fast_kernel(FastParams p
                             if (MODE == MODE_FP4 && ((zs >> e) & 1u)) {
                                 code = signbit(ue) ? 8u : 0u;          // magnitude zero either way: the sign of y = u / sqrt(b)
                             } else if (MODE == MODE_FP4) {
-                                const double y = ue / p.sqrt_b;
+                                const double y = over_sqrt_b(ue);
                                 code = e2m1_code_exact((s_src != 0.0) ? y / s_src : 0.0, signbit(y));
                             } else if (s_src != 0.0) {
-                                double qd = rint((ue / p.sqrt_b) / s_src);
+                                double qd = rint(over_sqrt_b(ue) / s_src);
                                 qd = fmin(fmax(qd, -8.0), 7.0);
                                 code = (uint32_t)((int)qd) & 0xFu;
                             }
@@ -1626,7 +1631,7 @@ __global__ void __launch_bounds__(FAST_THREADS, 1) perq_fast_kernel(FastParams p
                     }
                     if (lane == owner) {
                         int ex;
-                        (void)frexp(best / p.sqrt_b, &ex);
+                        (void)frexp(over_sqrt_b(best), &ex);
                         Eb = ex - 3 + 127;
                     }
                 }
@@ -1662,7 +1667,7 @@ __global__ void __launch_bounds__(FAST_THREADS, 1) perq_fast_kernel(FastParams p
                         }
                         if (q == m) {
                             int ex;
-                            (void)frexp(best / p.sqrt_b, &ex);
+                            (void)frexp(over_sqrt_b(best), &ex);
                             Eb = ex - 3 + 127;
                         }
                     }
@@ -1736,7 +1741,7 @@ __global__ void __launch_bounds__(FAST_THREADS, 1) perq_fast_kernel(FastParams p
                         const double ue = exact_coord_fast<BF>(bp, i, lane);
                         if (lane == 0) {
                             const int E = (int)((wsrc >> (8 * ((e >> 3) ^ fsrc))) & 0xFFu) - 127;
-                            const double y = ue / p.sqrt_b;
+                            const double y = over_sqrt_b(ue);
                             const uint32_t code = e2m1_code_exact(scalbn(y, -E), signbit(y));
                             uint8_t *bp = code_gen + (elem >> 1);
                             *bp = (elem & 1) ? (uint8_t)((*bp & 0x0F) | (code << 4)) : (uint8_t)((*bp & 0xF0) | code);
