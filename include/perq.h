@@ -245,9 +245,15 @@ int perq_massdiff_perm_device(const float *chan_abs_sum, int32_t d, int32_t b, i
  * perq_device_error -- reads (synchronously, cudaMemcpyFromSymbol) the library's device-side
  * error word on the current device into *flags_host.  0 = no error.  Bit 0 is set when a
  * bounded wait inside a kernel ran out (an asynchronous copy that never completed); the
- * kernel then stops early and its outputs are incomplete.  The word is never cleared.
+ * kernel then stops early and its outputs are incomplete.  Kernels only ever set bits; the
+ * word keeps them until perq_device_error_clear.
+ *
+ * perq_device_error_clear -- writes 0 to that word on the current device (synchronously,
+ * cudaMemcpyToSymbol), so that a later read reports only what happened since.  Call it with no
+ * kernel of the library in flight on the device, or a bit set concurrently may be lost.
  */
 int perq_device_error(uint32_t *flags_host);
+int perq_device_error_clear(void);
 
 /* Text for a status code (static storage).  Library version = major*10000 + minor*100 + patch. */
 const char *perq_status_string(int status);

@@ -58,6 +58,8 @@ def load() -> C.CDLL:
         lib.perq_massdiff_perm_device.argtypes = [vp, i32, i32, vp, vp, sz, vp]
         lib.perq_device_error.argtypes = [C.POINTER(C.c_uint32)]
         lib.perq_device_error.restype = C.c_int
+        lib.perq_device_error_clear.argtypes = []
+        lib.perq_device_error_clear.restype = C.c_int
         lib.perq_status_string.argtypes = [C.c_int]
         lib.perq_status_string.restype = C.c_char_p
         lib.perq_version.restype = C.c_int
@@ -214,6 +216,11 @@ def perq_device_error() -> int:
     v = C.c_uint32(0)
     _check(load().perq_device_error(C.byref(v)), "perq_device_error")
     return int(v.value)
+
+
+def perq_device_error_clear() -> None:
+    """Zeroes the device-side error word of the current device; synchronises."""
+    _check(load().perq_device_error_clear(), "perq_device_error_clear")
 
 
 def perq_massdiff_perm_device(chan_abs_sum: torch.Tensor, b: int, perm: Optional[torch.Tensor] = None,

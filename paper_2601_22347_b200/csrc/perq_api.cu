@@ -563,6 +563,12 @@ int perq_device_error(uint32_t *flags_host)
     return PERQ_OK;
 }
 
+int perq_device_error_clear(void)
+{
+    const unsigned int zero = 0;
+    return cudaMemcpyToSymbol(perq::g_perq_device_error, &zero, sizeof zero) == cudaSuccess ? PERQ_OK : PERQ_ERR_CUDA;
+}
+
 int perq_massdiff_perm_device(const float *chan_abs_sum, int32_t d, int32_t b, int32_t *perm, void *workspace,
                               size_t workspace_bytes, void *stream)
 {

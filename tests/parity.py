@@ -62,7 +62,7 @@ def compare_quantized(fmt: str, gpu_codes, gpu_scales, ora: dict) -> dict:
         pre = ora["pre"][idx]
         if fmt == "int4_asym":
             step = np.abs(g[idx].astype(np.int64) - o[idx].astype(np.int64))
-            near = np.abs(np.abs(pre - np.floor(pre)) - 0.5) < TIE_WINDOW * np.maximum(1.0, np.abs(pre) / 8.0)
+            near = np.abs(np.abs(pre - np.floor(pre)) - 0.5) < TIE_WINDOW
         elif fmt == "int4":
             step = np.abs(int4_values(g[idx]) - int4_values(o[idx]))
             near = np.abs(np.abs(pre - np.floor(pre)) - 0.5) < TIE_WINDOW

@@ -21,6 +21,14 @@ def B():
     return binding
 
 
+@pytest.fixture(autouse=True)
+def clean_error_word(B):
+    """Every test starts from a cleared device error word and must leave it clear."""
+    B.perq_device_error_clear()
+    yield
+    assert B.perq_device_error() == 0
+
+
 def to_dev(bits: np.ndarray) -> torch.Tensor:
     return torch.from_numpy(bits.view(np.int16).copy()).cuda().view(torch.bfloat16)
 
