@@ -16,6 +16,7 @@
 
 #include "perq_generic.cuh"
 #include "perq_fast.cuh"
+#include "perq_tok.cuh"
 #include "perq_stats.cuh"
 #include "perq_diag.cuh"
 #include "perq_massdiff.cuh"
@@ -203,6 +204,38 @@ int launch_fast_long(int xb, int G, const perq::FastParams &p, int grid, cudaStr
     }
 }
 
+// Lean per-token kernel: INT4 or E2M1 with one scale per token, unpermuted, d in {1024, 2048, 4096, 8192}, b <= 128.
+template <int LOG2B, int MODE, int LOG2G>
+int launch_tok_inst(const perq::FastParams &p, int grid, cudaStream_t st)
+{
+    auto kernel = perq::perq_tok_kernel<LOG2B, MODE, LOG2G>;
+    if (int rc = allow_smem(kernel, perq::TokSmem::total)) return rc;
+    kernel<<<grid, perq::FAST_THREADS, perq::TokSmem::total, st>>>(p);
+    return cudaGetLastError() == cudaSuccess ? PERQ_OK : PERQ_ERR_CUDA;
+}
+
+template <int MODE, int LOG2G>
+int launch_tok_b(int log2b, const perq::FastParams &p, int grid, cudaStream_t st)
+{
+    switch (log2b) {
+    case 4: return launch_tok_inst<4, MODE, LOG2G>(p, grid, st);
+    case 5: return launch_tok_inst<5, MODE, LOG2G>(p, grid, st);
+    case 6: return launch_tok_inst<6, MODE, LOG2G>(p, grid, st);
+    default: return launch_tok_inst<7, MODE, LOG2G>(p, grid, st);
+    }
+}
+
+template <int MODE>
+int launch_tok(int G, int log2b, const perq::FastParams &p, int grid, cudaStream_t st)
+{
+    switch (G) {
+    case 1: return launch_tok_b<MODE, 0>(log2b, p, grid, st);
+    case 2: return launch_tok_b<MODE, 1>(log2b, p, grid, st);
+    case 4: return launch_tok_b<MODE, 2>(log2b, p, grid, st);
+    default: return launch_tok_b<MODE, 3>(log2b, p, grid, st);
+    }
+}
+
 // The fast kernel covers d % 1024 == 0 with b <= 128 and scales per token (d / 1024 in {1,2,4,8}),
 // per 128 (INT4) or per 32 (MXFP4), with a permutation also d <= 16384; and b == d in {1024 .. 8192}
 // without a permutation, per token or MXFP4.  Returns -1 if it does not apply.
@@ -256,6 +289,10 @@ int try_launch_fast(const void *x, const int32_t *perm, int64_t T, int32_t d, in
     const int groups_per_cta = perq::FAST_WARPS / G;
     const long long want = (units + groups_per_cta - 1) / groups_per_cta;
     const int grid = (int)std::min<long long>(want, sms);
+    if ((mode == perq::MODE_TOKEN || mode == perq::MODE_FP4) && !permuted && !full && !longb &&
+        (segs == 1 || segs == 2 || segs == 4 || segs == 8))
+        return mode == perq::MODE_TOKEN ? launch_tok<perq::MODE_TOKEN>(segs, ilog2(b), p, grid, st)
+                                        : launch_tok<perq::MODE_FP4>(segs, ilog2(b), p, grid, st);
     if (full)
         return mode == perq::MODE_MX ? launch_fast_full<perq::MODE_MX>(G, p, grid, st)
                                      : launch_fast_full<perq::MODE_TOKEN>(G, p, grid, st);

@@ -145,6 +145,14 @@ __device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity)
     }
     return false;
 }
+// The common case costs one poll; the bounded loop is entered only when that poll fails.
+__device__ __forceinline__ bool mbar_wait_fast(uint32_t bar, uint32_t parity)
+{
+    uint32_t done;
+    asm volatile("{ .reg .pred p; mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2; selp.u32 %0, 1, 0, p; }"
+                 : "=r"(done) : "r"(bar), "r"(parity) : "memory");
+    return done != 0u || mbar_wait(bar, parity);
+}
 __device__ __forceinline__ void mbar_arrive(uint32_t bar)
 {
     asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];" ::"r"(bar) : "memory");
@@ -711,7 +719,11 @@ __global__ void __launch_bounds__(FAST_THREADS, 1) perq_fast_kernel(FastParams p
     const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
     const int g = lane >> 2, q = lane & 3;
     const int group = RUNTIME_G ? warp / G : warp >> (LOG2G < 0 ? 0 : LOG2G);
-    const int w_in_g = warp - group * G;
+    // Position of this warp in its row group, rotated by the group index.  Warps are handed to the SM's four
+    // schedulers by warp index, and for many inputs the same position of every row does the extra per-row
+    // work (the segment that holds the outlier channel finds the exact maximum; position 0 issues the
+    // loads): without the rotation those warps of all groups would share one scheduler.
+    const int w_in_g = (warp - group * G + group) % G;
     const unsigned qmask = 0xFu << (lane & 28);
     const float err_rel = (!FULLV ? FAST_ERR_K : LOG2BF >= 10 ? FAST_ERR_K_FULL : FAST_ERR_K_LONG) * (float)LOG2BF * TWO_M24;
     // u / sqrt(b) as the definition computes it.  For an even log2(b) the divisor is a power of two: the
@@ -797,25 +809,38 @@ __global__ void __launch_bounds__(FAST_THREADS, 1) perq_fast_kernel(FastParams p
     // sign to fold into the quantisation multiplier of class k (none once the true signs are restored)
     auto qsgn = [&](int k) { return FULLV ? 1.0f : sgn[k]; };
 
-    const uint16_t *xin = p.x;               // unit u starts at xin + u * G * SEG_ELEMS
+    // This group's units are first, first + stride, ...: n_units of them.  Addresses advance by increments
+    // (the loop is bound by the number of instructions it issues).
+    const uint32_t n_units = (p.units_total - first + stride - 1) / stride;
+    const uint32_t refill_end = n_units > (uint32_t)NST ? n_units - NST : 0u;      // iterations 1 .. refill_end load a unit
+    const size_t unit_step = (size_t)stride * ((size_t)G * SEG_ELEMS);
+    const uint16_t *xload = p.x + (size_t)first * ((size_t)G * SEG_ELEMS);         // leader: the next unit to load
     // prologue: fill the ring
     if (leader) {
 #pragma unroll
         for (int s = 0; s < NST; ++s) {
-            const uint32_t u = first + (uint32_t)s * stride;
-            if (u < p.units_total) {
+            if ((uint32_t)s < n_units) {
                 mbar_expect_tx(full_base + s * 8, UNIT_BYTES);
-                bulk_load(stage_base + s * UNIT_BYTES, xin + (size_t)u * (G * SEG_ELEMS), UNIT_BYTES, full_base + s * 8);
+                bulk_load(stage_base + s * UNIT_BYTES, xload, UNIT_BYTES, full_base + s * 8);
+                xload += unit_step;
             }
         }
     }
+    // quantisation multipliers of the sign classes, up to the scale range's factor (a sign change is exact, so
+    // inv * (sgn * (1 +- delta)) are the same floats as (sgn * inv) * (1 +- delta))
+    const float q_delta = 16.0f * err_rel + 5.0e-7f;
+    float q_cp[NCLS], q_cm[NCLS];
+#pragma unroll
+    for (int k = 0; k < NCLS; ++k) { q_cp[k] = qsgn(k) * (1.0f + q_delta); q_cm[k] = qsgn(k) * (1.0f - q_delta); }
 
-    uint32_t it = 0;
-    for (uint32_t unit = first; unit < p.units_total; unit += stride, ++it) {
+    uint8_t *code_out = p.out_codes + ((size_t)first * G + w_in_g) * SEG_CODE_BYTES;   // this warp's codes of the current unit
+    const size_t code_out_step = (size_t)stride * G * SEG_CODE_BYTES;
+    uint32_t unit = first;
+    for (uint32_t it = 0; it < n_units; ++it, unit += stride, code_out += code_out_step) {
         const uint32_t stage = it % NST;
         const uint32_t parity = (it / NST) & 1u;
         const uint32_t par2 = it & 1u;
-        if (!mbar_wait(full_base + stage * 8, parity)) {
+        if (!mbar_wait_fast(full_base + stage * 8, parity)) {
             if (lane == 0) atomicOr(&g_perq_device_error, 1u);
             return;
         }
@@ -860,7 +885,7 @@ __global__ void __launch_bounds__(FAST_THREADS, 1) perq_fast_kernel(FastParams p
 
         // ---- H_16 on the tensor cores; v[s][h] = outputs (2h, 2h+1) of this lane's four of slot s
         f32x2 v[8][2];
-        {
+        auto h16_tensor = [&](f32x2 (&w)[8][2]) {
             const uint32_t a0 = seg_addr + lm0;
 #pragma unroll
             for (int t = 0; t < 4; ++t) {
@@ -871,44 +896,46 @@ __global__ void __launch_bounds__(FAST_THREADS, 1) perq_fast_kernel(FastParams p
                 float c0[4], c1[4];
                 mma_bf16(c0, a, hb[0][0], hb[0][1]);
                 mma_bf16(c1, a, hb[1][0], hb[1][1]);
-                v[2 * t][0] = pack2(c0[0], c0[1]);
-                v[2 * t][1] = pack2(c1[0], c1[1]);
-                v[2 * t + 1][0] = pack2(c0[2], c0[3]);
-                v[2 * t + 1][1] = pack2(c1[2], c1[3]);
+                w[2 * t][0] = pack2(c0[0], c0[1]);
+                w[2 * t][1] = pack2(c1[0], c1[1]);
+                w[2 * t + 1][0] = pack2(c0[2], c0[3]);
+                w[2 * t + 1][1] = pack2(c1[2], c1[3]);
             }
-        }
+        };
+        // the butterfly stages over the slot bits inside a block (packed add/sub)
+        auto slot_stages = [&](f32x2 (&w)[8][2]) {
+#pragma unroll
+            for (int t = 0; t < CB; ++t) {
+#pragma unroll
+                for (int s = 0; s < 8; ++s) {
+                    if ((s & (1 << t)) == 0) {
+#pragma unroll
+                        for (int h = 0; h < 2; ++h) {
+                            const f32x2 a = w[s][h], c = w[s | (1 << t)][h];
+                            w[s][h] = add2(a, c);
+                            w[s | (1 << t)][h] = sub2(a, c);
+                        }
+                    }
+                }
+            }
+        };
+        h16_tensor(v);
         // refill the stage the previous iteration used (every warp of the group is past it now:
         // for G == 1 because this warp is, for G > 1 after the named barrier below)
         auto refill = [&]() {
-            if (leader && it > 0) {
-                const uint32_t u = unit + (NST - 1) * stride;
-                if (u < p.units_total && u > unit) {
-                    const uint32_t ps = (it - 1) % NST;
-                    // permuted rows are read until the end of an iteration: wait until every warp is done
-                    if (PERM && !mbar_wait(empty_base + ps * 8, ((it - 1) / NST) & 1u)) atomicOr(&g_perq_device_error, 4u);
-                    mbar_expect_tx(full_base + ps * 8, UNIT_BYTES);
-                    bulk_load(stage_base + ps * UNIT_BYTES, xin + (size_t)u * (G * SEG_ELEMS), UNIT_BYTES,
-                              full_base + ps * 8);
-                }
+            if (leader && it - 1u < refill_end) {        // it >= 1 and unit it + NST - 1 exists (it - 1 wraps for it == 0)
+                const uint32_t ps = (it - 1) % NST;
+                // permuted rows are read until the end of an iteration: wait until every warp is done
+                if (PERM && !mbar_wait(empty_base + ps * 8, ((it - 1) / NST) & 1u)) atomicOr(&g_perq_device_error, 4u);
+                mbar_expect_tx(full_base + ps * 8, UNIT_BYTES);
+                bulk_load(stage_base + ps * UNIT_BYTES, xload, UNIT_BYTES, full_base + ps * 8);
+                xload += unit_step;
             }
         };
         if (G == 1 || (!TOK && WBITS == 0)) refill();
 
-        // ---- remaining butterfly stages over the slot bits inside a block (packed add/sub)
-#pragma unroll
-        for (int t = 0; t < CB; ++t) {
-#pragma unroll
-            for (int s = 0; s < 8; ++s) {
-                if ((s & (1 << t)) == 0) {
-#pragma unroll
-                    for (int h = 0; h < 2; ++h) {
-                        const f32x2 a = v[s][h], c = v[s | (1 << t)][h];
-                        v[s][h] = add2(a, c);
-                        v[s | (1 << t)][h] = sub2(a, c);
-                    }
-                }
-            }
-        }
+        // ---- remaining butterfly stages over the slot bits inside a block
+        slot_stages(v);
 
         if (FULLV) {
             // ---- the rest of a full-vector butterfly.  First the true signs (the relabelling signs
@@ -1013,7 +1040,7 @@ __global__ void __launch_bounds__(FAST_THREADS, 1) perq_fast_kernel(FastParams p
             const uint32_t pidx = par2 * FAST_WARPS + group;
             float hi_row, lo_row, hm = hw, lm = lw;
             if (G > 1) {
-                if (lane == 0) { wmax[par2 * FAST_WARPS + warp] = hw; wmin[par2 * FAST_WARPS + warp] = lw; }
+                if (lane == 0) { wmax[par2 * FAST_WARPS + group * G + w_in_g] = hw; wmin[par2 * FAST_WARPS + group * G + w_in_g] = lw; }
                 named_barrier(1 + group, G * 32);
                 hm = (lane < G) ? wmax[par2 * FAST_WARPS + group * G + lane] : -INF;
                 lm = (lane < G) ? wmin[par2 * FAST_WARPS + group * G + lane] : INF;
@@ -1333,7 +1360,7 @@ __global__ void __launch_bounds__(FAST_THREADS, 1) perq_fast_kernel(FastParams p
                 const float aw = warp_max_f32(lane_max);
                 unsigned candw;
                 if (G > 1) {
-                    if (lane == 0) wmax[par2 * FAST_WARPS + warp] = aw;
+                    if (lane == 0) wmax[par2 * FAST_WARPS + group * G + w_in_g] = aw;
                     named_barrier(1 + group, G * 32);
                     const float am = (lane < G) ? wmax[par2 * FAST_WARPS + group * G + lane] : 0.0f;
                     a32 = warp_max_f32(am);
@@ -1350,51 +1377,9 @@ __global__ void __launch_bounds__(FAST_THREADS, 1) perq_fast_kernel(FastParams p
                 if (ncand == 0 && leader) reinterpret_cast<float *>(p.out_scales)[unit] = 0.0f;
             }
 
-            // ---- quantise: packed fp32 multiply-add against the magic constant, with the multiplier
-            // nudged up and down by the error bound; elements whose two codes differ are resolved exactly
-            const float inv = (a32 > 0.0f) ? fminf(__fdividef(7.0f, a32), 3.0e38f) : 0.0f;
-            const float delta = 16.0f * err_rel + 5.0e-7f;
-            f32x2 mul_p[NCLS], mul_m[NCLS];
-#pragma unroll
-            for (int k = 0; k < NCLS; ++k) {
-                const float mp = qsgn(k) * inv * (1.0f + delta), mm = qsgn(k) * inv * (1.0f - delta);
-                mul_p[k] = pack2(mp, mp);
-                mul_m[k] = pack2(mm, mm);
-            }
-            const f32x2 magic2 = pack2(MAGIC, MAGIC);
-            uint32_t tie_any = 0u;
-            uint32_t xw[MODE == MODE_FP4 ? 8 : 1];     // FP4: per slot, the XOR of the two code words (kept for the fix-up)
-            // E2M1 elements: the value scaled to [-7, 7] plus / minus an additive window, converted twice
-            const float tau = (a32 > 0.0f) ? 8.0f * err_rel + 4.0e-6f : 0.0f;
-            const f32x2 tau_p2 = pack2(tau, tau), tau_m2 = pack2(-tau, -tau);
-            f32x2 mul_c[NCLS];
-#pragma unroll
-            for (int k = 0; k < NCLS; ++k) mul_c[k] = pack2(qsgn(k) * inv, qsgn(k) * inv);
-#pragma unroll
-            for (int s = 0; s < 8; ++s) {
-                const int k = s & 3 & PM;
-                if (MODE == MODE_FP4) {
-                    const f32x2 up0 = fma2(v[s][0], mul_c[k], tau_p2), up1 = fma2(v[s][1], mul_c[k], tau_p2);
-                    const f32x2 dn0 = fma2(v[s][0], mul_c[k], tau_m2), dn1 = fma2(v[s][1], mul_c[k], tau_m2);
-                    const uint32_t pu = cvt_e2m1x4(up0.x, up0.y, up1.x, up1.y);
-                    const uint32_t pd = cvt_e2m1x4(dn0.x, dn0.y, dn1.x, dn1.y);
-                    xw[MODE == MODE_FP4 ? s : 0] = pu ^ pd;
-                    tie_any |= pu ^ pd;
-                    sts_code<(3 & ~PM)>(code_addr0, s, pu);
-                    continue;
-                }
-                const f32x2 tp0 = fma2(v[s][0], mul_p[k], magic2), tp1 = fma2(v[s][1], mul_p[k], magic2);
-                const f32x2 tm0 = fma2(v[s][0], mul_m[k], magic2), tm1 = fma2(v[s][1], mul_m[k], magic2);
-                const uint32_t pp = ((__float_as_uint(tp1.y) * 16u + __float_as_uint(tp1.x)) * 16u + __float_as_uint(tp0.y)) * 16u
-                                    + __float_as_uint(tp0.x);
-                const uint32_t pm = ((__float_as_uint(tm1.y) * 16u + __float_as_uint(tm1.x)) * 16u + __float_as_uint(tm0.y)) * 16u
-                                    + __float_as_uint(tm0.x);
-                tie_any |= pp ^ pm;          // low 16 bits: the four codes (offset by 8) under either multiplier
-                sts_code<(3 & ~PM)>(code_addr0, s, pp ^ 0x8888u);
-            }
-            tie_any &= 0xffffu;
-
             // ---- per token: the exact row maximum and the stored scale, by the candidate warps only
+            // (before the quantiser, while the rotated values are live anyway: placed after it, the block kept all of
+            // them in registers through the quantiser's loop)
             if (TOK && is_cand) {
                 const float thr_row = a32 * (1.0f - 2.0f * err_rel - 2.4e-7f);
                 slot_maxima();
@@ -1454,12 +1439,64 @@ __global__ void __launch_bounds__(FAST_THREADS, 1) perq_fast_kernel(FastParams p
                 }
             }
 
+            // ---- quantise: packed fp32 multiply-add against the magic constant, with the multiplier
+            // nudged up and down by the error bound; elements whose two codes differ are resolved exactly
+            const float inv = (a32 > 0.0f) ? fminf(__fdividef(7.0f, a32), 3.0e38f) : 0.0f;
+            f32x2 mul_p[NCLS], mul_m[NCLS];
+#pragma unroll
+            for (int k = 0; k < NCLS; ++k) {
+                const float mp = inv * q_cp[k], mm = inv * q_cm[k];
+                mul_p[k] = pack2(mp, mp);
+                mul_m[k] = pack2(mm, mm);
+            }
+            const f32x2 magic2 = pack2(MAGIC, MAGIC);
+            uint32_t tie_any = 0u;
+            uint32_t xw[MODE == MODE_FP4 ? 8 : 1];     // FP4: per slot, the XOR of the two code words (kept for the fix-up)
+            // E2M1 elements: the value scaled to [-7, 7] plus / minus an additive window, converted twice
+            const float tau = (a32 > 0.0f) ? 8.0f * err_rel + 4.0e-6f : 0.0f;
+            const f32x2 tau_p2 = pack2(tau, tau), tau_m2 = pack2(-tau, -tau);
+            f32x2 mul_c[NCLS];
+#pragma unroll
+            for (int k = 0; k < NCLS; ++k) mul_c[k] = pack2(qsgn(k) * inv, qsgn(k) * inv);
+#pragma unroll
+            for (int s = 0; s < 8; ++s) {
+                const int k = s & 3 & PM;
+                if (MODE == MODE_FP4) {
+                    const f32x2 up0 = fma2(v[s][0], mul_c[k], tau_p2), up1 = fma2(v[s][1], mul_c[k], tau_p2);
+                    const f32x2 dn0 = fma2(v[s][0], mul_c[k], tau_m2), dn1 = fma2(v[s][1], mul_c[k], tau_m2);
+                    const uint32_t pu = cvt_e2m1x4(up0.x, up0.y, up1.x, up1.y);
+                    const uint32_t pd = cvt_e2m1x4(dn0.x, dn0.y, dn1.x, dn1.y);
+                    xw[MODE == MODE_FP4 ? s : 0] = pu ^ pd;
+                    tie_any |= pu ^ pd;
+                    sts_code<(3 & ~PM)>(code_addr0, s, pu);
+                    continue;
+                }
+                const f32x2 tp0 = fma2(v[s][0], mul_p[k], magic2), tp1 = fma2(v[s][1], mul_p[k], magic2);
+                const f32x2 tm0 = fma2(v[s][0], mul_m[k], magic2), tm1 = fma2(v[s][1], mul_m[k], magic2);
+                const uint32_t pp = ((__float_as_uint(tp1.y) * 16u + __float_as_uint(tp1.x)) * 16u + __float_as_uint(tp0.y)) * 16u
+                                    + __float_as_uint(tp0.x);
+                const uint32_t pm = ((__float_as_uint(tm1.y) * 16u + __float_as_uint(tm1.x)) * 16u + __float_as_uint(tm0.y)) * 16u
+                                    + __float_as_uint(tm0.x);
+                tie_any |= pp ^ pm;          // low 16 bits: the four codes (offset by 8) under either multiplier
+                sts_code<(3 & ~PM)>(code_addr0, s, pp ^ 0x8888u);
+            }
+            tie_any &= 0xffffu;
+
             // ---- exact resolution of near ties (rare)
             if (__any_sync(0xffffffffu, tie_any != 0u)) {
                 // flagged elements; FP4: from the kept difference words, and zm marks those whose two codes differ
                 // in the sign alone (both magnitudes are zero: they need the sign of the exact value, not the scale
                 // and none of its fp64 divisions)
                 uint32_t fm = 0u, zm = 0u;
+                // The rotated values are formed again from the staged segment: had this rare path used the
+                // quantiser's, they would stay in registers until here in every iteration.  (Blocks that span
+                // lanes or warps cannot be redone by one warp on its own: those variants keep the values.)
+                f32x2 vr[8][2];
+                if (!FULLV) {
+                    h16_tensor(vr);
+                    slot_stages(vr);
+                }
+                f32x2 (&vq)[8][2] = FULLV ? v : vr;
                 if (tie_any != 0u) {
 #pragma unroll
                     for (int s = 0; s < 8; ++s) {
@@ -1474,8 +1511,8 @@ __global__ void __launch_bounds__(FAST_THREADS, 1) perq_fast_kernel(FastParams p
                             }
                             continue;
                         }
-                        const f32x2 tp0 = fma2(v[s][0], mul_p[k], magic2), tp1 = fma2(v[s][1], mul_p[k], magic2);
-                        const f32x2 tm0 = fma2(v[s][0], mul_m[k], magic2), tm1 = fma2(v[s][1], mul_m[k], magic2);
+                        const f32x2 tp0 = fma2(vq[s][0], mul_p[k], magic2), tp1 = fma2(vq[s][1], mul_p[k], magic2);
+                        const f32x2 tm0 = fma2(vq[s][0], mul_m[k], magic2), tm1 = fma2(vq[s][1], mul_m[k], magic2);
                         const float t[4] = {tp0.x, tp0.y, tp1.x, tp1.y}, u[4] = {tm0.x, tm0.y, tm1.x, tm1.y};
 #pragma unroll
                         for (int j = 0; j < 4; ++j) fm |= (t[j] != u[j]) ? (1u << (4 * s + j)) : 0u;
@@ -1524,7 +1561,10 @@ __global__ void __launch_bounds__(FAST_THREADS, 1) perq_fast_kernel(FastParams p
                     }
                     const double a_src = __longlong_as_double((long long)ab_src);
                     // (sign-only fix-ups do not use the scale: spare them its two fp64 divisions)
-                    const double s_src = (MODE == MODE_FP4 && (fs & ~zs) == 0u) ? 0.0 : over_sqrt_b(a_src) / 7.0;
+                    // (symmetric INT4 decides most elements without it, see below)
+                    const bool want_s = (MODE == MODE_FP4) ? (fs & ~zs) != 0u : false;
+                    double s_src = want_s ? over_sqrt_b(a_src) / 7.0 : 0.0;
+                    bool have_s = want_s;
                     while (fs) {
                         const int e = __ffs(fs) - 1;
                         fs &= fs - 1;
@@ -1540,10 +1580,25 @@ __global__ void __launch_bounds__(FAST_THREADS, 1) perq_fast_kernel(FastParams p
                             } else if (MODE == MODE_FP4) {
                                 const double y = over_sqrt_b(ue);
                                 code = e2m1_code_exact((s_src != 0.0) ? y / s_src : 0.0, signbit(y));
-                            } else if (s_src != 0.0) {
-                                double qd = rint(over_sqrt_b(ue) / s_src);
-                                qd = fmin(fmax(qd, -8.0), 7.0);
-                                code = (uint32_t)((int)qd) & 0xFu;
+                            } else if (a_src != 0.0) {
+                                // The staged code kp comes from the multiplier nudged away from zero, the other
+                                // candidate is one step towards zero, the tie between them at |y / s| = |kp| - 1/2.
+                                // y / s = 7 u / a: the side is the sign of 14 |u| - (2 |kp| - 1) a, two fp64
+                                // products whose rounding errors are far below the margin asked for here.  Only
+                                // an exact or all but exact tie takes the definition's own sequence of operations
+                                // (three fp64 divisions), which then lands on exact halves where the definition does.
+                                const uint32_t nib = (code_gen[elem >> 1] >> ((elem & 1) * 4)) & 0xFu;
+                                const int kp = (int)(nib ^ 8u) - 8;
+                                const int mag = kp < 0 ? -kp : kp;
+                                const double diff = 14.0 * fabs(ue) - (double)(2 * mag - 1) * a_src;
+                                if (mag >= 1 && fabs(diff) > a_src * 1.0e-12) {
+                                    code = (uint32_t)(diff > 0.0 ? kp : (kp < 0 ? kp + 1 : kp - 1)) & 0xFu;
+                                } else {
+                                    if (!have_s) { s_src = over_sqrt_b(a_src) / 7.0; have_s = true; }
+                                    double qd = rint(over_sqrt_b(ue) / s_src);
+                                    qd = fmin(fmax(qd, -8.0), 7.0);
+                                    code = (uint32_t)((int)qd) & 0xFu;
+                                }
                             }
                             uint8_t *bp = code_gen + (elem >> 1);
                             *bp = (elem & 1) ? (uint8_t)((*bp & 0x0F) | (code << 4)) : (uint8_t)((*bp & 0xF0) | code);
@@ -1756,7 +1811,7 @@ __global__ void __launch_bounds__(FAST_THREADS, 1) perq_fast_kernel(FastParams p
         fence_async_smem();
         __syncwarp();
         if (lane == 0) {
-            bulk_store(p.out_codes + seg_index * SEG_CODE_BYTES, code_buf, SEG_CODE_BYTES);
+            bulk_store(code_out, code_buf, SEG_CODE_BYTES);
             if (PERM) mbar_arrive(empty_base + stage * 8);     // this warp no longer reads the staged row
         }
     }
