@@ -35,9 +35,33 @@ FALLBACK_HBM_GBS = 6650.0
 T_HEAD, D_HEAD, B_HEAD, FMT_HEAD, GROUP_HEAD = 16384, 4096, 32, "int4", 0
 ORACLE_FMT = {"int4": 0, "mxfp4": 1, "fp4": 3}     # format numbers of oracle/perq_oracle.c
 
-# DRAM traffic per token (dram__bytes_read.sum + dram__bytes_write.sum) / T of the headline
-# kernel from an ncu capture; None until a capture of the current kernel exists.  See profiles/.
-NCU_TRAFFIC_BYTES_PER_TOKEN = (135.27e6 + 17.92e6) / 16384   # mean of the two captured launches   # profiles/perq_fast_kernel_cfg4_b32_int4.md
+# DRAM traffic of one launch of the headline kernel (dram__bytes_read.sum + dram__bytes_write.sum from an ncu
+# capture) is kept in a small tracked file together with a hash of the kernel sources it was captured on;
+# when the sources have changed since, the bench reports no traffic figure.
+TRAFFIC_FILE = os.path.join(ROOT, "paper_2601_22347_b200", "ncu_traffic.json")
+
+
+def kernel_sources_hash():
+    import hashlib
+    csrc = os.path.join(ROOT, "paper_2601_22347_b200", "csrc")
+    h = hashlib.sha256()
+    for name in sorted(os.listdir(csrc)):
+        with open(os.path.join(csrc, name), "rb") as f:
+            h.update(name.encode() + b"\0" + f.read())
+    return h.hexdigest()
+
+
+def captured_traffic(fmt):
+    """Bytes per launch from the last ncu capture of this format's headline kernel, or None if there is none
+    for the kernel sources as they are now."""
+    try:
+        with open(TRAFFIC_FILE) as f:
+            rec = json.load(f)
+        if rec.get("sources_sha256") != kernel_sources_hash():
+            return None
+        return rec.get("dram_bytes_per_launch", {}).get(fmt)
+    except Exception:
+        return None
 
 
 def measured_peak():
@@ -163,6 +187,15 @@ def main():
     FMT_HEAD, GROUP_HEAD = args.fmt, (32 if args.fmt == "mxfp4" else 0)
     if args.impl == "reference":
         return run_reference(args)
+    if args.gpus > 1 and "WORLD_SIZE" not in os.environ:
+        # started plainly with --gpus N: become the launcher of N ranks (one per GPU) of this same command
+        import socket
+        with socket.socket() as sock:
+            sock.bind(("127.0.0.1", 0))
+            port = sock.getsockname()[1]
+        cmd = [sys.executable, "-m", "torch.distributed.run", "--nnodes=1", "--nproc-per-node", str(args.gpus),
+               "--master-addr", "127.0.0.1", "--master-port", str(port), os.path.abspath(__file__)] + sys.argv[1:]
+        return subprocess.call(cmd)
 
     import numpy as np
     import torch
@@ -171,6 +204,9 @@ def main():
     world = int(os.environ.get("WORLD_SIZE", "1"))
     rank = int(os.environ.get("RANK", "0"))
     local_rank = int(os.environ.get("LOCAL_RANK", "0"))
+    if world != args.gpus:
+        sys.stderr.write("bench.py: --gpus %d but WORLD_SIZE is %d\n" % (args.gpus, world))
+        return 2
     assert torch.cuda.is_available(), "bench.py needs a CUDA device (no CPU fallback)"
     torch.cuda.set_device(local_rank)
     dist = None
@@ -220,9 +256,14 @@ def main():
     # launch would itself add a few microseconds to each 40 us step.
     marks = sorted(set([0, args.steps] + [args.steps * k // 8 for k in range(1, 8)]))
     ev = {m: torch.cuda.Event(enable_timing=True) for m in marks}
+    # a few untimed launches are queued first, so that the first event is recorded behind running work and a
+    # short run does not time the start of the queue
+    LEAD = 8
+    for i in range(LEAD):
+        step(i)
     ev[0].record()
     for i in range(args.steps):
-        step(i)
+        step(LEAD + i)
         if i + 1 in ev:
             ev[i + 1].record()
     barrier()
@@ -265,11 +306,28 @@ def main():
     achieved = bytes_per_step / (launch_ms * 1e-3) / 1e9
     roofline = {"bound": "hbm", "achieved": achieved, "peak": peak, "unit": "GB/s", "frac": achieved / peak,
                 "peak_kind": "of " + peak_kind, "frac_of_nominal_8TBs": achieved / NOMINAL_HBM_GBS,
-                "traffic": None if NCU_TRAFFIC_BYTES_PER_TOKEN is None else NCU_TRAFFIC_BYTES_PER_TOKEN * T_HEAD,
+                "traffic": captured_traffic(FMT_HEAD),
                 "algorithmic_bytes_per_launch": bytes_per_step, "kernel_ms": launch_ms,
                 "kernel_ms_by_eighth_of_the_run": [round(v, 5) for v in per_launch_ms]}
 
     sweep = []
+    check_rows = None
+    if not args.no_cpu_baseline:
+        # beside every timed variant: a few rows of the last call's outputs against the oracle (part of the CPU leg)
+        from oracle import perq_oracle
+        perq_oracle.build()
+        sys.path.insert(0, os.path.join(ROOT, "tests"))
+        from parity import compare_quantized
+
+        def check_rows(x_dev, perm, b, f, grp, codes, scales, n=16):
+            T = x_dev.shape[0]
+            rows = np.unique(np.linspace(0, T - 1, num=min(n, T)).astype(np.int64))
+            rt = torch.from_numpy(rows).to(x_dev.device)
+            bits = x_dev[rt].view(torch.int16).cpu().numpy().view(np.uint16)
+            ora = perq_oracle.rotate_quantize(bits, perm, b, B.FMT_BY_NAME[f], grp, want_pre=True)
+            rep = compare_quantized(f, codes[rt].cpu().numpy(), scales[rt].cpu().numpy(), ora)
+            return {"parity_rows_checked": int(rows.size), "tie_window_exemptions": rep["code_mismatch_exempt"]}
+
     if not args.no_sweep:
         def time_calls(fn, n=30, warm=5):
             for i in range(warm):
@@ -292,9 +350,14 @@ def main():
                                                                  out_codes=o[i % RING][0], out_scales=o[i % RING][1]))
                 by = bytes_per_token(D_HEAD, f, grp) * T_HEAD
                 gbs = by / (ms * 1e-3) / 1e9
-                sweep.append({"call": "perq_rotate_quantize", "T": T_HEAD, "d": D_HEAD, "b": bb, "fmt": f, "group": grp,
-                              "ms": ms, "GB/s": gbs, "frac_of_" + peak_kind: gbs / peak,
-                              "frac_of_nominal_8TBs": gbs / NOMINAL_HBM_GBS, "Mtokens/s": T_HEAD / ms / 1e3})
+                row = {"call": "perq_rotate_quantize", "T": T_HEAD, "d": D_HEAD, "b": bb, "fmt": f, "group": grp,
+                       "ms": ms, "GB/s": gbs, "frac_of_" + peak_kind: gbs / peak,
+                       "frac_of_nominal_8TBs": gbs / NOMINAL_HBM_GBS, "Mtokens/s": T_HEAD / ms / 1e3}
+                if check_rows is not None:
+                    B.perq_rotate_quantize(xs[0], None, bb, fcode, grp, out_codes=o[0][0], out_scales=o[0][1])
+                    torch.cuda.synchronize()
+                    row.update(check_rows(xs[0], None, bb, f, grp, o[0][0], o[0][1]))
+                sweep.append(row)
             del o
         # the calibration statistic on the MLP down-projection shape (T=4096 x d=8192, b=32)
         w3 = inputs.config3(T=4096)
@@ -339,6 +402,10 @@ def main():
                 row["us_graph_replay"] = gms * 1e3
                 row["GB/s_graph_replay"] = by / (gms * 1e-3) / 1e9
                 del graph
+            if check_rows is not None:
+                B.perq_rotate_quantize(xr[0], pd, b, fcode, grp, out_codes=orr[0][0], out_scales=orr[0][1])
+                torch.cuda.synchronize()
+                row.update(check_rows(xr[0], perm, b, f, grp, orr[0][0], orr[0][1]))
             sweep.append(row)
 
         w1 = inputs.config1()
@@ -362,8 +429,6 @@ def main():
 
     cpu_baseline = None
     if not args.no_cpu_baseline:
-        from oracle import perq_oracle
-        perq_oracle.build()
         rows = 4096
         wb = inputs.config4(T=rows, b=B_HEAD, fmt=FMT_HEAD)
         perq_oracle.rotate_quantize(wb.x[:256], None, B_HEAD, ORACLE_FMT[FMT_HEAD], GROUP_HEAD)

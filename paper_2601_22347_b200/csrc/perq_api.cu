@@ -204,7 +204,7 @@ int launch_fast_long(int xb, int G, const perq::FastParams &p, int grid, cudaStr
     }
 }
 
-// Lean per-token kernel: INT4 or E2M1 with one scale per token, unpermuted, d in {1024, 2048, 4096, 8192}, b <= 128.
+// Lean per-token kernel: INT4 or E2M1 with one scale per token, unpermuted, d in {2048, 4096, 8192}, b <= 128.
 template <int LOG2B, int MODE, int LOG2G>
 int launch_tok_inst(const perq::FastParams &p, int grid, cudaStream_t st)
 {
@@ -226,13 +226,12 @@ int launch_tok_b(int log2b, const perq::FastParams &p, int grid, cudaStream_t st
 }
 
 template <int MODE>
-int launch_tok(int G, int log2b, const perq::FastParams &p, int grid, cudaStream_t st)
+int launch_tok(int segs, int log2b, const perq::FastParams &p, int grid, cudaStream_t st)
 {
-    switch (G) {
-    case 1: return launch_tok_b<MODE, 0>(log2b, p, grid, st);
-    case 2: return launch_tok_b<MODE, 1>(log2b, p, grid, st);
-    case 4: return launch_tok_b<MODE, 2>(log2b, p, grid, st);
-    default: return launch_tok_b<MODE, 3>(log2b, p, grid, st);
+    switch (segs) {                                      // two segments per warp
+    case 2: return launch_tok_b<MODE, 0>(log2b, p, grid, st);
+    case 4: return launch_tok_b<MODE, 1>(log2b, p, grid, st);
+    default: return launch_tok_b<MODE, 2>(log2b, p, grid, st);
     }
 }
 
@@ -290,9 +289,12 @@ int try_launch_fast(const void *x, const int32_t *perm, int64_t T, int32_t d, in
     const long long want = (units + groups_per_cta - 1) / groups_per_cta;
     const int grid = (int)std::min<long long>(want, sms);
     if ((mode == perq::MODE_TOKEN || mode == perq::MODE_FP4) && !permuted && !full && !longb &&
-        (segs == 1 || segs == 2 || segs == 4 || segs == 8))
-        return mode == perq::MODE_TOKEN ? launch_tok<perq::MODE_TOKEN>(segs, ilog2(b), p, grid, st)
-                                        : launch_tok<perq::MODE_FP4>(segs, ilog2(b), p, grid, st);
+        (segs == 2 || segs == 4 || segs == 8)) {
+        const int tok_groups = perq::FAST_WARPS / (segs / perq::TOK_SPW);       // rows in flight per CTA
+        const int tok_grid = (int)std::min<long long>((T + tok_groups - 1) / tok_groups, sms);
+        return mode == perq::MODE_TOKEN ? launch_tok<perq::MODE_TOKEN>(segs, ilog2(b), p, tok_grid, st)
+                                        : launch_tok<perq::MODE_FP4>(segs, ilog2(b), p, tok_grid, st);
+    }
     if (full)
         return mode == perq::MODE_MX ? launch_fast_full<perq::MODE_MX>(G, p, grid, st)
                                      : launch_fast_full<perq::MODE_TOKEN>(G, p, grid, st);

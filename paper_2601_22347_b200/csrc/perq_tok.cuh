@@ -1,11 +1,16 @@
-// Per-token rotate+quantize kernel with a lean inner loop: unpermuted rows of d = G * 1024 channels
-// (G in {1, 2, 4, 8}), Hadamard blocks of 16 .. 128, symmetric INT4 or E2M1 codes with one fp32 scale per
-// token.  Same data path, lane layout, error model and exactness rules as perq_fast.cuh (whose helpers it
+// Per-token rotate+quantize kernel with a lean inner loop: unpermuted rows of d = 2048, 4096 or 8192
+// channels, Hadamard blocks of 16 .. 128, symmetric INT4 or E2M1 codes with one fp32 scale per token.  Same data path, lane layout, error model and exactness rules as perq_fast.cuh (whose helpers it
 // uses); what differs is where the rare work lives, because this kernel is bound by the number of warp
 // instructions an iteration issues (measured: about 0.15 us of a 16384 x 4096 call per instruction and
 // 1024-element segment), and because the G warps of a row move in lockstep (one named barrier per row), so
 // work that only one of them does delays all of them:
 //
+//   * A warp owns two adjacent 1024-element segments of a row, and a row is shared by W = d / 2048 warps.
+//     What an iteration costs once -- the wait for the staged row, the exchange of maxima around the row's
+//     named barrier, the refill of the ring, the fence and the bulk store of the packed codes, the loop's
+//     own bookkeeping: about a hundred instructions -- is paid per two segments.  The first segment's rotated
+//     values are not kept while the second one's maximum is formed: it is rotated again (28 instructions)
+//     after the second one is quantised.
 //   * The warps of a row share nothing but their fp32 maxima (one 4-byte word each, exchanged around the
 //     row's named barrier).  The warp that holds the row maximum pins it to one lane and one pair of slots
 //     (8 outputs) from the four pair maxima it has anyway, and appends a record; the exact scale is derived
@@ -21,16 +26,21 @@
 
 namespace perq {
 
+constexpr int TOK_SPW = 2;                    // adjacent segments of a row per warp
+constexpr int TOK_NSTAGE = 3;                 // ring stages (rows) per group of warps
+
+// Shared memory, relative to a 1024-byte aligned base: 16 warps x 3 stages x 2 segments of 2 KB, one 1 KB
+// code staging buffer per warp, the ring's mbarriers, the warp maxima, the deferred scale records.
 struct TokSmem {
-    static constexpr size_t stages = 0;                                                  // 16 warps x 4 stages x 2 KB
-    static constexpr size_t codes = stages + (size_t)FAST_WARPS * FAST_NSTAGE * SEG_BYTES;   // 2 x 512 B per warp
-    static constexpr size_t full = codes + (size_t)FAST_WARPS * 2 * SEG_CODE_BYTES;      // [groups][4] mbarriers
-    static constexpr size_t xch = full + (size_t)FAST_WARPS * FAST_NSTAGE * 8;           // [2][16] fp32 warp maxima (8 bytes apart)
-    static constexpr size_t wreq = xch + (size_t)2 * FAST_WARPS * 8;                     // [16][32] u64 deferred scale records
-    static constexpr size_t used = wreq + (size_t)FAST_WARPS * 32 * 8;
+    static constexpr size_t stages = 0;
+    static constexpr size_t codes = stages + (size_t)FAST_WARPS * TOK_NSTAGE * TOK_SPW * SEG_BYTES;
+    static constexpr size_t full = codes + (size_t)FAST_WARPS * TOK_SPW * SEG_CODE_BYTES;
+    static constexpr size_t xch = full + (size_t)FAST_WARPS * TOK_NSTAGE * 8;            // [2][16] fp32 warp maxima (8 bytes apart)
+    static constexpr size_t wreq = xch + (size_t)2 * FAST_WARPS * 8;                     // [16][16] u64 deferred scale records
+    static constexpr size_t used = wreq + (size_t)FAST_WARPS * 16 * 8;
     static constexpr size_t total = used + 1024;                                         // room to align the base
 };
-
+constexpr uint32_t TOK_MAX_RECORDS = 16;
 
 // Per-lane constants of the data layout (see perq_fast.cuh): Hadamard operand of the tensor-core stage,
 // ldmatrix source offset, position of the lane's code piece, relabelling signs.
@@ -208,28 +218,28 @@ __device__ __noinline__ void tok_serve_records(const uint16_t *x, float *out_sca
 }
 
 // The exact largest magnitude of a staged row (bit pattern of a non-negative double, the same in every
-// lane), by one warp: every segment whose fp32 maximum is within the error bound of the row's is rotated
-// again and its candidate slots are evaluated in fp64 from the bf16 inputs.  xch holds the G fp32 warp
-// maxima of the row (G = 1: pass nullptr; the row is the segment).  Rare: rows whose maximum is not pinned
-// to one pair of slots, and warps that need the exact maximum for a fix-up.
-template <int LOG2B, int LOG2G>
+// lane), by one warp: every segment of a warp whose fp32 maximum is within the error bound of the row's is
+// rotated again and its candidate slots are evaluated in fp64 from the bf16 inputs.  xch holds the fp32
+// maxima of the row's W warps, 8 bytes apart (W = 1: not read); a warp owns TOK_SPW adjacent segments.
+// Rare: rows whose maximum is not pinned to one pair of slots, and warps that need the exact maximum for
+// a fix-up.
+template <int LOG2B, int LOG2W>
 __device__ __noinline__ unsigned long long tok_row_exact_max(uint32_t row_addr, const uint16_t *raw_row, const uint32_t *xch,
-                                                             float a32, float thr_row, int lane)
+                                                             float thr_row, int lane)
 {
-    constexpr int G = 1 << LOG2G;
+    constexpr int W = 1 << LOG2W;
     TokLane<LOG2B> L;
     L.init(lane);
     unsigned long long best = 0ull;
 #pragma unroll 1
-    for (int w = 0; w < G; ++w) {
-        const float am = (G > 1) ? __uint_as_float(xch[2 * w]) : a32;
-        if (!(am >= thr_row)) continue;
+    for (int sgm = 0; sgm < W * TOK_SPW; ++sgm) {
+        if (W > 1 && !(__uint_as_float(xch[2 * (sgm / TOK_SPW)]) >= thr_row)) continue;
         f32x2 v[8][2];
-        tok_rotate<LOG2B>(row_addr + (uint32_t)w * SEG_BYTES, L, v);
+        tok_rotate<LOG2B>(row_addr + (uint32_t)sgm * SEG_BYTES, L, v);
         float ms[8];
 #pragma unroll
         for (int s = 0; s < 8; ++s) ms[s] = fmaxf(max3abs(fabsf(v[s][0].x), v[s][0].y, v[s][1].x), fabsf(v[s][1].y));
-        const unsigned long long wb = exact_max_of_candidates<LOG2B, 0>(raw_row + (size_t)w * SEG_ELEMS, 0, ms, thr_row, lane);
+        const unsigned long long wb = exact_max_of_candidates<LOG2B, 0>(raw_row + (size_t)sgm * SEG_ELEMS, 0, ms, thr_row, lane);
         best = wb > best ? wb : best;
     }
     return best;
@@ -238,14 +248,14 @@ __device__ __noinline__ unsigned long long tok_row_exact_max(uint32_t row_addr, 
 // Exact resolution of the elements whose two-sided rounding test failed (rare).  The rotated values and
 // the two code sets are formed again from the staged segment; the exact row maximum, unless this warp has it
 // already (known), is derived from the staged row.
-template <int LOG2B, int MODE, int LOG2G>
+template <int LOG2B, int MODE, int LOG2W>
 __device__ __noinline__ void tok_fix_ties(uint32_t seg_addr, const uint16_t *seg, uint32_t row_addr, const uint16_t *raw_row,
                                           const uint32_t *xch, uint8_t *code_gen, float inv, float a32, float thr_row,
                                           double sqrt_b, bool known, unsigned long long a_bits, int lane)
 {
     constexpr int B = 1 << LOG2B;
     constexpr int PM = (1 << (LOG2B - 4)) - 1;
-        constexpr float MAGIC = 12582920.0f;
+    constexpr float MAGIC = 12582920.0f;
     const float err_rel = FAST_ERR_K * (float)LOG2B * TWO_M24;
     auto over_sqrt_b = [&](double u) -> double {
         return (LOG2B % 2 == 0) ? u * (1.0 / (double)(1 << (LOG2B / 2))) : u / sqrt_b;
@@ -286,7 +296,7 @@ __device__ __noinline__ void tok_fix_ties(uint32_t seg_addr, const uint16_t *seg
     }
     // the exact row maximum (sign-only fix-ups of E2M1 codes do not need it)
     const bool need_scale = (MODE != MODE_FP4) || __any_sync(0xffffffffu, (fm & ~zm) != 0u);
-    if (need_scale && !known) a_bits = tok_row_exact_max<LOG2B, LOG2G>(row_addr, raw_row, xch, a32, thr_row, lane);
+    if (need_scale && !known) a_bits = tok_row_exact_max<LOG2B, LOG2W>(row_addr, raw_row, xch, thr_row, lane);
     const double a_src = __longlong_as_double((long long)a_bits);
     __syncwarp();
     double s_row = 0.0;
@@ -338,36 +348,38 @@ __device__ __noinline__ void tok_fix_ties(uint32_t seg_addr, const uint16_t *seg
     }
 }
 
-template <int LOG2B, int MODE, int LOG2G>
+template <int LOG2B, int MODE, int LOG2W>
 __global__ void __launch_bounds__(FAST_THREADS, 1) perq_tok_kernel(FastParams p)
 {
     static_assert(MODE == MODE_TOKEN || MODE == MODE_FP4, "one scale per token");
-    static_assert(LOG2B >= 4 && LOG2B <= 7 && LOG2G >= 0 && LOG2G <= 3, "blocks inside a segment, rows of 1, 2, 4 or 8 segments");
-    constexpr int G = 1 << LOG2G;
-    constexpr int GROUPS = FAST_WARPS / G;
+    static_assert(LOG2B >= 4 && LOG2B <= 7 && LOG2W >= 0 && LOG2W <= 2, "blocks inside a segment, rows of 2, 4 or 8 segments");
+    constexpr int W = 1 << LOG2W;                 // warps per row
+    constexpr int GROUPS = FAST_WARPS / W;
     constexpr int PM = (1 << (LOG2B - 4)) - 1;
     constexpr int NCLS = (PM & 3) + 1;
-    constexpr int NST = FAST_NSTAGE;
-    constexpr uint32_t UNIT_BYTES = (uint32_t)G * SEG_BYTES;
+    constexpr int NST = TOK_NSTAGE;
+    constexpr uint32_t UNIT_BYTES = (uint32_t)(W * TOK_SPW) * SEG_BYTES;
+    constexpr uint32_t UNIT_ELEMS = (uint32_t)(W * TOK_SPW) * SEG_ELEMS;
     constexpr float MAGIC = 12582920.0f;          // 1.5 * 2^23 + 8: low nibble of the sum = code + 8
     extern __shared__ __align__(128) unsigned char tsmem_raw[];
     unsigned char *tsmem = tsmem_raw + ((1024u - (smem_u32(tsmem_raw) & 1023u)) & 1023u);
 
     const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
-    const int group = warp >> LOG2G;
+    const int group = warp >> LOG2W;
     // position in the row, rotated by the group index (the same position of every row tends to do the per-row
     // extra work; warps go to the four schedulers by warp index)
-    const int w_in_g = (warp + group) & (G - 1);
+    const int w_in_g = (warp + group) & (W - 1);
     const float err_rel = FAST_ERR_K * (float)LOG2B * TWO_M24;
     const float thr_factor = 1.0f - 2.0f * err_rel - 2.4e-7f;
     const float delta = 16.0f * err_rel + 5.0e-7f;
 
     const uint32_t smem_base = smem_u32(tsmem);
     const uint32_t stage_base = smem_base + (uint32_t)TokSmem::stages + (uint32_t)group * (NST * UNIT_BYTES);
-    const uint32_t seg_base = stage_base + (uint32_t)w_in_g * SEG_BYTES;
+    const uint32_t seg_base = stage_base + (uint32_t)w_in_g * (TOK_SPW * SEG_BYTES);
     const uint32_t full_base = smem_base + (uint32_t)TokSmem::full + (uint32_t)group * (NST * 8);
-    const uint32_t xch_group = smem_base + (uint32_t)TokSmem::xch + (uint32_t)(group * G) * 8;
-    unsigned long long *wreq = reinterpret_cast<unsigned long long *>(tsmem + TokSmem::wreq) + warp * 32;
+    const uint32_t code_buf = smem_base + (uint32_t)TokSmem::codes + (uint32_t)warp * (TOK_SPW * SEG_CODE_BYTES);
+    const uint32_t xch_group = smem_base + (uint32_t)TokSmem::xch + (uint32_t)(group * W) * 8;
+    unsigned long long *wreq = reinterpret_cast<unsigned long long *>(tsmem + TokSmem::wreq) + warp * TOK_MAX_RECORDS;
 
     if (tid < FAST_WARPS * NST) mbar_init(smem_base + (uint32_t)TokSmem::full + tid * 8, 1);
     if (tid == 0) asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
@@ -377,7 +389,7 @@ __global__ void __launch_bounds__(FAST_THREADS, 1) perq_tok_kernel(FastParams p)
     const uint32_t stride = gridDim.x * GROUPS;
     if (first >= p.units_total) return;          // whole groups leave together
     const uint32_t n_units = (p.units_total - first + stride - 1) / stride;
-    const uint32_t refill_end = n_units > (uint32_t)NST ? n_units - NST : 0u;     // iterations 1 .. refill_end load a unit
+    const uint32_t refill_end = n_units > (uint32_t)NST ? n_units - NST : 0u;     // iterations 1 .. refill_end load a row
     const bool leader = (w_in_g == 0) && (lane == 0);
 
     TokLane<LOG2B> L;
@@ -389,10 +401,10 @@ __global__ void __launch_bounds__(FAST_THREADS, 1) perq_tok_kernel(FastParams p)
     for (int c = 0; c < NCLS; ++c) { cp[c] = L.sgn[c] * (1.0f + delta); cm[c] = L.sgn[c] * (1.0f - delta); }
 
     // running addresses
-    const size_t unit_step_elems = (size_t)stride * (G * SEG_ELEMS);
-    const uint16_t *xload = p.x + (size_t)first * (G * SEG_ELEMS);             // leader: source of the next unit to load
-    uint8_t *outp = p.out_codes + ((size_t)first * G + w_in_g) * SEG_CODE_BYTES;
-    const size_t out_step = (size_t)stride * G * SEG_CODE_BYTES;
+    const size_t unit_step_elems = (size_t)stride * UNIT_ELEMS;
+    const uint16_t *xload = p.x + (size_t)first * UNIT_ELEMS;                  // leader: source of the next row to load
+    uint8_t *outp = p.out_codes + ((size_t)first * (W * TOK_SPW) + (size_t)w_in_g * TOK_SPW) * SEG_CODE_BYTES;
+    const size_t out_step = (size_t)stride * (W * TOK_SPW) * SEG_CODE_BYTES;
     float *scales = reinterpret_cast<float *>(p.out_scales);
     if (leader) {
 #pragma unroll
@@ -404,25 +416,11 @@ __global__ void __launch_bounds__(FAST_THREADS, 1) perq_tok_kernel(FastParams p)
             }
         }
     }
-    // this iteration's code staging buffer and exchange words: they alternate
-    uint32_t code_buf = smem_base + (uint32_t)TokSmem::codes + (uint32_t)warp * (2 * SEG_CODE_BYTES);
-    uint32_t xch_it = xch_group;
+    uint32_t xch_it = xch_group;                 // this iteration's exchange words: two sets alternate
+    uint32_t stage = 0, parity = 0;              // ring position of this iteration
 
-    uint32_t nreq = 0;                           // records waiting in wreq (the same in every lane)
-    uint32_t unit = first;
-    bool ok = true;
-    for (uint32_t it = 0; it < n_units; ++it, unit += stride, outp += out_step, code_buf ^= SEG_CODE_BYTES, xch_it ^= FAST_WARPS * 8) {
-        const uint32_t stage = it & (NST - 1);
-        const uint32_t bar = full_base + stage * 8, parity = (it / NST) & 1u;
-        if (!mbar_try_once(bar, parity) && !mbar_wait(bar, parity)) { ok = false; break; }
-        const uint32_t row_addr = stage_base + stage * UNIT_BYTES;
-        const uint32_t seg_addr = seg_base + stage * UNIT_BYTES;
-
-        f32x2 v[8][2];
-        tok_rotate<LOG2B>(seg_addr, L, v);
-
-        // ---- magnitude maxima of the four slot pairs, of the lane, of the warp, of the row
-        float gm[4];
+    // magnitude maxima of the four slot pairs of a segment's rotated values
+    auto pair_maxima = [&](const f32x2 (&v)[8][2], float (&gm)[4]) {
 #pragma unroll
         for (int m = 0; m < 4; ++m) {
             float a = max3abs(fabsf(v[2 * m][0].x), v[2 * m][0].y, v[2 * m][1].x);
@@ -430,88 +428,15 @@ __global__ void __launch_bounds__(FAST_THREADS, 1) perq_tok_kernel(FastParams p)
             a = max3abs(a, v[2 * m + 1][0].y, v[2 * m + 1][1].x);
             gm[m] = fmaxf(a, fabsf(v[2 * m + 1][1].y));
         }
-        const float lane_max = fmaxf(fmaxf(gm[0], gm[1]), fmaxf(gm[2], gm[3]));
-        const float aw = warp_max_f32(lane_max);
-        float a32 = aw;
-        if (G > 1) {
-            if (lane == 0) asm volatile("st.shared.b32 [%0], %1;" ::"r"(xch_it + (uint32_t)w_in_g * 8), "r"(__float_as_uint(aw)) : "memory");
-            named_barrier(1 + group, G * 32);
-            uint32_t am_bits;
-            asm volatile("ld.shared.b32 %0, [%1];" : "=r"(am_bits) : "r"(xch_it + (uint32_t)(lane & (G - 1)) * 8) : "memory");
-            a32 = warp_max_f32(__uint_as_float(am_bits));          // (every lane reads one of the row's G words)
-        }
-        // every warp of the group is past the stage of the previous iteration: lane 0 of the first warp refills it
-        {
-            const uint32_t ps = (it - 1u) & (NST - 1);
-            const bool go = leader && (it - 1u < refill_end);     // it >= 1 and unit it + NST - 1 exists (it - 1 wraps for it == 0)
-            bulk_load_if(go, stage_base + ps * UNIT_BYTES, xload, UNIT_BYTES, full_base + ps * 8);
-            if (go) xload += unit_step_elems;
-        }
-        const float thr_row = a32 * thr_factor;
-
-        // ---- the warp that holds the row maximum: pin it to one lane and one pair of slots, record it
-        bool known = !(a32 > 0.0f);              // this warp holds the exact row maximum in a_bits
-        unsigned long long a_bits = 0ull;
-        if (aw >= thr_row) {
-            if (a32 > 0.0f) {
-                bool pinned = false;
-                if (G == 1 || aw == a32) {       // (ties between warps and near ties take the general path below)
-                    const unsigned cl = __ballot_sync(0xffffffffu, lane_max >= thr_row);
-                    const uint32_t c0 = gm[0] >= thr_row ? 1u : 0u, c1 = gm[1] >= thr_row ? 1u : 0u;
-                    const uint32_t c2 = gm[2] >= thr_row ? 1u : 0u, c3 = gm[3] >= thr_row ? 1u : 0u;
-                    const int src = __ffs(cl) - 1;
-                    const uint32_t packed = __shfl_sync(0xffffffffu, (c1 + 2u * c2 + 3u * c3) | ((c0 + c1 + c2 + c3) << 4), src & 31);
-                    bool alone = (cl & (cl - 1)) == 0u && (packed >> 4) == 1u;
-                    if (G > 1) {                 // no other warp of the row within the bound
-                        uint32_t ob;
-                        asm volatile("ld.shared.b32 %0, [%1];" : "=r"(ob) : "r"(xch_it + (uint32_t)(lane & (G - 1)) * 8) : "memory");
-                        alone = alone && __popc(__ballot_sync(0xffffffffu, lane < G && __uint_as_float(ob) >= thr_row)) == 1;
-                    }
-                    if (alone) {
-                        // slots 2m, 2m+1 of lane group sg are the chunks 8 sg + ((2m, 2m+1) ^ relabelling): one aligned pair
-                        const uint32_t sg = (uint32_t)src >> 2, m = packed & 3u;
-                        const uint32_t chunk = sg * 8 + (((2 * m) ^ (sg & 3u & ~(uint32_t)PM)) & ~1u);
-                        const uint32_t pos = (uint32_t)(w_in_g * SEG_ELEMS) + chunk * 16 + 4 * ((uint32_t)src & 3u);
-                        if (lane == 0) wreq[nreq] = ((unsigned long long)unit << 32) | pos;
-                        if (++nreq == 32u) {
-                            tok_serve_records<LOG2B>(p.x, scales, p.d, p.inv_7_sqrt_b, wreq, nreq, lane);
-                            nreq = 0;
-                        }
-                        pinned = true;
-                    }
-                }
-                if (!pinned) {
-                    // several candidates: the first warp of the row that is within the bound derives the exact
-                    // maximum of the whole row and stores the scale
-                    bool mine = true;
-                    if (G > 1) {
-                        uint32_t ob;
-                        asm volatile("ld.shared.b32 %0, [%1];" : "=r"(ob) : "r"(xch_it + (uint32_t)(lane & (G - 1)) * 8) : "memory");
-                        const unsigned cw = __ballot_sync(0xffffffffu, lane < G && __uint_as_float(ob) >= thr_row);
-                        mine = (__ffs(cw) - 1) == w_in_g;
-                    }
-                    if (mine) {
-                        const uint16_t *raw_row = reinterpret_cast<const uint16_t *>(tsmem + TokSmem::stages) + (row_addr - smem_base - (uint32_t)TokSmem::stages) / 2;
-                        a_bits = tok_row_exact_max<LOG2B, LOG2G>(row_addr, raw_row, reinterpret_cast<const uint32_t *>(tsmem + TokSmem::xch) + (xch_it - smem_base - (uint32_t)TokSmem::xch) / 4,
-                                                                 a32, thr_row, lane);
-                        known = true;
-                        if (lane == 0) scales[unit] = (a_bits == 0ull) ? 0.0f : (float)(__longlong_as_double((long long)a_bits) * p.inv_7_sqrt_b);
-                    }
-                }
-            } else if (leader) {
-                scales[unit] = 0.0f;             // a zero row
-            }
-        }
-
-        // ---- quantise: packed fp32 multiply-add against the magic constant, with the multiplier nudged up and
-        // down by the error bound (E2M1: the scaled value plus and minus an additive window, converted twice)
-        const float inv = (a32 > 0.0f) ? fminf(__fdividef(7.0f, a32), 3.0e38f) : 0.0f;
-        const uint32_t code_addr0 = code_buf + L.code_lane;
-        bulk_store_wait_read<1>();           // the store that last read this staging buffer has drained
-        __syncwarp();
+    };
+    // Quantise a segment's rotated values into the staging buffer at code_addr0 (+ this lane's offset):
+    // packed fp32 multiply-add against the magic constant, with the multiplier nudged up and down by the
+    // error bound (E2M1: the scaled value plus and minus an additive window, converted twice).  Returns the
+    // OR of the differences between the two code sets.
+    auto quantise = [&](const f32x2 (&v)[8][2], float inv, uint32_t code_addr0) -> uint32_t {
         uint32_t tie_any = 0u;
         if (MODE == MODE_FP4) {
-            const float tau = (a32 > 0.0f) ? 8.0f * err_rel + 4.0e-6f : 0.0f;
+            const float tau = (inv > 0.0f) ? 8.0f * err_rel + 4.0e-6f : 0.0f;
             const f32x2 tau_p2 = pack2(tau, tau), tau_m2 = pack2(-tau, -tau);
             f32x2 mul_c[NCLS];
 #pragma unroll
@@ -548,21 +473,133 @@ __global__ void __launch_bounds__(FAST_THREADS, 1) perq_tok_kernel(FastParams p)
                 sts_code<(3 & ~PM)>(code_addr0, s, pp ^ 0x8888u);
             }
         }
-        if (__any_sync(0xffffffffu, (tie_any & 0xffffu) != 0u)) {
+        return tie_any & 0xffffu;
+    };
+
+    uint32_t nreq = 0;                           // records waiting in wreq (the same in every lane)
+    uint32_t unit = first;
+    bool ok = true;
+    for (uint32_t it = 0; it < n_units; ++it, unit += stride, outp += out_step, xch_it ^= FAST_WARPS * 8) {
+        const uint32_t bar = full_base + stage * 8;
+        if (!mbar_try_once(bar, parity) && !mbar_wait(bar, parity)) { ok = false; break; }
+        const uint32_t row_addr = stage_base + stage * UNIT_BYTES;
+        const uint32_t seg_addr = seg_base + stage * UNIT_BYTES;          // this warp's first segment; the second follows
+
+        // ---- first segment: pair maxima only; second segment: its rotated values stay
+        f32x2 v[8][2];
+        float gm[2][4];
+        tok_rotate<LOG2B>(seg_addr, L, v);
+        pair_maxima(v, gm[0]);
+        tok_rotate<LOG2B>(seg_addr + SEG_BYTES, L, v);
+        pair_maxima(v, gm[1]);
+        // (a tournament, whose intermediate winners the candidate warp uses again below)
+        const float q0 = fmaxf(gm[0][0], gm[0][1]), q1 = fmaxf(gm[0][2], gm[0][3]);
+        const float q2 = fmaxf(gm[1][0], gm[1][1]), q3 = fmaxf(gm[1][2], gm[1][3]);
+        const float s0 = fmaxf(q0, q1), s1 = fmaxf(q2, q3);
+        const float lane_max = fmaxf(s0, s1);
+        const float aw = warp_max_f32(lane_max);
+        float a32 = aw;
+        if (W > 1) {
+            if (lane == 0) asm volatile("st.shared.b32 [%0], %1;" ::"r"(xch_it + (uint32_t)w_in_g * 8), "r"(__float_as_uint(aw)) : "memory");
+            named_barrier(1 + group, W * 32);
+            uint32_t am_bits;
+            asm volatile("ld.shared.b32 %0, [%1];" : "=r"(am_bits) : "r"(xch_it + (uint32_t)(lane & (W - 1)) * 8) : "memory");
+            a32 = warp_max_f32(__uint_as_float(am_bits));          // (every lane reads one of the row's W words)
+        }
+        // every warp of the group is past the stage of the previous iteration: lane 0 of the first warp refills it
+        if (w_in_g == 0) {
+            const uint32_t ps = stage == 0 ? (uint32_t)(NST - 1) : stage - 1u;
+            const bool go = (lane == 0) && (it - 1u < refill_end);     // it >= 1 and row it + NST - 1 exists (it - 1 wraps for it == 0)
+            bulk_load_if(go, stage_base + ps * UNIT_BYTES, xload, UNIT_BYTES, full_base + ps * 8);
+            if (go) xload += unit_step_elems;
+        }
+        const float thr_row = a32 * thr_factor;
+
+        // ---- the warp that holds the row maximum: pin it to one lane and one pair of slots, record it
+        bool known = !(a32 > 0.0f);              // this warp holds the exact row maximum in a_bits
+        unsigned long long a_bits = 0ull;
+        if (aw >= thr_row) {
+            if (a32 > 0.0f) {
+                bool pinned = false;
+                if (W == 1 || aw == a32) {       // (ties between warps and near ties take the general path below)
+                    const unsigned cl = __ballot_sync(0xffffffffu, lane_max >= thr_row);
+                    // the largest of the tournament's seven losers is the lane's second largest pair maximum
+                    const float r01 = fmaxf(fminf(gm[0][0], gm[0][1]), fminf(gm[0][2], gm[0][3]));
+                    const float r23 = fmaxf(fminf(gm[1][0], gm[1][1]), fminf(gm[1][2], gm[1][3]));
+                    const float second = fmaxf(fmaxf(r01, r23), fmaxf(fmaxf(fminf(q0, q1), fminf(q2, q3)), fminf(s0, s1)));
+                    // index 4h + m of the one pair maximum that reaches the bound (meaningless if there are several)
+                    const uint32_t idx = (s1 >= thr_row ? 4u : 0u) | ((q1 >= thr_row || q3 >= thr_row) ? 2u : 0u) |
+                                         ((gm[0][1] >= thr_row || gm[0][3] >= thr_row || gm[1][1] >= thr_row || gm[1][3] >= thr_row) ? 1u : 0u);
+                    const int src = __ffs(cl) - 1;
+                    const uint32_t packed = __shfl_sync(0xffffffffu, idx | (second < thr_row ? 16u : 0u), src & 31);
+                    bool alone = (cl & (cl - 1)) == 0u && (packed >> 4) == 1u;
+                    if (W > 1) {                 // no other warp of the row within the bound
+                        uint32_t ob;
+                        asm volatile("ld.shared.b32 %0, [%1];" : "=r"(ob) : "r"(xch_it + (uint32_t)(lane & (W - 1)) * 8) : "memory");
+                        alone = alone && __popc(__ballot_sync(0xffffffffu, lane < W && __uint_as_float(ob) >= thr_row)) == 1;
+                    }
+                    if (alone) {
+                        // slots 2m, 2m+1 of lane group sg are the chunks 8 sg + ((2m, 2m+1) ^ relabelling): one aligned pair
+                        const uint32_t sg = (uint32_t)src >> 2, m = packed & 3u, h = (packed >> 2) & 1u;
+                        const uint32_t chunk = sg * 8 + (((2 * m) ^ (sg & 3u & ~(uint32_t)PM)) & ~1u);
+                        const uint32_t pos = (uint32_t)(w_in_g * TOK_SPW + h) * SEG_ELEMS + chunk * 16 + 4 * ((uint32_t)src & 3u);
+                        if (lane == 0) wreq[nreq] = ((unsigned long long)unit << 32) | pos;
+                        if (++nreq == TOK_MAX_RECORDS) {
+                            tok_serve_records<LOG2B>(p.x, scales, p.d, p.inv_7_sqrt_b, wreq, nreq, lane);
+                            nreq = 0;
+                        }
+                        pinned = true;
+                    }
+                }
+                if (!pinned) {
+                    // several candidates: the first warp of the row that is within the bound derives the exact
+                    // maximum of the whole row and stores the scale
+                    bool mine = true;
+                    if (W > 1) {
+                        uint32_t ob;
+                        asm volatile("ld.shared.b32 %0, [%1];" : "=r"(ob) : "r"(xch_it + (uint32_t)(lane & (W - 1)) * 8) : "memory");
+                        const unsigned cw = __ballot_sync(0xffffffffu, lane < W && __uint_as_float(ob) >= thr_row);
+                        mine = (__ffs(cw) - 1) == w_in_g;
+                    }
+                    if (mine) {
+                        const uint16_t *raw_row = reinterpret_cast<const uint16_t *>(tsmem + TokSmem::stages) + (row_addr - smem_base - (uint32_t)TokSmem::stages) / 2;
+                        a_bits = tok_row_exact_max<LOG2B, LOG2W>(row_addr, raw_row, reinterpret_cast<const uint32_t *>(tsmem + TokSmem::xch) + (xch_it - smem_base - (uint32_t)TokSmem::xch) / 4,
+                                                                 thr_row, lane);
+                        known = true;
+                        if (lane == 0) scales[unit] = (a_bits == 0ull) ? 0.0f : (float)(__longlong_as_double((long long)a_bits) * p.inv_7_sqrt_b);
+                    }
+                }
+            } else if (leader) {
+                scales[unit] = 0.0f;             // a zero row
+            }
+        }
+
+        // ---- quantise the second segment (its values are live), rotate the first one again, quantise it
+        const float inv = (a32 > 0.0f) ? fminf(__fdividef(7.0f, a32), 3.0e38f) : 0.0f;
+        bulk_store_wait_read<0>();           // the store of the previous iteration has read the staging buffer
+        __syncwarp();
+        const uint32_t tie1 = quantise(v, inv, code_buf + SEG_CODE_BYTES + L.code_lane);
+        tok_rotate<LOG2B>(seg_addr, L, v);
+        const uint32_t tie0 = quantise(v, inv, code_buf + L.code_lane);
+        if (__any_sync(0xffffffffu, (tie0 | tie1) != 0u)) {
             const uint16_t *stage_gen = reinterpret_cast<const uint16_t *>(tsmem + TokSmem::stages);
             const uint16_t *seg = stage_gen + (seg_addr - smem_base - (uint32_t)TokSmem::stages) / 2;
             const uint16_t *raw_row = stage_gen + (row_addr - smem_base - (uint32_t)TokSmem::stages) / 2;
             uint8_t *code_gen = tsmem + TokSmem::codes + (code_buf - smem_base - (uint32_t)TokSmem::codes);
+            const uint32_t *xw = reinterpret_cast<const uint32_t *>(tsmem + TokSmem::xch) + (xch_it - smem_base - (uint32_t)TokSmem::xch) / 4;
             __syncwarp();
-            tok_fix_ties<LOG2B, MODE, LOG2G>(seg_addr, seg, row_addr, raw_row,
-                                             reinterpret_cast<const uint32_t *>(tsmem + TokSmem::xch) + (xch_it - smem_base - (uint32_t)TokSmem::xch) / 4,
-                                             code_gen, inv, a32, thr_row, p.sqrt_b, known, a_bits, lane);
+            if (__any_sync(0xffffffffu, tie0 != 0u))
+                tok_fix_ties<LOG2B, MODE, LOG2W>(seg_addr, seg, row_addr, raw_row, xw, code_gen, inv, a32, thr_row, p.sqrt_b, known, a_bits, lane);
+            if (__any_sync(0xffffffffu, tie1 != 0u))
+                tok_fix_ties<LOG2B, MODE, LOG2W>(seg_addr + SEG_BYTES, seg + SEG_ELEMS, row_addr, raw_row, xw, code_gen + SEG_CODE_BYTES, inv, a32,
+                                                 thr_row, p.sqrt_b, known, a_bits, lane);
         }
 
-        // ---- packed codes: shared staging -> global
+        // ---- packed codes of both segments: shared staging -> global
         fence_async_smem();
         __syncwarp();
-        bulk_store_if(lane == 0, outp, code_buf, SEG_CODE_BYTES);
+        bulk_store_if(lane == 0, outp, code_buf, TOK_SPW * SEG_CODE_BYTES);
+        if (++stage == (uint32_t)NST) { stage = 0; parity ^= 1u; }
     }
     // A load that never completed ends the loop for every warp of the group at the same iteration (they poll
     // the same barrier), so nobody is left behind at the named barrier; the error word tells the host.

@@ -43,11 +43,14 @@ def clean_error_word(B):
 def units_per_group(T, d, b, fmt, group, permuted):
     """Units (rows, or 1024-element segments) that the busiest warp group of the persistent kernel handles.
     A unit is a whole row when the warps of a row are coupled (per-token scales, a permutation, a block that
-    spans the row), else a single segment; a CTA holds 16 // G groups of G warps."""
+    spans the row), else a single segment; a CTA holds 16 // G groups of G warps.  (The records of deferred
+    scales are served when 32 have gathered, 16 in the lean per-token kernel.)"""
     assert d % SEG == 0
     segs = d // SEG
     per_token = fmt in ("fp4", "int4_asym") or (fmt == "int4" and group in (0, d))
     G = segs if (per_token or permuted or (b == d and b > 128)) else 1
+    if fmt in ("int4", "fp4") and per_token and not permuted and b <= 128 and segs in (2, 4, 8):
+        G = segs // 2        # the lean per-token kernel: a warp owns two adjacent segments of a row
     units = T * segs // G
     groups_per_cta = WARPS_PER_CTA // G
     grid = min((units + groups_per_cta - 1) // groups_per_cta, SMS)
