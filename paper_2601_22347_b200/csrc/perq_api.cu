@@ -92,6 +92,25 @@ int allow_smem(K kernel, size_t bytes)
     return PERQ_OK;
 }
 
+// Launch with programmatic stream serialization: the kernel may be set up while its predecessor in the stream
+// is still running (its prologue overlaps the predecessor's tail); every kernel launched this way calls
+// griddep_wait() before its first global memory access, so stream order is kept for all data.
+template <typename P>
+cudaError_t launch_overlapped(void (*kernel)(P), int grid, int block, size_t smem, cudaStream_t st, const P &params)
+{
+    cudaLaunchConfig_t cfg = {};
+    cfg.gridDim = dim3((unsigned)grid);
+    cfg.blockDim = dim3((unsigned)block);
+    cfg.dynamicSmemBytes = smem;
+    cfg.stream = st;
+    cudaLaunchAttribute attr[1];
+    attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+    attr[0].val.programmaticStreamSerializationAllowed = 1;
+    cfg.attrs = attr;
+    cfg.numAttrs = 1;
+    return cudaLaunchKernelEx(&cfg, kernel, params);
+}
+
 int launch_generic(const void *x, const int32_t *perm, int64_t T, int32_t d, int32_t b, int32_t fmt, int g,
                    void *out_codes, void *out_scales, cudaStream_t st)
 {
@@ -124,8 +143,11 @@ int launch_fast_inst(const perq::FastParams &p, int grid, cudaStream_t st)
     auto kernel = perq::perq_fast_kernel<LOG2B, MODE, LOG2G, PERM, XB>;
     const size_t smem = PERM ? perq::FastSmem::total_perm : XB > 3 ? perq::FastSmem::total_full : perq::FastSmem::total;
     if (int rc = allow_smem(kernel, smem)) return rc;
-    kernel<<<grid, perq::FAST_THREADS, smem, st>>>(p);
-    return cudaGetLastError() == cudaSuccess ? PERQ_OK : PERQ_ERR_CUDA;
+    if (launch_overlapped(kernel, grid, perq::FAST_THREADS, smem, st, p) != cudaSuccess) {
+        (void)cudaGetLastError();
+        return PERQ_ERR_CUDA;
+    }
+    return PERQ_OK;
 }
 
 template <int MODE, int LOG2G, bool PERM>
@@ -210,8 +232,11 @@ int launch_tok_inst(const perq::FastParams &p, int grid, cudaStream_t st)
 {
     auto kernel = perq::perq_tok_kernel<LOG2B, MODE, LOG2G>;
     if (int rc = allow_smem(kernel, perq::TokSmem::total)) return rc;
-    kernel<<<grid, perq::FAST_THREADS, perq::TokSmem::total, st>>>(p);
-    return cudaGetLastError() == cudaSuccess ? PERQ_OK : PERQ_ERR_CUDA;
+    if (launch_overlapped(kernel, grid, perq::FAST_THREADS, perq::TokSmem::total, st, p) != cudaSuccess) {
+        (void)cudaGetLastError();
+        return PERQ_ERR_CUDA;
+    }
+    return PERQ_OK;
 }
 
 template <int MODE, int LOG2G>

@@ -172,6 +172,13 @@ __device__ __forceinline__ void bulk_store_wait_read()
 {
     asm volatile("cp.async.bulk.wait_group.read %0;" ::"n"(N) : "memory");
 }
+// Programmatic dependent launch: a kernel launched with programmatic stream serialization may start while
+// its predecessor in the stream is still running; it must not touch global memory before griddep_wait(),
+// which returns once the predecessor has completed and its writes are visible (at once when there is none,
+// or when the launch did not ask for the overlap).  griddep_launch() lets the successor's CTAs be scheduled
+// as soon as this grid's CTAs have all passed it or exited.
+__device__ __forceinline__ void griddep_wait() { asm volatile("griddepcontrol.wait;" ::: "memory"); }
+__device__ __forceinline__ void griddep_launch() { asm volatile("griddepcontrol.launch_dependents;" ::: "memory"); }
 __device__ __forceinline__ void fence_async_smem() { asm volatile("fence.proxy.async.shared::cta;" ::: "memory"); }
 
 __device__ __forceinline__ void ldmatrix_x4(uint32_t (&r)[4], uint32_t addr)
@@ -757,6 +764,8 @@ __global__ void __launch_bounds__(FAST_THREADS, 1) perq_fast_kernel(FastParams p
         mbar_init(smem_u32(fsmem + FastSmem::full) + tid * 8, 1);
         if (PERM) mbar_init(smem_u32(fsmem + FastSmem::empty) + tid * 8, (uint32_t)G);
     }
+    griddep_wait();             // nothing above reads or writes global memory
+    griddep_launch();           // the stream's next kernel may be set up on every SM this grid has left (it waits like this one)
     if (PERM) {     // the permutation as byte offsets into a staged row; out-of-range entries are clamped
         uint16_t *pt = reinterpret_cast<uint16_t *>(fsmem + FastSmem::perm_tab);
         if ((reinterpret_cast<uintptr_t>(p.perm) & 15u) == 0) {      // four entries per load, all loads independent

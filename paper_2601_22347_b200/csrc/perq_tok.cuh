@@ -384,6 +384,8 @@ __global__ void __launch_bounds__(FAST_THREADS, 1) perq_tok_kernel(FastParams p)
     if (tid < FAST_WARPS * NST) mbar_init(smem_base + (uint32_t)TokSmem::full + tid * 8, 1);
     if (tid == 0) asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
     __syncthreads();
+    griddep_wait();             // nothing above reads or writes global memory
+    griddep_launch();           // the stream's next kernel may be set up on every SM this grid has left (it waits like this one)
 
     const uint32_t first = blockIdx.x * GROUPS + group;
     const uint32_t stride = gridDim.x * GROUPS;
