@@ -14,7 +14,8 @@
  * fix -- "parity unpinned" for: nibble order inside a byte, the all-zero-range
  * convention (scale 0, codes 0), sign of values that quantise to zero in E2M1, the
  * MX shared-exponent reading floor(log2 amax) - 2 versus 2^floor(log2(amax/6)), and the
- * tie-breaks of the greedy permutation.
+ * tie-breaks of the greedy permutation.  perq_oracle_swiglu rounds the product once to bf16 (a reading: the
+ * paper's figure gives the formula, not a storage precision).
  *
  * Rows are independent; `#pragma omp parallel for` over rows is the only parallelism.
  */
@@ -337,6 +338,48 @@ int perq_oracle_quantize_fp4(const double *y, int64_t T, int32_t d, uint8_t *cod
             pack_row(c, d, codes + (size_t)t * (d / 2));
         }
         free(c);
+    }
+    return 0;
+}
+
+/* ---------------------------------------------------------------- gated activation in front of the path
+ * Fig. "permutation-equivariance" (the feedforward network of a transformer block): the online rotation's
+ * input is h = Swish(x W_gate) (.) (x W_up), an elementwise product of the Swish of one projection with the
+ * other; Swish(g) = g * sigmoid(g) = g / (1 + exp(-g)).  Here the two projections are given (bf16) and h is
+ * what a model would store: the real-valued product rounded ONCE to bf16, round to nearest even.
+ *
+ * double_to_bf16_rne rounds a finite double directly to bf16 (no intermediate float: two roundings could
+ * differ from one).  bf16 has 8 significant bits and the exponent range of binary32 (normal from 2^-126,
+ * subnormal quantum 2^-133); magnitudes that round beyond the largest finite bf16 become infinity. */
+static uint16_t double_to_bf16_rne(double v)
+{
+    uint16_t sign = (uint16_t)(signbit(v) ? 0x8000u : 0u);
+    double a = fabs(v);
+    if (a == 0.0) return sign;
+    int e;
+    (void)frexp(a, &e);                       /* a = m * 2^e, m in [0.5, 1): exponent of the leading bit is e - 1 */
+    int lead = e - 1;
+    if (lead < -126) lead = -126;             /* subnormal range: fixed quantum 2^-133 */
+    double q = nearbyint(ldexp(a, 7 - lead)); /* units of 2^(lead-7); ties to even under FE_TONEAREST */
+    if (q >= 256.0) { q = 128.0; lead += 1; } /* rounded up to the next power of two */
+    if (lead > 127) return (uint16_t)(sign | 0x7F80u);
+    uint32_t qi = (uint32_t)q;                /* 0 .. 255; below 128 only in the subnormal range */
+    if (qi < 128u) return (uint16_t)(sign | qi);
+    return (uint16_t)(sign | ((uint32_t)(lead + 127) << 7) | (qi - 128u));
+}
+
+int perq_oracle_swiglu(const uint16_t *gate, const uint16_t *up, int64_t T, int32_t d, uint16_t *h)
+{
+    if (T < 0 || d <= 0 || !gate || !up || !h) return 1;
+    fesetround(FE_TONEAREST);
+#pragma omp parallel for schedule(static)
+    for (int64_t t = 0; t < T; ++t) {
+        for (int32_t i = 0; i < d; ++i) {
+            const double g = bf16_to_double(gate[(size_t)t * d + i]);
+            const double u = bf16_to_double(up[(size_t)t * d + i]);
+            const double swish = g / (1.0 + exp(-g));
+            h[(size_t)t * d + i] = double_to_bf16_rne(swish * u);
+        }
     }
     return 0;
 }

@@ -155,6 +155,16 @@ def rotate_quantize(x, perm, b: int, fmt: int, group: int, want_y: bool = False,
     return out
 
 
+def swiglu(gate, up) -> np.ndarray:
+    """h = Swish(gate) * up in fp64, rounded once to bf16 (round to nearest even); bf16 bit patterns in and out."""
+    gate = _x(gate); up = _x(up)
+    assert gate.shape == up.shape
+    T, d = gate.shape
+    h = np.empty((T, d), np.uint16)
+    _check(_load().perq_oracle_swiglu(_p(gate), _p(up), C.c_int64(T), C.c_int32(d), _p(h)), "swiglu")
+    return h
+
+
 def block_l1_stats(x, perm, b: int):
     """Returns (chan_abs_sum[d], block_l1_mean[d/b], token_max_block_l1[T]) in fp64."""
     x = _x(x); perm = _perm(perm)
