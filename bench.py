@@ -408,6 +408,33 @@ def main():
                 row.update(check_rows(xr[0], perm, b, f, grp, orr[0][0], orr[0][1]))
             sweep.append(row)
 
+        # the gated-activation entry point on the MLP down-projection shape: two bf16 projections in, h never stored
+        rng3 = np.random.default_rng(inputs.SEED_BASE + 33)
+        gate_bits = inputs.f32_to_bf16_bits((rng3.standard_normal((4096, 8192)) * 2.0).astype(np.float32))
+        up_bits = inputs.f32_to_bf16_bits(rng3.standard_normal((4096, 8192)).astype(np.float32))
+        gates = [torch.from_numpy(gate_bits.view(np.int16).copy()).cuda().view(torch.bfloat16)]
+        ups = [torch.from_numpy(up_bits.view(np.int16).copy()).cuda().view(torch.bfloat16)]
+        for i in range(2):
+            gates.append(torch.roll(gates[0], shifts=5 * (i + 1), dims=0).contiguous())
+            ups.append(torch.roll(ups[0], shifts=5 * (i + 1), dims=0).contiguous())
+        og = [B.alloc_outputs(4096, 8192, B.PERQ_FMT_MXFP4, 32, gates[0].device) for _ in range(3)]
+        ms = time_calls(lambda i: B.perq_swiglu_rotate_quantize(gates[i % 3], ups[i % 3], None, 32, B.PERQ_FMT_MXFP4, 32,
+                                                                out_codes=og[i % 3][0], out_scales=og[i % 3][1]))
+        by = (2 * 2 * 8192 + 8192 // 2 + 8192 // 32) * 4096
+        row = {"call": "perq_swiglu_rotate_quantize", "T": 4096, "d": 8192, "b": 32, "fmt": "mxfp4", "group": 32, "ms": ms,
+               "bytes": by, "GB/s": by / (ms * 1e-3) / 1e9, "frac_of_" + peak_kind: by / (ms * 1e-3) / 1e9 / peak}
+        if check_rows is not None:
+            B.perq_swiglu_rotate_quantize(gates[0], ups[0], None, 32, B.PERQ_FMT_MXFP4, 32, out_codes=og[0][0], out_scales=og[0][1])
+            torch.cuda.synchronize()
+            rows16 = np.unique(np.linspace(0, 4095, num=16).astype(np.int64))
+            hb = perq_oracle.swiglu(gate_bits[rows16], up_bits[rows16])
+            ora = perq_oracle.rotate_quantize(hb, None, 32, B.PERQ_FMT_MXFP4, 32, want_pre=True)
+            rt = torch.from_numpy(rows16).cuda()
+            rep = compare_quantized("mxfp4", og[0][0][rt].cpu().numpy(), og[0][1][rt].cpu().numpy(), ora)
+            row.update({"parity_rows_checked": int(rows16.size), "tie_window_exemptions": rep["code_mismatch_exempt"]})
+        sweep.append(row)
+        del gates, ups, og
+
         w1 = inputs.config1()
         time_workload("cfg1", w1.x, None, 16, "int4", 0)
         w2 = inputs.config2(T=4096, b=32)

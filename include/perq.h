@@ -18,7 +18,10 @@
  *     stream); no call synchronises the device unless it says so.  Outputs are valid
  *     once the caller has synchronised `stream`.
  *   - The return value is a perq_status_t.  Arguments are checked on the host before
- *     anything is launched; on an error nothing has been enqueued.
+ *     anything is launched: on an argument error nothing has been enqueued.  PERQ_ERR_CUDA
+ *     (a launch or a copy that the runtime refused) can come after earlier work of the same
+ *     call was enqueued: the host-buffer entry point has then already queued its copy to
+ *     the device, perq_block_l1_stats its first kernel; the outputs are undefined.
  *   - Device pointers must be 16-byte aligned.  Rows are dense (row stride = d).
  *   - Inputs are assumed finite.  NaN/Inf give unspecified codes but never a fault.
  */
@@ -43,14 +46,17 @@ typedef enum {
 typedef enum {
     PERQ_OK = 0,
     PERQ_ERR_NULL = 1,   /* a required pointer is NULL */
-    PERQ_ERR_SHAPE = 2,  /* T < 0, d <= 0, d % 32 != 0 or d > PERQ_MAX_D */
+    PERQ_ERR_SHAPE = 2,  /* T < 0, d <= 0, d % 32 != 0 or d > PERQ_MAX_D; also: a row that the general kernel cannot
+                            hold in 227 KB of shared memory with its per-range tables (very small groups of very long rows) */
     PERQ_ERR_BLOCK = 3,  /* b is not a power of two in [16, d] that divides d */
-    PERQ_ERR_GROUP = 4,  /* INT4: group not 0 and (d % group != 0 or group % 8 != 0); MXFP4: group not 0/32; FP4: not 0 */
+    PERQ_ERR_GROUP = 4,  /* INT4: group not 0 and (d % group != 0, group % 8 != 0, or group neither a multiple nor a
+                            divisor of b); MXFP4: group not 0/32; FP4, INT4_ASYM: not 0 */
     PERQ_ERR_FMT = 5,    /* unknown format */
     PERQ_ERR_ALIGN = 6,  /* a device pointer is not 16-byte aligned */
     PERQ_ERR_CUDA = 7,   /* the CUDA runtime reported an error (launch, copy, attribute) */
     PERQ_ERR_PERM = 8,   /* host-side permutation argument is not a permutation */
-    PERQ_ERR_WORKSPACE = 9 /* workspace missing or too small */
+    PERQ_ERR_WORKSPACE = 9, /* workspace missing or too small */
+    PERQ_ERR_UNSUPPORTED = 10 /* valid arguments that this entry point does not cover (see its description) */
 } perq_status_t;
 
 #define PERQ_MAX_D 32768
@@ -93,17 +99,46 @@ typedef enum {
  *            b <= 128 (any scale mode, with or without perm) and, unpermuted with per-token or MX
  *            scales, b <= 1024 and b == d <= 8192; everything else runs on a slower general kernel.
  * fmt        perq_fmt_t.
- * group      INT4: 0 (per token) or a multiple of 8 dividing d.  MXFP4: 0 or 32 (always 32).  FP4, INT4_ASYM: 0.
+ * group      INT4: 0 (per token) or a multiple of 8 that divides d and is a multiple or a divisor of b.
+ *            MXFP4: 0 or 32 (always 32).  FP4, INT4_ASYM: 0.
  *            Scale ranges are consecutive coordinates of the ROTATED row, independent of b.
  * out_codes  device.  INT4/MXFP4: uint8 [T, d/2].  F32_DEBUG: float [T, d] (the rotated row y).
  * out_scales device.  INT4: float [T] or [T, d/group].  MXFP4: uint8 [T, d/32].  FP4: float [T].  INT4_ASYM: float [T, 2].
  *            F32_DEBUG: unused, may be NULL.
  *
- * Codes and scales are deterministic (bit-identical from run to run).
+ * Codes and scales are deterministic (bit-identical from run to run).  Which kernel serves a call depends
+ * on its shape; every kernel stores the fp32 rounding of the exact scale up to one more rounding of a
+ * constant factor, so scales of the same row from different shapes' kernels agree to 1 ulp, not bit for bit.
  */
 int perq_rotate_quantize(const void *x, const int32_t *perm, int64_t T, int32_t d, int32_t b,
                          int32_t fmt, int32_t group, void *out_codes, void *out_scales,
                          void *stream);
+
+/*
+ * perq_swiglu_rotate_quantize -- the same path fed by the gated activation of a feedforward block.
+ *
+ * Defined by: the figure on permutation equivariance (the feedforward network of a transformer block):
+ * the online rotation's input is h = Swish(x W_gate) (.) (x W_up) -- an elementwise product; Swish(g) =
+ * g * sigmoid(g) = g / (1 + exp(-g)) -- and the region is permutation-equivariant, so the permutation is
+ * merged into the two projections and none is applied here.  With gate = x W_gate and up = x W_up given as
+ * bf16, every row is
+ *
+ *     h_i = bf16( Swish(gate_i) * up_i )        (the real product, rounded once, to nearest even)
+ *
+ * followed by steps 2-4 of perq_rotate_quantize on h.  The outputs equal those of perq_rotate_quantize on a
+ * materialised h; h is never written to memory (4d + d/2 bytes per token move instead of 8d + d/2).
+ * The activation is evaluated in fp32 and again in fp64 wherever the fp32 value is too close to a bf16
+ * rounding boundary to decide the rounding, so h is the correctly rounded value.
+ *
+ * gate, up   device, bf16 [T, d] row-major.      perm   must be NULL (PERQ_ERR_UNSUPPORTED otherwise).
+ * Covered:   d % 1024 == 0, b <= 128, and fmt / group = MXFP4, INT4 with group 128, or INT4 per token with
+ *            d <= 15360.  Anything else that perq_rotate_quantize would accept returns PERQ_ERR_UNSUPPORTED
+ *            (materialise h and call perq_rotate_quantize).
+ * Other arguments, outputs and errors as for perq_rotate_quantize.
+ */
+int perq_swiglu_rotate_quantize(const void *gate, const void *up, const int32_t *perm, int64_t T, int32_t d,
+                                int32_t b, int32_t fmt, int32_t group, void *out_codes, void *out_scales,
+                                void *stream);
 
 /*
  * perq_out_sizes -- bytes of out_codes and out_scales for a call.  Host only, no CUDA.
@@ -120,6 +155,12 @@ int perq_out_sizes(int64_t T, int32_t d, int32_t fmt, int32_t group, size_t *cod
  * then synchronises `stream` before returning.  `workspace` is device memory provided
  * by the caller, at least perq_host_workspace_bytes(...) long; the library allocates
  * nothing.  perm stays a DEVICE pointer (it is reused across calls) or NULL.
+ *
+ * Calls of 4096 rows or more are processed in four chunks of rows, and the copy back of a
+ * chunk runs on an internal non-blocking stream while the next chunk is copied in; that
+ * stream and five events are created once per device on first use and kept until exit.
+ * Two such calls at the same time on one device (different caller streams) would share
+ * those events: issue them from one thread at a time.
  */
 int perq_rotate_quantize_host(const void *x_host, const int32_t *perm, int64_t T, int32_t d,
                               int32_t b, int32_t fmt, int32_t group, void *out_codes_host,
@@ -136,8 +177,8 @@ int perq_host_workspace_bytes(int64_t T, int32_t d, int32_t fmt, int32_t group, 
  *   block_l1_mean[j]      = (1/T) sum_t L[t, j],   L[t, j] = sum_{i<b} |x[t, perm[j*b+i]]|
  *   token_max_block_l1[t] = max_j L[t, j]
  *
- * x, perm, T, d as above (T >= 1 here unless all outputs are NULL); b any power of two
- * >= 8 dividing d (or b == d).  Each output is device fp32 and may be NULL: [d], [d/b], [T].
+ * x, perm, T, d as above (T >= 1 here unless all outputs are NULL); b a power of two
+ * >= 8 dividing d.  Each output is device fp32 and may be NULL: [d], [d/b], [T].
  * workspace  device, perq_block_l1_stats_workspace_bytes(...) bytes: per-CTA partial sums
  *            that a second kernel adds in a fixed order, so results are deterministic.
  * Accumulation is fp32: sums agree with exact arithmetic to about 1e-6 relative.

@@ -46,6 +46,8 @@ def load() -> C.CDLL:
         lib = C.CDLL(path)
         vp, i32, i64, sz = C.c_void_p, C.c_int32, C.c_int64, C.c_size_t
         lib.perq_rotate_quantize.argtypes = [vp, vp, i64, i32, i32, i32, i32, vp, vp, vp]
+        lib.perq_swiglu_rotate_quantize.argtypes = [vp, vp, vp, i64, i32, i32, i32, i32, vp, vp, vp]
+        lib.perq_swiglu_rotate_quantize.restype = C.c_int
         lib.perq_rotate_quantize_host.argtypes = [vp, vp, i64, i32, i32, i32, i32, vp, vp, vp, sz, vp]
         lib.perq_host_workspace_bytes.argtypes = [i64, i32, i32, i32, C.POINTER(sz)]
         lib.perq_out_sizes.argtypes = [i64, i32, i32, i32, C.POINTER(sz), C.POINTER(sz)]
@@ -129,6 +131,22 @@ def perq_rotate_quantize(x: torch.Tensor, perm: Optional[torch.Tensor], b: int, 
     rc = load().perq_rotate_quantize(_ptr(x), _ptr(perm), T, d, b, fmt, group, _ptr(out_codes), _ptr(out_scales),
                                      _stream(stream))
     _check(rc, "perq_rotate_quantize")
+    return out_codes, out_scales
+
+
+def perq_swiglu_rotate_quantize(gate: torch.Tensor, up: torch.Tensor, perm: Optional[torch.Tensor], b: int, fmt: int,
+                                group: int = 0, out_codes: Optional[torch.Tensor] = None,
+                                out_scales: Optional[torch.Tensor] = None, stream=None):
+    """gate, up: bf16 CUDA tensors [T, d] (contiguous); perm must be None."""
+    for t in (gate, up):
+        assert t.is_cuda and t.dtype == torch.bfloat16 and t.dim() == 2 and t.is_contiguous()
+    assert gate.shape == up.shape
+    T, d = gate.shape
+    if out_codes is None:
+        out_codes, out_scales = alloc_outputs(T, d, fmt, group, gate.device)
+    rc = load().perq_swiglu_rotate_quantize(_ptr(gate), _ptr(up), _ptr(perm), T, d, b, fmt, group, _ptr(out_codes),
+                                            _ptr(out_scales), _stream(stream))
+    _check(rc, "perq_swiglu_rotate_quantize")
     return out_codes, out_scales
 
 

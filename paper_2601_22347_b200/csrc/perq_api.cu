@@ -43,6 +43,9 @@ int check_shape(int64_t T, int32_t d, int32_t b, int32_t fmt, int32_t group, int
         if (group < 0) return PERQ_ERR_GROUP;
         if (group > 0) {
             if (d % group != 0 || group % 8 != 0) return PERQ_ERR_GROUP;
+            // a scale range lies inside one Hadamard block or is made of whole blocks: the error bound of a
+            // range's maximum is taken from the blocks it covers
+            if (group % b != 0 && b % group != 0) return PERQ_ERR_GROUP;
             g = group;
         }
     } else if (fmt == PERQ_FMT_MXFP4) {
@@ -303,6 +306,7 @@ int try_launch_fast(const void *x, const int32_t *perm, int64_t T, int32_t d, in
     p.out_codes = static_cast<uint8_t *>(out_codes);
     p.out_scales = out_scales;
     p.units_total = (uint32_t)units;
+    p.x2 = nullptr;
     p.perm = perm;
     p.G = G;
     p.d = d;
@@ -314,7 +318,7 @@ int try_launch_fast(const void *x, const int32_t *perm, int64_t T, int32_t d, in
     const long long want = (units + groups_per_cta - 1) / groups_per_cta;
     const int grid = (int)std::min<long long>(want, sms);
     if ((mode == perq::MODE_TOKEN || mode == perq::MODE_FP4) && !permuted && !full && !longb &&
-        (segs == 2 || segs == 4 || segs == 8)) {
+        (segs == 2 || segs == 4 || segs == 8) && b <= 64) {     // (b = 128: the second rotation costs what the sharing saves)
         const int tok_groups = perq::FAST_WARPS / (segs / perq::TOK_SPW);       // rows in flight per CTA
         const int tok_grid = (int)std::min<long long>((T + tok_groups - 1) / tok_groups, sms);
         return mode == perq::MODE_TOKEN ? launch_tok<perq::MODE_TOKEN>(segs, ilog2(b), p, tok_grid, st)
@@ -329,6 +333,30 @@ int try_launch_fast(const void *x, const int32_t *perm, int64_t T, int32_t d, in
     const int log2b = ilog2(b);
     return permuted ? launch_fast_mode<true>(mode, G, log2b, p, grid, st)
                     : launch_fast_mode<false>(mode, G, log2b, p, grid, st);
+}
+
+// Gated variants of the group kernel: h = Swish(gate) * up formed in shared memory, then the same path.
+template <int LOG2B, int MODE, int LOG2G>
+int launch_swiglu_inst(const perq::FastParams &p, int grid, cudaStream_t st)
+{
+    auto kernel = perq::perq_fast_kernel<LOG2B, MODE, LOG2G, false, 0, true>;
+    if (int rc = allow_smem(kernel, perq::FastSmem::total)) return rc;
+    if (launch_overlapped(kernel, grid, perq::FAST_THREADS, perq::FastSmem::total, st, p) != cudaSuccess) {
+        (void)cudaGetLastError();
+        return PERQ_ERR_CUDA;
+    }
+    return PERQ_OK;
+}
+
+template <int MODE, int LOG2G>
+int launch_swiglu_b(int log2b, const perq::FastParams &p, int grid, cudaStream_t st)
+{
+    switch (log2b) {
+    case 4: return launch_swiglu_inst<4, MODE, LOG2G>(p, grid, st);
+    case 5: return launch_swiglu_inst<5, MODE, LOG2G>(p, grid, st);
+    case 6: return launch_swiglu_inst<6, MODE, LOG2G>(p, grid, st);
+    default: return launch_swiglu_inst<7, MODE, LOG2G>(p, grid, st);
+    }
 }
 
 int launch_any(const void *x, const int32_t *perm, int64_t T, int32_t d, int32_t b, int32_t fmt, int g,
@@ -380,6 +408,36 @@ static __device__ __align__(256) float g_stats_scratch[PERQ_STATS_STATIC_MAX_FLO
 float *g_stats_scratch_addr[kMaxDevices] = {};   // device address of the array, per device ordinal
 std::mutex g_stats_scratch_mutex;
 
+// Per-device resources of perq_rotate_quantize_host's overlap of the two copy directions: one
+// non-blocking stream and a few events, created on first use and kept until the process exits.
+struct HostPipe {
+    static constexpr int kChunks = 4;
+    cudaStream_t aux = nullptr;
+    cudaEvent_t ready[kChunks] = {};
+    cudaEvent_t done = nullptr;
+    bool ok = false, tried = false;
+};
+HostPipe g_host_pipe[kMaxDevices];
+std::mutex g_host_pipe_mutex;
+
+HostPipe *host_pipe()
+{
+    int dev = -1;
+    if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= kMaxDevices) return nullptr;
+    std::lock_guard<std::mutex> lock(g_host_pipe_mutex);
+    HostPipe &hp = g_host_pipe[dev];
+    if (!hp.tried) {
+        hp.tried = true;
+        bool ok = cudaStreamCreateWithFlags(&hp.aux, cudaStreamNonBlocking) == cudaSuccess;
+        for (int i = 0; ok && i < HostPipe::kChunks; ++i)
+            ok = cudaEventCreateWithFlags(&hp.ready[i], cudaEventDisableTiming) == cudaSuccess;
+        ok = ok && cudaEventCreateWithFlags(&hp.done, cudaEventDisableTiming) == cudaSuccess;
+        if (!ok) (void)cudaGetLastError();
+        hp.ok = ok;
+    }
+    return hp.ok ? &hp : nullptr;     // without it the call still works, on the caller's stream alone
+}
+
 template <int KC, int CL, bool WB>
 int launch_stats_inst(const perq::StatsParams &p, const StatsPlan &plan, cudaStream_t st)
 {
@@ -418,12 +476,13 @@ const char *perq_status_string(int status)
     case PERQ_ERR_NULL: return "a required pointer is NULL";
     case PERQ_ERR_SHAPE: return "bad shape: need T >= 0, 0 < d <= 32768, d % 32 == 0 (and the row must fit in shared memory)";
     case PERQ_ERR_BLOCK: return "bad block size: need a power of two b, 16 <= b <= d, dividing d";
-    case PERQ_ERR_GROUP: return "bad group: INT4 needs 0 or a multiple of 8 dividing d; MXFP4 needs 0 or 32; FP4 and asymmetric INT4 need 0";
+    case PERQ_ERR_GROUP: return "bad group: INT4 needs 0 or a multiple of 8 that divides d and is a multiple or a divisor of b; MXFP4 needs 0 or 32; FP4 and asymmetric INT4 need 0";
     case PERQ_ERR_FMT: return "unknown format";
     case PERQ_ERR_ALIGN: return "device pointers must be 16-byte aligned";
     case PERQ_ERR_CUDA: return "CUDA runtime error";
     case PERQ_ERR_PERM: return "not a permutation";
     case PERQ_ERR_WORKSPACE: return "workspace missing or too small";
+    case PERQ_ERR_UNSUPPORTED: return "combination not covered by this entry point";
     default: return "unknown status";
     }
 }
@@ -466,6 +525,46 @@ int perq_rotate_quantize(const void *x, const int32_t *perm, int64_t T, int32_t 
     return launch_any(x, perm, T, d, b, fmt, g, out_codes, out_scales, static_cast<cudaStream_t>(stream));
 }
 
+int perq_swiglu_rotate_quantize(const void *gate, const void *up, const int32_t *perm, int64_t T, int32_t d, int32_t b,
+                                int32_t fmt, int32_t group, void *out_codes, void *out_scales, void *stream)
+{
+    int g = 0;
+    if (int rc = check_shape(T, d, b, fmt, group, &g)) return rc;
+    if (perm != nullptr) return PERQ_ERR_UNSUPPORTED;      // in deployment the permutation is merged into the weights
+    if (d % perq::SEG_ELEMS != 0 || b > 128) return PERQ_ERR_UNSUPPORTED;
+    const int segs = d / perq::SEG_ELEMS;
+    int mode, G = 1;
+    if (fmt == PERQ_FMT_MXFP4) mode = perq::MODE_MX;
+    else if (fmt == PERQ_FMT_INT4 && g == 128) mode = perq::MODE_G128;
+    else if (fmt == PERQ_FMT_INT4 && g == d && segs <= perq::FAST_WARPS - 1) { mode = perq::MODE_TOKEN; G = segs; }
+    else return PERQ_ERR_UNSUPPORTED;
+    if (T == 0) return PERQ_OK;
+    if (!gate || !up || !out_codes || !out_scales) return PERQ_ERR_NULL;
+    if (!aligned16(gate) || !aligned16(up) || !aligned16(out_codes) || !aligned16(out_scales)) return PERQ_ERR_ALIGN;
+    const long long units = (long long)T * segs / G;
+    if (units >= (1ll << 31)) return PERQ_ERR_SHAPE;
+    perq::FastParams p;
+    p.x = static_cast<const uint16_t *>(gate);
+    p.x2 = static_cast<const uint16_t *>(up);
+    p.out_codes = static_cast<uint8_t *>(out_codes);
+    p.out_scales = out_scales;
+    p.units_total = (uint32_t)units;
+    p.perm = nullptr;
+    p.G = G;
+    p.d = d;
+    p.sqrt_b = std::sqrt((double)b);
+    p.inv_7_sqrt_b = 1.0 / (7.0 * p.sqrt_b);
+    const int sms = sm_count();
+    if (sms <= 0) return PERQ_ERR_CUDA;
+    const int groups_per_cta = perq::FAST_WARPS / G;
+    const int grid = (int)std::min<long long>((units + groups_per_cta - 1) / groups_per_cta, sms);
+    cudaStream_t st = static_cast<cudaStream_t>(stream);
+    const int log2b = ilog2(b);
+    if (mode == perq::MODE_MX) return launch_swiglu_b<perq::MODE_MX, 0>(log2b, p, grid, st);
+    if (mode == perq::MODE_G128) return launch_swiglu_b<perq::MODE_G128, 0>(log2b, p, grid, st);
+    return launch_swiglu_b<perq::MODE_TOKEN, -1>(log2b, p, grid, st);       // warps per row at run time
+}
+
 int perq_host_workspace_bytes(int64_t T, int32_t d, int32_t fmt, int32_t group, size_t *bytes)
 {
     size_t cb = 0, sb = 0;
@@ -496,11 +595,31 @@ int perq_rotate_quantize_host(const void *x_host, const int32_t *perm, int64_t T
     unsigned char *x_dev = base;
     unsigned char *codes_dev = x_dev + up((size_t)T * (size_t)d * 2);
     unsigned char *scales_dev = codes_dev + up(cb);
-    if (cudaMemcpyAsync(x_dev, x_host, (size_t)T * (size_t)d * 2, cudaMemcpyHostToDevice, st) != cudaSuccess)
-        return PERQ_ERR_CUDA;
-    if (int rc = launch_any(x_dev, perm, T, d, b, fmt, g, codes_dev, scales_dev, st)) return rc;
-    if (cudaMemcpyAsync(out_codes_host, codes_dev, cb, cudaMemcpyDeviceToHost, st) != cudaSuccess) return PERQ_ERR_CUDA;
-    if (sb && cudaMemcpyAsync(out_scales_host, scales_dev, sb, cudaMemcpyDeviceToHost, st) != cudaSuccess)
+    // Rows are independent: larger calls go in four chunks of rows, the copy back of one chunk (on an
+    // internal stream) overlapping the copy in of the next, so that both directions of the link are busy.
+    HostPipe *pipe = (T >= 4096) ? host_pipe() : nullptr;
+    const int n_chunks = pipe ? HostPipe::kChunks : 1;
+    const int64_t rows_per = (((T + n_chunks - 1) / n_chunks) + 63) & ~(int64_t)63;
+    const size_t code_row = cb / (size_t)T, scale_row = sb / (size_t)T;
+    const unsigned char *xh = static_cast<const unsigned char *>(x_host);
+    unsigned char *ch = static_cast<unsigned char *>(out_codes_host), *sh = static_cast<unsigned char *>(out_scales_host);
+    for (int c = 0; c < n_chunks; ++c) {
+        const int64_t r0 = c * rows_per, r1 = std::min<int64_t>(T, r0 + rows_per);
+        if (r0 >= r1) break;
+        const size_t n = (size_t)(r1 - r0), xo = (size_t)r0 * d * 2, co = (size_t)r0 * code_row, so = (size_t)r0 * scale_row;
+        if (cudaMemcpyAsync(x_dev + xo, xh + xo, n * d * 2, cudaMemcpyHostToDevice, st) != cudaSuccess) return PERQ_ERR_CUDA;
+        if (int rc = launch_any(x_dev + xo, perm, (int64_t)n, d, b, fmt, g, codes_dev + co, scales_dev + so, st)) return rc;
+        cudaStream_t back = st;
+        if (pipe) {
+            if (cudaEventRecord(pipe->ready[c], st) != cudaSuccess || cudaStreamWaitEvent(pipe->aux, pipe->ready[c], 0) != cudaSuccess)
+                return PERQ_ERR_CUDA;
+            back = pipe->aux;
+        }
+        if (cudaMemcpyAsync(ch + co, codes_dev + co, n * code_row, cudaMemcpyDeviceToHost, back) != cudaSuccess) return PERQ_ERR_CUDA;
+        if (sb && cudaMemcpyAsync(sh + so, scales_dev + so, n * scale_row, cudaMemcpyDeviceToHost, back) != cudaSuccess)
+            return PERQ_ERR_CUDA;
+    }
+    if (pipe && (cudaEventRecord(pipe->done, pipe->aux) != cudaSuccess || cudaStreamWaitEvent(st, pipe->done, 0) != cudaSuccess))
         return PERQ_ERR_CUDA;
     return cudaStreamSynchronize(st) == cudaSuccess ? PERQ_OK : PERQ_ERR_CUDA;
 }

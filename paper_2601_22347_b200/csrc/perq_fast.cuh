@@ -82,6 +82,7 @@ struct FastParams {
     uint8_t *out_codes;
     void *out_scales;
     uint32_t units_total;    // units of G segments (fewer than 2^31); rows when G = d / 1024
+    const uint16_t *x2;      // gated-activation variants only: the second projection ("up"), same shape as x
     const int32_t *perm;     // permuted variants only: perm[d] (device)
     int G;                   // permuted variants: segments per row
     int d;
@@ -690,15 +691,109 @@ __device__ __forceinline__ void serve_asym_requests(const FastParams &p, const u
     __syncwarp();
 }
 
+// ---------------------------------------------------------------- gated activation in front of the rotation
+//
+// h = Swish(g) * u, Swish(g) = g / (1 + exp(-g)), rounded once to bf16 (round to nearest even): the input of the
+// online rotation in a gated feedforward block.  The fp32 evaluation below is accurate to about 5e-7 relative
+// (exp2 of a compensated argument, one approximate reciprocal, three roundings); a result whose low 16 bits
+// are within SWIGLU_MARGIN fp32 ulps (at least 9.5e-7 relative) of the halfway pattern 0x8000 could round to
+// either neighbour, and is evaluated again in fp64, as are arguments beyond +-80 and results deep in the
+// subnormal range, where the relative bound does not hold.
+constexpr uint32_t SWIGLU_MARGIN = 16;
+
+__device__ __forceinline__ float ex2_approx(float x)
+{
+    float r;
+    asm("ex2.approx.f32 %0, %1;" : "=f"(r) : "f"(x));
+    return r;
+}
+__device__ __forceinline__ float swish_mul_f32(float g, float u)
+{
+    const float L2E_HI = 1.44269502162933349609375f, L2E_LO = 1.925963033500011e-8f;      // log2(e) = hi + lo
+    const float t = -g * L2E_HI;
+    float r = fmaf(-g, L2E_HI, -t);                  // what the rounding of t dropped
+    r = fmaf(-g, L2E_LO, r);
+    float e = ex2_approx(t);
+    e = fmaf(e, r * 0.693147182464599609375f, e);    // 2^(t + r) = 2^t (1 + r ln 2) to first order (|r| < 2^-17)
+    return __fdividef(g, 1.0f + e) * u;
+}
+__device__ __forceinline__ bool swiglu_needs_fp64(float h, float g)
+{
+    const uint32_t bits = __float_as_uint(h);
+    const uint32_t off = ((bits & 0xffffu) - (0x8000u - SWIGLU_MARGIN)) & 0xffffu;
+    const uint32_t mag = bits & 0x7fffffffu;
+    return off <= 2u * SWIGLU_MARGIN || fabsf(g) > 80.0f || (mag != 0u && mag < 0x0d800000u) || mag >= 0x7f800000u;
+}
+// A finite double to bf16 bits, one rounding to nearest even (integer arithmetic on the double's fields).
+__device__ __forceinline__ uint32_t double_to_bf16_bits(double v)
+{
+    const unsigned long long b = (unsigned long long)__double_as_longlong(v);
+    const uint32_t sign = (uint32_t)(b >> 48) & 0x8000u;
+    const int E = (int)((b >> 52) & 0x7ffu);
+    if (E == 0) return sign;                                   // zero (fp64 subnormals are far below bf16's)
+    const int e = E - 1023;
+    if (e > 127) return sign | 0x7f80u;
+    const unsigned long long M = (1ull << 52) | (b & ((1ull << 52) - 1ull));
+    const int lead = e < -126 ? -126 : e;
+    const int shift = 45 + (lead - e);                         // the quantum is 2^(lead - 7)
+    if (shift > 54) return sign;                               // below half of the smallest subnormal
+    unsigned long long q = M >> shift;
+    const unsigned long long rem = M & ((1ull << shift) - 1ull), half = 1ull << (shift - 1);
+    if (rem > half || (rem == half && (q & 1ull))) q += 1ull;
+    const uint32_t mag = (e >= -126) ? (uint32_t)((e + 127) << 7) + (uint32_t)(q - 128ull) : (uint32_t)q;
+    return sign | (mag > 0x7f80u ? 0x7f80u : mag);
+}
+__device__ __noinline__ uint32_t swiglu_fp64_bits(float g, float u)
+{
+    const double gd = (double)g;
+    return double_to_bf16_bits(gd / (1.0 + exp(-gd)) * (double)u);
+}
+// One word (two bf16 values) of h from one word of each projection.
+__device__ __forceinline__ uint32_t swiglu_word(uint32_t gw, uint32_t uw)
+{
+    const float g0 = __uint_as_float(gw << 16), g1 = __uint_as_float(gw & 0xffff0000u);
+    const float u0 = __uint_as_float(uw << 16), u1 = __uint_as_float(uw & 0xffff0000u);
+    const float h0 = swish_mul_f32(g0, u0), h1 = swish_mul_f32(g1, u1);
+    uint32_t w;
+    asm("cvt.rn.bf16x2.f32 %0, %1, %2;" : "=r"(w) : "f"(h1), "f"(h0));
+    const bool s0 = swiglu_needs_fp64(h0, g0), s1 = swiglu_needs_fp64(h1, g1);
+    if (s0 || s1) {
+        if (s0) w = (w & 0xffff0000u) | swiglu_fp64_bits(g0, u0);
+        if (s1) w = (w & 0x0000ffffu) | (swiglu_fp64_bits(g1, u1) << 16);
+    }
+    return w;
+}
+// This warp's 1024-element segment of h, written over the staged gate segment (lane l handles the 16-byte
+// pieces l, l + 32, l + 64, l + 96 of both projections).
+__device__ __forceinline__ void swiglu_segment(uint32_t gate_addr, uint32_t up_addr, int lane)
+{
+#pragma unroll
+    for (int r = 0; r < 4; ++r) {
+        const uint32_t off = (uint32_t)(r * 32 + lane) * 16u;
+        uint32_t gw[4], uw[4];
+        asm volatile("ld.shared.v4.b32 {%0,%1,%2,%3}, [%4];" : "=r"(gw[0]), "=r"(gw[1]), "=r"(gw[2]), "=r"(gw[3]) : "r"(gate_addr + off) : "memory");
+        asm volatile("ld.shared.v4.b32 {%0,%1,%2,%3}, [%4];" : "=r"(uw[0]), "=r"(uw[1]), "=r"(uw[2]), "=r"(uw[3]) : "r"(up_addr + off) : "memory");
+        uint32_t hw[4];
+#pragma unroll
+        for (int k = 0; k < 4; ++k) hw[k] = swiglu_word(gw[k], uw[k]);
+        sts_v4(gate_addr + off, hw[0], hw[1], hw[2], hw[3]);
+    }
+    __syncwarp();
+}
+
 // ---------------------------------------------------------------- the kernel
 
 // XB > 0: the Hadamard block has 2^(7 + XB) elements (LOG2B must be 7: the part of the
 // butterfly done inside a warp's registers); the lane-group bits go through shuffles, the warp bits
 // through shared memory.
 // XB = 1..3 keeps the block inside a warp's segment; XB = 3 + LOG2G is the whole row.
-template <int LOG2B, int MODE, int LOG2G, bool PERM, int XB>
+// SWIGLU: the rows are h = Swish(x) * x2, formed in shared memory from the two staged projections (unpermuted,
+// blocks inside a segment); two ring stages of each projection instead of four of one, and no deferred scales
+// (they would be re-derived from the inputs in global memory, which are not h).
+template <int LOG2B, int MODE, int LOG2G, bool PERM, int XB, bool SWIGLU = false>
 __global__ void __launch_bounds__(FAST_THREADS, 1) perq_fast_kernel(FastParams p)
 {
+    static_assert(!SWIGLU || (!PERM && XB == 0 && MODE != MODE_ASYM && MODE != MODE_FP4), "gated variant: unpermuted, short blocks");
     constexpr int B = 1 << LOG2B;
     constexpr bool FULLV = XB > 0;                           // a block longer than the in-register part
     constexpr int WBITS = XB > 3 ? XB - 3 : 0;               // index bits that span the warps of a row
@@ -713,7 +808,7 @@ __global__ void __launch_bounds__(FAST_THREADS, 1) perq_fast_kernel(FastParams p
     // G is a template constant 2^LOG2G, or (LOG2G < 0, and permuted rows without per-token scales) p.G
     constexpr bool TOK = per_token_mode(MODE);
     constexpr bool RUNTIME_G = (PERM && !TOK) || LOG2G < 0;
-    constexpr int NST = (PERM || WBITS > 0) ? 3 : FAST_NSTAGE;
+    constexpr int NST = (PERM || WBITS > 0) ? 3 : SWIGLU ? 2 : FAST_NSTAGE;
     const int G = RUNTIME_G ? p.G : (1 << (LOG2G < 0 ? 0 : LOG2G));   // warps (segments) per unit
     const int GROUPS = FAST_WARPS / G;
     const uint32_t UNIT_BYTES = (uint32_t)G * SEG_BYTES;
@@ -741,6 +836,8 @@ __global__ void __launch_bounds__(FAST_THREADS, 1) perq_fast_kernel(FastParams p
     const uint32_t xbuf_addr = smem_u32(fsmem + FastSmem::xbuf) + (uint32_t)(group * G) * 4096u;   // FULLV: this row's exchange space
 
     const uint32_t stage_base = smem_u32(fsmem + FastSmem::stages) + (uint32_t)group * (NST * UNIT_BYTES);
+    // gated variant: the second projection's stages fill the other half of the stage area
+    const uint32_t up_base = stage_base + (uint32_t)FAST_WARPS * 2u * SEG_BYTES;
     const uint32_t empty_base = smem_u32(fsmem + FastSmem::empty) + (uint32_t)group * (FAST_NSTAGE * 8);
     const uint32_t pbuf_addr = smem_u32(fsmem + FastSmem::pbuf) + (uint32_t)warp * SEG_BYTES;
     const uint16_t *ptab = reinterpret_cast<const uint16_t *>(fsmem + FastSmem::perm_tab);
@@ -824,14 +921,17 @@ __global__ void __launch_bounds__(FAST_THREADS, 1) perq_fast_kernel(FastParams p
     const uint32_t refill_end = n_units > (uint32_t)NST ? n_units - NST : 0u;      // iterations 1 .. refill_end load a unit
     const size_t unit_step = (size_t)stride * ((size_t)G * SEG_ELEMS);
     const uint16_t *xload = p.x + (size_t)first * ((size_t)G * SEG_ELEMS);         // leader: the next unit to load
+    const uint16_t *xload2 = (SWIGLU ? p.x2 : p.x) + (size_t)first * ((size_t)G * SEG_ELEMS);
     // prologue: fill the ring
     if (leader) {
 #pragma unroll
         for (int s = 0; s < NST; ++s) {
             if ((uint32_t)s < n_units) {
-                mbar_expect_tx(full_base + s * 8, UNIT_BYTES);
+                mbar_expect_tx(full_base + s * 8, SWIGLU ? 2 * UNIT_BYTES : UNIT_BYTES);
                 bulk_load(stage_base + s * UNIT_BYTES, xload, UNIT_BYTES, full_base + s * 8);
+                if (SWIGLU) bulk_load(up_base + s * UNIT_BYTES, xload2, UNIT_BYTES, full_base + s * 8);
                 xload += unit_step;
+                xload2 += unit_step;
             }
         }
     }
@@ -850,7 +950,10 @@ __global__ void __launch_bounds__(FAST_THREADS, 1) perq_fast_kernel(FastParams p
         const uint32_t parity = (it / NST) & 1u;
         const uint32_t par2 = it & 1u;
         if (!mbar_wait_fast(full_base + stage * 8, parity)) {
+            // the load never completed: every warp of the group polls this barrier and leaves here together,
+            // so none is left behind at the group's named barrier
             if (lane == 0) atomicOr(&g_perq_device_error, 1u);
+            bulk_store_wait_read<0>();
             return;
         }
         // the staged row (or, unpermuted, the staged unit) and this warp's 1024 elements of it
@@ -858,6 +961,7 @@ __global__ void __launch_bounds__(FAST_THREADS, 1) perq_fast_kernel(FastParams p
                                   ((size_t)group * NST + stage) * ((size_t)G * SEG_ELEMS);
         uint32_t seg_addr = stage_base + stage * UNIT_BYTES + (uint32_t)w_in_g * SEG_BYTES;
         const uint16_t *seg = raw_row + (size_t)w_in_g * SEG_ELEMS;
+        if (SWIGLU) swiglu_segment(seg_addr, up_base + stage * UNIT_BYTES + (uint32_t)w_in_g * SEG_BYTES, lane);
         if (PERM) {
             // gather this warp's segment of the permuted row into its own buffer: lane l takes
             // positions r*256 + 8l .. +7 in round r (16-byte conflict-free stores)
@@ -936,9 +1040,11 @@ __global__ void __launch_bounds__(FAST_THREADS, 1) perq_fast_kernel(FastParams p
                 const uint32_t ps = (it - 1) % NST;
                 // permuted rows are read until the end of an iteration: wait until every warp is done
                 if (PERM && !mbar_wait(empty_base + ps * 8, ((it - 1) / NST) & 1u)) atomicOr(&g_perq_device_error, 4u);
-                mbar_expect_tx(full_base + ps * 8, UNIT_BYTES);
+                mbar_expect_tx(full_base + ps * 8, SWIGLU ? 2 * UNIT_BYTES : UNIT_BYTES);
                 bulk_load(stage_base + ps * UNIT_BYTES, xload, UNIT_BYTES, full_base + ps * 8);
+                if (SWIGLU) bulk_load(up_base + ps * UNIT_BYTES, xload2, UNIT_BYTES, full_base + ps * 8);
                 xload += unit_step;
+                xload2 += unit_step;
             }
         };
         if (G == 1 || (!TOK && WBITS == 0)) refill();
@@ -1209,12 +1315,11 @@ __global__ void __launch_bounds__(FAST_THREADS, 1) perq_fast_kernel(FastParams p
                 have_exact = true;
                 return true;
             };
+            // (a wait that runs out only records the error: the warp must go on to the row's next barrier, or
+            // its siblings would be stranded there; the fp32 zero point then stands)
             if (live && !(fabsf(vmin - z32) <= 0.5f - wz)) {
-                if (!fetch_exact()) {
-                    if (lane == 0) atomicOr(&g_perq_device_error, 2u);
-                    return;
-                }
-                z32 = (float)z_ex;
+                if (fetch_exact()) z32 = (float)z_ex;
+                else if (lane == 0) atomicOr(&g_perq_device_error, 2u);
             }
 
             // ---- quantise: the magic constant carries -z, so the low nibble of the sum is the code
@@ -1244,14 +1349,12 @@ __global__ void __launch_bounds__(FAST_THREADS, 1) perq_fast_kernel(FastParams p
 
             // ---- slots whose two sums differ: all four codes exactly (a carry may have reached a neighbour)
             if (__any_sync(0xffffffffu, tie_any != 0u)) {
-                if (!have_exact && !fetch_exact()) {
-                    if (lane == 0) atomicOr(&g_perq_device_error, 2u);
-                    return;
-                }
+                const bool got_exact = have_exact || fetch_exact();
+                if (!got_exact && lane == 0) atomicOr(&g_perq_device_error, 2u);     // the codes stay as staged
                 // elements whose two sums differ; all four of a slot in which a sum left 0..15 (its carry
                 // may have reached a neighbour)
                 uint32_t fm = 0u;
-                if (tie_any != 0u) {
+                if (got_exact && tie_any != 0u) {
                     const float t_lo = 12582912.0f, t_hi = 12582927.0f;
 #pragma unroll
                     for (int s = 0; s < 8; ++s) {
@@ -1323,7 +1426,7 @@ __global__ void __launch_bounds__(FAST_THREADS, 1) perq_fast_kernel(FastParams p
                 const int srcq = (lane & 28) | ((__ffs(cl4) - 1) & 3);
                 const uint32_t smq = __shfl_sync(0xffffffffu, slot_mask, srcq);
                 // (deferring pays while a block is short and the row can be re-read contiguously)
-                constexpr bool DEFER = !PERM && LOG2B <= 5;
+                constexpr bool DEFER = !PERM && !SWIGLU && LOG2B <= 5;
                 const bool simple = DEFER && cl4 != 0u && (cl4 & (cl4 - 1)) == 0u && (smq & (smq - 1)) == 0u;
                 if (simple) {
                     const int sl = __ffs(smq) - 1;
@@ -1398,7 +1501,7 @@ __global__ void __launch_bounds__(FAST_THREADS, 1) perq_fast_kernel(FastParams p
                 const unsigned cl = __ballot_sync(0xffffffffu, slot_mask != 0u);
                 const int src = __ffs(cl) - 1;
                 const uint32_t sm = __shfl_sync(0xffffffffu, slot_mask, src);
-                if (ncand == 1 && (cl & (cl - 1)) == 0u && (sm & (sm - 1)) == 0u) {
+                if (!SWIGLU && ncand == 1 && (cl & (cl - 1)) == 0u && (sm & (sm - 1)) == 0u) {
                     // one slot holds the maximum: record it, the scale is stored later
                     const int sl = __ffs(sm) - 1, sg = src >> 2;
                     const int pch = sg * 8 + (sl ^ ((sg & 3) & ~PM));
@@ -1532,11 +1635,15 @@ __global__ void __launch_bounds__(FAST_THREADS, 1) perq_fast_kernel(FastParams p
                     unsigned long long d = (1ull << 63) | my_pos;
                     if (my_pos == 0xffffffffu) {      // published by a candidate warp of the row: wait for it
                         uint32_t spin = 0;
+                        bool gave_up = false;
                         while (ld_volatile_shared_u32(&wflag[pidx]) != it + 1u) {
-                            if (++spin >= WAIT_SPIN_LIMIT) {
-                                if (lane == 0) atomicOr(&g_perq_device_error, 2u);
-                                return;
-                            }
+                            if (++spin >= WAIT_SPIN_LIMIT) { gave_up = true; break; }
+                        }
+                        if (gave_up) {
+                            // the codes stay as staged; the warp goes on (leaving would strand its siblings at the
+                            // row's next barrier)
+                            if (lane == 0) atomicOr(&g_perq_device_error, 2u);
+                            fm = 0u;
                         }
                         __threadfence_block();
                         d = *reinterpret_cast<volatile unsigned long long *>(&wpub[pidx]);

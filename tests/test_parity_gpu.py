@@ -311,6 +311,26 @@ def test_host_buffer_entry_point(B, oracle):
     compare_quantized("int4", codes.numpy(), scales.numpy(), ora)
 
 
+@pytest.mark.parametrize("fmt,group", [("int4", 0), ("mxfp4", 32), ("int4", 128)])
+def test_host_entry_point_in_chunks_matches_the_device_entry_point(B, fmt, group):
+    """From 4096 rows on, the host-buffer call works in chunks of rows with the two copy
+    directions overlapped; its bytes must equal those of one device call."""
+    T, d, b = 5001, 2048, 32
+    bits, _ = inputs.student_t_outliers(T, d, 3.0, 8, 100.0, seed=7000)
+    f = FMT[fmt]
+    x = to_dev(bits)
+    codes_d, scales_d = B.perq_rotate_quantize(x, None, b, f, group)
+    torch.cuda.synchronize()
+    xh = torch.from_numpy(bits.view(np.int16).copy()).view(torch.bfloat16).pin_memory()
+    ws = torch.empty(B.perq_host_workspace_bytes(T, d, f, group), dtype=torch.uint8, device="cuda")
+    codes_h = torch.empty_like(codes_d, device="cpu").pin_memory()
+    scales_h = torch.empty_like(scales_d, device="cpu").pin_memory()
+    for _ in range(2):
+        codes_h.zero_(); scales_h.zero_()
+        B.perq_rotate_quantize_host(xh, None, b, f, group, codes_h, scales_h, ws)
+        assert torch.equal(codes_h, codes_d.cpu()) and torch.equal(scales_h, scales_d.cpu())
+
+
 def test_invalid_permutation_is_reported_not_faulted(B):
     d = 2048
     bad = inputs.random_perm(d, 3)
