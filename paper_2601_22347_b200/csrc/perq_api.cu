@@ -17,6 +17,7 @@
 #include "perq_generic.cuh"
 #include "perq_fast.cuh"
 #include "perq_tok.cuh"
+#include "perq_mx.cuh"
 #include "perq_stats.cuh"
 #include "perq_diag.cuh"
 #include "perq_massdiff.cuh"
@@ -229,6 +230,29 @@ int launch_fast_long(int xb, int G, const perq::FastParams &p, int grid, cudaStr
     }
 }
 
+// Lean MXFP4 kernel: unpermuted, d % 2048 == 0, b <= 128 (a warp's unit is two adjacent segments).
+template <int LOG2B>
+int launch_mx_inst(const perq::FastParams &p, int grid, cudaStream_t st)
+{
+    auto kernel = perq::perq_mx_kernel<LOG2B>;
+    if (int rc = allow_smem(kernel, perq::MxSmem::total)) return rc;
+    if (launch_overlapped(kernel, grid, perq::FAST_THREADS, perq::MxSmem::total, st, p) != cudaSuccess) {
+        (void)cudaGetLastError();
+        return PERQ_ERR_CUDA;
+    }
+    return PERQ_OK;
+}
+
+int launch_mx(int log2b, const perq::FastParams &p, int grid, cudaStream_t st)
+{
+    switch (log2b) {
+    case 4: return launch_mx_inst<4>(p, grid, st);
+    case 5: return launch_mx_inst<5>(p, grid, st);
+    case 6: return launch_mx_inst<6>(p, grid, st);
+    default: return launch_mx_inst<7>(p, grid, st);
+    }
+}
+
 // Lean per-token kernel: INT4 or E2M1 with one scale per token, unpermuted, d in {2048, 4096, 8192}, b <= 128.
 template <int LOG2B, int MODE, int LOG2G>
 int launch_tok_inst(const perq::FastParams &p, int grid, cudaStream_t st)
@@ -323,6 +347,12 @@ int try_launch_fast(const void *x, const int32_t *perm, int64_t T, int32_t d, in
         const int tok_grid = (int)std::min<long long>((T + tok_groups - 1) / tok_groups, sms);
         return mode == perq::MODE_TOKEN ? launch_tok<perq::MODE_TOKEN>(segs, ilog2(b), p, tok_grid, st)
                                         : launch_tok<perq::MODE_FP4>(segs, ilog2(b), p, tok_grid, st);
+    }
+    if (mode == perq::MODE_MX && !permuted && !full && !longb && segs % perq::MX_SPW == 0) {
+        const long long mx_units = (long long)T * segs / perq::MX_SPW;
+        p.units_total = (uint32_t)mx_units;
+        const int mx_grid = (int)std::min<long long>((mx_units + perq::FAST_WARPS - 1) / perq::FAST_WARPS, sms);
+        return launch_mx(ilog2(b), p, mx_grid, st);
     }
     if (full)
         return mode == perq::MODE_MX ? launch_fast_full<perq::MODE_MX>(G, p, grid, st)

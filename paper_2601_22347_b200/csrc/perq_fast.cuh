@@ -299,8 +299,19 @@ __device__ __forceinline__ float max3abs(float acc, float a, float b) { return f
 __device__ __forceinline__ uint32_t cvt_e2m1x4(float a, float b, float c, float d)
 {
     uint32_t r;
-    asm("{ .reg .b8 t0, t1; .reg .b16 h; cvt.rn.satfinite.e2m1x2.f32 t0, %2, %1; cvt.rn.satfinite.e2m1x2.f32 t1, %4, %3; "
-        "mov.b16 h, {t0, t1}; cvt.u32.u16 %0, h; }" : "=r"(r) : "f"(a), "f"(b), "f"(c), "f"(d));
+    asm("{ .reg .b8 t0, t1; .reg .b32 w0, w1; cvt.rn.satfinite.e2m1x2.f32 t0, %2, %1; cvt.rn.satfinite.e2m1x2.f32 t1, %4, %3; "
+        "cvt.u32.u8 w0, t0; cvt.u32.u8 w1, t1; mad.lo.u32 %0, w1, 256, w0; }" : "=r"(r) : "f"(a), "f"(b), "f"(c), "f"(d));
+    return r;
+}
+
+// Eight fp32 values -> two sets of four E2M1 codes in one word: bits 0..15 from (a0..a3), bits 16..31 from
+// (b0..b3), first operand of a set in its lowest nibble.
+__device__ __forceinline__ uint32_t cvt_e2m1x4_pair(float a0, float a1, float a2, float a3, float b0, float b1, float b2, float b3)
+{
+    uint32_t r;
+    asm("{ .reg .b8 t0, t1, t2, t3; cvt.rn.satfinite.e2m1x2.f32 t0, %2, %1; cvt.rn.satfinite.e2m1x2.f32 t1, %4, %3; "
+        "cvt.rn.satfinite.e2m1x2.f32 t2, %6, %5; cvt.rn.satfinite.e2m1x2.f32 t3, %8, %7; mov.b32 %0, {t0, t1, t2, t3}; }"
+        : "=r"(r) : "f"(a0), "f"(a1), "f"(a2), "f"(a3), "f"(b0), "f"(b1), "f"(b2), "f"(b3));
     return r;
 }
 

@@ -52,6 +52,8 @@ def units_per_group(T, d, b, fmt, group, permuted):
     if fmt in ("int4", "fp4") and per_token and not permuted and b <= 128 and segs in (2, 4, 8):
         G = segs // 2        # the lean per-token kernel: a warp owns two adjacent segments of a row
     units = T * segs // G
+    if fmt == "mxfp4" and not permuted and b <= 128 and segs % 2 == 0:
+        units //= 2          # the lean MXFP4 kernel: a warp's unit is two adjacent segments
     groups_per_cta = WARPS_PER_CTA // G
     grid = min((units + groups_per_cta - 1) // groups_per_cta, SMS)
     return -(-units // (grid * groups_per_cta))
