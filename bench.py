@@ -46,6 +46,8 @@ def kernel_sources_hash():
     csrc = os.path.join(ROOT, "paper_2601_22347_b200", "csrc")
     h = hashlib.sha256()
     for name in sorted(os.listdir(csrc)):
+        if not os.path.isfile(os.path.join(csrc, name)):
+            continue
         with open(os.path.join(csrc, name), "rb") as f:
             h.update(name.encode() + b"\0" + f.read())
     return h.hexdigest()

@@ -545,3 +545,59 @@ int perq_oracle_massdiff_perm(const double *chan_abs_sum, int32_t d, int32_t b, 
     free(order); free(mass); free(fill);
     return 0;
 }
+
+/* ---------------------------------------------------------------- comparison permutations
+ * Appendix C, paragraph "Permutations" (Table "permute_fn_ablations"): "absmax" permutes coordinates in
+ * descending order of the maximum absolute value observed over the calibration sample; "ZigZag" assigns
+ * coordinates to blocks in a zigzag pattern over a coordinate-wise l-infinity statistic (the cited method's
+ * strategy; Sec. 4.2 mentions it as the alternative to MassDiff).  The paper prints neither procedure.
+ * Readings taken here (parity unpinned against the authors' code): both visit channels by descending
+ * statistic, equal values by ascending channel; absmax returns that order; ZigZag deals the visiting order to
+ * the n = d / b blocks back and forth -- ranks 0..n-1 to blocks 0..n-1, ranks n..2n-1 to blocks n-1..0, and so
+ * on -- so that every block receives one channel of every round and block j's r-th slot is round r.
+ *
+ * chan_abs_max[c] = max_t |x[t, c]| is the statistic of both. */
+int perq_oracle_chan_abs_max(const uint16_t *x, int64_t T, int32_t d, double *chan_abs_max)
+{
+    if (T < 0 || d <= 0 || !x || !chan_abs_max) return 1;
+    for (int32_t c = 0; c < d; ++c) chan_abs_max[c] = 0.0;
+    for (int64_t t = 0; t < T; ++t)
+        for (int32_t c = 0; c < d; ++c) {
+            const double a = fabs(bf16_to_double(x[(size_t)t * d + c]));
+            if (a > chan_abs_max[c]) chan_abs_max[c] = a;
+        }
+    return 0;
+}
+
+/* visiting order: descending statistic, equal values by ascending channel (insertion sort: stable) */
+static void descending_order(const double *stat, int32_t d, int32_t *order)
+{
+    for (int32_t i = 0; i < d; ++i) {
+        int32_t k = i;
+        while (k > 0 && stat[order[k - 1]] < stat[i]) { order[k] = order[k - 1]; --k; }
+        order[k] = i;
+    }
+}
+
+int perq_oracle_absmax_perm(const double *chan_abs_max, int32_t d, int32_t *perm)
+{
+    if (d <= 0 || !chan_abs_max || !perm) return 1;
+    descending_order(chan_abs_max, d, perm);
+    return 0;
+}
+
+int perq_oracle_zigzag_perm(const double *chan_abs_max, int32_t d, int32_t b, int32_t *perm)
+{
+    if (d <= 0 || b <= 0 || d % b != 0 || !chan_abs_max || !perm) return 1;
+    int32_t *order = (int32_t *)malloc(sizeof(int32_t) * (size_t)d);
+    if (!order) return 3;
+    descending_order(chan_abs_max, d, order);
+    const int32_t n = d / b;
+    for (int32_t r = 0; r < d; ++r) {
+        const int32_t round = r / n, pos = r % n;
+        const int32_t block = (round % 2 == 0) ? pos : n - 1 - pos;
+        perm[(size_t)block * b + round] = order[r];
+    }
+    free(order);
+    return 0;
+}

@@ -193,3 +193,26 @@ def massdiff_perm(chan_abs_sum, b: int) -> np.ndarray:
     perm = np.empty(d, np.int32)
     _check(_load().perq_oracle_massdiff_perm(_p(a), C.c_int32(d), C.c_int32(b), _p(perm)), "massdiff_perm")
     return perm
+
+
+def chan_abs_max(x) -> np.ndarray:
+    """max_t |x[t, c]| per channel, fp64."""
+    x = _x(x)
+    T, d = x.shape
+    out = np.empty(d, np.float64)
+    _check(_load().perq_oracle_chan_abs_max(_p(x), C.c_int64(T), C.c_int32(d), _p(out)), "chan_abs_max")
+    return out
+
+
+def absmax_perm(stat) -> np.ndarray:
+    a = np.ascontiguousarray(stat, dtype=np.float64)
+    perm = np.empty(a.shape[0], np.int32)
+    _check(_load().perq_oracle_absmax_perm(_p(a), C.c_int32(a.shape[0]), _p(perm)), "absmax_perm")
+    return perm
+
+
+def zigzag_perm(stat, b: int) -> np.ndarray:
+    a = np.ascontiguousarray(stat, dtype=np.float64)
+    perm = np.empty(a.shape[0], np.int32)
+    _check(_load().perq_oracle_zigzag_perm(_p(a), C.c_int32(a.shape[0]), C.c_int32(b), _p(perm)), "zigzag_perm")
+    return perm
