@@ -266,6 +266,25 @@ int perq_validate_perm(const int32_t *perm, int32_t d, int32_t *status_dev, void
 int perq_massdiff_perm(const float *chan_abs_sum_host, int32_t d, int32_t b, int32_t *perm_host);
 
 /*
+ * perq_chan_abs_max, perq_absmax_perm, perq_zigzag_perm -- the permutations the paper compares MassDiff with
+ * (Appendix C, paragraph "Permutations", Table "permute_fn_ablations"; Sec. 4.2 on the zigzag assignment).
+ *
+ *   perq_chan_abs_max   device: chan_abs_max[c] = max_t |x[t, c]| (float [d], written in full; x bf16 [T, d]
+ *                       device, 16-byte aligned; d % 32 == 0).  Enqueues a memset and one kernel on `stream`.
+ *   perq_absmax_perm    host only: the channels in descending order of that maximum (equal values: lower
+ *                       channel first).
+ *   perq_zigzag_perm    host only: the same visiting order dealt to the n = d / b blocks back and forth
+ *                       (ranks 0..n-1 to blocks 0..n-1, ranks n..2n-1 to blocks n-1..0, ...); slot r of
+ *                       block j holds the channel that round r gave it: perm[j*b + r].
+ * The paper prints neither procedure; these are the readings this library takes.  Host arrays: float [d] in,
+ * int32 [d] out; the result is a `perm` argument of perq_rotate_quantize / perq_block_l1_stats.
+ * Errors: NULL, SHAPE, BLOCK (b < 1 or d % b != 0), ALIGN, CUDA.
+ */
+int perq_chan_abs_max(const void *x, int64_t T, int32_t d, float *chan_abs_max, void *stream);
+int perq_absmax_perm(const float *chan_abs_max_host, int32_t d, int32_t *perm_host);
+int perq_zigzag_perm(const float *chan_abs_max_host, int32_t d, int32_t b, int32_t *perm_host);
+
+/*
  * perq_massdiff_perm_device -- Algorithm 1 (MassDiff) on the device: the same permutation as
  * perq_massdiff_perm, entry for entry, from a device array, so that a calibration pass (statistic ->
  * permutation -> permuted rotate+quantize) needs no copy to the host.

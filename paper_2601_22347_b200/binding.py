@@ -58,6 +58,11 @@ def load() -> C.CDLL:
         lib.perq_validate_perm.argtypes = [vp, i32, vp, vp]
         lib.perq_massdiff_perm.argtypes = [vp, i32, i32, vp]
         lib.perq_massdiff_perm_device.argtypes = [vp, i32, i32, vp, vp, sz, vp]
+        lib.perq_chan_abs_max.argtypes = [vp, i64, i32, vp, vp]
+        lib.perq_absmax_perm.argtypes = [vp, i32, vp]
+        lib.perq_zigzag_perm.argtypes = [vp, i32, i32, vp]
+        for name in ("perq_chan_abs_max", "perq_absmax_perm", "perq_zigzag_perm"):
+            getattr(lib, name).restype = C.c_int
         lib.perq_device_error.argtypes = [C.POINTER(C.c_uint32)]
         lib.perq_device_error.restype = C.c_int
         lib.perq_device_error_clear.argtypes = []
@@ -253,6 +258,32 @@ def perq_massdiff_perm_device(chan_abs_sum: torch.Tensor, b: int, perm: Optional
     _check(load().perq_massdiff_perm_device(_ptr(chan_abs_sum), d, b, _ptr(perm), _ptr(workspace),
                                             workspace.numel() * workspace.element_size(), _stream(stream)),
            "perq_massdiff_perm_device")
+    return perm
+
+
+def perq_chan_abs_max(x: torch.Tensor, out: Optional[torch.Tensor] = None, stream=None) -> torch.Tensor:
+    """x: bf16 CUDA tensor [T, d]; returns fp32 CUDA tensor [d] (nothing is synchronised)."""
+    assert x.is_cuda and x.dtype == torch.bfloat16 and x.dim() == 2 and x.is_contiguous()
+    T, d = x.shape
+    if out is None:
+        out = torch.empty(d, dtype=torch.float32, device=x.device)
+    _check(load().perq_chan_abs_max(_ptr(x), T, d, _ptr(out), _stream(stream)), "perq_chan_abs_max")
+    return out
+
+
+def perq_absmax_perm(chan_abs_max_host: np.ndarray) -> np.ndarray:
+    """Host only.  float32 [d] numpy array in, int32 [d] out."""
+    a = np.ascontiguousarray(chan_abs_max_host, dtype=np.float32)
+    perm = np.empty(a.shape[0], np.int32)
+    _check(load().perq_absmax_perm(a.ctypes.data_as(C.c_void_p), a.shape[0], perm.ctypes.data_as(C.c_void_p)), "perq_absmax_perm")
+    return perm
+
+
+def perq_zigzag_perm(chan_abs_max_host: np.ndarray, b: int) -> np.ndarray:
+    """Host only.  float32 [d] numpy array in, int32 [d] out."""
+    a = np.ascontiguousarray(chan_abs_max_host, dtype=np.float32)
+    perm = np.empty(a.shape[0], np.int32)
+    _check(load().perq_zigzag_perm(a.ctypes.data_as(C.c_void_p), a.shape[0], b, perm.ctypes.data_as(C.c_void_p)), "perq_zigzag_perm")
     return perm
 
 

@@ -800,6 +800,59 @@ int perq_massdiff_perm_device(const float *chan_abs_sum, int32_t d, int32_t b, i
     return cudaGetLastError() == cudaSuccess ? PERQ_OK : PERQ_ERR_CUDA;
 }
 
+int perq_chan_abs_max(const void *x, int64_t T, int32_t d, float *chan_abs_max, void *stream)
+{
+    if (T < 0 || d <= 0 || d % 32 != 0 || d > PERQ_MAX_D) return PERQ_ERR_SHAPE;
+    if (!chan_abs_max || (T > 0 && !x)) return PERQ_ERR_NULL;
+    if (!aligned16(x) || (reinterpret_cast<uintptr_t>(chan_abs_max) & 3u) != 0) return PERQ_ERR_ALIGN;
+    cudaStream_t st = static_cast<cudaStream_t>(stream);
+    if (cudaMemsetAsync(chan_abs_max, 0, (size_t)d * sizeof(float), st) != cudaSuccess) return PERQ_ERR_CUDA;
+    if (T == 0) return PERQ_OK;
+    const int col_ctas = (d / 8 + 255) / 256;
+    const long long want_slabs = std::max<long long>(1, (4ll * 148 + col_ctas - 1) / col_ctas);
+    const long long rows_per = std::max<long long>(8, (T + want_slabs - 1) / want_slabs);
+    const long long slabs = (T + rows_per - 1) / rows_per;
+    if (slabs > 65535) return PERQ_ERR_SHAPE;
+    perq::perq_chan_abs_max_kernel<<<dim3((unsigned)col_ctas, (unsigned)slabs), 256, 0, st>>>(
+        static_cast<const uint16_t *>(x), (long long)T, d, (int)rows_per, chan_abs_max);
+    return cudaGetLastError() == cudaSuccess ? PERQ_OK : PERQ_ERR_CUDA;
+}
+
+namespace {
+// channels by descending statistic, equal values by ascending channel
+std::vector<int32_t> descending_channels(const float *stat, int32_t d)
+{
+    std::vector<int32_t> order(d);
+    for (int i = 0; i < d; ++i) order[i] = i;
+    std::stable_sort(order.begin(), order.end(), [&](int32_t l, int32_t r) { return stat[l] > stat[r]; });
+    return order;
+}
+}  // namespace
+
+int perq_absmax_perm(const float *chan_abs_max_host, int32_t d, int32_t *perm_host)
+{
+    if (!chan_abs_max_host || !perm_host) return PERQ_ERR_NULL;
+    if (d <= 0) return PERQ_ERR_SHAPE;
+    const std::vector<int32_t> order = descending_channels(chan_abs_max_host, d);
+    std::copy(order.begin(), order.end(), perm_host);
+    return PERQ_OK;
+}
+
+int perq_zigzag_perm(const float *chan_abs_max_host, int32_t d, int32_t b, int32_t *perm_host)
+{
+    if (!chan_abs_max_host || !perm_host) return PERQ_ERR_NULL;
+    if (d <= 0) return PERQ_ERR_SHAPE;
+    if (b < 1 || d % b != 0) return PERQ_ERR_BLOCK;
+    const std::vector<int32_t> order = descending_channels(chan_abs_max_host, d);
+    const int32_t n = d / b;
+    for (int32_t r = 0; r < d; ++r) {
+        const int32_t round = r / n, pos = r - round * n;
+        const int32_t block = (round & 1) ? n - 1 - pos : pos;       // forwards over the blocks, then back
+        perm_host[(size_t)block * b + round] = order[r];
+    }
+    return PERQ_OK;
+}
+
 int perq_massdiff_perm(const float *chan_abs_sum_host, int32_t d, int32_t b, int32_t *perm_host)
 {
     if (!chan_abs_sum_host || !perm_host) return PERQ_ERR_NULL;

@@ -266,6 +266,36 @@ __global__ void __launch_bounds__(256) perq_stats_reduce_kernel(const float *ws_
 }
 
 // perm[0..d) is a permutation?  status: bit0 = out of range, bit1 = duplicate.
+// Per-channel maximum magnitude over the rows: chan_abs_max[c] = max_t |x[t, c]| (the statistic of the absmax and
+// zigzag comparison permutations).  A CTA takes a slab of rows and 2048 channels; a thread keeps the maxima of
+// eight adjacent channels as bf16 magnitude patterns (which order like the values), two per word, and merges
+// them into the output with atomicMax on the fp32 bit patterns (non-negative floats order like unsigned
+// integers; a maximum does not depend on the order of its operands: deterministic).  out must be zero on entry.
+__global__ void __launch_bounds__(256) perq_chan_abs_max_kernel(const uint16_t *x, long long T, int d, int rows_per_cta, float *out)
+{
+    const int c0 = (blockIdx.x * 256 + threadIdx.x) * 8;
+    if (c0 >= d) return;
+    const long long t0 = (long long)blockIdx.y * rows_per_cta;
+    const long long t1 = min(T, t0 + rows_per_cta);
+    uint32_t m[4] = {0u, 0u, 0u, 0u};
+    const uint4 *src = reinterpret_cast<const uint4 *>(x + t0 * d + c0);
+    const size_t step = (size_t)d / 8;
+#pragma unroll 4
+    for (long long t = t0; t < t1; ++t, src += step) {
+        const uint4 w = __ldg(src);
+        m[0] = __vmaxu2(m[0], w.x & 0x7fff7fffu);
+        m[1] = __vmaxu2(m[1], w.y & 0x7fff7fffu);
+        m[2] = __vmaxu2(m[2], w.z & 0x7fff7fffu);
+        m[3] = __vmaxu2(m[3], w.w & 0x7fff7fffu);
+    }
+    uint32_t *o = reinterpret_cast<uint32_t *>(out) + c0;
+#pragma unroll
+    for (int k = 0; k < 4; ++k) {
+        atomicMax(o + 2 * k, m[k] << 16);
+        atomicMax(o + 2 * k + 1, m[k] & 0xffff0000u);
+    }
+}
+
 __global__ void perq_validate_perm_kernel(const int32_t *perm, int d, int32_t *status)
 {
     extern __shared__ uint32_t bitmap[];

@@ -130,3 +130,15 @@ def test_host_massdiff_hand_example(lib):
     assert B.perq_massdiff_perm(np.array([9, 8, 7, 6, 5, 4, 3, 2], np.float32), 4).tolist() == [0, 3, 4, 7, 1, 2, 5, 6]
     with pytest.raises(B.PerqError):
         B.perq_massdiff_perm(np.ones(10, np.float32), 4)
+
+
+def test_comparison_permutations_match_the_oracle(oracle):
+    from paper_2601_22347_b200 import binding as B
+    rng = np.random.default_rng(77)
+    for d, b in ((256, 16), (2048, 32), (96, 8), (64, 64)):
+        s = (rng.exponential(size=d) * np.where(rng.random(d) < 0.05, 40.0, 1.0)).astype(np.float32)
+        s[rng.integers(0, d, 8)] = s[0]
+        assert np.array_equal(B.perq_absmax_perm(s), oracle.absmax_perm(s.astype(np.float64)))
+        assert np.array_equal(B.perq_zigzag_perm(s, b), oracle.zigzag_perm(s.astype(np.float64), b))
+    with pytest.raises(RuntimeError):
+        B.perq_zigzag_perm(np.ones(10, np.float32), 4)

@@ -729,3 +729,15 @@ def test_calibration_pass_stays_on_the_device(B, oracle):
     assert np.array_equal(perm.cpu().numpy(), ref_perm)
     ora = oracle.rotate_quantize(w.x, ref_perm, 32, FMT["mxfp4"], 32, want_pre=True)
     compare_quantized("mxfp4", codes.cpu().numpy(), scales.cpu().numpy(), ora)
+
+
+@pytest.mark.parametrize("T,d", [(1, 64), (37, 2048), (4096, 8192), (1000, 14336), (5, 32768)])
+def test_chan_abs_max_and_the_comparison_permutations(B, oracle, T, d):
+    bits, _ = inputs.student_t_outliers(T, d, 3.0, max(1, d // 512), 100.0, seed=9500 + d)
+    got = B.perq_chan_abs_max(to_dev(bits))
+    torch.cuda.synchronize()
+    ref = oracle.chan_abs_max(bits)
+    assert np.array_equal(got.cpu().numpy().astype(np.float64), ref)        # a maximum of bf16 magnitudes: exact
+    b = 32
+    assert np.array_equal(B.perq_zigzag_perm(got.cpu().numpy(), b), oracle.zigzag_perm(ref, b))
+    assert np.array_equal(B.perq_absmax_perm(got.cpu().numpy()), oracle.absmax_perm(ref))
