@@ -1,9 +1,10 @@
 // Per-token rotate+quantize kernel with a lean inner loop: unpermuted rows of d = 2048, 4096 or 8192
-// channels, Hadamard blocks of 16 .. 128, symmetric INT4 or E2M1 codes with one fp32 scale per token.  Same data path, lane layout, error model and exactness rules as perq_fast.cuh (whose helpers it
-// uses); what differs is where the rare work lives, because this kernel is bound by the number of warp
-// instructions an iteration issues (measured: about 0.15 us of a 16384 x 4096 call per instruction and
-// 1024-element segment), and because the G warps of a row move in lockstep (one named barrier per row), so
-// work that only one of them does delays all of them:
+// channels, Hadamard blocks of 16 .. 128, symmetric INT4 or E2M1 codes with one fp32 scale per token.
+//
+// Same data path, lane layout, error model and exactness rules as perq_fast.cuh (whose helpers it uses).
+// What differs is the loop around a segment: this path is bound by the number of warp instructions it issues
+// (measured: 0.1 to 0.2 us of a 16384 x 4096 call per instruction and 1024-element segment), and a good half
+// of the group kernel's instructions were not the rotation, the maxima or the quantiser:
 //
 //   * A warp owns two adjacent 1024-element segments of a row, and a row is shared by W = d / 2048 warps.
 //     What an iteration costs once -- the wait for the staged row, the exchange of maxima around the row's
