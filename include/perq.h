@@ -109,6 +109,9 @@ typedef enum {
  * Codes and scales are deterministic (bit-identical from run to run).  Which kernel serves a call depends
  * on its shape; every kernel stores the fp32 rounding of the exact scale up to one more rounding of a
  * constant factor, so scales of the same row from different shapes' kernels agree to 1 ulp, not bit for bit.
+ * Range limit: a token whose largest |y| lies below about 2^-120 (every input subnormal or nearly so) gets
+ * the exact scale but all-zero INT4/FP4 codes from the tensor-core kernels, because the fp32 reciprocal of
+ * such a scale overflows; the definition would give +-7 at the maximum.
  */
 int perq_rotate_quantize(const void *x, const int32_t *perm, int64_t T, int32_t d, int32_t b,
                          int32_t fmt, int32_t group, void *out_codes, void *out_scales,
