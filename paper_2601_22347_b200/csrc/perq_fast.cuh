@@ -705,35 +705,46 @@ __device__ __forceinline__ void serve_asym_requests(const FastParams &p, const u
 // ---------------------------------------------------------------- gated activation in front of the rotation
 //
 // h = Swish(g) * u, Swish(g) = g / (1 + exp(-g)), rounded once to bf16 (round to nearest even): the input of the
-// online rotation in a gated feedforward block.  The fp32 evaluation below is accurate to about 5e-7 relative
-// (exp2 of a compensated argument, one approximate reciprocal, three roundings); a result whose low 16 bits
-// are within SWIGLU_MARGIN fp32 ulps (at least 9.5e-7 relative) of the halfway pattern 0x8000 could round to
-// either neighbour, and is evaluated again in fp64, as are arguments beyond +-80 and results deep in the
-// subnormal range, where the relative bound does not hold.
-constexpr uint32_t SWIGLU_MARGIN = 16;
-
-__device__ __forceinline__ float ex2_approx(float x)
+// online rotation in a gated feedforward block.  The fp32 evaluation below works on pairs (packed fp32
+// instructions) and is accurate to 11 * 2^-24 = 6.6e-7 relative wherever no intermediate leaves the normal
+// range: exp2 of a compensated argument (2^-22 for the approximation, 2^-24 each for the correction factor and
+// its product; weighted by e / (1 + e) <= 1), the sum 1 + e (2^-24), one approximate reciprocal (2^-23), two
+// products (2^-24 each).  A result whose low half-word lies in
+// [0x7fe0, 0x801f] -- within 31 fp32 ulps, at least 1.8e-6 relative, of the halfway pattern 0x8000 -- could
+// round to either neighbour and is evaluated again in fp64; so is every result that is zero, below 2^-100 or
+// not finite, which covers the arguments whose exponential or reciprocal left the normal range (they give a
+// zero or an infinity here) and the subnormal results, where the relative bound does not hold.
+__device__ __forceinline__ float ex2_ftz(float x)
 {
     float r;
-    asm("ex2.approx.f32 %0, %1;" : "=f"(r) : "f"(x));
+    asm("ex2.approx.ftz.f32 %0, %1;" : "=f"(r) : "f"(x));
     return r;
 }
-__device__ __forceinline__ float swish_mul_f32(float g, float u)
+__device__ __forceinline__ float rcp_ftz(float x)
+{
+    float r;
+    asm("rcp.approx.ftz.f32 %0, %1;" : "=f"(r) : "f"(x));
+    return r;
+}
+__device__ __forceinline__ f32x2 swish_mul2(f32x2 g, f32x2 u)
 {
     const float L2E_HI = 1.44269502162933349609375f, L2E_LO = 1.925963033500011e-8f;      // log2(e) = hi + lo
-    const float t = -g * L2E_HI;
-    float r = fmaf(-g, L2E_HI, -t);                  // what the rounding of t dropped
-    r = fmaf(-g, L2E_LO, r);
-    float e = ex2_approx(t);
-    e = fmaf(e, r * 0.693147182464599609375f, e);    // 2^(t + r) = 2^t (1 + r ln 2) to first order (|r| < 2^-17)
-    return __fdividef(g, 1.0f + e) * u;
+    const float LN2 = 0.693147182464599609375f;
+    const f32x2 tp = mul2(g, pack2(L2E_HI, L2E_HI));                 // -t, rounded
+    f32x2 r = fma2(g, pack2(-L2E_HI, -L2E_HI), tp);                  // t_exact - t: what the rounding dropped
+    r = fma2(g, pack2(-L2E_LO, -L2E_LO), r);
+    f32x2 e = pack2(ex2_ftz(-tp.x), ex2_ftz(-tp.y));
+    // 2^(t + r) = 2^t (1 + r ln 2) to first order (|r| < 2^-17); as a product, so that an infinite 2^t stays one
+    e = mul2(e, fma2(r, pack2(LN2, LN2), pack2(1.0f, 1.0f)));
+    const f32x2 den = add2(e, pack2(1.0f, 1.0f));
+    const f32x2 rc = pack2(rcp_ftz(den.x), rcp_ftz(den.y));
+    return mul2(mul2(g, rc), u);                                     // (finite inputs never give a NaN in this order)
 }
-__device__ __forceinline__ bool swiglu_needs_fp64(float h, float g)
+// zero if and only if the low half-word of an fp32 pattern lies in [0x7fe0, 0x801f]
+__device__ __forceinline__ uint32_t swiglu_midpoint_key(float h) { return ((__float_as_uint(h) + 0x20u) & 0xffc0u) ^ 0x8000u; }
+__device__ __forceinline__ bool swiglu_needs_fp64(float h)
 {
-    const uint32_t bits = __float_as_uint(h);
-    const uint32_t off = ((bits & 0xffffu) - (0x8000u - SWIGLU_MARGIN)) & 0xffffu;
-    const uint32_t mag = bits & 0x7fffffffu;
-    return off <= 2u * SWIGLU_MARGIN || fabsf(g) > 80.0f || (mag != 0u && mag < 0x0d800000u) || mag >= 0x7f800000u;
+    return swiglu_midpoint_key(h) == 0u || !(fabsf(h) >= 0x1p-100f) || !(fabsf(h) <= 3.4028234663852886e38f);
 }
 // A finite double to bf16 bits, one rounding to nearest even (integer arithmetic on the double's fields).
 __device__ __forceinline__ uint32_t double_to_bf16_bits(double v)
@@ -756,23 +767,38 @@ __device__ __forceinline__ uint32_t double_to_bf16_bits(double v)
 }
 __device__ __noinline__ uint32_t swiglu_fp64_bits(float g, float u)
 {
+    if (g == 0.0f || u == 0.0f) return ((__float_as_uint(g) ^ __float_as_uint(u)) >> 16) & 0x8000u;      // a signed zero
     const double gd = (double)g;
     return double_to_bf16_bits(gd / (1.0 + exp(-gd)) * (double)u);
 }
-// One word (two bf16 values) of h from one word of each projection.
-__device__ __forceinline__ uint32_t swiglu_word(uint32_t gw, uint32_t uw)
+// Eight values of h (one 16-byte piece, four words of two bf16) from the matching pieces of the projections.
+// The three reasons for the fp64 route are reduced over the piece (one integer minimum, the smallest and the
+// largest magnitude) and tested once.
+__device__ __forceinline__ void swiglu_piece(const uint32_t (&gw)[4], const uint32_t (&uw)[4], uint32_t (&hw)[4])
 {
-    const float g0 = __uint_as_float(gw << 16), g1 = __uint_as_float(gw & 0xffff0000u);
-    const float u0 = __uint_as_float(uw << 16), u1 = __uint_as_float(uw & 0xffff0000u);
-    const float h0 = swish_mul_f32(g0, u0), h1 = swish_mul_f32(g1, u1);
-    uint32_t w;
-    asm("cvt.rn.bf16x2.f32 %0, %1, %2;" : "=r"(w) : "f"(h1), "f"(h0));
-    const bool s0 = swiglu_needs_fp64(h0, g0), s1 = swiglu_needs_fp64(h1, g1);
-    if (s0 || s1) {
-        if (s0) w = (w & 0xffff0000u) | swiglu_fp64_bits(g0, u0);
-        if (s1) w = (w & 0x0000ffffu) | (swiglu_fp64_bits(g1, u1) << 16);
+    f32x2 h[4];
+    uint32_t key = 0xffffffffu;
+    float lo = 3.0e38f, hi = 0.0f;
+#pragma unroll
+    for (int k = 0; k < 4; ++k) {
+        const f32x2 g = pack2(__uint_as_float(gw[k] << 16), __uint_as_float(gw[k] & 0xffff0000u));
+        const f32x2 u = pack2(__uint_as_float(uw[k] << 16), __uint_as_float(uw[k] & 0xffff0000u));
+        h[k] = swish_mul2(g, u);
+        asm("cvt.rn.bf16x2.f32 %0, %1, %2;" : "=r"(hw[k]) : "f"(h[k].y), "f"(h[k].x));
+        key = min(key, min(swiglu_midpoint_key(h[k].x), swiglu_midpoint_key(h[k].y)));
+        lo = fminf(fminf(lo, fabsf(h[k].x)), fabsf(h[k].y));
+        hi = fmaxf(fmaxf(hi, fabsf(h[k].x)), fabsf(h[k].y));
     }
-    return w;
+    if (key == 0u || !(lo >= 0x1p-100f) || !(hi <= 3.4028234663852886e38f)) {       // rare
+#pragma unroll
+        for (int k = 0; k < 4; ++k) {
+            if (swiglu_needs_fp64(h[k].x))
+                hw[k] = (hw[k] & 0xffff0000u) | swiglu_fp64_bits(__uint_as_float(gw[k] << 16), __uint_as_float(uw[k] << 16));
+            if (swiglu_needs_fp64(h[k].y))
+                hw[k] = (hw[k] & 0x0000ffffu) |
+                        (swiglu_fp64_bits(__uint_as_float(gw[k] & 0xffff0000u), __uint_as_float(uw[k] & 0xffff0000u)) << 16);
+        }
+    }
 }
 // This warp's 1024-element segment of h, written over the staged gate segment (lane l handles the 16-byte
 // pieces l, l + 32, l + 64, l + 96 of both projections).
@@ -785,8 +811,7 @@ __device__ __forceinline__ void swiglu_segment(uint32_t gate_addr, uint32_t up_a
         asm volatile("ld.shared.v4.b32 {%0,%1,%2,%3}, [%4];" : "=r"(gw[0]), "=r"(gw[1]), "=r"(gw[2]), "=r"(gw[3]) : "r"(gate_addr + off) : "memory");
         asm volatile("ld.shared.v4.b32 {%0,%1,%2,%3}, [%4];" : "=r"(uw[0]), "=r"(uw[1]), "=r"(uw[2]), "=r"(uw[3]) : "r"(up_addr + off) : "memory");
         uint32_t hw[4];
-#pragma unroll
-        for (int k = 0; k < 4; ++k) hw[k] = swiglu_word(gw[k], uw[k]);
+        swiglu_piece(gw, uw, hw);
         sts_v4(gate_addr + off, hw[0], hw[1], hw[2], hw[3]);
     }
     __syncwarp();
