@@ -295,10 +295,16 @@ __device__ __noinline__ void tok_fix_ties(uint32_t seg_addr, const uint16_t *seg
             for (int e = 0; e < 4; ++e) fm |= (t[e] != u[e]) ? (1u << (4 * s + e)) : 0u;
         }
     }
-    // the exact row maximum (sign-only fix-ups of E2M1 codes do not need it)
-    const bool need_scale = (MODE != MODE_FP4) || __any_sync(0xffffffffu, (fm & ~zm) != 0u);
-    if (need_scale && !known) a_bits = tok_row_exact_max<LOG2B, LOG2W>(row_addr, raw_row, xch, thr_row, lane);
-    const double a_src = __longlong_as_double((long long)a_bits);
+    // The exact row maximum a.  E2M1 codes need it unless only signs are in doubt.  INT4 codes mostly do not:
+    // the fp32 maximum a32 brackets it, a32 (1 - a_unc) <= a <= a32 (1 + a_unc) (the largest fp32 value and the
+    // largest exact value are both within the error bound of each other's element), which decides every element
+    // that is not within that bracket of its tie -- about fifteen in sixteen of the elements that get here,
+    // whose window is sixteen times wider.  It is derived from the staged row only when an element asks for it.
+    const float a_unc = 1.0625f * err_rel + 2.4e-7f;
+    if (MODE == MODE_FP4 && !known && __any_sync(0xffffffffu, (fm & ~zm) != 0u)) {
+        a_bits = tok_row_exact_max<LOG2B, LOG2W>(row_addr, raw_row, xch, thr_row, lane);
+        known = true;
+    }
     __syncwarp();
     double s_row = 0.0;
     bool have_s = false;
@@ -313,34 +319,57 @@ __device__ __noinline__ void tok_fix_ties(uint32_t seg_addr, const uint16_t *seg
             fs &= fs - 1;
             int blk_elem, i, elem;
             locate<LOG2B>(src >> 2, src & 3, e, blk_elem, i, elem);
-            const double ue = exact_coord_fast<B>(seg + blk_elem, i, lane);
-            if (lane == 0) {
-                uint32_t code = 0u;
-                if (MODE == MODE_FP4 && ((zs >> e) & 1u)) {
+            // (lane 0's sum for everybody: the lanes add in different orders, and the branches below must not differ)
+            const double ue = __shfl_sync(0xffffffffu, exact_coord_fast<B>(seg + blk_elem, i, lane), 0);
+            uint32_t code = 0u;
+            if (MODE == MODE_FP4) {
+                if ((zs >> e) & 1u) {
                     code = signbit(ue) ? 8u : 0u;          // magnitude zero either way: the sign of y = u / sqrt(b)
-                } else if (MODE == MODE_FP4) {
+                } else {
+                    const double a_src = __longlong_as_double((long long)a_bits);
                     if (!have_s) { s_row = over_sqrt_b(a_src) / 7.0; have_s = true; }
                     const double y = over_sqrt_b(ue);
                     code = e2m1_code_exact((s_row != 0.0) ? y / s_row : 0.0, signbit(y));
-                } else if (a_src != 0.0) {
-                    // The staged code kp comes from the multiplier nudged away from zero, the other candidate is one
-                    // step towards zero, the tie between them at |y / s| = |kp| - 1/2.  y / s = 7 u / a: the side is the
-                    // sign of 14 |u| - (2 |kp| - 1) a, two fp64 products whose rounding errors are far below the margin
-                    // asked for here.  Only an exact or all but exact tie takes the definition's own sequence of
-                    // operations (fp64 divisions), which lands on exact halves where the definition does.
-                    const uint32_t nib = (code_gen[elem >> 1] >> ((elem & 1) * 4)) & 0xFu;
-                    const int kp = (int)(nib ^ 8u) - 8;
-                    const int mag = kp < 0 ? -kp : kp;
-                    const double diff = 14.0 * fabs(ue) - (double)(2 * mag - 1) * a_src;
+                }
+            } else if (a32 > 0.0f) {
+                // The staged code kp comes from the multiplier nudged away from zero, the other candidate is one
+                // step towards zero, the tie between them at |y / s| = |kp| - 1/2.  y / s = 7 u / a: the side is the
+                // sign of 14 |u| - (2 |kp| - 1) a, two fp64 products whose rounding errors are far below the margins
+                // asked for here.  Only an exact or all but exact tie takes the definition's own sequence of
+                // operations (fp64 divisions), which lands on exact halves where the definition does.
+                // (read by one lane and handed round: every lane takes the same branches below, and none reads the
+                // byte after lane 0 has rewritten it)
+                const uint32_t nib = __shfl_sync(0xffffffffu, (uint32_t)(code_gen[elem >> 1] >> ((elem & 1) * 4)) & 0xFu, 0);
+                const int kp = (int)(nib ^ 8u) - 8;
+                const int mag = kp < 0 ? -kp : kp;
+                const double lhs = 14.0 * fabs(ue), wgt = (double)(2 * mag - 1);
+                const uint32_t towards_zero = (uint32_t)(kp < 0 ? kp + 1 : kp - 1) & 0xFu;
+                bool decided = false;
+                if (!known && mag >= 1) {
+                    const double d32 = lhs - wgt * (double)a32;
+                    if (fabs(d32) > wgt * (double)a32 * (double)a_unc) {
+                        code = d32 > 0.0 ? ((uint32_t)kp & 0xFu) : towards_zero;
+                        decided = true;
+                    }
+                }
+                if (!decided) {                            // (warp-uniform: every lane holds the same operands)
+                    if (!known) {
+                        a_bits = tok_row_exact_max<LOG2B, LOG2W>(row_addr, raw_row, xch, thr_row, lane);
+                        known = true;
+                    }
+                    const double a_src = __longlong_as_double((long long)a_bits);
+                    const double diff = lhs - wgt * a_src;
                     if (mag >= 1 && fabs(diff) > a_src * 1.0e-12) {
-                        code = (uint32_t)(diff > 0.0 ? kp : (kp < 0 ? kp + 1 : kp - 1)) & 0xFu;
-                    } else {
+                        code = diff > 0.0 ? ((uint32_t)kp & 0xFu) : towards_zero;
+                    } else if (a_src != 0.0) {
                         if (!have_s) { s_row = over_sqrt_b(a_src) / 7.0; have_s = true; }
                         double qd = rint(over_sqrt_b(ue) / s_row);
                         qd = fmin(fmax(qd, -8.0), 7.0);
                         code = (uint32_t)((int)qd) & 0xFu;
                     }
                 }
+            }
+            if (lane == 0) {
                 uint8_t *bp = code_gen + (elem >> 1);
                 *bp = (elem & 1) ? (uint8_t)((*bp & 0x0F) | (code << 4)) : (uint8_t)((*bp & 0xF0) | code);
             }
