@@ -139,7 +139,7 @@ struct MxQuant {
             const float c_m = __shfl_sync(0xffffffffu, c, (lane & 28) | m);
             const float t_m = __shfl_sync(0xffffffffu, tau, (lane & 28) | m);
             tau_p[m] = pack2(t_m, t_m);
-            tau_m[m] = pack2(-t_m, -t_m);
+            tau_m[m] = pack2(0.0f - t_m, 0.0f - t_m);       // +0 for a zero window: (-0) + (+0) = +0 on both sides
 #pragma unroll
             for (int h = 0; h < 2; ++h) {
                 const float mc = L.sgn[(2 * m + h) & 3 & PM] * c_m;
@@ -290,7 +290,8 @@ __global__ void __launch_bounds__(FAST_THREADS, 1) perq_mx_kernel(FastParams p)
             else c = __uint_as_float((uint32_t)min(max(254 - Eb - (LOG2B - 1) / 2, 1), 254) << 23) * 0.70710678118654752f;
             uint32_t byte = (uint32_t)Eb;
             if (!(a32 > 0.0f)) { c = 0.0f; byte = 0u; }
-            const float tau = 2.0f * err_rel * bref * c + 2.0e-6f;
+            // (an all-zero block is exact: no window, so that its zeros are not flagged for their sign)
+            const float tau = (bref > 0.0f) ? 2.0f * err_rel * bref * c + 2.0e-6f : 0.0f;
             // scale bytes of the quad's four groups: slot pair m is chunk pair m ^ (f >> 1)
             uint32_t word = byte << (8 * (q ^ (((g & 3) & ~PM) >> 1)));
             word |= __shfl_xor_sync(0xffffffffu, word, 1);

@@ -268,7 +268,7 @@ __device__ __noinline__ void tok_fix_ties(uint32_t seg_addr, const uint16_t *seg
     const float delta = 16.0f * err_rel + 5.0e-7f;
     const float tau = (a32 > 0.0f) ? 8.0f * err_rel + 4.0e-6f : 0.0f;
     const f32x2 magic2 = pack2(MAGIC, MAGIC);
-    const f32x2 tau_p2 = pack2(tau, tau), tau_m2 = pack2(-tau, -tau);
+    const f32x2 tau_p2 = pack2(tau, tau), tau_m2 = pack2(0.0f - tau, 0.0f - tau);     // (+0 for a zero row)
     uint32_t fm = 0u, zm = 0u;
 #pragma unroll
     for (int s = 0; s < 8; ++s) {
@@ -301,6 +301,28 @@ __device__ __noinline__ void tok_fix_ties(uint32_t seg_addr, const uint16_t *seg
     // that is not within that bracket of its tie -- about fifteen in sixteen of the elements that get here,
     // whose window is sixteen times wider.  It is derived from the staged row only when an element asks for it.
     const float a_unc = 1.0625f * err_rel + 2.4e-7f;
+    if (MODE == MODE_FP4) {
+        // The zeros of an all-zero block (padded channels) are exact, and the staged code +0 is theirs: drop
+        // their flags (the window of the loop's test is the same for every block of the row).  A block is 2^CB
+        // slots of the four lanes of a quad.
+        constexpr int CB = LOG2B - 4;
+        float bm[8];
+#pragma unroll
+        for (int s = 0; s < 8; ++s) bm[s] = fmaxf(max3abs(fabsf(v[s][0].x), v[s][0].y, v[s][1].x), fabsf(v[s][1].y));
+#pragma unroll
+        for (int s = 0; s < 8; s += (1 << CB)) {
+            float m = bm[s];
+#pragma unroll
+            for (int k = 1; k < (1 << CB); ++k) m = fmaxf(m, bm[s + k]);
+            m = fmaxf(m, __shfl_xor_sync(0xffffffffu, m, 1));
+            m = fmaxf(m, __shfl_xor_sync(0xffffffffu, m, 2));
+            if (m == 0.0f) {
+#pragma unroll
+                for (int k = 0; k < (1 << CB); ++k) fm &= ~(0xFu << (4 * (s + k)));
+            }
+        }
+        if (!__any_sync(0xffffffffu, fm != 0u)) return;
+    }
     if (MODE == MODE_FP4 && !known && __any_sync(0xffffffffu, (fm & ~zm) != 0u)) {
         a_bits = tok_row_exact_max<LOG2B, LOG2W>(row_addr, raw_row, xch, thr_row, lane);
         known = true;
@@ -469,7 +491,7 @@ __global__ void __launch_bounds__(FAST_THREADS, 1) perq_tok_kernel(FastParams p)
         uint32_t tie_any = 0u;
         if (MODE == MODE_FP4) {
             const float tau = (inv > 0.0f) ? 8.0f * err_rel + 4.0e-6f : 0.0f;
-            const f32x2 tau_p2 = pack2(tau, tau), tau_m2 = pack2(-tau, -tau);
+            const f32x2 tau_p2 = pack2(tau, tau), tau_m2 = pack2(0.0f - tau, 0.0f - tau);     // (+0 for a zero row)
             f32x2 mul_c[NCLS];
 #pragma unroll
             for (int c = 0; c < NCLS; ++c) mul_c[c] = pack2(L.sgn[c] * inv, L.sgn[c] * inv);

@@ -189,6 +189,54 @@ def test_zero_rows_and_zero_groups(B, oracle):
     assert not codes[1].any() and not scales[1].any()
 
 
+@pytest.mark.parametrize("fmt,group", [("int4", 0), ("int4", 128), ("mxfp4", 32), ("fp4", 0), ("int4_asym", 0)])
+@pytest.mark.parametrize("d,b", [(4096, 32), (2048, 16), (8192, 64), (3072, 128)])
+def test_padded_rows_and_padded_channels(B, oracle, d, b, fmt, group):
+    """Zero rows (padding tokens) and all-zero blocks (padding channels) between dense rows: exact zeros take the
+    code +0 and the scale of an empty range, through the persistent kernels' main loops (many rows per group)."""
+    T = 640
+    bits, _ = inputs.laplace_outliers(T, d, 4, 200.0, seed=11)
+    bits[::3] = 0                                  # every third row
+    bits[:, 2 * b:3 * b] = 0                       # one Hadamard block of every row
+    bits[5::7, d // 2:] = 0                        # the second half of some rows
+    bits[:, 7] = 0                                 # one zero channel inside a dense block
+    w = inputs.Workload(name="padded", x=bits, perm=None, b=b, fmt=fmt, group=group, seed=11)
+    check(B, oracle, w)
+    codes, scales = run_gpu(B, w)
+    assert not codes[0].any()
+    if fmt != "int4_asym":
+        assert not scales[0].any()
+
+
+@pytest.mark.parametrize("fmt,group", [("int4", 0), ("mxfp4", 32), ("fp4", 0)])
+def test_padding_does_not_slow_a_call_down(B, fmt, group):
+    """Exact zeros must stay on the fast path of the rounding test: a call on padded rows may not take several
+    times as long as the same call on dense rows (an E2M1 zero flagged for its sign goes to the exact path)."""
+    T, d, b = 4096, 4096, 32
+    dense, _ = inputs.laplace_outliers(T, d, 4, 200.0, seed=12)
+    padded = dense.copy()
+    padded[::2] = 0
+    padded[:, 64:96] = 0
+
+    def timed(bits):
+        x = to_dev(bits)
+        oc, os_ = B.alloc_outputs(T, d, FMT[fmt], group, x.device)
+        for _ in range(3):
+            B.perq_rotate_quantize(x, None, b, FMT[fmt], group, out_codes=oc, out_scales=os_)
+        torch.cuda.synchronize()
+        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        e0.record()
+        for _ in range(20):
+            B.perq_rotate_quantize(x, None, b, FMT[fmt], group, out_codes=oc, out_scales=os_)
+        e1.record()
+        torch.cuda.synchronize()
+        return e0.elapsed_time(e1) / 20
+
+    t_dense, t_padded = timed(dense), timed(padded)
+    print("%s: dense %.1f us, padded %.1f us" % (fmt, 1e3 * t_dense, 1e3 * t_padded))
+    assert t_padded < 2.5 * t_dense
+
+
 def test_single_huge_outlier_and_basis_rows(B, oracle):
     d = 2048
     x = np.zeros((6, d), np.float32)
