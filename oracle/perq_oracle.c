@@ -15,7 +15,9 @@
  * convention (scale 0, codes 0), sign of values that quantise to zero in E2M1, the
  * MX shared-exponent reading floor(log2 amax) - 2 versus 2^floor(log2(amax/6)), and the
  * tie-breaks of the greedy permutation.  perq_oracle_swiglu rounds the product once to bf16 (a reading: the
- * paper's figure gives the formula, not a storage precision).
+ * paper's figure gives the formula, not a storage precision).  perq_oracle_hadamard_base: "parity unpinned"
+ * against the authors' base matrices of order 12 / 28 / 76, which the paper does not print (Paley's second
+ * construction is taken; H H^T = n I, symmetry and the Kronecker structure are pinned).
  *
  * Rows are independent; `#pragma omp parallel for` over rows is the only parallelism.
  */
@@ -57,14 +59,83 @@ int perq_oracle_num_threads(void)
 /* ---------------------------------------------------------------- Hadamard matrix
  * Notation paragraph: R is a normalised Hadamard matrix, columns of unit l2 norm and
  * entries +-1/sqrt(k).  The Sylvester construction in natural order has entry (k,i)
- * equal to (-1)^{popcount(k AND i)}.  This writes the UNNORMALISED +-1 matrix, b*b
- * signed bytes, row-major. */
+ * equal to (-1)^{popcount(k AND i)}.
+ *
+ * Appendix A.1 (non-power-of-2 rotation): d = k t with t the largest odd factor of d; R is
+ * built from k' = log2(k) - 2 recursive (Sylvester) applications of a 4t-dimensional base
+ * matrix, so the computation is k' radix-2 stages and 2^k' independent 4t-dimensional
+ * rotations of ADJACENT inputs:  H_d = H_{2^k'} (x) H_{4t}, entry (k, i) =
+ * (-1)^{popcount(k/4t AND i/4t)} * H_{4t}[k mod 4t][i mod 4t].
+ * The paper does not print its base matrices (H_12, H_28, H_76): PARITY UNPINNED against the
+ * authors' matrix.  Reading taken here: Paley's second construction for 4t = 2(q + 1), q a
+ * prime with q = 1 (mod 4) -- q = 5, 13, 37 give exactly the three orders the paper's table of
+ * non-power-of-2 dimensions needs (also 36 and 60).  With chi the quadratic character mod q
+ * (chi(0) = 0, chi(a) = 1 for a non-zero square, -1 otherwise) and the symmetric conference
+ * matrix S of order q + 1 (S_00 = 0, S_0j = S_j0 = 1, S_ij = chi(i - j) for i, j >= 1), every
+ * zero of S becomes the 2x2 block [[1, -1], [-1, -1]] and every entry +-1 becomes
+ * +-[[1, 1], [1, -1]].  What the mathematics fixes, H H^T = n I, is pinned in the tests.
+ *
+ * Both functions write the UNNORMALISED +-1 matrix, row-major signed bytes. */
+int perq_oracle_hadamard_base(int32_t n, int8_t *H)
+{
+    if (n < 4 || n % 4 != 0 || !H) return 1;
+    const int32_t q = n / 2 - 1;
+    if (q % 4 != 1) return 1;
+    for (int32_t f = 2; f * f <= q; ++f)
+        if (q % f == 0) return 1;                       /* prime fields only */
+    int8_t *chi = (int8_t *)malloc((size_t)q);
+    if (!chi) return 3;
+    for (int32_t a = 0; a < q; ++a) chi[a] = -1;
+    chi[0] = 0;
+    for (int32_t a = 1; a < q; ++a) chi[(a * a) % q] = 1;
+    for (int32_t i = 0; i <= q; ++i) {
+        for (int32_t j = 0; j <= q; ++j) {
+            int s;
+            if (i == 0 && j == 0) s = 0;
+            else if (i == 0 || j == 0) s = 1;
+            else s = chi[((i - j) % q + q) % q];
+            int8_t *blk = H + (size_t)(2 * i) * n + 2 * j;
+            if (s == 0) {
+                blk[0] = 1;  blk[1] = -1;
+                blk[n] = -1; blk[n + 1] = -1;
+            } else {
+                blk[0] = (int8_t)s; blk[1] = (int8_t)s;
+                blk[n] = (int8_t)s; blk[n + 1] = (int8_t)-s;
+            }
+        }
+    }
+    free(chi);
+    return 0;
+}
+
+/* order of the base matrix of a b-dimensional rotation: 1 for a power of two (Sylvester all the
+ * way down), else 4t with t the odd part of b; 0 if b has no such factorisation (k < 4). */
+static int32_t base_order(int32_t b)
+{
+    if (b < 1) return 0;
+    int32_t t = b;
+    while ((t & 1) == 0) t >>= 1;
+    if (t == 1) return 1;
+    return (b % (4 * t) == 0) ? 4 * t : 0;
+}
+
 int perq_oracle_hadamard_pm1(int32_t b, int8_t *H)
 {
-    if (b < 1 || (b & (b - 1)) != 0 || !H) return 1;
+    const int32_t n = base_order(b);
+    if (n == 0 || !H) return 1;
+    int8_t *base = (int8_t *)malloc((size_t)n * n);
+    if (!base) return 3;
+    if (n == 1) base[0] = 1;
+    else {
+        const int rc = perq_oracle_hadamard_base(n, base);
+        if (rc) { free(base); return rc; }
+    }
     for (int32_t k = 0; k < b; ++k)
-        for (int32_t i = 0; i < b; ++i)
-            H[(size_t)k * b + i] = (popcount32((uint32_t)(k & i)) & 1) ? -1 : 1;
+        for (int32_t i = 0; i < b; ++i) {
+            const int8_t e = base[(size_t)(k % n) * n + (i % n)];
+            H[(size_t)k * b + i] = (popcount32((uint32_t)((k / n) & (i / n))) & 1) ? (int8_t)-e : e;
+        }
+    free(base);
     return 0;
 }
 
@@ -76,17 +147,19 @@ int perq_oracle_hadamard_pm1(int32_t b, int8_t *H)
  *
  * y[t, j*b + i] = (1/sqrt(b)) * sum_{k<b} x'[t, j*b + k] * H[k][i],  x'[i] = x[perm[i]].
  * The sum is an explicit matrix-vector product (k ascending), no butterfly.
- * perm == NULL is the identity.  b may be any power of two >= 1 that divides d. */
+ * perm == NULL is the identity.  b may be any power of two >= 1 that divides d, or b = d for a
+ * d that is not a power of two (Appendix A.1; the matrix of perq_oracle_hadamard_pm1). */
 int perq_oracle_rotate(const uint16_t *x, const int32_t *perm, int64_t T, int32_t d,
                        int32_t b, double *y)
 {
-    if (!x || !y || T < 0 || d <= 0 || b < 1 || (b & (b - 1)) != 0 || d % b != 0) return 1;
+    if (!x || !y || T < 0 || d <= 0 || b < 1 || d % b != 0) return 1;
+    if ((b & (b - 1)) != 0 && b != d) return 1;          /* other orders only as the full-vector rotation */
     if (perm)
         for (int32_t i = 0; i < d; ++i)
             if (perm[i] < 0 || perm[i] >= d) return 2;
     int8_t *H = (int8_t *)malloc((size_t)b * b);
     if (!H) return 3;
-    perq_oracle_hadamard_pm1(b, H);
+    if (perq_oracle_hadamard_pm1(b, H)) { free(H); return 1; }
     const double sqrt_b = sqrt((double)b);
     int fail = 0;
 #pragma omp parallel

@@ -62,6 +62,13 @@ def hadamard_pm1(b: int) -> np.ndarray:
     return H
 
 
+def hadamard_base(n: int) -> np.ndarray:
+    """Base matrix of order n = 4t of the non-power-of-2 rotation (Appendix A.1; Paley's second construction)."""
+    H = np.empty((n, n), np.int8)
+    _check(_load().perq_oracle_hadamard_base(C.c_int32(n), _p(H)), "hadamard_base")
+    return H
+
+
 def _x(x):
     x = np.ascontiguousarray(x, dtype=np.uint16)
     assert x.ndim == 2

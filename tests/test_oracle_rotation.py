@@ -158,3 +158,91 @@ def test_op_count_table():
     assert len(rows) == 16
     for _, d, b, ops in rows:
         assert butterfly_add_sub_per_token(int(d), int(b)) == int(ops)
+
+
+# ------------------------------------------------------------------ full-vector rotation of a non-power-of-2 dimension
+
+def _paley2_by_kron(q: int) -> np.ndarray:
+    """Textbook form of Paley's second construction, by another route than the oracle's loops: Euler's criterion
+    for the quadratic character and H = S (x) [[1, 1], [1, -1]] + I (x) [[1, -1], [-1, -1]]."""
+    chi = [0] + [1 if pow(a, (q - 1) // 2, q) == 1 else -1 for a in range(1, q)]
+    S = np.zeros((q + 1, q + 1), np.int64)
+    S[0, 1:] = 1
+    S[1:, 0] = 1
+    for i in range(q):
+        for j in range(q):
+            S[1 + i, 1 + j] = chi[(i - j) % q]
+    return np.kron(S, np.array([[1, 1], [1, -1]])) + np.kron(np.eye(q + 1, dtype=np.int64), np.array([[1, -1], [-1, -1]]))
+
+
+@pytest.mark.parametrize("n", [12, 28, 36, 60, 76])
+def test_base_matrix_is_hadamard(oracle, n):
+    """What the mathematics fixes about the base matrix of order 4t (the paper does not print its own)."""
+    H = oracle.hadamard_base(n).astype(np.int64)
+    assert set(np.unique(H).tolist()) == {-1, 1}
+    assert np.array_equal(H @ H.T, n * np.eye(n, dtype=np.int64))
+    assert np.array_equal(H.T @ H, n * np.eye(n, dtype=np.int64))
+    assert np.array_equal(H, H.T)
+    assert np.array_equal(H, _paley2_by_kron(n // 2 - 1))
+
+
+@pytest.mark.parametrize("n", [8, 20, 44, 52, 14, 3])
+def test_orders_without_a_base_matrix_are_refused(oracle, n):
+    with pytest.raises(Exception):
+        oracle.hadamard_base(n)
+
+
+@pytest.mark.parametrize("d", [48, 112, 3072, 1216])
+def test_non_po2_matrix_is_sylvester_kron_base(oracle, d):
+    """H_d = H_{2^k'} (x) H_{4t}: k' butterfly stages over strides of 4t, rotations of 4t ADJACENT inputs."""
+    import scipy.linalg
+    t = d
+    while t % 2 == 0:
+        t //= 2
+    n = 4 * t
+    H = oracle.hadamard_pm1(d).astype(np.int64)
+    assert np.array_equal(H, np.kron(scipy.linalg.hadamard(d // n).astype(np.int64), oracle.hadamard_base(n).astype(np.int64)))
+    if d <= 1216:
+        assert np.array_equal(H @ H.T, d * np.eye(d, dtype=np.int64))
+
+
+def test_non_po2_rotation_closed_forms(oracle):
+    rng = np.random.default_rng(41)
+    for d in (48, 112, 3072):
+        x = rng.standard_normal((5, d)).astype(np.float32)
+        bits = inputs.f32_to_bf16_bits(x)
+        xb = inputs.bf16_to_f64(bits)
+        y = oracle.rotate(bits, None, d)
+        H = oracle.hadamard_pm1(d).astype(np.float64)
+        np.testing.assert_allclose(y, xb @ H / np.sqrt(d), rtol=0, atol=1e-12 * np.abs(xb).sum(axis=1).max())
+        # orthogonal and (H symmetric) an involution; the full-vector bound of Sec. 3
+        np.testing.assert_allclose((y * y).sum(axis=1), (xb * xb).sum(axis=1), rtol=1e-12)
+        np.testing.assert_allclose(y @ H / np.sqrt(d), xb, atol=1e-12 * np.abs(xb).sum(axis=1).max())
+        assert (np.abs(y).max(axis=1) <= np.abs(xb).sum(axis=1) / np.sqrt(d) * (1 + 1e-12)).all()
+        # a unit vector returns a row of H
+        e = np.zeros((1, d), np.float32)
+        e[0, 17] = 1.0
+        np.testing.assert_array_equal(oracle.rotate(inputs.f32_to_bf16_bits(e), None, d)[0] * np.sqrt(d), H[17])
+    # a permutation is applied before the rotation
+    p = inputs.random_perm(112, 5)
+    bits = inputs.f32_to_bf16_bits(rng.standard_normal((2, 112)).astype(np.float32))
+    np.testing.assert_array_equal(oracle.rotate(bits, p, 112), oracle.rotate(bits[:, p], None, 112))
+    with pytest.raises(Exception):
+        oracle.rotate(bits, None, 56)             # a non-power-of-2 block inside a longer row
+
+
+def test_non_po2_op_count_table():
+    """The three add/sub counts of the paper's Table "non-po2-ops" for its five dimensions."""
+    import os
+    from paper_2601_22347_b200.roofline import full_vector_add_sub_per_token, non_po2_factors
+    here = os.path.dirname(__file__)
+    rows = [l.split() for l in open(os.path.join(here, "golden", "non_po2_op_counts.txt")) if l.strip() and not l.startswith("#")]
+    assert len(rows) == 5
+
+    def printed(v):
+        return "%.2fM" % (v / 1e6) if v >= 1e6 else "%.2fK" % (v / 1e3)
+
+    for _, d, kp, n, dense, mixed, ours in rows:
+        assert non_po2_factors(int(d)) == (int(kp), int(n))
+        assert tuple(printed(v) for v in full_vector_add_sub_per_token(int(d))) == (dense, mixed, ours)
+    assert non_po2_factors(4096) is None
