@@ -455,6 +455,10 @@ def main():
         for T5 in (1, 16, 128, 1024, 16384):
             w5 = inputs.config5(T=T5, b=32)
             time_workload("cfg5", w5.x, w5.perm, 32, "int4", 128)
+        # full-vector rotation of a width that is not a power of two (14336 = 2^9 x 28, general kernel)
+        w5 = inputs.config5(T=1024, b=32)
+        time_workload("cfg5 width, full-vector 2^9 x 28", w5.x, None, 14336, "int4", 0)
+        time_workload("cfg5 width, full-vector 2^9 x 28", w5.x, None, 14336, "mxfp4", 32)
 
     cpu_baseline = None
     if not args.no_cpu_baseline:

@@ -48,7 +48,7 @@ typedef enum {
     PERQ_ERR_NULL = 1,   /* a required pointer is NULL */
     PERQ_ERR_SHAPE = 2,  /* T < 0, d <= 0, d % 32 != 0 or d > PERQ_MAX_D; also: a row that the general kernel cannot
                             hold in 227 KB of shared memory with its per-range tables (very small groups of very long rows) */
-    PERQ_ERR_BLOCK = 3,  /* b is not a power of two in [16, d] that divides d */
+    PERQ_ERR_BLOCK = 3,  /* b is neither a power of two in [16, d] that divides d nor (perq_rotate_quantize) a supported b == d = 2^k * 4t */
     PERQ_ERR_GROUP = 4,  /* INT4: group not 0 and (d % group != 0, group % 8 != 0, or group neither a multiple nor a
                             divisor of b); MXFP4: group not 0/32; FP4, INT4_ASYM: not 0 */
     PERQ_ERR_FMT = 5,    /* unknown format */
@@ -94,8 +94,16 @@ typedef enum {
  *            perq_validate_perm to check a permutation beforehand.
  * T, d       rows and channels.  T == 0 is a no-op (pointers are then not looked at).
  *            d % 32 == 0, d <= PERQ_MAX_D.
- * b          a power of two, 16 <= b <= d, with d % b == 0 (b == d is the full-vector rotation and
- *            needs d itself to be a power of two).  The tensor-core kernels cover d % 1024 == 0 with
+ * b          a power of two, 16 <= b <= d, with d % b == 0 (b == d is the full-vector rotation); or, for a d
+ *            that is not a power of two, b == d = 2^k' * 4t with t the odd part of d and 4t one of 12, 28,
+ *            36, 60, 76 (Appendix A.1, "An Optimized Non-Power-of-2 Hadamard Rotation": Llama-3-8B's
+ *            14336 = 2^9 * 28, Qwen3's 3072 / 6144 / 12288 = 2^k' * 12 and 9728 = 2^7 * 76).  Step 2 is then
+ *            y_i = d^{-1/2} sum_k (-1)^{popcount(floor(i/4t) & floor(k/4t))} B[i mod 4t][k mod 4t] x'_k: rotations
+ *            of 4t ADJACENT inputs by a +-1 base matrix B, then k' butterfly stages over strides of 4t.  The
+ *            paper does not print its base matrices; B is Paley's second construction for the prime
+ *            q = 2t - 1 (symmetric, B B^T = 4t I), so codes need not equal those of another implementation's
+ *            matrix.  Other non-power-of-two b, and such a b inside a longer row: PERQ_ERR_BLOCK.
+ *            The tensor-core kernels cover d % 1024 == 0 with
  *            b <= 128 (any scale mode, with or without perm) and, unpermuted with per-token or MX
  *            scales, b <= 1024 and b == d <= 8192; everything else runs on a slower general kernel.
  * fmt        perq_fmt_t.

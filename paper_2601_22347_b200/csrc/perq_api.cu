@@ -7,12 +7,14 @@
 #include <map>
 #include <cmath>
 #include <cstdint>
+#include <cstring>
 #include <mutex>
 #include <queue>
 #include <utility>
 #include <vector>
 
 #include <cuda_runtime.h>
+#include <cstring>
 
 #include "perq_generic.cuh"
 #include "perq_fast.cuh"
@@ -31,14 +33,57 @@ inline bool is_pow2(long long v) { return v > 0 && (v & (v - 1)) == 0; }
 inline int ilog2(int v) { int l = 0; while ((1 << l) < v) ++l; return l; }
 inline bool aligned16(const void *p) { return (reinterpret_cast<uintptr_t>(p) & 15u) == 0; }
 
-// Common shape checks.  On success *g_out is the effective scale-range length.
-int check_shape(int64_t T, int32_t d, int32_t b, int32_t fmt, int32_t group, int *g_out)
+// Order of the base matrix of a b-dimensional Hadamard rotation (Appendix A.1: b = 2^k' * 4t, t the odd part
+// of b): 0 for a power of two (Sylvester all the way), 4t when this library has a base matrix of that order
+// (Paley's second construction: 4t = 2 (q + 1) with q = 5, 13, 17, 29 or 37), -1 otherwise.
+int base_order(int32_t b)
+{
+    if (b < 1) return -1;
+    if (is_pow2(b)) return 0;
+    int t = b;
+    while ((t & 1) == 0) t >>= 1;
+    const int n = 4 * t;
+    if (b % n != 0) return -1;
+    return (n == 12 || n == 28 || n == 36 || n == 60 || n == 76) ? n : -1;
+}
+
+// Rows of the +-1 base matrix of order n = 2 (q + 1) as bit masks (bit c of row r set: entry -1).  Paley's
+// second construction: chi = quadratic character mod the prime q = 1 (mod 4); S = symmetric conference matrix
+// of order q + 1 (zero corner, ones along the first row and column, chi(i - j) elsewhere); a zero of S becomes
+// [[1, -1], [-1, -1]], an entry s = +-1 becomes s [[1, 1], [1, -1]].
+void base_matrix_rows(int n, uint32_t (*rows)[3])
+{
+    const int q = n / 2 - 1;
+    int chi[64];
+    for (int a = 0; a < q; ++a) chi[a] = -1;
+    chi[0] = 0;
+    for (int a = 1; a < q; ++a) chi[(a * a) % q] = 1;
+    for (int r = 0; r < n; ++r) rows[r][0] = rows[r][1] = rows[r][2] = 0u;
+    auto set_neg = [&](int r, int c) { rows[r][c >> 5] |= 1u << (c & 31); };
+    for (int i = 0; i <= q; ++i) {
+        for (int j = 0; j <= q; ++j) {
+            const int sv = (i == 0 && j == 0) ? 0 : (i == 0 || j == 0) ? 1 : chi[((i - j) % q + q) % q];
+            const int r = 2 * i, c = 2 * j;
+            if (sv == 0) { set_neg(r, c + 1); set_neg(r + 1, c); set_neg(r + 1, c + 1); }
+            else if (sv > 0) { set_neg(r + 1, c + 1); }
+            else { set_neg(r, c); set_neg(r, c + 1); set_neg(r + 1, c); }
+        }
+    }
+}
+
+// Common shape checks.  On success *g_out is the effective scale-range length.  Block sizes that are not a
+// power of two are accepted only where the caller can run them (non_po2_ok) and only as b == d.
+int check_shape(int64_t T, int32_t d, int32_t b, int32_t fmt, int32_t group, int *g_out, bool non_po2_ok = false)
 {
     if (T < 0 || d <= 0 || d % 32 != 0 || d > PERQ_MAX_D) return PERQ_ERR_SHAPE;
     if (fmt != PERQ_FMT_INT4 && fmt != PERQ_FMT_MXFP4 && fmt != PERQ_FMT_F32_DEBUG && fmt != PERQ_FMT_FP4 &&
         fmt != PERQ_FMT_INT4_ASYM)
         return PERQ_ERR_FMT;
-    if (!is_pow2(b) || b < 16 || b > d || d % b != 0) return PERQ_ERR_BLOCK;
+    if (!is_pow2(b)) {
+        if (!non_po2_ok || b != d || base_order(b) <= 0) return PERQ_ERR_BLOCK;
+    } else if (b < 16 || b > d || d % b != 0) {
+        return PERQ_ERR_BLOCK;
+    }
     int g = d;
     if (fmt == PERQ_FMT_INT4) {
         if (group < 0) return PERQ_ERR_GROUP;
@@ -123,14 +168,19 @@ int launch_generic(const void *x, const int32_t *perm, int64_t T, int32_t d, int
     p.perm = perm;
     p.T = T;
     p.d = d;
-    p.log2b = ilog2(b);
+    const int n0 = base_order(b);
+    if (n0 < 0) return PERQ_ERR_BLOCK;
+    p.base_n = n0;
+    p.log2b = ilog2(n0 ? b / n0 : b);
+    std::memset(p.hrow, 0, sizeof(p.hrow));
+    if (n0) base_matrix_rows(n0, p.hrow);
     p.fmt = fmt;
     p.g = g;
     p.out_codes = out_codes;
     p.out_scales = out_scales;
     p.sqrt_b = std::sqrt((double)b);
     p.inv_sqrt_b = (float)(1.0 / p.sqrt_b);
-    const perq::GenSmem lay(d, g, p.log2b);
+    const perq::GenSmem lay(d, g, p.log2b, n0);
     if (lay.total > kMaxSmem) return PERQ_ERR_SHAPE;
     if (int rc = allow_smem(perq::perq_generic_kernel, lay.total)) return rc;
     const int sms = sm_count();
@@ -392,8 +442,10 @@ int launch_swiglu_b(int log2b, const perq::FastParams &p, int grid, cudaStream_t
 int launch_any(const void *x, const int32_t *perm, int64_t T, int32_t d, int32_t b, int32_t fmt, int g,
                void *out_codes, void *out_scales, cudaStream_t st)
 {
-    const int rc = try_launch_fast(x, perm, T, d, b, fmt, g, out_codes, out_scales, st);
-    if (rc >= 0) return rc;
+    if (is_pow2(b)) {
+        const int rc = try_launch_fast(x, perm, T, d, b, fmt, g, out_codes, out_scales, st);
+        if (rc >= 0) return rc;
+    }
     return launch_generic(x, perm, T, d, b, fmt, g, out_codes, out_scales, st);
 }
 
@@ -505,7 +557,7 @@ const char *perq_status_string(int status)
     case PERQ_OK: return "ok";
     case PERQ_ERR_NULL: return "a required pointer is NULL";
     case PERQ_ERR_SHAPE: return "bad shape: need T >= 0, 0 < d <= 32768, d % 32 == 0 (and the row must fit in shared memory)";
-    case PERQ_ERR_BLOCK: return "bad block size: need a power of two b, 16 <= b <= d, dividing d";
+    case PERQ_ERR_BLOCK: return "bad block size: need a power of two b, 16 <= b <= d, dividing d (perq_rotate_quantize also takes b == d = 2^k * 4t with 4t = 12, 28, 36, 60 or 76)";
     case PERQ_ERR_GROUP: return "bad group: INT4 needs 0 or a multiple of 8 that divides d and is a multiple or a divisor of b; MXFP4 needs 0 or 32; FP4 and asymmetric INT4 need 0";
     case PERQ_ERR_FMT: return "unknown format";
     case PERQ_ERR_ALIGN: return "device pointers must be 16-byte aligned";
@@ -548,7 +600,7 @@ int perq_rotate_quantize(const void *x, const int32_t *perm, int64_t T, int32_t 
                          int32_t group, void *out_codes, void *out_scales, void *stream)
 {
     int g = 0;
-    if (int rc = check_shape(T, d, b, fmt, group, &g)) return rc;
+    if (int rc = check_shape(T, d, b, fmt, group, &g, true)) return rc;
     if (T == 0) return PERQ_OK;   // nothing to read or write: pointers may be anything
     if (!x || !out_codes || (fmt != PERQ_FMT_F32_DEBUG && !out_scales)) return PERQ_ERR_NULL;
     if (!aligned16(x) || !aligned16(out_codes) || !aligned16(out_scales) || !aligned16(perm)) return PERQ_ERR_ALIGN;
@@ -610,7 +662,7 @@ int perq_rotate_quantize_host(const void *x_host, const int32_t *perm, int64_t T
                               void *workspace, size_t workspace_bytes, void *stream)
 {
     int g = 0;
-    if (int rc = check_shape(T, d, b, fmt, group, &g)) return rc;
+    if (int rc = check_shape(T, d, b, fmt, group, &g, true)) return rc;
     if (T == 0) return PERQ_OK;
     if (!x_host || !out_codes_host || (fmt != PERQ_FMT_F32_DEBUG && !out_scales_host)) return PERQ_ERR_NULL;
     size_t need = 0, cb = 0, sb = 0;

@@ -25,6 +25,7 @@ constexpr int GEN_WARPS = GEN_THREADS / 32;
 constexpr int TIE_CAP = 1024;
 constexpr float ERR_K = 8.0f;                 // safety factor on the fp32 butterfly error model
 constexpr float TWO_M24 = 5.9604644775390625e-8f;
+constexpr int GEN_MAX_BASE = 76;              // largest base matrix of a non-power-of-2 rotation (3 words of sign bits)
 
 struct GenParams {
     const uint16_t *x;
@@ -38,17 +39,23 @@ struct GenParams {
     void *out_scales;
     float inv_sqrt_b;
     double sqrt_b;
+    // Full-vector rotation of a row whose length is not a power of two: d = 2^log2b * base_n, H_d =
+    // H_{2^log2b} (x) H_{base_n} (rotations of base_n ADJACENT inputs, then butterflies over strides of base_n).
+    // base_n = 0: Sylvester blocks of 2^log2b.  hrow[r] holds row r of the +-1 base matrix, bit c set = -1.
+    int base_n;
+    uint32_t hrow[GEN_MAX_BASE][3];
 };
 
 // Shared-memory carve-up, computed identically on host (for the launch) and device.
 struct GenSmem {
-    size_t xs, ub, codes, r_max, r_thr, r_mul, r_aux, r_E, b_max, ties, asym, total;
-    __host__ __device__ GenSmem(int d, int g, int log2b)
+    size_t xs, ub, ub2, codes, r_max, r_thr, r_mul, r_aux, r_E, b_max, ties, asym, total;
+    __host__ __device__ GenSmem(int d, int g, int log2b, int base_n)
     {
-        const size_t nr = (size_t)(d / g), nb = (size_t)(d >> log2b);
+        const size_t nr = (size_t)(d / g), nb = base_n ? 1 : (size_t)(d >> log2b);
         size_t o = 0;
         xs = o;    o += (size_t)d * 2;
         ub = o;    o += (size_t)d * 4;
+        ub2 = o;   o += base_n ? (size_t)d * 4 : 0;      // transposed copy for the butterflies over strides of base_n
         codes = o; o += (size_t)d / 2;
         o = (o + 15) & ~(size_t)15;
         r_aux = o; o += nr * 8;
@@ -121,26 +128,52 @@ __device__ __forceinline__ void radix_pass(float *ub, int d, int s, int tid)
     }
 }
 
-// Exact value of one unnormalised output coordinate, sum_k (-1)^{popcount(ii & k)} x'_k over
-// the coordinate's block, evaluated by a whole warp in fp64.
-__device__ __forceinline__ double exact_coord_warp(const uint16_t *xs, int blk_base, int b, int ii, int lane)
+// Exact value of one unnormalised output coordinate, sum_k H[k][ii] x'_k over the coordinate's block,
+// evaluated by a whole warp in fp64.  Sylvester blocks: H[k][ii] = (-1)^{popcount(ii & k)}.  With a base
+// matrix of order n0 (one block: the row): H[k][ii] = (-1)^{popcount(k / n0 & ii / n0)} * base[ii % n0][k % n0].
+__device__ __forceinline__ double exact_coord_warp(const GenParams &p, const uint16_t *xs, int blk_base, int b, int ii, int lane)
 {
     double acc = 0.0;
-    for (int k = lane; k < b; k += 32) {
-        const double v = bf16_to_f64(xs[blk_base + k]);
-        acc += (__popc(ii & k) & 1) ? -v : v;
+    if (p.base_n == 0) {
+        for (int k = lane; k < b; k += 32) {
+            const double v = bf16_to_f64(xs[blk_base + k]);
+            acc += (__popc(ii & k) & 1) ? -v : v;
+        }
+    } else {
+        const int n0 = p.base_n, i2 = ii / n0, r = ii - i2 * n0;
+        const uint32_t h0 = p.hrow[r][0], h1 = p.hrow[r][1], h2 = p.hrow[r][2];
+        int k2 = lane / n0, c = lane - k2 * n0;
+        for (int k = lane; k < b; k += 32) {
+            const double v = bf16_to_f64(xs[k]);
+            const uint32_t hw = c < 32 ? h0 : (c < 64 ? h1 : h2);
+            const uint32_t neg = (__popc(i2 & k2) ^ (hw >> (c & 31))) & 1u;
+            acc += neg ? -v : v;
+            c += 32;
+            while (c >= n0) { c -= n0; ++k2; }
+        }
     }
 #pragma unroll
     for (int o = 16; o > 0; o >>= 1) acc += __shfl_xor_sync(0xffffffffu, acc, o);
     return acc;
 }
 
-__device__ __forceinline__ double exact_coord_thread(const uint16_t *xs, int blk_base, int b, int ii)
+__device__ __forceinline__ double exact_coord_thread(const GenParams &p, const uint16_t *xs, int blk_base, int b, int ii)
 {
     double acc = 0.0;
-    for (int k = 0; k < b; ++k) {
-        const double v = bf16_to_f64(xs[blk_base + k]);
-        acc += (__popc(ii & k) & 1) ? -v : v;
+    if (p.base_n == 0) {
+        for (int k = 0; k < b; ++k) {
+            const double v = bf16_to_f64(xs[blk_base + k]);
+            acc += (__popc(ii & k) & 1) ? -v : v;
+        }
+    } else {
+        const int n0 = p.base_n, i2 = ii / n0, r = ii - i2 * n0;
+        int k2 = 0, c = 0;
+        for (int k = 0; k < b; ++k) {
+            const double v = bf16_to_f64(xs[k]);
+            const uint32_t neg = (__popc(i2 & k2) ^ (p.hrow[r][c >> 5] >> (c & 31))) & 1u;
+            acc += neg ? -v : v;
+            if (++c == n0) { c = 0; ++k2; }
+        }
     }
     return acc;
 }
@@ -207,9 +240,11 @@ __device__ __forceinline__ uint32_t exact_code(const GenParams &p, double u, dou
 __global__ void __launch_bounds__(GEN_THREADS) perq_generic_kernel(GenParams p)
 {
     extern __shared__ __align__(16) unsigned char smem[];
-    const int d = p.d, L = p.log2b, b = 1 << L, g = p.g;
-    const int nr = d / g, nb = d >> L, nchunks = d >> 3;
-    const GenSmem lay(d, g, L);
+    const int d = p.d, L = p.log2b, n0 = p.base_n, b = n0 ? d : 1 << L, g = p.g;
+    const int LB = n0 ? 30 : L;               // shift from an element index to its Hadamard block (one block with a base matrix)
+    const int bmask = n0 ? 0x3fffffff : b - 1;
+    const int nr = d / g, nb = n0 ? 1 : d >> L, nchunks = d >> 3;
+    const GenSmem lay(d, g, L, n0);
     uint16_t *xs = (uint16_t *)(smem + lay.xs);
     float *ub = (float *)(smem + lay.ub);
     uint32_t *codes = (uint32_t *)(smem + lay.codes);
@@ -223,7 +258,8 @@ __global__ void __launch_bounds__(GEN_THREADS) perq_generic_kernel(GenParams p)
     int *tie_count = tie_list + TIE_CAP;
 
     const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
-    const float err_rel = ERR_K * (float)L * TWO_M24;   // |u32 - u| <= err_rel * (block max |u32|)
+    // |u32 - u| <= err_rel * (block max |u32|); a base matrix adds a sequential sum of n0 terms to the L stages
+    const float err_rel = ERR_K * (float)(n0 ? L + n0 - 1 : L) * TWO_M24;
 
     for (long long row = blockIdx.x; row < p.T; row += gridDim.x) {
         // ---- A. row -> shared memory, through the permutation gather if there is one
@@ -246,20 +282,50 @@ __global__ void __launch_bounds__(GEN_THREADS) perq_generic_kernel(GenParams p)
         __syncthreads();
 
         // ---- B. butterfly: index bits 0..2 in registers, the rest in passes over shared memory
-        for (int c = tid; c < nchunks; c += GEN_THREADS) {
-            const uint4 w = ((const uint4 *)xs)[c];
-            float v[8] = {bf16lo(w.x), bf16hi(w.x), bf16lo(w.y), bf16hi(w.y),
-                          bf16lo(w.z), bf16hi(w.z), bf16lo(w.w), bf16hi(w.w)};
-            butterfly_regs<3>(v);
-            ((float4 *)ub)[2 * c] = make_float4(v[0], v[1], v[2], v[3]);
-            ((float4 *)ub)[2 * c + 1] = make_float4(v[4], v[5], v[6], v[7]);
-        }
-        __syncthreads();
-        for (int s = 3; s < L; s += 3) {
-            const int R = min(3, L - s);
-            if (R == 3) radix_pass<3>(ub, d, s, tid);
-            else if (R == 2) radix_pass<2>(ub, d, s, tid);
-            else radix_pass<1>(ub, d, s, tid);
+        if (n0 == 0) {
+            for (int c = tid; c < nchunks; c += GEN_THREADS) {
+                const uint4 w = ((const uint4 *)xs)[c];
+                float v[8] = {bf16lo(w.x), bf16hi(w.x), bf16lo(w.y), bf16hi(w.y),
+                              bf16lo(w.z), bf16hi(w.z), bf16lo(w.w), bf16hi(w.w)};
+                butterfly_regs<3>(v);
+                ((float4 *)ub)[2 * c] = make_float4(v[0], v[1], v[2], v[3]);
+                ((float4 *)ub)[2 * c + 1] = make_float4(v[4], v[5], v[6], v[7]);
+            }
+            __syncthreads();
+            for (int s = 3; s < L; s += 3) {
+                const int R = min(3, L - s);
+                if (R == 3) radix_pass<3>(ub, d, s, tid);
+                else if (R == 2) radix_pass<2>(ub, d, s, tid);
+                else radix_pass<1>(ub, d, s, tid);
+                __syncthreads();
+            }
+        } else {
+            // ---- B'. base matrix: every group of n0 adjacent inputs is multiplied by the +-1 base matrix (one
+            // thread per group, k ascending), the results stored transposed (output r of all groups contiguous);
+            // then the L butterfly stages over the group index, and the transpose back.
+            float *ub2 = (float *)(smem + lay.ub2);
+            const int K = 1 << L;
+            for (int grp = tid; grp < K; grp += GEN_THREADS) {
+                float xin[GEN_MAX_BASE];
+                for (int c = 0; c < n0; ++c) xin[c] = __uint_as_float((uint32_t)xs[grp * n0 + c] << 16);
+                for (int r = 0; r < n0; ++r) {
+                    float acc = 0.0f;
+                    for (int c = 0; c < n0; ++c) {
+                        const bool neg = (p.hrow[r][c >> 5] >> (c & 31)) & 1u;
+                        acc += neg ? -xin[c] : xin[c];
+                    }
+                    ub2[r * K + grp] = acc;
+                }
+            }
+            __syncthreads();
+            for (int s = 0; s < L; s += 3) {
+                const int R = min(3, L - s);
+                if (R == 3) radix_pass<3>(ub2, d, s, tid);
+                else if (R == 2) radix_pass<2>(ub2, d, s, tid);
+                else radix_pass<1>(ub2, d, s, tid);
+                __syncthreads();
+            }
+            for (int j = tid; j < d; j += GEN_THREADS) ub[(j & (K - 1)) * n0 + (j >> L)] = ub2[j];
             __syncthreads();
         }
 
@@ -286,7 +352,7 @@ __global__ void __launch_bounds__(GEN_THREADS) perq_generic_kernel(GenParams p)
                 const float lo = fminf(fminf(fminf(a.x, a.y), fminf(a.z, a.w)), fminf(fminf(e.x, e.y), fminf(e.z, e.w)));
                 atomicMax(&r_max[0], ord32(hi));
                 atomicMin(&cmin[0], ord32(lo));
-                atomicMax(&b_max[(c * 8) >> L], __float_as_uint(fmaxf(fabsf(hi), fabsf(lo))));
+                atomicMax(&b_max[(c * 8) >> LB], __float_as_uint(fmaxf(fabsf(hi), fabsf(lo))));
             }
             __syncthreads();
             const float mx32 = unord32(r_max[0]), mn32 = unord32(cmin[0]);
@@ -298,7 +364,7 @@ __global__ void __launch_bounds__(GEN_THREADS) perq_generic_kernel(GenParams p)
                 while (m) {
                     const int ic = i0 + (__ffs(m) - 1);
                     m &= m - 1;
-                    const double u = exact_coord_warp(xs, (ic >> L) << L, b, ic & (b - 1), lane);
+                    const double u = exact_coord_warp(p, xs, (ic >> LB) << LB, b, ic & bmask, lane);
                     if (lane == 0) { atomicMax(&asym[0], ord64(u)); atomicMin(&asym[1], ord64(u)); }
                 }
             }
@@ -321,14 +387,14 @@ __global__ void __launch_bounds__(GEN_THREADS) perq_generic_kernel(GenParams p)
             const float m = fmaxf(fmaxf(fmaxf(fabsf(a.x), fabsf(a.y)), fmaxf(fabsf(a.z), fabsf(a.w))),
                                   fmaxf(fmaxf(fabsf(e.x), fabsf(e.y)), fmaxf(fabsf(e.z), fabsf(e.w))));
             atomicMax(&r_max[(c * 8) / g], __float_as_uint(m));
-            atomicMax(&b_max[(c * 8) >> L], __float_as_uint(m));
+            atomicMax(&b_max[(c * 8) >> LB], __float_as_uint(m));
         }
         __syncthreads();
 
         // ---- D. which ranges need their absmax re-derived exactly, and from which elements
         for (int r = tid; p.fmt != 4 && r < nr; r += GEN_THREADS) {
             const float rm = __uint_as_float(r_max[r]);
-            const float bm = (g >= b) ? rm : __uint_as_float(b_max[(r * g) >> L]);
+            const float bm = (g >= b) ? rm : __uint_as_float(b_max[(r * g) >> LB]);
             const float err = err_rel * bm;
             bool need = rm > 0.0f;
             if (need && p.fmt == 1) {
@@ -357,7 +423,7 @@ __global__ void __launch_bounds__(GEN_THREADS) perq_generic_kernel(GenParams p)
                     while (m) {
                         const int ic = i0 + (__ffs(m) - 1);
                         m &= m - 1;
-                        const double u = exact_coord_warp(xs, (ic >> L) << L, b, ic & (b - 1), lane);
+                        const double u = exact_coord_warp(p, xs, (ic >> LB) << LB, b, ic & bmask, lane);
                         if (lane == 0) atomicMax(&r_aux[r], (unsigned long long)__double_as_longlong(fabs(u)));
                     }
                 }
@@ -394,7 +460,7 @@ __global__ void __launch_bounds__(GEN_THREADS) perq_generic_kernel(GenParams p)
         for (int c = tid; c < nchunks; c += GEN_THREADS) {
             const int i0 = c * 8, r = i0 / g;
             const float mul = r_mul[r];
-            const float tau_abs = err_rel * __uint_as_float(b_max[i0 >> L]) * mul;
+            const float tau_abs = err_rel * __uint_as_float(b_max[i0 >> LB]) * mul;
             const float4 a = ((const float4 *)ub)[2 * c], e = ((const float4 *)ub)[2 * c + 1];
             const float u[8] = {a.x, a.y, a.z, a.w, e.x, e.y, e.z, e.w};
             uint32_t word = 0u, flags = 0u;
@@ -433,7 +499,7 @@ __global__ void __launch_bounds__(GEN_THREADS) perq_generic_kernel(GenParams p)
                     tie_list[pos] = i0 + k;
                 } else {   // list full: resolve here, single-threaded
                     const int i = i0 + k;
-                    const double ue = exact_coord_thread(xs, (i >> L) << L, b, i & (b - 1));
+                    const double ue = exact_coord_thread(p, xs, (i >> LB) << LB, b, i & bmask);
                     const uint32_t code = (p.fmt == 4)
                         ? exact_code(p, ue, __longlong_as_double((long long)asym[2]), 0, __longlong_as_double((long long)asym[3]))
                         : exact_code(p, ue, __longlong_as_double((long long)r_aux[r]), r_E[r]);
@@ -449,7 +515,7 @@ __global__ void __launch_bounds__(GEN_THREADS) perq_generic_kernel(GenParams p)
             const int n = min(*tie_count, TIE_CAP);
             for (int t = warp; t < n; t += GEN_WARPS) {
                 const int i = tie_list[t], r = i / g;
-                const double ue = exact_coord_warp(xs, (i >> L) << L, b, i & (b - 1), lane);
+                const double ue = exact_coord_warp(p, xs, (i >> LB) << LB, b, i & bmask, lane);
                 if (lane == 0) {
                     const uint32_t code = (p.fmt == 4)
                         ? exact_code(p, ue, __longlong_as_double((long long)asym[2]), 0, __longlong_as_double((long long)asym[3]))

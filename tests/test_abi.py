@@ -71,7 +71,12 @@ def test_argument_validation_happens_before_any_launch(lib):
     assert call(p, None, 4, 4096, 24, 0, 0, p, p) == 3           # b not a power of two
     assert call(p, None, 4, 4096, 8192, 0, 0, p, p) == 3         # b larger than d
     assert call(p, None, 4, 12288, 8192, 0, 0, p, p) == 3        # b does not divide d
-    assert call(p, None, 4, 14336, 14336, 0, 0, p, p) == 3       # full vector needs a power of two
+    assert call(p, None, 4, 5120, 5120, 0, 0, p, p) == 3         # 2^8 * 20: no base matrix of order 20
+    assert call(p, None, 4, 14336, 28, 0, 0, p, p) == 3          # a base-matrix block only as the whole row
+    assert call(p, None, 4, 14336, 7168, 0, 0, p, p) == 3
+    assert call(p, None, 0, 14336, 14336, 0, 0, p, p) == 0       # 2^9 * 28 as the whole row: accepted (T == 0)
+    assert call(p, None, 0, 9728, 9728, 1, 32, p, p) == 0        # 2^7 * 76
+    assert call(p, None, 0, 3072, 3072, 3, 0, p, p) == 0         # 2^8 * 12
     assert call(p, None, 4, 4096, 32, 0, 12, p, p) == 4          # group % 8
     assert call(p, None, 4, 4096, 32, 0, 24, p, p) == 4          # group does not divide d
     assert call(p, None, 4, 4096, 32, 1, 64, p, p) == 4          # MX group must be 32
@@ -97,6 +102,7 @@ def test_token_diagnostics_validation(lib):
     assert f(fake, None, 4, 2048, 32, None, None) == 1
     assert f(fake, None, 4, 2050, 32, fake, None) == 2
     assert f(fake, None, 4, 2048, 8, fake, None) == 3          # blocks of at least 16
+    assert f(fake, None, 4, 3072, 3072, fake, None) == 3       # power-of-two blocks only
     assert f(C.c_void_p(0x1008), None, 4, 2048, 32, fake, None) == 6
     assert f(fake, None, 0, 2048, 32, fake, None) == 0          # T = 0: nothing to do
 

@@ -152,7 +152,8 @@ def test_fast_path_exact_ties(B, oracle):
 # ------------------------------------------------------------------ rotated values (debug format)
 
 @pytest.mark.parametrize("d,b,perm", [(2048, 16, False), (2048, 128, True), (4096, 4096, False),
-                                      (14336, 64, True), (8192, 32, False), (2048, 2048, True)])
+                                      (14336, 64, True), (8192, 32, False), (2048, 2048, True),
+                                      (3072, 3072, False), (14336, 14336, True), (9728, 9728, False)])
 def test_rotated_values(B, oracle, d, b, perm):
     bits, _ = inputs.laplace_outliers(48, d, 4, 200.0, seed=77 + d + b)
     p = inputs.random_perm(d, 78) if perm else None
@@ -235,6 +236,19 @@ def test_padding_does_not_slow_a_call_down(B, fmt, group):
     t_dense, t_padded = timed(dense), timed(padded)
     print("%s: dense %.1f us, padded %.1f us" % (fmt, 1e3 * t_dense, 1e3 * t_padded))
     assert t_padded < 2.5 * t_dense
+
+
+@pytest.mark.parametrize("fmt,group", [("int4", 0), ("int4", 128), ("mxfp4", 32), ("fp4", 0), ("int4_asym", 0)])
+@pytest.mark.parametrize("d,T,perm", [(3072, 40, False), (14336, 6, False), (9728, 5, True), (6144, 300, False), (12288, 9, True)])
+def test_full_vector_rotation_of_rows_that_are_not_a_power_of_two(B, oracle, d, T, perm, fmt, group):
+    """b = d = 2^k' * 4t (Appendix A.1: Llama-3-8B's 14336 = 2^9 * 28, Qwen3's 3072 / 6144 / 12288 = 2^k' * 12 and
+    9728 = 2^7 * 76): base-matrix rotations of adjacent inputs, then butterflies, every format."""
+    bits, _ = inputs.laplace_outliers(T, d, 4, 200.0, seed=500 + d)
+    bits[1] = 0
+    if T > 3:
+        bits[3, : d // 2] = 0
+    w = inputs.Workload("non-po2 full vector", bits, inputs.random_perm(d, 9) if perm else None, d, fmt, group, 0)
+    check(B, oracle, w)
 
 
 def test_single_huge_outlier_and_basis_rows(B, oracle):
