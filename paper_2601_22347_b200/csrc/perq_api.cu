@@ -20,6 +20,7 @@
 #include "perq_fast.cuh"
 #include "perq_tok.cuh"
 #include "perq_mx.cuh"
+#include "perq_full.cuh"
 #include "perq_stats.cuh"
 #include "perq_diag.cuh"
 #include "perq_massdiff.cuh"
@@ -303,6 +304,29 @@ int launch_mx(int log2b, const perq::FastParams &p, int grid, cudaStream_t st)
     }
 }
 
+// Full-vector kernel (b = d = 1024, 2048 or 4096): one round trip through shared memory for the chunk-index bits.
+template <int LOG2D, int MODE>
+int launch_full_inst(const perq::FastParams &p, int grid, cudaStream_t st)
+{
+    auto kernel = perq::perq_full_kernel<LOG2D, MODE>;
+    if (int rc = allow_smem(kernel, perq::FullSmem::total)) return rc;
+    if (launch_overlapped(kernel, grid, perq::FAST_THREADS, perq::FullSmem::total, st, p) != cudaSuccess) {
+        (void)cudaGetLastError();
+        return PERQ_ERR_CUDA;
+    }
+    return PERQ_OK;
+}
+
+template <int MODE>
+int launch_full(int segs, const perq::FastParams &p, int grid, cudaStream_t st)
+{
+    switch (segs) {
+    case 1: return launch_full_inst<10, MODE>(p, grid, st);
+    case 2: return launch_full_inst<11, MODE>(p, grid, st);
+    default: return launch_full_inst<12, MODE>(p, grid, st);
+    }
+}
+
 // Lean per-token kernel: INT4 or E2M1 with one scale per token, unpermuted, d in {2048, 4096, 8192}, b <= 128.
 template <int LOG2B, int MODE, int LOG2G>
 int launch_tok_inst(const perq::FastParams &p, int grid, cudaStream_t st)
@@ -404,6 +428,8 @@ int try_launch_fast(const void *x, const int32_t *perm, int64_t T, int32_t d, in
         const int mx_grid = (int)std::min<long long>((mx_units + perq::FAST_WARPS - 1) / perq::FAST_WARPS, sms);
         return launch_mx(ilog2(b), p, mx_grid, st);
     }
+    if (full && mode == perq::MODE_MX && segs <= 4)          // (units are rows; grid as computed above)
+        return launch_full<perq::MODE_MX>(segs, p, grid, st);
     if (full)
         return mode == perq::MODE_MX ? launch_fast_full<perq::MODE_MX>(G, p, grid, st)
                                      : launch_fast_full<perq::MODE_TOKEN>(G, p, grid, st);
