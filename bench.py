@@ -36,18 +36,17 @@ T_HEAD, D_HEAD, B_HEAD, FMT_HEAD, GROUP_HEAD = 16384, 4096, 32, "int4", 0
 ORACLE_FMT = {"int4": 0, "mxfp4": 1, "fp4": 3}     # format numbers of oracle/perq_oracle.c
 
 # DRAM traffic of one launch of the headline kernel (dram__bytes_read.sum + dram__bytes_write.sum from an ncu
-# capture) is kept in a small tracked file together with a hash of the kernel sources it was captured on;
+# capture) is kept in a small tracked file together with the names and a hash of the sources that kernel is compiled from;
 # when the sources have changed since, the bench reports no traffic figure.
 TRAFFIC_FILE = os.path.join(ROOT, "paper_2601_22347_b200", "ncu_traffic.json")
 
 
-def kernel_sources_hash():
+def kernel_sources_hash(names):
+    """SHA-256 over the named files of csrc/ (the sources a captured kernel is compiled from)."""
     import hashlib
     csrc = os.path.join(ROOT, "paper_2601_22347_b200", "csrc")
     h = hashlib.sha256()
-    for name in sorted(os.listdir(csrc)):
-        if not os.path.isfile(os.path.join(csrc, name)):
-            continue
+    for name in sorted(names):
         with open(os.path.join(csrc, name), "rb") as f:
             h.update(name.encode() + b"\0" + f.read())
     return h.hexdigest()
@@ -55,13 +54,13 @@ def kernel_sources_hash():
 
 def captured_traffic(fmt):
     """Bytes per launch from the last ncu capture of this format's headline kernel, or None if there is none
-    for the kernel sources as they are now."""
+    for that kernel's sources as they are now."""
     try:
         with open(TRAFFIC_FILE) as f:
-            rec = json.load(f)
-        if rec.get("sources_sha256") != kernel_sources_hash():
+            rec = json.load(f).get(fmt)
+        if rec is None or rec.get("sources_sha256") != kernel_sources_hash(rec["sources"]):
             return None
-        return rec.get("dram_bytes_per_launch", {}).get(fmt)
+        return rec.get("dram_bytes_per_launch")
     except Exception:
         return None
 
