@@ -46,9 +46,14 @@ struct GenParams {
     uint32_t hrow[GEN_MAX_BASE][3];
 };
 
+// Base matrix in shared memory for the tensor-core stage: NP output columns (a multiple of 8), rows of KP + 8
+// bf16 (KP = inputs padded to a multiple of 16; the 8 extra keep the fragment loads off one bank).
+__host__ __device__ constexpr int gen_base_np(int n0) { return (n0 + 7) / 8 * 8; }
+__host__ __device__ constexpr int gen_base_ldk(int n0) { return (n0 + 15) / 16 * 16 + 8; }
+
 // Shared-memory carve-up, computed identically on host (for the launch) and device.
 struct GenSmem {
-    size_t xs, ub, ub2, codes, r_max, r_thr, r_mul, r_aux, r_E, b_max, ties, asym, total;
+    size_t xs, ub, ub2, bmat, codes, r_max, r_thr, r_mul, r_aux, r_E, b_max, ties, asym, total;
     __host__ __device__ GenSmem(int d, int g, int log2b, int base_n)
     {
         const size_t nr = (size_t)(d / g), nb = base_n ? 1 : (size_t)(d >> log2b);
@@ -56,6 +61,7 @@ struct GenSmem {
         xs = o;    o += (size_t)d * 2;
         ub = o;    o += (size_t)d * 4;
         ub2 = o;   o += base_n ? (size_t)d * 4 : 0;      // transposed copy for the butterflies over strides of base_n
+        bmat = o;  o += base_n ? (size_t)gen_base_np(base_n) * gen_base_ldk(base_n) * 2 : 0;   // base matrix, bf16, [n][k]
         codes = o; o += (size_t)d / 2;
         o = (o + 15) & ~(size_t)15;
         r_aux = o; o += nr * 8;
@@ -126,6 +132,14 @@ __device__ __forceinline__ void radix_pass(float *ub, int d, int s, int tid)
 #pragma unroll
         for (int e = 0; e < (1 << R); ++e) ub[base + (e << s)] = v[e];
     }
+}
+
+// d += a * b, one m16n8k16 tile: bf16 operands (a: 16 x 16 row-major fragment, b: 16 x 8), fp32 accumulators.
+__device__ __forceinline__ void gen_mma_bf16(float (&c)[4], const uint32_t (&a)[4], uint32_t b0, uint32_t b1)
+{
+    asm volatile("mma.sync.aligned.m16n8k16.row.col.f32.bf16.bf16.f32 {%0,%1,%2,%3}, {%4,%5,%6,%7}, {%8,%9}, {%0,%1,%2,%3};"
+                 : "+f"(c[0]), "+f"(c[1]), "+f"(c[2]), "+f"(c[3])
+                 : "r"(a[0]), "r"(a[1]), "r"(a[2]), "r"(a[3]), "r"(b0), "r"(b1));
 }
 
 // Exact value of one unnormalised output coordinate, sum_k H[k][ii] x'_k over the coordinate's block,
@@ -261,6 +275,17 @@ __global__ void __launch_bounds__(GEN_THREADS) perq_generic_kernel(GenParams p)
     // |u32 - u| <= err_rel * (block max |u32|); a base matrix adds a sequential sum of n0 terms to the L stages
     const float err_rel = ERR_K * (float)(n0 ? L + n0 - 1 : L) * TWO_M24;
 
+    if (n0) {   // base matrix as bf16 +-1 (0 in the padding), [output n][input k]: B[k][n] = base[n][k] (symmetric)
+        uint16_t *bmw = (uint16_t *)(smem + lay.bmat);
+        const int NP = gen_base_np(n0), LDK = gen_base_ldk(n0);
+        for (int e = tid; e < NP * LDK; e += GEN_THREADS) {
+            const int n = e / LDK, k = e - n * LDK;
+            uint16_t v = 0;
+            if (n < n0 && k < n0) v = ((p.hrow[n][k >> 5] >> (k & 31)) & 1u) ? 0xBF80 : 0x3F80;
+            bmw[e] = v;
+        }
+        __syncthreads();
+    }
     for (long long row = blockIdx.x; row < p.T; row += gridDim.x) {
         // ---- A. row -> shared memory, through the permutation gather if there is one
         const uint4 *src = (const uint4 *)(p.x + (size_t)row * d);
@@ -300,21 +325,39 @@ __global__ void __launch_bounds__(GEN_THREADS) perq_generic_kernel(GenParams p)
                 __syncthreads();
             }
         } else {
-            // ---- B'. base matrix: every group of n0 adjacent inputs is multiplied by the +-1 base matrix (one
-            // thread per group, k ascending), the results stored transposed (output r of all groups contiguous);
-            // then the L butterfly stages over the group index, and the transpose back.
+            // ---- B'. base matrix: the groups of n0 adjacent inputs times the +-1 base matrix -- a dense contraction,
+            // on the tensor cores: m16n8k16 tiles over 16 groups x 8 outputs, bf16 operands (products exact), fp32
+            // accumulators.  A warp takes 16 groups at a time, keeps their input fragments (the bf16 row in shared
+            // memory read as 32-bit pairs, zero beyond n0) and walks the output tiles; results are stored
+            // transposed (output r of all groups contiguous).  Then the L butterfly stages over the group index,
+            // and the transpose back.
             float *ub2 = (float *)(smem + lay.ub2);
+            const uint16_t *bm = (const uint16_t *)(smem + lay.bmat);
             const int K = 1 << L;
-            for (int grp = tid; grp < K; grp += GEN_THREADS) {
-                float xin[GEN_MAX_BASE];
-                for (int c = 0; c < n0; ++c) xin[c] = __uint_as_float((uint32_t)xs[grp * n0 + c] << 16);
-                for (int r = 0; r < n0; ++r) {
-                    float acc = 0.0f;
-                    for (int c = 0; c < n0; ++c) {
-                        const bool neg = (p.hrow[r][c >> 5] >> (c & 31)) & 1u;
-                        acc += neg ? -xin[c] : xin[c];
+            const int KT = (n0 + 15) >> 4, NT = (n0 + 7) >> 3, LDK = gen_base_ldk(n0);
+            const int fg = lane >> 2, fq = lane & 3;
+            for (int mt = warp; mt * 16 < K; mt += GEN_WARPS) {
+                uint32_t afr[(GEN_MAX_BASE + 15) / 16][4];
+#pragma unroll
+                for (int kt = 0; kt < (GEN_MAX_BASE + 15) / 16; ++kt) {
+#pragma unroll
+                    for (int h = 0; h < 4; ++h) {
+                        const int grp = mt * 16 + fg + 8 * (h & 1), kk = kt * 16 + 2 * fq + 8 * (h >> 1);
+                        afr[kt][h] = (kt < KT && grp < K && kk < n0) ? *(const uint32_t *)(xs + grp * n0 + kk) : 0u;
                     }
-                    ub2[r * K + grp] = acc;
+                }
+                for (int nt = 0; nt < NT; ++nt) {
+                    float c[4] = {0.0f, 0.0f, 0.0f, 0.0f};
+                    const uint16_t *brow = bm + (nt * 8 + fg) * LDK + 2 * fq;
+#pragma unroll
+                    for (int kt = 0; kt < (GEN_MAX_BASE + 15) / 16; ++kt) {
+                        if (kt < KT) gen_mma_bf16(c, afr[kt], *(const uint32_t *)(brow + kt * 16), *(const uint32_t *)(brow + kt * 16 + 8));
+                    }
+#pragma unroll
+                    for (int h = 0; h < 4; ++h) {
+                        const int grp = mt * 16 + fg + 8 * (h >> 1), r = nt * 8 + 2 * fq + (h & 1);
+                        if (grp < K && r < n0) ub2[r * K + grp] = c[h];
+                    }
                 }
             }
             __syncthreads();
